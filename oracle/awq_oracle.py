@@ -1,0 +1,239 @@
+"""CPU oracle for the W4A16 group-wise linear layer.  TEST INFRASTRUCTURE ONLY.
+
+Nothing in the product path may import this module: it exists so that the CUDA kernels
+can be checked against a plain, slow, independent statement of what they must compute.
+It shares no code with the CUDA path (no headers, tables, helpers or constants); it is
+written in numpy, every fp32 step being a single IEEE-754 binary32 operation (numpy
+ufuncs on float32 arrays do not contract into fused multiply-adds) and the linear layer
+being evaluated in fp64.
+
+What is computed, and where it comes from
+-----------------------------------------
+* channel_scale      s = s_X ** alpha, per input channel                     (Eq. 5)
+* quantize           w' = w * s folded into the weight (Eq. 3, Eq. 4), then the
+                     group-wise round-to-nearest grid Delta * Round(w'/Delta)   (Eq. 2),
+                     in the asymmetric min/max form with an integer zero point in
+                     [0, 15] and Delta stored in fp16 (Sec. 3.2: "Delta and x are
+                     represented in FP16").
+* pack_* / unpack_*  eight 4-bit codes per 32-bit word in the order
+                     w{0,2,4,6,1,3,5,7} (Sec. 4.2, SIMD-aware weight packing), inside
+                     a 128-row x 64-column tile whose 16-byte pieces are ordered for a
+                     warp-wide register fragment; see `qweight_location`.
+* dequantize         (q - z) * Delta, exact in fp64.
+* linear             y = x . dequant(Wq)^T in fp64 (Sec. 4.2, on-the-fly weight
+                     dequantization followed by the matrix product; here unfused).
+
+Readings adopted where the paper is silent
+------------------------------------------
+The paper's Eq. 2 is the symmetric abs-max grid.  The deployed form asked for here is
+asymmetric: Delta = (max - min) / 15, z = Round(-min / Delta) clamped to [0, 15],
+q = clamp(Round(w'/Delta) + z, 0, 15).  Round is round-half-to-even in fp32; Delta is
+rounded to fp16 *before* it is used, so that quantize and dequantize use the same grid; the
+group's raw min and max are used (the range is not widened to contain 0); a degenerate
+group (Delta rounds to 0 or is not finite) takes Delta = 1.  w * s stays in fp32.
+Parity for these asymmetric details is unpinned by the paper (it prints no worked numeric
+example of Q); they are pinned by closed-form invariants, grid-aligned round trips and
+brute-force enumeration in tests/test_oracle_pins.py.
+"""
+from __future__ import annotations
+
+import numpy as np
+
+TILE_ROWS = 128          # output channels per packed tile
+TILE_COLS = 64           # input channels per packed tile
+WORDS_PER_TILE = TILE_ROWS * TILE_COLS // 8
+# Nibble position (bits 4p..4p+3) of element slot e inside a word: slot order read from
+# the low nibble upwards is {0,2,4,6,1,3,5,7} (Sec. 4.2).
+NIBBLE_OF_SLOT = (0, 4, 1, 5, 2, 6, 3, 7)
+
+
+# --------------------------------------------------------------------------- Eq. 5
+def channel_scale(act_mean_abs, alpha: float) -> np.ndarray:
+    """s_k = a_k ** alpha as fp32 [K]  (Eq. 5: s = s_X^alpha).
+
+    alpha = 0 means "do not scale" (s = 1).  A statistic that is not finite or not
+    positive gives s_k = 1.  alpha = 1 is the identity and alpha = 0.5 the correctly
+    rounded fp32 square root; any other alpha is the fp64 power rounded once to fp32.
+    """
+    alpha = float(alpha)
+    if not (0.0 <= alpha <= 1.0):
+        raise ValueError("alpha must lie in [0, 1]")
+    a = np.asarray(act_mean_abs, dtype=np.float32)
+    if alpha == 0.0:
+        return np.ones(a.shape, dtype=np.float32)
+    ok = np.isfinite(a) & (a > 0)
+    safe = np.where(ok, a, np.float32(1.0)).astype(np.float32)
+    if alpha == 1.0:
+        s = safe
+    elif alpha == 0.5:
+        s = np.sqrt(safe, dtype=np.float32)
+    else:
+        s = np.power(safe.astype(np.float64), alpha).astype(np.float32)
+    return np.where(ok, s, np.float32(1.0)).astype(np.float32)
+
+
+# --------------------------------------------------------------------- Eq. 2 - Eq. 4
+def quantize(W, s, group: int):
+    """Group-wise asymmetric INT4 round-to-nearest of W * diag(s).
+
+    W fp16 [N][K]; s fp32 [K]; groups are `group` consecutive input channels of one
+    output row.  Returns (codes u8 [N][K], zeros u8 [N][K/group], scales fp16 [N][K/group]).
+    """
+    W = np.asarray(W)
+    assert W.dtype == np.float16 and W.ndim == 2
+    N, K = W.shape
+    assert K % group == 0
+    ng = K // group
+    s = np.asarray(s, dtype=np.float32)
+    assert s.shape == (K,)
+
+    codes = np.empty((N, K), dtype=np.uint8)
+    zeros = np.empty((N, ng), dtype=np.uint8)
+    scales = np.empty((N, ng), dtype=np.float16)
+    rows = max(1, (1 << 23) // K)                       # bound the fp32 temporaries
+    f15, f0 = np.float32(15.0), np.float32(0.0)
+    for r0 in range(0, N, rows):
+        r1 = min(N, r0 + rows)
+        wp = W[r0:r1].astype(np.float32) * s[None, :]   # Eq. 3: w * s, one fp32 multiply
+        wg = wp.reshape(r1 - r0, ng, group)
+        mn = wg.min(axis=2)
+        mx = wg.max(axis=2)
+        with np.errstate(over="ignore", invalid="ignore", divide="ignore"):
+            d16 = ((mx - mn) / f15).astype(np.float16)  # Delta, stored in fp16
+            bad = ~np.isfinite(d16) | (d16 == 0)
+            d16 = np.where(bad, np.float16(1.0), d16).astype(np.float16)
+            d = d16.astype(np.float32)
+            z = np.clip(np.rint((-mn) / d), f0, f15)    # zero point, half-to-even
+            q = np.rint(wg / d[:, :, None]) + z[:, :, None]   # Eq. 2: Round(w / Delta)
+            q = np.clip(q, f0, f15)
+        codes[r0:r1] = q.reshape(r1 - r0, K).astype(np.uint8)
+        zeros[r0:r1] = z.astype(np.uint8)
+        scales[r0:r1] = d16
+    return codes, zeros, scales
+
+
+# ------------------------------------------------------------------- packed layout
+def qweight_location(n: int, k: int, K: int):
+    """(word index, nibble position) of code (n, k) in the packed weight array.
+
+    Tiles of 128 output rows x 64 input columns are stored whole (1024 words), row-slab
+    major: tile = (n // 128) * (K // 64) + k // 64.  A tile is 8 bands of 16 rows; a band
+    is 32 pieces of 16 bytes; piece (g, t) holds rows g and g+8 of the band and columns
+    16t .. 16t+15 of the tile.  Word j of a piece holds columns 16t+4j .. 16t+4j+3 of both
+    rows in the slot order (g,c0) (g,c1) (g+8,c0) (g+8,c1) (g,c2) (g,c3) (g+8,c2) (g+8,c3),
+    and slot e sits at nibble NIBBLE_OF_SLOT[e].
+    """
+    tile = (n // TILE_ROWS) * (K // TILE_COLS) + k // TILE_COLS
+    r, c = n % TILE_ROWS, k % TILE_COLS
+    band, rr = r // 16, r % 16
+    g, h = rr % 8, rr // 8
+    t, j, i = c // 16, (c % 16) // 4, c % 4
+    word = tile * WORDS_PER_TILE + band * 128 + (g * 4 + t) * 4 + j
+    slot = (i // 2) * 4 + h * 2 + (i % 2)
+    return word, NIBBLE_OF_SLOT[slot]
+
+
+def zeros_location(n: int, gi: int, N: int):
+    """(byte index, nibble position) of the zero point of row n, group gi.
+
+    One byte holds the zero points of rows g (low nibble) and g+8 (high nibble) of a
+    16-row band; bands follow each other along N, groups along the outer axis.
+    """
+    band, rr = n // 16, n % 16
+    return gi * (N // 2) + band * 8 + rr % 8, rr // 8
+
+
+def pack_qweight(codes) -> np.ndarray:
+    """codes u8 [N][K] -> uint32 [N*K/8] in the layout of `qweight_location`."""
+    codes = np.asarray(codes, dtype=np.uint8)
+    N, K = codes.shape
+    assert N % TILE_ROWS == 0 and K % TILE_COLS == 0
+    # axes: R, band, h, g, C, t, j, ihi, ilo
+    a = codes.reshape(N // 128, 8, 2, 8, K // 64, 4, 4, 2, 2)
+    # -> R, C, band, g, t, j, ihi, h, ilo   (the last three are the slot bits, high to low)
+    a = a.transpose(0, 4, 1, 3, 5, 6, 7, 2, 8).reshape(-1, 8).astype(np.uint32)
+    words = np.zeros(a.shape[0], dtype=np.uint32)
+    for slot in range(8):
+        words |= a[:, slot] << np.uint32(4 * NIBBLE_OF_SLOT[slot])
+    return words
+
+
+def unpack_qweight(words, N: int, K: int) -> np.ndarray:
+    """Inverse of pack_qweight."""
+    words = np.asarray(words, dtype=np.uint32).reshape(-1)
+    assert words.size == N * K // 8
+    a = np.empty((words.size, 8), dtype=np.uint8)
+    for slot in range(8):
+        a[:, slot] = (words >> np.uint32(4 * NIBBLE_OF_SLOT[slot])) & np.uint32(0xF)
+    a = a.reshape(N // 128, K // 64, 8, 8, 4, 4, 2, 2, 2)
+    return a.transpose(0, 2, 7, 3, 1, 4, 5, 6, 8).reshape(N, K)
+
+
+def pack_zeros(zeros) -> np.ndarray:
+    """zeros u8 [N][ng] -> u8 [ng][N/2] in the layout of `zeros_location`."""
+    zeros = np.asarray(zeros, dtype=np.uint8)
+    N, ng = zeros.shape
+    a = zeros.T.reshape(ng, N // 16, 2, 8)              # gi, band, h, g
+    return (a[:, :, 0, :] | (a[:, :, 1, :] << 4)).reshape(ng, N // 2).astype(np.uint8)
+
+
+def unpack_zeros(packed, N: int, ng: int) -> np.ndarray:
+    p = np.asarray(packed, dtype=np.uint8).reshape(ng, N // 16, 8)
+    a = np.stack([p & 0xF, p >> 4], axis=2)             # gi, band, h, g
+    return a.reshape(ng, N).T.copy()
+
+
+def pack_scales(scales) -> np.ndarray:
+    """scales fp16 [N][ng] -> fp16 [ng][N] (group-major)."""
+    return np.ascontiguousarray(np.asarray(scales, dtype=np.float16).T)
+
+
+def quantize_pack(W, act_mean_abs, alpha: float, group: int):
+    """The whole offline step: returns (qweight u32, scales fp16 [ng][N], zeros u8 [ng][N/2])."""
+    K = W.shape[1]
+    a = np.ones(K, np.float32) if act_mean_abs is None else act_mean_abs
+    codes, zeros, scales = quantize(W, channel_scale(a, alpha), group)
+    return pack_qweight(codes), pack_scales(scales), pack_zeros(zeros)
+
+
+# ----------------------------------------------------------------- dequantize, multiply
+def dequantize(codes, zeros, scales, group: int) -> np.ndarray:
+    """Wdq[n][k] = (q - z) * Delta in fp64 (exact: a 5-bit integer times an fp16 value)."""
+    N, K = codes.shape
+    ng = K // group
+    q = codes.reshape(N, ng, group).astype(np.float64)
+    z = np.asarray(zeros, dtype=np.float64)[:, :, None]
+    d = np.asarray(scales, dtype=np.float16).astype(np.float64)[:, :, None]
+    return ((q - z) * d).reshape(N, K)
+
+
+def linear(x, Wdq) -> np.ndarray:
+    """y[m][n] = sum_k x[m][k] * Wdq[n][k] in fp64; x is fp16 and already divided by s."""
+    x = np.asarray(x)
+    assert x.dtype == np.float16
+    return x.astype(np.float64) @ np.asarray(Wdq, dtype=np.float64).T
+
+
+def linear_from_packed(x, qweight, scales_gn, zeros_packed, N: int, K: int, group: int,
+                       rows=None) -> np.ndarray:
+    """Dequantize-then-multiply starting from the packed arrays (optionally only the
+    output channels listed in `rows`, for sampled checks at sizes where the full product
+    is too slow)."""
+    ng = K // group
+    codes = unpack_qweight(qweight, N, K)
+    zeros = unpack_zeros(zeros_packed, N, ng)
+    scales = np.asarray(scales_gn, dtype=np.float16).reshape(ng, N).T
+    if rows is not None:
+        codes, zeros, scales = codes[rows], zeros[rows], scales[rows]
+    return linear(x, dequantize(codes, zeros, scales, group))
+
+
+def parity_errors(y, y_ref):
+    """(relative L2 error, max abs error / max |y_ref|) of y against the fp64 reference."""
+    y = np.asarray(y, dtype=np.float64)
+    y_ref = np.asarray(y_ref, dtype=np.float64)
+    den = np.linalg.norm(y_ref)
+    amax = np.abs(y_ref).max() if y_ref.size else 0.0
+    rel = np.linalg.norm(y - y_ref) / den if den > 0 else float(np.linalg.norm(y - y_ref))
+    mx = np.abs(y - y_ref).max() / amax if amax > 0 else float(np.abs(y - y_ref).max(initial=0.0))
+    return float(rel), float(mx)

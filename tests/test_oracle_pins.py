@@ -1,0 +1,408 @@
+"""Pins for the CPU oracle: each test checks oracle/awq_oracle.py against something fixed
+by the paper or by mathematics (closed forms, exact special cases, brute force), never
+against the oracle's own formula retyped and never against the CUDA path."""
+import itertools
+import os
+import struct
+from fractions import Fraction
+
+import numpy as np
+import pytest
+
+from oracle import awq_oracle as orc
+from paper_2306_00978_b200 import synth
+
+
+# ----------------------------------------------------------------------------- helpers
+def _f16_rne_bits(x: float) -> int:
+    """Independent fp32 -> fp16 round-to-nearest-even on the bit patterns (no numpy cast)."""
+    b = struct.unpack("<I", struct.pack("<f", x))[0]
+    sign = (b >> 16) & 0x8000
+    exp = (b >> 23) & 0xFF
+    man = b & 0x7FFFFF
+    if exp == 0xFF:
+        return sign | 0x7C00 | (0x200 if man else 0)
+    e = exp - 127
+    if e > 15:
+        return sign | 0x7C00
+    if e >= -14:
+        m = man | 0x800000
+        shift = 13
+        he = e + 15
+    else:
+        if e < -25:
+            return sign
+        m = man | 0x800000
+        shift = 13 + (-14 - e)
+        he = 0
+    q, r = m >> shift, m & ((1 << shift) - 1)
+    half = 1 << (shift - 1)
+    if r > half or (r == half and (q & 1)):
+        q += 1
+    if he == 0:
+        return sign | q                       # a carry into bit 10 becomes the smallest normal
+    q -= 0x400
+    out = (he << 10) + q                      # a mantissa carry increments the exponent
+    return sign | min(out, 0x7C00)
+
+
+def _golden(path):
+    rows = {}
+    with open(path) as f:
+        for line in f:
+            line = line.strip()
+            if line and not line.startswith("#"):
+                k, *v = line.split()
+                rows[k] = v
+    return rows
+
+
+def _grid_aligned(rng, N, K, G, exps=(-6, -9)):
+    """W = (q - z) * 2^-e with codes 0 and 15 present in every group: exactly representable."""
+    ng = K // G
+    q = rng.integers(0, 16, size=(N, ng, G), dtype=np.int64)
+    q[:, :, 0], q[:, :, 1] = 0, 15
+    q = rng.permuted(q, axis=2)
+    z = rng.integers(0, 16, size=(N, ng), dtype=np.int64)
+    e = rng.integers(exps[1], exps[0] + 1, size=(N, ng))
+    d = np.ldexp(1.0, e)
+    W = ((q - z[:, :, None]) * d[:, :, None]).reshape(N, K)
+    W16 = W.astype(np.float16)
+    assert np.array_equal(W16.astype(np.float64), W)
+    return W16, q.reshape(N, K).astype(np.uint8), z.astype(np.uint8), d.astype(np.float16)
+
+
+# ------------------------------------------------------------------- rounding primitives
+def test_round_half_to_even_table():
+    # the quantizer's Round(.) must be half-to-even (np.rint), not half-away (np.round is
+    # also half-to-even in numpy, so pin the values themselves)
+    x = np.array([0.5, 1.5, 2.5, -0.5, -1.5, 3.5, 6.5, 7.5], dtype=np.float32)
+    assert np.rint(x).tolist() == [0.0, 2.0, 2.0, -0.0, -2.0, 4.0, 6.0, 8.0]
+    # observable through the oracle: Delta = 1, min = -7 -> z = 7; w = 0.5, 1.5, 2.5 -> 0, 2, 2
+    W = np.array([[-7, 8, 0.5, 1.5, 2.5, -0.5, -1.5, 3.5]], dtype=np.float16)
+    codes, zeros, scales = orc.quantize(W, np.ones(8, np.float32), 8)
+    assert float(scales[0, 0]) == 1.0 and int(zeros[0, 0]) == 7
+    assert codes[0].tolist() == [0, 15, 7, 9, 9, 7, 5, 11]
+
+
+def test_fp16_rounding_matches_bit_level_definition():
+    rng = np.random.default_rng(1)
+    bits = rng.integers(0, 2**32, size=200_000, dtype=np.uint64).astype(np.uint32)
+    specials = np.array([0x33000000, 0x33000001, 0x33800000, 0x387FC000, 0x387FE000, 0x387FF000,
+                         0x477FE000, 0x477FEFFF, 0x477FF000, 0x3F801000, 0x3F803000, 0x3F802FFF,
+                         0x38800000, 0x00000001, 0x80000000], dtype=np.uint32)
+    bits = np.concatenate([bits, specials])
+    x = bits.view(np.float32)
+    x = x[np.isfinite(x)]
+    with np.errstate(over="ignore"):
+        got = x.astype(np.float16).view(np.uint16)
+    sample = np.concatenate([np.arange(0, 2000), np.arange(x.size - specials.size, x.size)])
+    for i in sample:
+        assert int(got[i]) == _f16_rne_bits(float(x[i])), hex(int(x[i:i + 1].view(np.uint32)[0]))
+
+
+# ------------------------------------------------------------------------ Eq. 5: s = s_X^a
+def test_channel_scale_special_cases():
+    a = np.array([1.0, 4.0, 16.0, 0.25, 0.0, -3.0, np.inf, np.nan, 2.0], dtype=np.float32)
+    assert orc.channel_scale(a, 0.0).tolist() == [1.0] * 9            # 0 = "do not scale"
+    s1 = orc.channel_scale(a, 1.0)
+    assert s1[:4].tolist() == [1.0, 4.0, 16.0, 0.25] and s1[4:8].tolist() == [1.0] * 4
+    sh = orc.channel_scale(a, 0.5)
+    assert sh[:4].tolist() == [1.0, 2.0, 4.0, 0.5] and sh[4:8].tolist() == [1.0] * 4
+    assert sh[8] == np.float32(np.sqrt(2.0))
+    # general alpha: exact powers of two, and agreement with exact rational roots
+    sq = orc.channel_scale(np.array([16.0, 81.0], np.float32), 0.25)
+    assert sq.tolist() == [2.0, 3.0]
+    with pytest.raises(ValueError):
+        orc.channel_scale(a, 1.5)
+
+
+# ---------------------------------------------------- Eq. 2: grid-aligned weights round-trip
+@pytest.mark.parametrize("G", [64, 128])
+def test_grid_aligned_round_trip(G):
+    rng = np.random.default_rng(7)
+    N, K = 128, 4 * G
+    W, q, z, d = _grid_aligned(rng, N, K, G)
+    codes, zeros, scales = orc.quantize(W, orc.channel_scale(np.ones(K, np.float32), 0.0), G)
+    assert np.array_equal(codes, q)
+    assert np.array_equal(zeros, z)
+    assert np.array_equal(scales.view(np.uint16), d.view(np.uint16))
+    back = orc.dequantize(codes, zeros, scales, G)
+    assert np.array_equal(back, W.astype(np.float64))                   # bit-for-bit
+
+
+# ------------------------------------- Eq. 3/4: Q(W diag(s)) (diag(s)^-1 x) = W x when exact
+def test_scaling_equivalence_exact_case():
+    rng = np.random.default_rng(11)
+    N, K, G, M = 128, 256, 128, 3
+    Ws, _, _, _ = _grid_aligned(rng, N, K, G, exps=(-5, -7))             # this is W * s
+    a = rng.choice(np.array([1.0, 4.0, 16.0], np.float32), size=K)
+    s = orc.channel_scale(a, 0.5)
+    assert set(np.unique(s).tolist()) <= {1.0, 2.0, 4.0}
+    W = (Ws.astype(np.float64) / s).astype(np.float16)                   # exact: powers of two
+    assert np.array_equal(W.astype(np.float64) * s, Ws.astype(np.float64))
+    x = (rng.integers(-64, 65, size=(M, K)) / 8.0).astype(np.float16)
+    xs = (x.astype(np.float32) / s[None, :]).astype(np.float16)
+    assert np.array_equal(xs.astype(np.float64) * s, x.astype(np.float64))
+    codes, zeros, scales = orc.quantize(W, s, G)
+    y = orc.linear(xs, orc.dequantize(codes, zeros, scales, G))
+    y_fp = x.astype(np.float64) @ W.astype(np.float64).T                 # the unquantized layer
+    assert np.abs(y - y_fp).max() <= 1e-13 * np.abs(y_fp).max()
+    # and the scale really matters: quantizing the *unscaled* W is not on its grid any more
+    c2, z2, s2 = orc.quantize(W, np.ones(K, np.float32), G)
+    assert np.abs(orc.dequantize(c2, z2, s2, G) - W.astype(np.float64)).max() > 0
+
+
+# ----------------------------------------------------------------- Sec. 4.2: the pack order
+def test_pack_order_worked_example(golden_dir):
+    g = _golden(os.path.join(golden_dir, "pack_order.txt"))
+    order = [int(v) for v in g["order"]]
+    want = int(g["word_for_codes_0_to_7"][0], 16)
+    # the slot stored at nibble p is order[p]
+    assert [orc.NIBBLE_OF_SLOT.index(p) for p in range(8)] == order
+    codes = np.zeros((128, 64), np.uint8)
+    # the eight slots of word 0 are rows 0 and 8, columns 0..3 of the first piece
+    slots = [(0, 0), (0, 1), (8, 0), (8, 1), (0, 2), (0, 3), (8, 2), (8, 3)]
+    for v, (n, k) in enumerate(slots):
+        codes[n, k] = v
+    words = orc.pack_qweight(codes)
+    assert int(words[0]) == want == 0x75316420
+    assert not words[1:].any()
+    # the two-at-a-time register conversion that motivates the order: masking the low
+    # nibble of each 16-bit half yields slots (0,1); shifting by 4, 8, 12 yields (2,3), (4,5), (6,7)
+    w = int(words[0])
+    pairs = [((w >> sh) & 0xF, (w >> (sh + 16)) & 0xF) for sh in (0, 4, 8, 12)]
+    assert pairs == [(0, 1), (2, 3), (4, 5), (6, 7)]
+
+
+def test_pack_matches_location_formula_and_round_trips():
+    rng = np.random.default_rng(3)
+    for N, K in [(128, 64), (256, 192)]:
+        codes = rng.integers(0, 16, size=(N, K), dtype=np.uint8)
+        words = orc.pack_qweight(codes)
+        ref = [0] * (N * K // 8)
+        seen = set()
+        for n in range(N):
+            for k in range(K):
+                wi, p = orc.qweight_location(n, k, K)
+                assert (wi, p) not in seen
+                seen.add((wi, p))
+                ref[wi] |= int(codes[n, k]) << (4 * p)
+        assert words.tolist() == ref
+        assert np.array_equal(orc.unpack_qweight(words, N, K), codes)
+    # a tile is 4096 contiguous bytes and tiles of one 128-row slab follow each other along K
+    assert orc.qweight_location(127, 63, 192)[0] == 1023
+    assert orc.qweight_location(0, 64, 192)[0] == 1024
+    assert orc.qweight_location(128, 0, 192)[0] == 3 * 1024
+
+
+def test_zero_and_scale_packing():
+    rng = np.random.default_rng(5)
+    N, ng = 256, 3
+    zeros = rng.integers(0, 16, size=(N, ng), dtype=np.uint8)
+    packed = orc.pack_zeros(zeros)
+    assert packed.shape == (ng, N // 2)
+    flat = packed.reshape(-1)
+    for n in range(N):
+        for gi in range(ng):
+            b, nib = orc.zeros_location(n, gi, N)
+            assert (int(flat[b]) >> (4 * nib)) & 0xF == int(zeros[n, gi])
+    assert np.array_equal(orc.unpack_zeros(packed, N, ng), zeros)
+    sc = rng.standard_normal((N, ng)).astype(np.float16)
+    assert np.array_equal(orc.pack_scales(sc)[2], sc[:, 2])
+
+
+# ------------------------------------------------------- dequantize-then-multiply, exactly
+def test_linear_special_cases():
+    rng = np.random.default_rng(13)
+    N, K, G, M = 128, 256, 128, 4
+    zeros = rng.integers(0, 16, size=(N, K // G), dtype=np.uint8)
+    scales = (rng.random((N, K // G)) * 0.01 + 0.001).astype(np.float16)
+    x = rng.standard_normal((M, K)).astype(np.float16)
+    codes = np.repeat(zeros, G, axis=1)                                  # every code = its zero point
+    y0 = orc.linear(x, orc.dequantize(codes, zeros, scales, G))
+    assert not y0.any()
+    n, k = 77, 200
+    codes2 = codes.copy()
+    codes2[n, k] = (int(zeros[n, 1]) + 5) % 16
+    diff = int(codes2[n, k]) - int(zeros[n, 1])
+    y1 = orc.linear(x, orc.dequantize(codes2, zeros, scales, G))
+    want = x[:, k].astype(np.float64) * diff * float(scales[n, 1])
+    assert np.array_equal(y1[:, n], want)
+    y1[:, n] = 0
+    assert not y1.any()
+    # linear in x
+    codes3 = rng.integers(0, 16, size=(N, K), dtype=np.uint8)
+    Wdq = orc.dequantize(codes3, zeros, scales, G)
+    xa = (rng.integers(-8, 9, size=(M, K))).astype(np.float16)
+    xb = (rng.integers(-8, 9, size=(M, K))).astype(np.float16)
+    lhs = orc.linear((xa + xb).astype(np.float16), Wdq)
+    assert np.allclose(lhs, orc.linear(xa, Wdq) + orc.linear(xb, Wdq), rtol=1e-12, atol=1e-12)
+
+
+def test_linear_against_explicit_sum():
+    rng = np.random.default_rng(17)
+    N, K, G, M = 128, 128, 64, 2
+    codes = rng.integers(0, 16, size=(N, K), dtype=np.uint8)
+    zeros = rng.integers(0, 16, size=(N, K // G), dtype=np.uint8)
+    scales = (rng.random((N, K // G)) * 0.01 + 0.001).astype(np.float16)
+    x = rng.standard_normal((M, K)).astype(np.float16)
+    y = orc.linear(x, orc.dequantize(codes, zeros, scales, G))
+    for m in range(M):
+        for n in range(0, N, 9):
+            acc = Fraction(0)
+            for k in range(K):
+                w = Fraction(int(codes[n, k]) - int(zeros[n, k // G])) * Fraction(float(scales[n, k // G]))
+                acc += Fraction(float(x[m, k])) * w
+            assert abs(y[m, n] - float(acc)) <= 1e-12 * max(1.0, abs(float(acc)))
+    # the packed entry point agrees, also on a subset of rows
+    qw, sc, zp = orc.pack_qweight(codes), orc.pack_scales(scales), orc.pack_zeros(zeros)
+    assert np.array_equal(orc.linear_from_packed(x, qw, sc, zp, N, K, G), y)
+    rows = np.array([3, 64, 127])
+    assert np.array_equal(orc.linear_from_packed(x, qw, sc, zp, N, K, G, rows=rows), y[:, rows])
+
+
+# --------------------------------------------------------------- brute force on tiny groups
+@pytest.mark.parametrize("G", [2, 3, 4])
+def test_brute_force_tiny_groups(G):
+    """For the oracle's own (Delta, z) the chosen codes must minimise the squared error over
+    all 16^G code vectors (exact rational arithmetic)."""
+    rng = np.random.default_rng(100 + G)
+    vals = (rng.integers(-40, 41, size=(40, G)) / 64.0).astype(np.float16)
+    vals = vals[(vals.max(axis=1) > 0) & (vals.min(axis=1) < 0)]
+    codes, zeros, scales = orc.quantize(vals, np.ones(G, np.float32), G)
+    for r in range(vals.shape[0]):
+        d, z = Fraction(float(scales[r, 0])), int(zeros[r, 0])
+        w = [Fraction(float(v)) for v in vals[r]]
+        err = lambda qs: sum((wi - (qi - z) * d) ** 2 for wi, qi in zip(w, qs))
+        best = min(err(qs) for qs in itertools.product(range(16), repeat=G))
+        assert err([int(c) for c in codes[r]]) <= best * (1 + Fraction(1, 2**20))
+
+
+# ------------------------------------------------------------ closed-form error invariants
+def _gaussian_case(seed, N, K):
+    return synth.weight(seed, N, K), synth.act_mean_abs(seed, K)
+
+
+@pytest.mark.parametrize("alpha,G", [(0.0, 128), (0.5, 128), (1.0, 64)])
+def test_error_bound_invariants(alpha, G):
+    N, K = 256, 1024
+    W, a = _gaussian_case(21, N, K)
+    s = orc.channel_scale(a, alpha)
+    codes, zeros, scales = orc.quantize(W, s, G)
+    wp = W.astype(np.float64) * s.astype(np.float64)
+    wg = wp.reshape(N, K // G, G)
+    d = scales.astype(np.float64)[:, :, None]
+    back = orc.dequantize(codes, zeros, scales, G).reshape(N, K // G, G)
+    straddle = (wg.min(axis=2) <= 0) & (wg.max(axis=2) >= 0)
+    assert straddle.all()                                  # Gaussian groups always straddle 0
+    bound = (0.5 + 15 * 2.0**-11) * d + 2.0**-22 * np.abs(wg) + 1e-12
+    assert (np.abs(wg - back) <= bound).all()
+    cg = codes.reshape(N, K // G, G)
+    imin, imax = wg.argmin(axis=2), wg.argmax(axis=2)
+    qmin = np.take_along_axis(cg, imin[:, :, None], axis=2)
+    qmax = np.take_along_axis(cg, imax[:, :, None], axis=2)
+    assert (qmin == 0).all()
+    assert np.isin(qmax, (14, 15)).all() and (qmax == 15).mean() > 0.9
+    # Delta is the fp16 rounding of range / 15
+    rng_ = (wg.max(axis=2) - wg.min(axis=2)) / 15.0
+    assert (np.abs(scales.astype(np.float64) - rng_) <= 2.0**-11 * rng_ * 1.0001).all()
+
+
+def test_round_error_statistics(golden_dir):
+    """Sec. 3.2: the rounding error is roughly uniform on [0, 0.5] with mean 0.25."""
+    g = _golden(os.path.join(golden_dir, "round_error_model.txt"))
+    N, K, G = 512, 1024, 128
+    W, a = _gaussian_case(22, N, K)
+    for alpha in (0.0, 0.5):
+        s = orc.channel_scale(a, alpha)
+        codes, zeros, scales = orc.quantize(W, s, G)
+        wp = (W.astype(np.float64) * s).reshape(N, K // G, G)
+        d = scales.astype(np.float64)[:, :, None]
+        back = orc.dequantize(codes, zeros, scales, G).reshape(N, K // G, G)
+        err = np.abs(wp - back) / d
+        inside = (codes.reshape(err.shape) > 0) & (codes.reshape(err.shape) < 15)
+        e = err[inside]
+        assert e.min() >= float(g["round_err_min"][0])
+        assert e.max() <= float(g["round_err_max"][0]) + 1e-6
+        assert abs(e.mean() - float(g["round_err_mean"][0])) < 0.01
+        hist, _ = np.histogram(e, bins=5, range=(0, 0.5))
+        assert hist.min() / hist.max() > 0.9                # flat
+
+
+def test_salient_channel_scaling_trend(golden_dir):
+    """Sec. 3.2 / Table 2: multiplying 1 % of the channels by s > 1 leaves most group
+    Deltas unchanged and shrinks those channels' error by (Delta'/Delta) / s."""
+    rows = []
+    with open(os.path.join(golden_dir, "scale_study_table2.txt")) as f:
+        for line in f:
+            if line.strip() and not line.startswith("#"):
+                rows.append([float(v) for v in line.split()])
+    for s_, _, ratio, ratio_over_s in rows:                # the table's own identity
+        assert abs(ratio / s_ - ratio_over_s) < 2e-3
+    N, K, G = 512, 2048, 128
+    W = synth.weight(23, N, K)
+    sal = synth.outlier_channels(23, K)
+    base_codes, base_z, base_d = orc.quantize(W, np.ones(K, np.float32), G)
+    base_err = np.abs(orc.dequantize(base_codes, base_z, base_d, G) - W.astype(np.float64))
+    prev_changed, prev_rel = -1.0, 2.0
+    for s_, *_ in rows[1:]:
+        s = np.ones(K, np.float32)
+        s[sal] = s_
+        c, z, d = orc.quantize(W, s, G)
+        changed = (d.view(np.uint16) != base_d.view(np.uint16)).mean()
+        ratio = (d.astype(np.float64) / base_d.astype(np.float64)).mean()
+        err = np.abs(orc.dequantize(c, z, d, G) / s.astype(np.float64) - W.astype(np.float64))
+        rel = err[:, sal].mean() / base_err[:, sal].mean()
+        assert changed > prev_changed and changed < 0.5     # a minority, growing with s
+        assert 1.0 <= ratio < 1.5
+        assert rel < prev_rel                               # salient error keeps falling
+        assert abs(rel - ratio / s_) < 0.15 * ratio / s_ + 0.05   # ~ (Delta'/Delta) / s
+        prev_changed, prev_rel = changed, rel
+
+
+def test_alpha_zero_ignores_statistics_and_output_bound():
+    N, K, G, M = 256, 1024, 128, 2
+    seed = 24
+    W, a = _gaussian_case(seed, N, K)
+    q0 = orc.quantize_pack(W, a, 0.0, G)
+    q1 = orc.quantize_pack(W, a * 7 + 1, 0.0, G)
+    q2 = orc.quantize_pack(W, None, 0.0, G)
+    for u, v, w in zip(q0, q1, q2):
+        assert np.array_equal(u, v) and np.array_equal(u, w)
+    for alpha in (0.0, 0.5, 1.0):
+        s = orc.channel_scale(a, alpha)
+        x = synth.activations(seed, M, K)
+        xs = (x.astype(np.float32) / s[None, :]).astype(np.float16)
+        codes, zeros, scales = orc.quantize(W, s, G)
+        y = orc.linear(xs, orc.dequantize(codes, zeros, scales, G))
+        y_fp = xs.astype(np.float64) @ (W.astype(np.float64) * s).T
+        dk = np.repeat(scales.astype(np.float64), G, axis=1)             # [N][K]
+        bound = np.abs(xs.astype(np.float64)) @ (0.508 * dk).T
+        assert (np.abs(y - y_fp) <= bound + 1e-9).all()
+        rel = np.linalg.norm(y - y_fp) / np.linalg.norm(y_fp)
+        assert rel < 0.2
+
+
+def test_activation_aware_scaling_reduces_output_error():
+    """The paper's claim in Sec. 3.2: scaling salient channels lowers the layer's output error
+    on activations with outlier channels (alpha = 0.5 beats plain round-to-nearest)."""
+    N, K, G, M = 512, 2048, 128, 16
+    seed = 25
+    W, a = _gaussian_case(seed, N, K)
+    x = synth.activations(seed, M, K)
+    y_fp = x.astype(np.float64) @ W.astype(np.float64).T
+    errs = {}
+    for alpha in (0.0, 0.5):
+        s = orc.channel_scale(a, alpha)
+        xs = (x.astype(np.float32) / s[None, :]).astype(np.float16)
+        codes, zeros, scales = orc.quantize(W, s, G)
+        y = orc.linear(xs, orc.dequantize(codes, zeros, scales, G))
+        errs[alpha] = np.linalg.norm(y - y_fp) / np.linalg.norm(y_fp)
+    assert errs[0.5] < 0.7 * errs[0.0]
+
+
+def test_parity_error_helper():
+    y_ref = np.array([[3.0, 4.0]])
+    rel, mx = orc.parity_errors(np.array([[3.0, 4.5]]), y_ref)
+    assert abs(rel - 0.1) < 1e-12 and abs(mx - 0.125) < 1e-12
