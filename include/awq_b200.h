@@ -1,0 +1,141 @@
+/*
+ * awq_b200.h - C ABI of the B200 (sm_100a) W4A16 group-wise linear layer.
+ *
+ * The layer is  y = x . dequant(Wq)^T  with  dequant(q) = (q - z) * Delta  per group of
+ * `group` consecutive input channels of one output row, where Wq was obtained by
+ * round-to-nearest quantization of W * diag(s),  s = s_X^alpha  (AWQ: Eq. 2 - Eq. 5 of the
+ * paper; the fused dequantize + matrix-vector / matrix-matrix product is its Sec. 4.2).
+ *
+ * Conventions for every call
+ *  - All data pointers are DEVICE pointers on the current CUDA device, 16-byte aligned,
+ *    owned by the caller.  The library keeps no pointer after a call returns, except the
+ *    workspace registered with awq_set_workspace.
+ *  - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ *    Calls enqueue work and return; they never synchronize unless stated.
+ *  - Return value: AWQ_OK (0) or a positive AwqStatus code.  Nothing is printed, thrown
+ *    or aborted.  awq_status_string() names a code.
+ *  - Shapes: N (output channels) a multiple of 128, K (input channels) a multiple of 128,
+ *    group 64 or 128, M >= 1.  W is fp16 [N][K] row-major, x fp16 [M][K] row-major,
+ *    y fp16 [M][N] row-major.
+ *
+ * Packed layout (layout version 1)
+ *  qweight: N*K/2 bytes.  Tiles of 128 rows x 64 columns are stored whole (4096 bytes),
+ *    tile index (n/128)*(K/64) + k/64.  A tile is 8 bands of 16 rows; a band is 32 pieces
+ *    of 16 bytes, piece index 4*g + t (g = 0..7, t = 0..3) holding rows g and g+8 of the
+ *    band and columns 16t..16t+15 of the tile.  32-bit word j of a piece holds columns
+ *    c = 16t+4j .. +3 of both rows as eight 4-bit slots
+ *      (g,c) (g,c+1) (g+8,c) (g+8,c+1) (g,c+2) (g,c+3) (g+8,c+2) (g+8,c+3),
+ *    slot e stored at bits 4p..4p+3 with p = {0,4,1,5,2,6,3,7}[e]  (read from the low
+ *    nibble up, the slots appear in the order 0,2,4,6,1,3,5,7 - the GPU order of Sec. 4.2).
+ *  scales: fp16 [K/group][N].
+ *  zeros:  (K/group) * N/2 bytes; byte gi*(N/2) + (n/16)*8 + (n%8) holds the zero point of
+ *    row n (n%16 < 8) in its low nibble and of row n+8 in its high nibble.
+ */
+#ifndef AWQ_B200_H_
+#define AWQ_B200_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum AwqStatus {
+    AWQ_OK = 0,
+    AWQ_ERR_NULL_POINTER = 1,
+    AWQ_ERR_BAD_SHAPE = 2,      /* N % 128, K % 128, K % group != 0, M < 1, or too large */
+    AWQ_ERR_BAD_GROUP = 3,      /* group not 64 or 128 */
+    AWQ_ERR_BAD_ALPHA = 4,      /* alpha outside [0, 1] or NaN */
+    AWQ_ERR_MISALIGNED = 5,     /* a pointer is not 16-byte aligned */
+    AWQ_ERR_NO_WORKSPACE = 6,   /* the call needs more workspace than was registered */
+    AWQ_ERR_WRONG_DEVICE = 7,   /* current device is not compute capability 10.x */
+    AWQ_ERR_CUDA = 8,           /* a CUDA runtime / driver call failed */
+    AWQ_ERR_TIMEOUT = 9,        /* a bounded device-side wait ran out (see awq_poll_status) */
+    AWQ_ERR_BAD_ARGUMENT = 10
+} AwqStatus;
+
+/* Which kernel awq_linear_path runs. */
+typedef enum AwqPath {
+    AWQ_PATH_AUTO = 0,          /* what awq_linear does: chosen from M */
+    AWQ_PATH_GEMV = 1,          /* fused dequant matrix-vector kernel, M <= 16 */
+    AWQ_PATH_GEMM = 2           /* tcgen05 tensor-core kernel, any M >= 1 */
+} AwqPath;
+
+/* Sizes of the packed arrays, in bytes (0 if the shape is not accepted). */
+size_t awq_qweight_bytes(int N, int K);
+size_t awq_scales_bytes(int N, int K, int group);
+size_t awq_zeros_bytes(int N, int K, int group);
+
+/*
+ * Offline step (Eq. 2 - Eq. 5): fold s = act_mean_abs^alpha into W, quantize each group of
+ * `group` input channels of each row to 4-bit codes with an fp16 scale Delta and an integer
+ * zero point in [0,15], and write the three packed arrays described above.
+ *   s_k = 1 if alpha == 0 or act_mean_abs[k] is not finite or <= 0, else act_mean_abs[k]^alpha
+ *         (alpha = 1: identity; alpha = 0.5: correctly rounded fp32 sqrt; else fp64 pow -> fp32)
+ *   w'  = fp32(W) * s_k                               (one fp32 multiply, kept in fp32)
+ *   Delta = fp16_rne((max w' - min w') / 15) over the group; 1.0 if that is 0 or not finite
+ *   z   = clamp(rne(-min w' / Delta), 0, 15)          (fp32 division, round half to even)
+ *   q   = clamp(rne(w' / Delta) + z, 0, 15)
+ * W: in, fp16 [N][K].  act_mean_abs: in, fp32 [K], may be NULL iff alpha == 0.
+ * qweight / scales / zeros: out, awq_*_bytes() bytes each, fully overwritten.
+ * The result is a pure function of the inputs (bit-reproducible).
+ */
+int awq_quantize_pack(const void* W, const float* act_mean_abs, float alpha, int group,
+                      void* qweight, void* scales, void* zeros, int N, int K, void* stream);
+
+/* Eq. 5 alone: s[k] as used by awq_quantize_pack.  s: out, fp32 [K]. */
+int awq_channel_scale(const float* act_mean_abs, float alpha, float* s, int K, void* stream);
+
+/*
+ * The layer itself (Sec. 4.2, on-the-fly dequantization fused into the product):
+ *   y[m][n] = sum_g Delta[g][n] * sum_{k in g} (q[n][k] - z[g][n]) * x[m][k],  stored as fp16.
+ * x must already be divided by s (the paper folds diag(s)^-1 into the previous operator).
+ * x: in, fp16 [M][K].  y: out, fp16 [M][N], fully overwritten; must not alias an input.
+ * M <= 8 runs the matrix-vector kernel (HBM-bound; exact integer (q - z) in fp16 into
+ * fp32 tensor-core accumulation, Delta applied in fp32 per group), larger M the tcgen05
+ * kernel ((q - z) * Delta rounded once to fp16, fp32 accumulation in tensor memory).
+ * The matrix-vector kernel splits K across thread blocks and combines the partial sums in a
+ * fixed order through the registered workspace: results are bit-reproducible.  Calls that
+ * use the workspace must not overlap on the GPU (issue them on one stream).
+ * Errors: AWQ_ERR_NO_WORKSPACE if awq_workspace_bytes(M,N,K,group) exceeds the registered
+ * size; shape / pointer errors as listed in AwqStatus.
+ */
+int awq_linear(const void* x, const void* qweight, const void* scales, const void* zeros,
+               void* y, int M, int N, int K, int group, void* stream);
+
+/* Same as awq_linear with the kernel forced (for the small-batch crossover measurement).
+ * AWQ_PATH_GEMV with M > 16 returns AWQ_ERR_BAD_SHAPE. */
+int awq_linear_path(const void* x, const void* qweight, const void* scales, const void* zeros,
+                    void* y, int M, int N, int K, int group, int path, void* stream);
+
+/* Workspace (scratch for split-K partial sums and arrival counters).
+ * awq_workspace_bytes: bytes awq_linear needs for this problem (0 if none).
+ * awq_set_workspace: registers caller-owned device memory for the current device; the first
+ * 4096 bytes are cleared with a synchronous cudaMemset.  Pass (NULL, 0) to unregister.
+ * The memory must stay valid until it is unregistered or replaced. */
+size_t awq_workspace_bytes(int M, int N, int K, int group);
+int awq_set_workspace(void* dev_ptr, size_t bytes);
+
+/* Test / debug: expand the packed arrays into canonical ones.
+ * codes: out u8 [N][K]; scales_nk: out fp16 bits [N][K/group]; zeros_nk: out u8 [N][K/group]. */
+int awq_unpack_canonical(const void* qweight, const void* scales, const void* zeros,
+                         int N, int K, int group,
+                         uint8_t* codes, uint16_t* scales_nk, uint8_t* zeros_nk, void* stream);
+
+/* Reads and clears the device status word of the current device (synchronizes the device).
+ * Returns AWQ_OK, or AWQ_ERR_TIMEOUT if a kernel gave up a bounded wait since the last poll
+ * (its output is then undefined), or AWQ_ERR_CUDA. */
+int awq_poll_status(void);
+
+const char* awq_status_string(int status);
+/* Text of the last CUDA error seen by the calling thread's library calls ("" if none). */
+const char* awq_last_cuda_error(void);
+int awq_layout_version(void);
+/* Number of kernels this library has launched in this process (all threads). */
+unsigned long long awq_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* AWQ_B200_H_ */

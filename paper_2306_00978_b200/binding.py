@@ -1,0 +1,169 @@
+"""Thin ctypes binding over the C ABI in include/awq_b200.h (argument marshalling only).
+
+torch supplies device memory and the current stream; every step of the layer runs in the
+CUDA library.  There is no fallback: if the library has not been built, or a call returns
+an error status, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Tuple
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libawq_b200.so")
+
+PATH_AUTO, PATH_GEMV, PATH_GEMM = 0, 1, 2
+
+EXPORTS = (
+    "awq_qweight_bytes", "awq_scales_bytes", "awq_zeros_bytes", "awq_quantize_pack",
+    "awq_channel_scale", "awq_linear", "awq_linear_path", "awq_workspace_bytes",
+    "awq_set_workspace", "awq_unpack_canonical", "awq_poll_status", "awq_status_string",
+    "awq_last_cuda_error", "awq_layout_version", "awq_launch_count",
+)
+
+_lib = None
+_workspace: dict = {}          # device index -> torch tensor registered with the library
+
+
+class AwqError(RuntimeError):
+    pass
+
+
+def lib() -> ctypes.CDLL:
+    """Loads the library on first use; raises if it is missing (no CPU or eager fallback)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise AwqError(f"{LIB_PATH} not found: build it with `python -m paper_2306_00978_b200.build`")
+    L = ctypes.CDLL(LIB_PATH)
+    vp, i, f, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_float, ctypes.c_size_t
+    L.awq_qweight_bytes.restype, L.awq_qweight_bytes.argtypes = sz, [i, i]
+    L.awq_scales_bytes.restype, L.awq_scales_bytes.argtypes = sz, [i, i, i]
+    L.awq_zeros_bytes.restype, L.awq_zeros_bytes.argtypes = sz, [i, i, i]
+    L.awq_quantize_pack.restype, L.awq_quantize_pack.argtypes = i, [vp, vp, f, i, vp, vp, vp, i, i, vp]
+    L.awq_channel_scale.restype, L.awq_channel_scale.argtypes = i, [vp, f, vp, i, vp]
+    L.awq_linear.restype, L.awq_linear.argtypes = i, [vp, vp, vp, vp, vp, i, i, i, i, vp]
+    L.awq_linear_path.restype, L.awq_linear_path.argtypes = i, [vp, vp, vp, vp, vp, i, i, i, i, i, vp]
+    L.awq_workspace_bytes.restype, L.awq_workspace_bytes.argtypes = sz, [i, i, i, i]
+    L.awq_set_workspace.restype, L.awq_set_workspace.argtypes = i, [vp, sz]
+    L.awq_unpack_canonical.restype, L.awq_unpack_canonical.argtypes = i, [vp, vp, vp, i, i, i, vp, vp, vp, vp]
+    L.awq_poll_status.restype, L.awq_poll_status.argtypes = i, []
+    L.awq_status_string.restype, L.awq_status_string.argtypes = ctypes.c_char_p, [i]
+    L.awq_last_cuda_error.restype, L.awq_last_cuda_error.argtypes = ctypes.c_char_p, []
+    L.awq_layout_version.restype, L.awq_layout_version.argtypes = i, []
+    L.awq_launch_count.restype, L.awq_launch_count.argtypes = ctypes.c_ulonglong, []
+    _lib = L
+    return L
+
+
+def _check(rc: int, what: str) -> None:
+    if rc != 0:
+        L = lib()
+        msg = L.awq_status_string(rc).decode()
+        extra = L.awq_last_cuda_error().decode()
+        raise AwqError(f"{what}: status {rc} ({msg}){' - ' + extra if extra and rc == 8 else ''}")
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _dev(t: torch.Tensor, dtype: torch.dtype, name: str) -> int:
+    if not t.is_cuda or t.dtype != dtype or not t.is_contiguous():
+        raise AwqError(f"{name}: expected a contiguous CUDA tensor of dtype {dtype}")
+    return t.data_ptr()
+
+
+def launch_count() -> int:
+    return int(lib().awq_launch_count())
+
+
+def packed_sizes(N: int, K: int, group: int) -> Tuple[int, int, int]:
+    L = lib()
+    sizes = (L.awq_qweight_bytes(N, K), L.awq_scales_bytes(N, K, group), L.awq_zeros_bytes(N, K, group))
+    if 0 in sizes:
+        raise AwqError(f"shape N={N}, K={K}, group={group} is not accepted")
+    return sizes
+
+
+def channel_scale(act_mean_abs: Optional[torch.Tensor], alpha: float, K: int) -> torch.Tensor:
+    """s = act_mean_abs ** alpha as the quantizer computes it (Eq. 5); fp32 [K] on the device."""
+    s = torch.empty(K, dtype=torch.float32, device="cuda")
+    a = 0 if act_mean_abs is None else _dev(act_mean_abs, torch.float32, "act_mean_abs")
+    _check(lib().awq_channel_scale(a, float(alpha), s.data_ptr(), K, _stream()), "awq_channel_scale")
+    return s
+
+
+def quantize_pack(W: torch.Tensor, act_mean_abs: Optional[torch.Tensor], alpha: float, group: int):
+    """awq_quantize_pack: returns (qweight u8 [N*K/2], scales fp16 [K/group][N], zeros u8 [K/group][N/2])."""
+    N, K = W.shape
+    qb, sb, zb = packed_sizes(N, K, group)
+    dev = W.device
+    qweight = torch.empty(qb, dtype=torch.uint8, device=dev)
+    scales = torch.empty((K // group, N), dtype=torch.float16, device=dev)
+    zeros = torch.empty((K // group, N // 2), dtype=torch.uint8, device=dev)
+    a = 0 if act_mean_abs is None else _dev(act_mean_abs, torch.float32, "act_mean_abs")
+    rc = lib().awq_quantize_pack(_dev(W, torch.float16, "W"), a, float(alpha), int(group),
+                                 qweight.data_ptr(), scales.data_ptr(), zeros.data_ptr(), N, K, _stream())
+    _check(rc, "awq_quantize_pack")
+    return qweight, scales, zeros
+
+
+def ensure_workspace(nbytes: int) -> None:
+    """Registers (growing if needed) a torch-allocated scratch buffer for the current device."""
+    if nbytes <= 0:
+        return
+    dev = torch.cuda.current_device()
+    cur = _workspace.get(dev)
+    if cur is not None and cur.numel() >= nbytes:
+        return
+    torch.cuda.synchronize()
+    buf = torch.empty(max(nbytes, 1 << 22), dtype=torch.uint8, device=f"cuda:{dev}")
+    _check(lib().awq_set_workspace(buf.data_ptr(), buf.numel()), "awq_set_workspace")
+    _workspace[dev] = buf
+
+
+def workspace_bytes(M: int, N: int, K: int, group: int) -> int:
+    return int(lib().awq_workspace_bytes(M, N, K, group))
+
+
+def linear(x: torch.Tensor, qweight: torch.Tensor, scales: torch.Tensor, zeros: torch.Tensor,
+           N: int, K: int, group: int, out: Optional[torch.Tensor] = None,
+           path: int = PATH_AUTO) -> torch.Tensor:
+    """awq_linear / awq_linear_path: y = x . dequant(Wq)^T, x fp16 [M][K] already divided by s."""
+    M = x.shape[0]
+    if x.shape[1] != K:
+        raise AwqError("x must be [M][K]")
+    y = out if out is not None else torch.empty((M, N), dtype=torch.float16, device=x.device)
+    if M <= 16 and path != PATH_GEMM:
+        ensure_workspace(workspace_bytes(M, N, K, group))
+    args = (_dev(x, torch.float16, "x"), _dev(qweight, torch.uint8, "qweight"),
+            _dev(scales, torch.float16, "scales"), _dev(zeros, torch.uint8, "zeros"),
+            _dev(y, torch.float16, "y"), M, N, K, int(group))
+    if path == PATH_AUTO:
+        rc = lib().awq_linear(*args, _stream())
+    else:
+        rc = lib().awq_linear_path(*args, int(path), _stream())
+    _check(rc, "awq_linear")
+    return y
+
+
+def unpack_canonical(qweight, scales, zeros, N: int, K: int, group: int):
+    """Expands the packed arrays: (codes u8 [N][K], scales fp16 [N][K/group], zeros u8 [N][K/group])."""
+    ng = K // group
+    codes = torch.empty((N, K), dtype=torch.uint8, device=qweight.device)
+    sc = torch.empty((N, ng), dtype=torch.float16, device=qweight.device)
+    zp = torch.empty((N, ng), dtype=torch.uint8, device=qweight.device)
+    rc = lib().awq_unpack_canonical(qweight.data_ptr(), scales.data_ptr(), zeros.data_ptr(), N, K, int(group),
+                                    codes.data_ptr(), sc.data_ptr(), zp.data_ptr(), _stream())
+    _check(rc, "awq_unpack_canonical")
+    return codes, sc, zp
+
+
+def poll_status() -> None:
+    """Synchronizes and raises if a kernel gave up a bounded wait since the last poll."""
+    _check(lib().awq_poll_status(), "awq_poll_status")

@@ -1,0 +1,221 @@
+// C ABI of the library: argument checks, dispatch, workspace and status bookkeeping.
+#include <atomic>
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <mutex>
+
+#include "common.cuh"
+
+namespace awq {
+
+namespace {
+
+constexpr int kMaxDevices = 64;
+std::atomic<unsigned long long> g_launches{0};
+thread_local char t_cuda_error[256] = "";
+
+struct DeviceState {
+    void* workspace = nullptr;
+    size_t workspace_bytes = 0;
+    unsigned int* status_word = nullptr;   // device address of g_status on this device
+    int cc_major = -1;
+};
+DeviceState g_dev[kMaxDevices];
+std::mutex g_mutex;
+
+__device__ unsigned int g_status;          // 0, or a code written by a kernel that gave up a wait
+
+int note_cuda(cudaError_t e) {
+    if (e == cudaSuccess) return AWQ_OK;
+    std::snprintf(t_cuda_error, sizeof(t_cuda_error), "%s: %s", cudaGetErrorName(e), cudaGetErrorString(e));
+    return AWQ_ERR_CUDA;
+}
+
+// Per-device set-up on first use: compute capability and the status word's device address.
+int device_state(DeviceState** out) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return note_cuda(e);
+    if (dev < 0 || dev >= kMaxDevices) return AWQ_ERR_WRONG_DEVICE;
+    std::lock_guard<std::mutex> lock(g_mutex);
+    DeviceState& d = g_dev[dev];
+    if (d.cc_major < 0) {
+        int major = 0;
+        e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+        if (e != cudaSuccess) return note_cuda(e);
+        if (major == 10) {
+            void* p = nullptr;
+            e = cudaGetSymbolAddress(&p, g_status);
+            if (e != cudaSuccess) return note_cuda(e);
+            e = cudaMemset(p, 0, sizeof(unsigned int));
+            if (e != cudaSuccess) return note_cuda(e);
+            d.status_word = reinterpret_cast<unsigned int*>(p);
+        }
+        d.cc_major = major;
+    }
+    if (d.cc_major != 10) return AWQ_ERR_WRONG_DEVICE;
+    *out = &d;
+    return AWQ_OK;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int check_shape(int N, int K, int group) {
+    if (group != 64 && group != 128) return AWQ_ERR_BAD_GROUP;
+    if (N < 128 || K < 128 || N % 128 != 0 || K % 128 != 0 || K % group != 0) return AWQ_ERR_BAD_SHAPE;
+    if (N / 128 > kMaxSlabs) return AWQ_ERR_BAD_SHAPE;
+    if ((long long)N * K > (1LL << 33)) return AWQ_ERR_BAD_SHAPE;
+    return AWQ_OK;
+}
+
+}  // namespace
+
+void count_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
+
+}  // namespace awq
+
+using namespace awq;
+
+extern "C" {
+
+size_t awq_qweight_bytes(int N, int K) {
+    return check_shape(N, K, 128) == AWQ_OK ? (size_t)N * K / 2 : 0;
+}
+size_t awq_scales_bytes(int N, int K, int group) {
+    return check_shape(N, K, group) == AWQ_OK ? (size_t)(K / group) * N * 2 : 0;
+}
+size_t awq_zeros_bytes(int N, int K, int group) {
+    return check_shape(N, K, group) == AWQ_OK ? (size_t)(K / group) * N / 2 : 0;
+}
+
+int awq_channel_scale(const float* act_mean_abs, float alpha, float* s, int K, void* stream) {
+    if (!(alpha >= 0.0f && alpha <= 1.0f)) return AWQ_ERR_BAD_ALPHA;
+    if (!s || (!act_mean_abs && alpha != 0.0f)) return AWQ_ERR_NULL_POINTER;
+    if (K < 1) return AWQ_ERR_BAD_SHAPE;
+    DeviceState* d;
+    if (int rc = device_state(&d)) return rc;
+    return note_cuda(launch_channel_scale(act_mean_abs, alpha, s, K, (cudaStream_t)stream));
+}
+
+int awq_quantize_pack(const void* W, const float* act_mean_abs, float alpha, int group,
+                      void* qweight, void* scales, void* zeros, int N, int K, void* stream) {
+    if (!(alpha >= 0.0f && alpha <= 1.0f)) return AWQ_ERR_BAD_ALPHA;
+    if (int rc = check_shape(N, K, group)) return rc;
+    if (!W || !qweight || !scales || !zeros || (!act_mean_abs && alpha != 0.0f)) return AWQ_ERR_NULL_POINTER;
+    if (!aligned16(W) || !aligned16(qweight) || !aligned16(scales) || !aligned16(zeros) ||
+        (reinterpret_cast<uintptr_t>(act_mean_abs) & 3u))
+        return AWQ_ERR_MISALIGNED;
+    DeviceState* d;
+    if (int rc = device_state(&d)) return rc;
+    return note_cuda(launch_quantize_pack(reinterpret_cast<const __half*>(W), act_mean_abs, alpha, group,
+                                          reinterpret_cast<uint32_t*>(qweight),
+                                          reinterpret_cast<__half*>(scales),
+                                          reinterpret_cast<uint8_t*>(zeros), N, K, (cudaStream_t)stream));
+}
+
+static int resolve_path(int M, int path) {
+    if (path == AWQ_PATH_AUTO) return M <= 8 ? AWQ_PATH_GEMV : AWQ_PATH_GEMM;
+    return path;
+}
+
+size_t awq_workspace_bytes(int M, int N, int K, int group) {
+    if (check_shape(N, K, group) != AWQ_OK || M < 1) return 0;
+    if (M > 16) return 0;
+    return gemv_plan(M, N, K, group).workspace_bytes;
+}
+
+int awq_set_workspace(void* dev_ptr, size_t bytes) {
+    DeviceState* d;
+    if (int rc = device_state(&d)) return rc;
+    if ((dev_ptr == nullptr) != (bytes == 0)) return AWQ_ERR_BAD_ARGUMENT;
+    if (dev_ptr) {
+        if (!aligned16(dev_ptr)) return AWQ_ERR_MISALIGNED;
+        if (bytes < kCounterBytes) return AWQ_ERR_BAD_ARGUMENT;
+        if (int rc = note_cuda(cudaMemset(dev_ptr, 0, kCounterBytes))) return rc;
+    }
+    std::lock_guard<std::mutex> lock(g_mutex);
+    d->workspace = dev_ptr;
+    d->workspace_bytes = bytes;
+    return AWQ_OK;
+}
+
+int awq_linear_path(const void* x, const void* qweight, const void* scales, const void* zeros,
+                    void* y, int M, int N, int K, int group, int path, void* stream) {
+    if (int rc = check_shape(N, K, group)) return rc;
+    if (M < 1 || (long long)M * K > (1LL << 40) || (long long)M * N > (1LL << 40)) return AWQ_ERR_BAD_SHAPE;
+    if (!x || !qweight || !scales || !zeros || !y) return AWQ_ERR_NULL_POINTER;
+    if (!aligned16(x) || !aligned16(qweight) || !aligned16(scales) || !aligned16(zeros) || !aligned16(y))
+        return AWQ_ERR_MISALIGNED;
+    if (path != AWQ_PATH_AUTO && path != AWQ_PATH_GEMV && path != AWQ_PATH_GEMM) return AWQ_ERR_BAD_ARGUMENT;
+    path = resolve_path(M, path);
+    if (path == AWQ_PATH_GEMV && M > 16) return AWQ_ERR_BAD_SHAPE;
+    DeviceState* d;
+    if (int rc = device_state(&d)) return rc;
+    const cudaStream_t st = (cudaStream_t)stream;
+    if (path == AWQ_PATH_GEMV) {
+        const GemvPlan plan = gemv_plan(M, N, K, group);
+        void* ws = nullptr;
+        if (plan.workspace_bytes) {
+            std::lock_guard<std::mutex> lock(g_mutex);
+            if (d->workspace_bytes < plan.workspace_bytes) return AWQ_ERR_NO_WORKSPACE;
+            ws = d->workspace;
+        }
+        return note_cuda(launch_gemv(x, qweight, scales, zeros, y, M, N, K, group, plan, ws, st));
+    }
+    return note_cuda(launch_gemm(x, qweight, scales, zeros, y, M, N, K, group, d->status_word, st));
+}
+
+int awq_linear(const void* x, const void* qweight, const void* scales, const void* zeros,
+               void* y, int M, int N, int K, int group, void* stream) {
+    return awq_linear_path(x, qweight, scales, zeros, y, M, N, K, group, AWQ_PATH_AUTO, stream);
+}
+
+int awq_unpack_canonical(const void* qweight, const void* scales, const void* zeros,
+                         int N, int K, int group,
+                         uint8_t* codes, uint16_t* scales_nk, uint8_t* zeros_nk, void* stream) {
+    if (int rc = check_shape(N, K, group)) return rc;
+    if (!qweight || !scales || !zeros || !codes || !scales_nk || !zeros_nk) return AWQ_ERR_NULL_POINTER;
+    DeviceState* d;
+    if (int rc = device_state(&d)) return rc;
+    return note_cuda(launch_unpack(reinterpret_cast<const uint32_t*>(qweight),
+                                   reinterpret_cast<const __half*>(scales),
+                                   reinterpret_cast<const uint8_t*>(zeros), N, K, group,
+                                   codes, scales_nk, zeros_nk, (cudaStream_t)stream));
+}
+
+int awq_poll_status(void) {
+    DeviceState* d;
+    if (int rc = device_state(&d)) return rc;
+    if (int rc = note_cuda(cudaDeviceSynchronize())) return rc;
+    unsigned int v = 0;
+    if (int rc = note_cuda(cudaMemcpy(&v, d->status_word, sizeof(v), cudaMemcpyDeviceToHost))) return rc;
+    if (v != 0) {
+        if (int rc = note_cuda(cudaMemset(d->status_word, 0, sizeof(v)))) return rc;
+        return AWQ_ERR_TIMEOUT;
+    }
+    return AWQ_OK;
+}
+
+const char* awq_status_string(int status) {
+    switch (status) {
+        case AWQ_OK: return "ok";
+        case AWQ_ERR_NULL_POINTER: return "null pointer";
+        case AWQ_ERR_BAD_SHAPE: return "bad shape (N, K multiples of 128; K % group == 0; M >= 1)";
+        case AWQ_ERR_BAD_GROUP: return "group must be 64 or 128";
+        case AWQ_ERR_BAD_ALPHA: return "alpha must lie in [0, 1]";
+        case AWQ_ERR_MISALIGNED: return "pointer not 16-byte aligned";
+        case AWQ_ERR_NO_WORKSPACE: return "registered workspace too small (see awq_workspace_bytes)";
+        case AWQ_ERR_WRONG_DEVICE: return "current device is not compute capability 10.x";
+        case AWQ_ERR_CUDA: return "CUDA call failed (see awq_last_cuda_error)";
+        case AWQ_ERR_TIMEOUT: return "a device-side wait ran out";
+        case AWQ_ERR_BAD_ARGUMENT: return "bad argument";
+        default: return "unknown status";
+    }
+}
+
+const char* awq_last_cuda_error(void) { return t_cuda_error; }
+int awq_layout_version(void) { return 1; }
+unsigned long long awq_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+}  // extern "C"

@@ -1,0 +1,51 @@
+// Shared declarations of the library's translation units (host side and launchers).
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_fp16.h>
+#include <stdint.h>
+#include "../../include/awq_b200.h"
+
+namespace awq {
+
+constexpr int kTileRows = 128;           // output channels per packed tile
+constexpr int kTileCols = 64;            // input channels per packed tile
+constexpr int kTileBytes = kTileRows * kTileCols / 2;
+constexpr size_t kCounterBytes = 4096;   // head of the workspace: split-K arrival counters
+constexpr int kMaxSlabs = int(kCounterBytes / sizeof(unsigned int));
+
+// alpha is classified on the host so that the device takes the exact branch.
+enum AlphaMode : int { kAlphaZero = 0, kAlphaOne = 1, kAlphaHalf = 2, kAlphaGeneral = 3 };
+
+inline AlphaMode alpha_mode(float alpha) {
+    if (alpha == 0.0f) return kAlphaZero;
+    if (alpha == 1.0f) return kAlphaOne;
+    if (alpha == 0.5f) return kAlphaHalf;
+    return kAlphaGeneral;
+}
+
+void count_launch();
+
+// launchers (each returns the cudaError_t of the launch)
+cudaError_t launch_channel_scale(const float* a, float alpha, float* s, int K, cudaStream_t st);
+cudaError_t launch_quantize_pack(const __half* W, const float* a, float alpha, int group,
+                                 uint32_t* qweight, __half* scales, uint8_t* zeros,
+                                 int N, int K, cudaStream_t st);
+cudaError_t launch_unpack(const uint32_t* qweight, const __half* scales, const uint8_t* zeros,
+                          int N, int K, int group, uint8_t* codes, uint16_t* scales_nk,
+                          uint8_t* zeros_nk, cudaStream_t st);
+
+struct GemvPlan {
+    int splits;          // thread blocks along K per 128-row slab
+    int ktiles_per_split;
+    size_t workspace_bytes;
+};
+GemvPlan gemv_plan(int M, int N, int K, int group);
+cudaError_t launch_gemv(const void* x, const void* qweight, const void* scales, const void* zeros,
+                        void* y, int M, int N, int K, int group, const GemvPlan& plan,
+                        void* workspace, cudaStream_t st);
+
+cudaError_t launch_gemm(const void* x, const void* qweight, const void* scales, const void* zeros,
+                        void* y, int M, int N, int K, int group, unsigned int* status_word,
+                        cudaStream_t st);
+
+}  // namespace awq

@@ -1,0 +1,450 @@
+// Prefill path of the layer (Sec. 4.2: fused dequantize + matrix-matrix product), sm_100a.
+//
+// The weights are the MMA's A operand (128 output channels = 128 TMEM lanes), the tokens
+// its N side (BN = 32..256 columns of the fp32 accumulator in tensor memory), so
+// D[n][m] = sum_k dequant(Wq)[n][k] * x[m][k] and the epilogue writes y[m][n] = D[n][m].
+//
+// One persistent thread block per SM, warp-specialised:
+//   warp 0      producer: per 64-wide k-block one TMA tensor copy of the x tile
+//               (BN x 64 fp16, 128-byte swizzle) and three bulk copies (4 KB packed weight
+//               tile, 256 B of fp16 scales, 64 B of zero points) into a ring of stages,
+//               completion counted on an mbarrier.
+//   warps 8-15  dequantizers: each lane takes its 16-byte packed piece (rows g, g+8 of its
+//               band, 16 columns), converts two codes at a time to exact fp16 (q - z),
+//               multiplies by Delta (one fp16 rounding) and stores four 16-byte pieces into
+//               the stage's A tile in the K-major 128-byte-swizzled layout the MMA reads.
+//   warp 1      one thread issues tcgen05.mma (kind::f16, M = 128, N = BN, K = 16, four per
+//               k-block), commits to the stage's "empty" barrier and, after the last
+//               k-block, to the accumulator's "full" barrier.
+//   warps 4-7   epilogue: tcgen05.ld 32 columns at a time, convert to fp16, store to y.
+//               Two accumulator buffers let the epilogue of one tile overlap the next main loop.
+//
+// Every wait is bounded (about two seconds of wall clock): a wait that runs out writes a code to
+// the status word, raises a block-wide flag, and every role leaves its loop; the block
+// then waits (bounded) for its own copies in flight, frees its tensor memory and returns.
+#include <cuda.h>
+
+#include <mutex>
+
+#include "common.cuh"
+
+namespace awq {
+
+namespace {
+
+constexpr int kGemmThreads = 512;
+constexpr int kBK = 64;
+constexpr int kATileBytes = 128 * kBK * 2;            // dequantized fp16 weight tile
+constexpr int kMetaBytes = 1024;                      // 256 B scales + 64 B zeros, padded to keep stages 1024-aligned
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;
+constexpr unsigned int kTimeoutCode = 0x57A17u;
+
+template <int BN> struct GemmCfg {
+    static constexpr int kXTileBytes = BN * kBK * 2;
+    static constexpr int kStageBytes = kXTileBytes + kATileBytes + kTileBytes + kMetaBytes;
+    static constexpr int kStagesRaw = (216 * 1024) / kStageBytes;
+    static constexpr int kStages = kStagesRaw > 8 ? 8 : kStagesRaw;
+    static constexpr int kTmemCols = 2 * BN < 32 ? 32 : 2 * BN;   // two accumulator buffers
+    static constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*align*/ + 256 /*barriers*/;
+    static constexpr uint32_t kTxBytes = kXTileBytes + kTileBytes + 256 + 64;
+};
+
+// ------------------------------------------------------------------ small PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+    return (uint32_t)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ unsigned long long global_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+
+struct WaitCtl {
+    unsigned int* status;            // device status word (global)
+    volatile unsigned int* abort;    // block-wide flag (shared)
+};
+
+// Bounded wait on an mbarrier phase.  Returns false if the block is giving up.
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, const WaitCtl& ctl) {
+    const unsigned long long t0 = global_ns();
+    for (unsigned int i = 1;; ++i) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((i & 63u) == 0u) {
+            if (*ctl.abort) return false;
+            if (global_ns() - t0 > kWaitLimitNs) {
+                *ctl.abort = 1u;
+                atomicExch(ctl.status, kTimeoutCode);
+                return false;
+            }
+        }
+    }
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const WaitCtl& ctl) {
+    if (mbar_try_wait(bar, parity)) return true;
+    return mbar_wait_slow(bar, parity, ctl);
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+        ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void fence_proxy_async_smem() {
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void umma_f16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                         uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+// Shared-memory matrix descriptor: K-major operand, 128-byte swizzle, rows of 128 bytes,
+// 8-row atoms 1024 bytes apart.
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((addr & 0x3FFFFu) >> 4);          // start address, 16-byte units
+    d |= (uint64_t)1 << 16;                           // leading byte offset (unused for swizzled K-major)
+    d |= (uint64_t)(1024 >> 4) << 32;                 // stride byte offset between 8-row atoms
+    d |= (uint64_t)1 << 46;                           // descriptor version (sm_100)
+    d |= (uint64_t)2 << 61;                           // layout: 128-byte swizzle
+    return d;
+}
+
+// Instruction descriptor: D fp32, A and B fp16, both K-major, M = 128, N = BN.
+__host__ __device__ constexpr uint32_t instr_desc(int bn) {
+    return (1u << 4) | (0u << 7) | (0u << 10) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+}
+
+__device__ __forceinline__ uint32_t hsub2_u32(uint32_t a, uint32_t b) {
+    uint32_t d; asm("sub.rn.f16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b)); return d;
+}
+__device__ __forceinline__ uint32_t hfma2_u32(uint32_t a, uint32_t b, uint32_t c) {
+    uint32_t d; asm("fma.rn.f16x2 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c)); return d;
+}
+__device__ __forceinline__ uint32_t hmul2_u32(uint32_t a, uint32_t b) {
+    uint32_t d; asm("mul.rn.f16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b)); return d;
+}
+
+__device__ __forceinline__ void tmem_ld_32cols(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// ------------------------------------------------------------------------- the kernel
+template <int G, int BN>
+__global__ void __launch_bounds__(kGemmThreads, 1)
+gemm_kernel(const __grid_constant__ CUtensorMap x_map, const unsigned char* __restrict__ qweight,
+            const __half* __restrict__ scales, const unsigned char* __restrict__ zeros,
+            __half* __restrict__ y, int M, int N, int K, unsigned int* status_word) {
+    using Cfg = GemmCfg<BN>;
+    constexpr int S = Cfg::kStages;
+    extern __shared__ unsigned char smem_dyn[];
+    __shared__ unsigned int s_abort;
+    __shared__ uint32_t s_tmem_base;
+
+    const uint32_t dyn = smem_u32(smem_dyn);
+    const uint32_t base = (dyn + 1023u) & ~1023u;                    // 1024-byte aligned stage ring
+    unsigned char* base_ptr = smem_dyn + (base - dyn);
+    // stage layout: [X tile | A tile | packed tile | scales(256) zeros(64) pad]
+    auto x_addr = [&](int s) { return base + (uint32_t)s * Cfg::kStageBytes; };
+    auto a_addr = [&](int s) { return x_addr(s) + Cfg::kXTileBytes; };
+    auto stage_ptr = [&](int s) { return base_ptr + (size_t)s * Cfg::kStageBytes; };
+    const uint32_t bars = base + (uint32_t)S * Cfg::kStageBytes;       // 8-byte barriers follow the ring
+    auto raw_full = [&](int s) { return bars + 8u * (uint32_t)s; };
+    auto a_full = [&](int s) { return bars + 8u * (uint32_t)(S + s); };
+    auto empty = [&](int s) { return bars + 8u * (uint32_t)(2 * S + s); };
+    auto acc_full = [&](int b) { return bars + 8u * (uint32_t)(3 * S + b); };
+    auto acc_empty = [&](int b) { return bars + 8u * (uint32_t)(3 * S + 2 + b); };
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int m_tiles = (M + BN - 1) / BN;
+    const int total_tiles = (N / 128) * m_tiles;
+    const int nkb = K / kBK;
+
+    if (threadIdx.x == 0) {
+        s_abort = 0u;
+        for (int s = 0; s < S; ++s) { mbar_init(raw_full(s), 1); mbar_init(a_full(s), 8); mbar_init(empty(s), 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(acc_full(b), 1); mbar_init(acc_empty(b), 4); }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(&s_tmem_base)), "r"((uint32_t)Cfg::kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = s_tmem_base;
+    const WaitCtl ctl{status_word, &s_abort};
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ producer
+        if (lane == 0) {
+            uint32_t stage = 0, phase = 0;
+            unsigned int issued = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+                const int slab = tile / m_tiles, mt = tile % m_tiles;
+                const unsigned char* wsrc = qweight + (size_t)slab * nkb * kTileBytes;
+                for (int kb = 0; kb < nkb; ++kb) {
+                    if (!mbar_wait(empty(stage), phase ^ 1u, ctl)) { ok = false; break; }
+                    const int gi = kb * kBK / G;
+                    const uint32_t bar = raw_full(stage);
+                    mbar_arrive_expect_tx(bar, Cfg::kTxBytes);
+                    tma_load_2d(x_addr(stage), &x_map, kb * kBK, mt * BN, bar);
+                    const uint32_t raw = a_addr(stage) + kATileBytes;
+                    bulk_load(raw, wsrc + (size_t)kb * kTileBytes, kTileBytes, bar);
+                    bulk_load(raw + kTileBytes, scales + (size_t)gi * N + slab * 128, 256, bar);
+                    bulk_load(raw + kTileBytes + 256, zeros + (size_t)gi * (N / 2) + slab * 64, 64, bar);
+                    ++issued;
+                    if (++stage == S) { stage = 0; phase ^= 1u; }
+                }
+            }
+            if (!ok) {
+                // giving up: let the copies already issued land before the block exits
+                const unsigned int pending = issued < (unsigned)S ? issued : (unsigned)S;
+                uint32_t st = stage, ph = phase;
+                for (unsigned int i = 0; i < pending; ++i) {
+                    if (st == 0) { st = S - 1; ph ^= 1u; } else { --st; }
+                    const unsigned long long t0 = global_ns();
+                    while (!mbar_try_wait(raw_full(st), ph) && global_ns() - t0 < 100000000ull) {}
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------------------------------------------------------- MMA issuer
+        if (lane == 0) {
+            constexpr uint32_t idesc = instr_desc(BN);
+            uint32_t stage = 0, phase = 0;
+            int local = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++local) {
+                const int b = local & 1;
+                const uint32_t use = (uint32_t)(local >> 1) & 1u;
+                if (!mbar_wait(acc_empty(b), use ^ 1u, ctl)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)(b * BN);
+                for (int kb = 0; kb < nkb; ++kb) {
+                    if (!mbar_wait(raw_full(stage), phase, ctl) || !mbar_wait(a_full(stage), phase, ctl)) {
+                        ok = false; break;
+                    }
+                    tc_fence_after();
+                    const uint64_t adesc = smem_desc_sw128(a_addr(stage));
+                    const uint64_t bdesc = smem_desc_sw128(x_addr(stage));
+#pragma unroll
+                    for (int k = 0; k < kBK / 16; ++k)       // +32 bytes per K = 16 step, 16-byte units
+                        umma_f16(d_tmem, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), idesc,
+                                 (kb | k) != 0 ? 1u : 0u);
+                    umma_commit(empty(stage));
+                    if (++stage == S) { stage = 0; phase ^= 1u; }
+                }
+                if (ok) umma_commit(acc_full(b));
+            }
+        }
+    } else if (warp >= 8) {
+        // -------------------------------------------------------------- dequantizers
+        const int band = warp - 8;
+        const int g = lane >> 2, t = lane & 3;
+        uint32_t stage = 0, phase = 0;
+        bool ok = true;
+        // destination of this lane's four 16-byte pieces inside the swizzled A tile
+        const uint32_t row_up = (uint32_t)(2 * band) * 1024u + (uint32_t)g * 128u;
+        const uint32_t row_lo = row_up + 1024u;
+        const uint32_t c0 = (uint32_t)((2 * t) ^ g) * 16u, c1 = (uint32_t)((2 * t + 1) ^ g) * 16u;
+        for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+            for (int kb = 0; kb < nkb; ++kb) {
+                ok = mbar_wait(raw_full(stage), phase, ctl);
+                ok = __all_sync(0xFFFFFFFFu, ok);
+                if (!ok) break;
+                const unsigned char* sp = stage_ptr(stage) + Cfg::kXTileBytes;
+                const unsigned char* raw = sp + kATileBytes;
+                const uint4 pk = *reinterpret_cast<const uint4*>(raw + band * 512 + lane * 16);
+                const __half* sc = reinterpret_cast<const __half*>(raw + kTileBytes);
+                const uint32_t du = __half_as_ushort(sc[band * 16 + g]);
+                const uint32_t dl = __half_as_ushort(sc[band * 16 + g + 8]);
+                const uint32_t zb = raw[kTileBytes + 256 + band * 8 + g];
+                const uint32_t d_up = du | (du << 16), d_lo = dl | (dl << 16);
+                const uint32_t zu = 0x6400u + (zb & 0xFu), zl = 0xD400u + ((zb >> 4) << 4);
+                const uint32_t zlo = zu | (zu << 16), zhi = zl | (zl << 16);
+                const uint32_t wds[4] = {pk.x, pk.y, pk.z, pk.w};
+                uint32_t up[8], lo[8];                 // rows g / g+8: columns 16t .. 16t+15 as fp16x2
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    constexpr uint32_t kMagic = 0x64006400u, kSixteenth = 0x2C002C00u;
+                    const uint32_t w = wds[j], w8 = w >> 8;
+                    up[2 * j] = hmul2_u32(hsub2_u32((w & 0x000F000Fu) | kMagic, zlo), d_up);
+                    lo[2 * j] = hmul2_u32(hfma2_u32((w & 0x00F000F0u) | kMagic, kSixteenth, zhi), d_lo);
+                    up[2 * j + 1] = hmul2_u32(hsub2_u32((w8 & 0x000F000Fu) | kMagic, zlo), d_up);
+                    lo[2 * j + 1] = hmul2_u32(hfma2_u32((w8 & 0x00F000F0u) | kMagic, kSixteenth, zhi), d_lo);
+                }
+                unsigned char* a_tile = const_cast<unsigned char*>(sp);
+                *reinterpret_cast<uint4*>(a_tile + row_up + c0) = make_uint4(up[0], up[1], up[2], up[3]);
+                *reinterpret_cast<uint4*>(a_tile + row_up + c1) = make_uint4(up[4], up[5], up[6], up[7]);
+                *reinterpret_cast<uint4*>(a_tile + row_lo + c0) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+                *reinterpret_cast<uint4*>(a_tile + row_lo + c1) = make_uint4(lo[4], lo[5], lo[6], lo[7]);
+                fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(a_full(stage));
+                if (++stage == S) { stage = 0; phase ^= 1u; }
+            }
+        }
+    } else if (warp >= 4) {
+        // ------------------------------------------------------------------ epilogue
+        const int quad = warp & 3;                     // TMEM lanes 32*quad .. +31
+        int local = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++local) {
+            const int slab = tile / m_tiles, mt = tile % m_tiles;
+            const int b = local & 1;
+            const uint32_t use = (uint32_t)(local >> 1) & 1u;
+            ok = mbar_wait(acc_full(b), use, ctl);
+            ok = __all_sync(0xFFFFFFFFu, ok);
+            if (!ok) break;
+            tc_fence_after();
+            const int n = slab * 128 + quad * 32 + lane;
+            const int m0 = mt * BN;
+            const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(b * BN);
+#pragma unroll 1
+            for (int c = 0; c < BN; c += 32) {
+                uint32_t r[32];
+                tmem_ld_32cols(taddr + (uint32_t)c, r);
+                tmem_ld_wait();
+#pragma unroll
+                for (int i = 0; i < 32; ++i) {
+                    const int m = m0 + c + i;
+                    if (m < M) y[(size_t)m * N + n] = __float2half_rn(__uint_as_float(r[i]));
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(acc_empty(b));
+        }
+    }
+
+    __syncwarp();
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;"
+                     ::"r"(tmem_base), "r"((uint32_t)Cfg::kTmemCols) : "memory");
+    }
+}
+
+// ------------------------------------------------------------------------------ host
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static std::once_flag once;
+    std::call_once(once, [] {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    });
+    return fn;
+}
+
+template <int G, int BN>
+cudaError_t launch_one(const CUtensorMap& map, const void* qweight, const void* scales, const void* zeros,
+                       void* y, int M, int N, int K, unsigned int* status_word, int sms, cudaStream_t st) {
+    using Cfg = GemmCfg<BN>;
+    static bool attr_done[64] = {};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (!attr_done[dev & 63]) {
+        cudaError_t e = cudaFuncSetAttribute(gemm_kernel<G, BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             Cfg::kSmemBytes);
+        if (e != cudaSuccess) return e;
+        attr_done[dev & 63] = true;
+    }
+    const int tiles = (N / 128) * ((M + BN - 1) / BN);
+    const int grid = tiles < sms ? tiles : sms;
+    gemm_kernel<G, BN><<<grid, kGemmThreads, Cfg::kSmemBytes, st>>>(
+        map, reinterpret_cast<const unsigned char*>(qweight), reinterpret_cast<const __half*>(scales),
+        reinterpret_cast<const unsigned char*>(zeros), reinterpret_cast<__half*>(y), M, N, K, status_word);
+    count_launch();
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_gemm(const void* x, const void* qweight, const void* scales, const void* zeros,
+                        void* y, int M, int N, int K, int group, unsigned int* status_word,
+                        cudaStream_t st) {
+    EncodeTiledFn enc = encode_fn();
+    if (!enc) return cudaErrorNotSupported;
+    const int bn = M > 128 ? 256 : M > 64 ? 128 : M > 32 ? 64 : 32;
+    CUtensorMap map;
+    const cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)M};
+    const cuuint64_t strides[1] = {(cuuint64_t)K * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)kBK, (cuuint32_t)bn};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUresult r = enc(&map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void*>(x), dims, strides, box,
+                           estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                           CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
+    int dev = 0, sms = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return e;
+#define AWQ_GEMM_CASE(GG, BNN) \
+    return launch_one<GG, BNN>(map, qweight, scales, zeros, y, M, N, K, status_word, sms, st)
+    if (group == 128) {
+        switch (bn) { case 256: AWQ_GEMM_CASE(128, 256); case 128: AWQ_GEMM_CASE(128, 128);
+                      case 64: AWQ_GEMM_CASE(128, 64); default: AWQ_GEMM_CASE(128, 32); }
+    } else {
+        switch (bn) { case 256: AWQ_GEMM_CASE(64, 256); case 128: AWQ_GEMM_CASE(64, 128);
+                      case 64: AWQ_GEMM_CASE(64, 64); default: AWQ_GEMM_CASE(64, 32); }
+    }
+#undef AWQ_GEMM_CASE
+}
+
+}  // namespace awq
