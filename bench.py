@@ -1,0 +1,440 @@
+#!/usr/bin/env python
+"""Benchmark of the W4A16 g128 linear layer on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+One step = the seven linear layers of one Llama-2-7B-shaped decoder layer at M = 1 (decode),
+each a single awq_linear call on packed INT4 weights resident in HBM; the step's weights
+rotate over several independently seeded layers so that consecutive steps never find their
+weights in L2.  The headline value is the algorithmic GB/s of that step (packed codes +
+scales + zero points + activations in and out, each moved once).  The same JSON line also
+carries the prefill GEMM at M = 2048 on the Llama-2-13B MLP shapes (TFLOP/s), the offline
+quantize+pack kernel, the roofline fraction of the dominant kernel, the end-to-end figure
+with host buffers, and the CPU oracle timed on a bounded sample.
+
+With N > 1 (torchrun) every rank runs an independent replica; the reported value is all
+ranks' bytes over the slowest rank's time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2306_00978_b200 import replicas, synth  # noqa: E402
+
+METRIC = "W4A16 g128 GEMV GB/s at M=1 (Llama-2-7B decoder-layer linears)"
+UNIT = "GB/s"
+GROUP = 128
+ALPHA = 0.5
+FALLBACK_HBM_GBS = 6650.0
+FALLBACK_BF16_TFLOPS = 1590.0
+NOMINAL_HBM_GBS = 8000.0
+NOMINAL_FP16_TFLOPS = 2250.0
+# DRAM bytes per launch of the dominant kernel from the ncu capture summarised under
+# profiles/ (None until a capture of the current kernel exists).
+NCU_TRAFFIC_BYTES_PER_LAUNCH = None
+
+
+def algorithmic_bytes(N: int, K: int, M: int, group: int = GROUP) -> int:
+    """codes + fp16 scales + 4-bit zero points + x in + y out, each moved once."""
+    return N * K // 2 + 2 * N * K // group + N * K // (2 * group) + 2 * M * K + 2 * M * N
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_tflops": float(p["bf16_tflops"]),
+                "bf16_tflops_sustained": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])),
+                "source": "measured"}
+    except Exception:
+        return {"hbm_gbs": FALLBACK_HBM_GBS, "bf16_tflops": FALLBACK_BF16_TFLOPS,
+                "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+# ------------------------------------------------------------------------------ clocks
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while a region runs."""
+
+    QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu_index = gpu_index
+        self.rows = []
+        self.proc = None
+        self.thread = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.gpu_index}", f"--query-gpu={self.QUERY}",
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) >= 7:
+                self.rows.append((time.time(), parts))
+
+    def stop(self):
+        if self.proc is not None:
+            self.proc.terminate()          # the exact process started above
+            try:
+                self.proc.wait(timeout=5)
+            except subprocess.TimeoutExpired:
+                self.proc.kill()
+        if self.thread is not None:
+            self.thread.join(timeout=5)
+
+    def summary(self, t0: float, t1: float):
+        rows = [r for (t, r) in self.rows if t0 <= t <= t1] or [r for (_, r) in self.rows]
+        if not rows:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        mhz, mx, reasons = [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for r in rows:
+            try:
+                mhz.append(float(r[0]))
+                mx.append(float(r[1]))
+            except ValueError:
+                continue
+            for name, v in zip(names, r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(mhz) if mhz else None,
+                "sm_max_mhz": max(mx) if mx else None, "reasons": sorted(reasons),
+                "samples": len(mhz)}
+
+
+# --------------------------------------------------------------------------- workload
+def build_layers(n_layers: int, seed0: int = 2000):
+    """Quantizes n_layers x 7 seeded Llama-2-7B-shaped matrices on the GPU (setup, untimed)."""
+    import torch
+    from paper_2306_00978_b200 import binding
+    layers = []
+    for li in range(n_layers):
+        lin = []
+        for idx, (name, K, N) in enumerate(synth.LLAMA2_7B_LAYER):
+            seed = seed0 + 16 * li + idx
+            W = torch.from_numpy(synth.weight(seed, N, K)).cuda()
+            a = torch.from_numpy(synth.act_mean_abs(seed, K)).cuda()
+            qw, sc, zp = binding.quantize_pack(W, a, ALPHA, GROUP)
+            s = binding.channel_scale(a, ALPHA, K)
+            x = torch.from_numpy(synth.activations(seed, 1, K)).cuda()
+            xs = (x.float() / s[None, :]).half().contiguous()     # the caller's x / s
+            x_host = xs.cpu().pin_memory()
+            y = torch.empty((1, N), dtype=torch.float16, device="cuda")
+            y_host = torch.empty((1, N), dtype=torch.float16).pin_memory()
+            lin.append(dict(name=name, N=N, K=K, qw=qw, sc=sc, zp=zp, x=xs, x_host=x_host,
+                            y=y, y_host=y_host, x_dev_in=torch.empty_like(xs)))
+            del W
+        layers.append(lin)
+    torch.cuda.synchronize()
+    return layers
+
+
+def run_step(layer):
+    from paper_2306_00978_b200 import binding
+    for l in layer:
+        binding.linear(l["x"], l["qw"], l["sc"], l["zp"], l["N"], l["K"], GROUP, out=l["y"])
+
+
+def run_step_e2e(layer):
+    """The same step through host buffers: x from pinned memory in, y back out, every call."""
+    from paper_2306_00978_b200 import binding
+    for l in layer:
+        l["x_dev_in"].copy_(l["x_host"], non_blocking=True)
+        binding.linear(l["x_dev_in"], l["qw"], l["sc"], l["zp"], l["N"], l["K"], GROUP, out=l["y"])
+        l["y_host"].copy_(l["y"], non_blocking=True)
+
+
+def timed_region(fn, layers, steps: int, warmup: int, device: str):
+    """W warm-up steps, then exactly `steps` steps between barrier+synchronize, CUDA events on
+    the launching stream; returns (seconds = max over ranks, launches)."""
+    import torch
+    from paper_2306_00978_b200 import binding
+    for i in range(warmup):
+        fn(layers[i % len(layers)])
+    torch.cuda.synchronize()
+    replicas.barrier()
+    torch.cuda.synchronize()
+    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    n0 = binding.launch_count()
+    t0 = time.time()
+    start.record()
+    for i in range(steps):
+        fn(layers[(warmup + i) % len(layers)])
+    end.record()
+    torch.cuda.synchronize()
+    t1 = time.time()
+    replicas.barrier()
+    launches = binding.launch_count() - n0
+    sec = start.elapsed_time(end) * 1e-3
+    return replicas.max_over_ranks(sec, device), launches, (t0, t1)
+
+
+def gemm_section(peaks, reps: int = 20):
+    """Prefill GEMM, M = 2048, Llama-2-13B MLP shapes: best-of-reps and mean TFLOP/s."""
+    import torch
+    from paper_2306_00978_b200 import binding
+    out = []
+    M = 2048
+    for idx, (name, K, N) in enumerate(synth.LLAMA2_13B_MLP):
+        seed = 3000 + idx
+        W = torch.from_numpy(synth.weight(seed, N, K)).cuda()
+        a = torch.from_numpy(synth.act_mean_abs(seed, K)).cuda()
+        qw, sc, zp = binding.quantize_pack(W, a, ALPHA, GROUP)
+        s = binding.channel_scale(a, ALPHA, K)
+        x = torch.from_numpy(synth.activations(seed, M, K)).cuda()
+        xs = (x.float() / s[None, :]).half().contiguous()
+        y = torch.empty((M, N), dtype=torch.float16, device="cuda")
+        del W
+        for _ in range(3):
+            binding.linear(xs, qw, sc, zp, N, K, GROUP, out=y)
+        torch.cuda.synchronize()
+        times = []
+        for _ in range(reps):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            binding.linear(xs, qw, sc, zp, N, K, GROUP, out=y)
+            e1.record()
+            torch.cuda.synchronize()
+            times.append(e0.elapsed_time(e1) * 1e-3)
+        binding.poll_status()
+        flops = 2.0 * M * N * K
+        best, mean = min(times), sum(times) / len(times)
+        out.append({"shape": f"{K}->{N}", "M": M, "tflops_best": flops / best / 1e12,
+                    "tflops_mean": flops / mean / 1e12, "ms_best": best * 1e3,
+                    "frac_of_measured_bf16_burst": flops / best / 1e12 / peaks["bf16_tflops"],
+                    "frac_of_nominal_2250": flops / best / 1e12 / NOMINAL_FP16_TFLOPS})
+    return out
+
+
+def quantize_section(peaks, reps: int = 10):
+    import torch
+    from paper_2306_00978_b200 import binding
+    N, K = 11008, 4096
+    W = torch.from_numpy(synth.weight(2004, N, K)).cuda()
+    a = torch.from_numpy(synth.act_mean_abs(2004, K)).cuda()
+    for _ in range(3):
+        binding.quantize_pack(W, a, ALPHA, GROUP)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(reps):
+        binding.quantize_pack(W, a, ALPHA, GROUP)
+    e1.record()
+    torch.cuda.synchronize()
+    sec = e0.elapsed_time(e1) * 1e-3 / reps
+    nbytes = 2 * N * K + 4 * K + N * K // 2 + 2 * N * K // GROUP + N * K // (2 * GROUP)
+    return {"shape": f"{K}->{N}", "gbs": nbytes / sec / 1e9, "ms": sec * 1e3,
+            "frac_of_hbm_peak": nbytes / sec / 1e9 / peaks["hbm_gbs"],
+            "note": "includes the output allocation of the Python binding"}
+
+
+# ------------------------------------------------------------------- oracle (CPU) arm
+def _oracle_layer_inputs(max_rows=None):
+    """Quantizes one decoder layer's matrices with the oracle; optionally only the first
+    `max_rows` output rows of each (whole 128-row slabs), to bound the work."""
+    from oracle import awq_oracle as orc
+    items = []
+    for idx, (name, K, N) in enumerate(synth.LLAMA2_7B_LAYER):
+        seed = 2000 + idx
+        n = N if max_rows is None else min(N, max_rows)
+        W = synth.weight(seed, N, K)[:n]
+        a = synth.act_mean_abs(seed, K)
+        s = orc.channel_scale(a, ALPHA)
+        x = synth.activations(seed, 1, K)
+        xs = (x.astype(np.float32) / s[None, :]).astype(np.float16)
+        qw, sc, zp = orc.quantize_pack(W, a, ALPHA, GROUP)
+        items.append((n, K, xs, qw, sc, zp))
+    return items
+
+
+def _oracle_step(items):
+    from oracle import awq_oracle as orc
+    for (n, K, xs, qw, sc, zp) in items:
+        orc.linear_from_packed(xs, qw, sc, zp, n, K, GROUP)
+
+
+def cpu_baseline(budget_s: float = 20.0):
+    """The oracle as it stands on the host cores, on a bounded sample of the same step."""
+    rows = 1024
+    items = _oracle_layer_inputs(max_rows=rows)
+    nbytes = sum(algorithmic_bytes(n, K, 1) for (n, K, *_rest) in items)
+    t0 = time.time()
+    reps = 0
+    while True:
+        _oracle_step(items)
+        reps += 1
+        if time.time() - t0 > budget_s * 0.5 or reps >= 3:
+            break
+    sec = (time.time() - t0) / reps
+    try:
+        from threadpoolctl import threadpool_info
+        cores = max([p.get("num_threads", 1) for p in threadpool_info()] or [1])
+    except Exception:
+        cores = os.cpu_count() or 1
+    return {"value": nbytes / sec / 1e9, "unit": UNIT, "cores": int(cores), "kind": "oracle",
+            "sample": f"first {rows} output rows of each of the 7 linears of one layer at M=1 "
+                      f"(unpack + fp64 dequantize + fp64 product), {reps} repetitions"}
+
+
+def reference_arm(args):
+    rank, world, _ = replicas.env_world()
+    if rank != 0:
+        return 0
+    steps, warmup = max(1, args.steps), max(0, args.warmup)
+    # size the per-step sample so that the whole run stays within a few minutes
+    budget = 150.0 / (steps + warmup)
+    rows = 1024
+    per_row_s = 12 * 1.7 / 4096           # about 1.7 s per 4096x4096 matrix on 8 cores
+    while rows > 128 and rows * per_row_s > budget:
+        rows //= 2
+    items = _oracle_layer_inputs(max_rows=rows)
+    nbytes = sum(algorithmic_bytes(n, K, 1) for (n, K, *_rest) in items)
+    for _ in range(warmup):
+        _oracle_step(items)
+    t0 = time.time()
+    for _ in range(steps):
+        _oracle_step(items)
+    sec = (time.time() - t0) / steps
+    try:
+        from threadpoolctl import threadpool_info
+        cores = max([p.get("num_threads", 1) for p in threadpool_info()] or [1])
+    except Exception:
+        cores = os.cpu_count() or 1
+    value = nbytes / sec / 1e9
+    sample = (f"each step = first {rows} output rows of each of the 7 linears of one layer at M=1 "
+              f"through the CPU oracle")
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": steps, "warmup": warmup, "ms_per_step": sec * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": "llama2-7b decoder-layer linears, M=1, g128, alpha=0.5 (bounded sample)",
+                       "rows_per_linear": rows},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": int(cores), "kind": "oracle",
+                             "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+    return 0
+
+
+# --------------------------------------------------------------------------------- main
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=100)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--layers", type=int, default=4, help="independently seeded layers to rotate over")
+    ap.add_argument("--skip-extras", action="store_true", help="only the headline step (for profiling)")
+    args = ap.parse_args()
+
+    if args.impl == "reference":
+        return reference_arm(args)
+
+    import torch
+    from paper_2306_00978_b200 import binding
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    rank, world, local_rank = replicas.env_world()
+    torch.cuda.set_device(local_rank)
+    device = f"cuda:{local_rank}"
+    replicas.init("nccl")
+    binding.lib()                                     # fail now if the library is missing
+    peaks = load_peaks()
+    warmup = max(3, args.warmup)
+    steps = max(1, args.steps)
+
+    layers = build_layers(args.layers)
+    step_bytes = sum(algorithmic_bytes(l["N"], l["K"], 1) for l in layers[0])
+    packed_bytes = sum(l["qw"].numel() + l["sc"].numel() * 2 + l["zp"].numel() for l in layers[0])
+
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    sec, launches, (w0, w1) = timed_region(run_step, layers, steps, warmup, device)
+    e2e_sec, _, _ = timed_region(run_step_e2e, layers, steps, warmup, device)
+    clocks = None
+    if rank == 0:
+        if w1 - w0 < 1.0:
+            # the timed region is too short for 100 ms clock samples: keep the same load
+            # running (untimed) for about a second and sample that instead
+            w0 = time.time()
+            while time.time() - w0 < 1.2:
+                for i in range(50):
+                    run_step(layers[i % len(layers)])
+                torch.cuda.synchronize()
+            w1 = time.time()
+            clocks_note = "sampled over ~1.2 s of the same steps run right after the timed region"
+        else:
+            clocks_note = "sampled during the timed region"
+        time.sleep(0.15)
+        sampler.stop()
+        clocks = sampler.summary(w0, w1)
+        clocks["note"] = clocks_note
+    binding.poll_status()
+
+    value = replicas.aggregate_throughput(step_bytes * steps, sec) / 1e9
+    e2e_value = replicas.aggregate_throughput(step_bytes * steps, e2e_sec) / 1e9
+    per_launch_s = sec / max(1, launches)
+    achieved = step_bytes * steps / sec / 1e9         # one GPU's algorithmic GB/s over the region
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warmup,
+        "ms_per_step": sec / steps * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f16 x int4 -> f32", "data": "synthetic",
+        "config": {"workload": "llama2-7b decoder-layer linears (q,k,v,o 4096->4096; gate,up 4096->11008; "
+                               "down 11008->4096), M=1, g128, alpha=0.5",
+                   "layers_rotated": args.layers, "packed_bytes_per_layer": packed_bytes,
+                   "l2_policy": f"weights rotate over {args.layers} layers "
+                                f"({args.layers * packed_bytes / 1e6:.0f} MB > 2 x 126 MB L2)",
+                   "algorithmic_bytes_per_step": step_bytes, "parallelism": f"replicas x{world}"},
+        "roofline": {"bound": "hbm", "kernel": "gemv_kernel<128,1>", "achieved": achieved,
+                     "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
+                     "peak_source": peaks["source"], "frac_of_nominal_8000": achieved / NOMINAL_HBM_GBS,
+                     "avg_launch_us": per_launch_s * 1e6, "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH},
+        "e2e": {"value": e2e_value, "unit": UNIT,
+                "h2d_bytes_per_step": sum(2 * l["K"] for l in layers[0]),
+                "d2h_bytes_per_step": sum(2 * l["N"] for l in layers[0])},
+        "gpu_launches": launches,
+        "clocks": clocks,
+    }
+    if rank == 0 and not args.skip_extras:
+        line["gemm_m2048"] = gemm_section(peaks)
+        line["quantize_pack"] = quantize_section(peaks)
+        if world == 1:
+            del layers
+            torch.cuda.empty_cache()
+            line["cpu_baseline"] = cpu_baseline()
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    replicas.barrier()
+    replicas.shutdown()
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())

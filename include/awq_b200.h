@@ -18,7 +18,7 @@
  *    group 64 or 128, M >= 1.  W is fp16 [N][K] row-major, x fp16 [M][K] row-major,
  *    y fp16 [M][N] row-major.
  *
- * Packed layout (layout version 1)
+ * Packed layout (layout version 2)
  *  qweight: N*K/2 bytes.  Tiles of 128 rows x 64 columns are stored whole (4096 bytes),
  *    tile index (n/128)*(K/64) + k/64.  A tile is 8 bands of 16 rows; a band is 32 pieces
  *    of 16 bytes, piece index 4*g + t (g = 0..7, t = 0..3) holding rows g and g+8 of the
@@ -27,9 +27,10 @@
  *      (g,c) (g,c+1) (g+8,c) (g+8,c+1) (g,c+2) (g,c+3) (g+8,c+2) (g+8,c+3),
  *    slot e stored at bits 4p..4p+3 with p = {0,4,1,5,2,6,3,7}[e]  (read from the low
  *    nibble up, the slots appear in the order 0,2,4,6,1,3,5,7 - the GPU order of Sec. 4.2).
- *  scales: fp16 [K/group][N].
- *  zeros:  (K/group) * N/2 bytes; byte gi*(N/2) + (n/16)*8 + (n%8) holds the zero point of
- *    row n (n%16 < 8) in its low nibble and of row n+8 in its high nibble.
+ *  scales: fp16 [N/128][K/group][128] (slab, group, row in slab): the parameters one slab
+ *    needs for consecutive groups are contiguous.
+ *  zeros:  bytes [N/128][K/group][64]; byte (n%128)/16*8 + n%8 of a (slab, group) block holds
+ *    the zero point of row n (n%16 < 8) in its low nibble and of row n+8 in its high nibble.
  */
 #ifndef AWQ_B200_H_
 #define AWQ_B200_H_

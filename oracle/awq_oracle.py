@@ -133,14 +133,21 @@ def qweight_location(n: int, k: int, K: int):
     return word, NIBBLE_OF_SLOT[slot]
 
 
-def zeros_location(n: int, gi: int, N: int):
-    """(byte index, nibble position) of the zero point of row n, group gi.
+def zeros_location(n: int, gi: int, ng: int):
+    """(byte index, nibble position) of the zero point of row n, group gi (ng groups per row).
 
-    One byte holds the zero points of rows g (low nibble) and g+8 (high nibble) of a
-    16-row band; bands follow each other along N, groups along the outer axis.
+    Zero points are stored slab by slab (128 rows), group by group: 64 bytes per (slab,
+    group).  One byte holds the zero points of rows g (low nibble) and g+8 (high nibble) of
+    a 16-row band.
     """
-    band, rr = n // 16, n % 16
-    return gi * (N // 2) + band * 8 + rr % 8, rr // 8
+    slab, r = n // TILE_ROWS, n % TILE_ROWS
+    band, rr = r // 16, r % 16
+    return (slab * ng + gi) * 64 + band * 8 + rr % 8, rr // 8
+
+
+def scales_location(n: int, gi: int, ng: int) -> int:
+    """Element index of Delta of row n, group gi: fp16 [N/128][ng][128] (slab, group, row)."""
+    return ((n // TILE_ROWS) * ng + gi) * TILE_ROWS + n % TILE_ROWS
 
 
 def pack_qweight(codes) -> np.ndarray:
@@ -170,26 +177,34 @@ def unpack_qweight(words, N: int, K: int) -> np.ndarray:
 
 
 def pack_zeros(zeros) -> np.ndarray:
-    """zeros u8 [N][ng] -> u8 [ng][N/2] in the layout of `zeros_location`."""
+    """zeros u8 [N][ng] -> u8 [N/128][ng][64] in the layout of `zeros_location`."""
     zeros = np.asarray(zeros, dtype=np.uint8)
     N, ng = zeros.shape
-    a = zeros.T.reshape(ng, N // 16, 2, 8)              # gi, band, h, g
-    return (a[:, :, 0, :] | (a[:, :, 1, :] << 4)).reshape(ng, N // 2).astype(np.uint8)
+    a = zeros.reshape(N // 128, 8, 2, 8, ng)            # slab, band, h, g, gi
+    a = a.transpose(0, 4, 1, 3, 2)                      # slab, gi, band, g, h
+    return (a[..., 0] | (a[..., 1] << 4)).reshape(N // 128, ng, 64).astype(np.uint8)
 
 
 def unpack_zeros(packed, N: int, ng: int) -> np.ndarray:
-    p = np.asarray(packed, dtype=np.uint8).reshape(ng, N // 16, 8)
-    a = np.stack([p & 0xF, p >> 4], axis=2)             # gi, band, h, g
-    return a.reshape(ng, N).T.copy()
+    p = np.asarray(packed, dtype=np.uint8).reshape(N // 128, ng, 8, 8)   # slab, gi, band, g
+    a = np.stack([p & 0xF, p >> 4], axis=-1)            # slab, gi, band, g, h
+    return a.transpose(0, 2, 4, 3, 1).reshape(N, ng).copy()
 
 
 def pack_scales(scales) -> np.ndarray:
-    """scales fp16 [N][ng] -> fp16 [ng][N] (group-major)."""
-    return np.ascontiguousarray(np.asarray(scales, dtype=np.float16).T)
+    """scales fp16 [N][ng] -> fp16 [N/128][ng][128] (slab, group, row)."""
+    sc = np.asarray(scales, dtype=np.float16)
+    N, ng = sc.shape
+    return np.ascontiguousarray(sc.reshape(N // 128, 128, ng).transpose(0, 2, 1))
+
+
+def unpack_scales(packed, N: int, ng: int) -> np.ndarray:
+    p = np.asarray(packed, dtype=np.float16).reshape(N // 128, ng, 128)
+    return np.ascontiguousarray(p.transpose(0, 2, 1).reshape(N, ng))
 
 
 def quantize_pack(W, act_mean_abs, alpha: float, group: int):
-    """The whole offline step: returns (qweight u32, scales fp16 [ng][N], zeros u8 [ng][N/2])."""
+    """The whole offline step: returns (qweight u32, scales fp16 [N/128][ng][128], zeros u8 [N/128][ng][64])."""
     K = W.shape[1]
     a = np.ones(K, np.float32) if act_mean_abs is None else act_mean_abs
     codes, zeros, scales = quantize(W, channel_scale(a, alpha), group)
@@ -222,7 +237,7 @@ def linear_from_packed(x, qweight, scales_gn, zeros_packed, N: int, K: int, grou
     ng = K // group
     codes = unpack_qweight(qweight, N, K)
     zeros = unpack_zeros(zeros_packed, N, ng)
-    scales = np.asarray(scales_gn, dtype=np.float16).reshape(ng, N).T
+    scales = unpack_scales(scales_gn, N, ng)
     if rows is not None:
         codes, zeros, scales = codes[rows], zeros[rows], scales[rows]
     return linear(x, dequantize(codes, zeros, scales, group))

@@ -99,13 +99,14 @@ def channel_scale(act_mean_abs: Optional[torch.Tensor], alpha: float, K: int) ->
 
 
 def quantize_pack(W: torch.Tensor, act_mean_abs: Optional[torch.Tensor], alpha: float, group: int):
-    """awq_quantize_pack: returns (qweight u8 [N*K/2], scales fp16 [K/group][N], zeros u8 [K/group][N/2])."""
+    """awq_quantize_pack: returns (qweight u8 [N*K/2], scales fp16 [N/128][K/group][128],
+    zeros u8 [N/128][K/group][64])."""
     N, K = W.shape
     qb, sb, zb = packed_sizes(N, K, group)
     dev = W.device
     qweight = torch.empty(qb, dtype=torch.uint8, device=dev)
-    scales = torch.empty((K // group, N), dtype=torch.float16, device=dev)
-    zeros = torch.empty((K // group, N // 2), dtype=torch.uint8, device=dev)
+    scales = torch.empty((N // 128, K // group, 128), dtype=torch.float16, device=dev)
+    zeros = torch.empty((N // 128, K // group, 64), dtype=torch.uint8, device=dev)
     a = 0 if act_mean_abs is None else _dev(act_mean_abs, torch.float32, "act_mean_abs")
     rc = lib().awq_quantize_pack(_dev(W, torch.float16, "W"), a, float(alpha), int(group),
                                  qweight.data_ptr(), scales.data_ptr(), zeros.data_ptr(), N, K, _stream())

@@ -34,31 +34,36 @@ def _stale() -> bool:
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    """Compile every kernel for sm_100a into one shared library; returns its path."""
-    if not force and not _stale():
+def build(force: bool = False, verbose: bool = False, out: str = LIB_PATH, extra=()) -> str:
+    """Compile every kernel for sm_100a into one shared library; returns its path.
+    `extra` are additional nvcc flags (e.g. -D switches for an experiment), `out` the library
+    to write."""
+    if not force and not _stale() and out == LIB_PATH:
         return LIB_PATH
     objs = []
     procs = []
     for src in SOURCES:
         obj = os.path.join(CSRC, src.replace(".cu", ".o"))
-        cmd = [_nvcc(), *NVCC_FLAGS, "-c", os.path.join(CSRC, src), "-o", obj]
+        cmd = [_nvcc(), *NVCC_FLAGS, *extra, "-c", os.path.join(CSRC, src), "-o", obj]
         if verbose:
             cmd.insert(1, "-Xptxas=-v")
         procs.append((src, subprocess.Popen(cmd, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)))
         objs.append(obj)
     failed = False
     for src, p in procs:
-        out, _ = p.communicate()
+        log, _ = p.communicate()
         if verbose or p.returncode != 0:
-            sys.stderr.write(out)
+            sys.stderr.write(log)
         failed |= p.returncode != 0
     if failed:
         raise RuntimeError("nvcc failed")
-    link = [_nvcc(), "-shared", "-o", LIB_PATH, *objs, "-lcudart", "-Xcompiler", "-fPIC"]
+    link = [_nvcc(), "-shared", "-o", out, *objs, "-lcudart", "-Xcompiler", "-fPIC"]
     subprocess.run(link, check=True)
-    return LIB_PATH
+    return out
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    _extra = tuple(a for a in sys.argv[1:] if a.startswith("-D"))
+    _out = [a[6:] for a in sys.argv[1:] if a.startswith("--out=")]
+    print(build(force="--force" in sys.argv or bool(_extra), verbose="-v" in sys.argv,
+                out=_out[0] if _out else LIB_PATH, extra=_extra))

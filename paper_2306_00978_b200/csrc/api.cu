@@ -20,6 +20,7 @@ struct DeviceState {
     size_t workspace_bytes = 0;
     unsigned int* status_word = nullptr;   // device address of g_status on this device
     int cc_major = -1;
+    int sms = 0;
 };
 DeviceState g_dev[kMaxDevices];
 std::mutex g_mutex;
@@ -52,6 +53,8 @@ int device_state(DeviceState** out) {
             if (e != cudaSuccess) return note_cuda(e);
             d.status_word = reinterpret_cast<unsigned int*>(p);
         }
+        e = cudaDeviceGetAttribute(&d.sms, cudaDevAttrMultiProcessorCount, dev);
+        if (e != cudaSuccess) return note_cuda(e);
         d.cc_major = major;
     }
     if (d.cc_major != 10) return AWQ_ERR_WRONG_DEVICE;
@@ -114,8 +117,8 @@ int awq_quantize_pack(const void* W, const float* act_mean_abs, float alpha, int
                                           reinterpret_cast<uint8_t*>(zeros), N, K, (cudaStream_t)stream));
 }
 
-static int resolve_path(int M, int path) {
-    if (path == AWQ_PATH_AUTO) return M <= 8 ? AWQ_PATH_GEMV : AWQ_PATH_GEMM;
+static int resolve_path(int M, int K, int path) {
+    if (path == AWQ_PATH_AUTO) return (M <= 8 && K <= 65536) ? AWQ_PATH_GEMV : AWQ_PATH_GEMM;
     return path;
 }
 
@@ -148,20 +151,21 @@ int awq_linear_path(const void* x, const void* qweight, const void* scales, cons
     if (!aligned16(x) || !aligned16(qweight) || !aligned16(scales) || !aligned16(zeros) || !aligned16(y))
         return AWQ_ERR_MISALIGNED;
     if (path != AWQ_PATH_AUTO && path != AWQ_PATH_GEMV && path != AWQ_PATH_GEMM) return AWQ_ERR_BAD_ARGUMENT;
-    path = resolve_path(M, path);
-    if (path == AWQ_PATH_GEMV && M > 16) return AWQ_ERR_BAD_SHAPE;
+    path = resolve_path(M, K, path);
+    if (path == AWQ_PATH_GEMV && (M > 16 || K > 65536)) return AWQ_ERR_BAD_SHAPE;
     DeviceState* d;
     if (int rc = device_state(&d)) return rc;
     const cudaStream_t st = (cudaStream_t)stream;
     if (path == AWQ_PATH_GEMV) {
         const GemvPlan plan = gemv_plan(M, N, K, group);
         void* ws = nullptr;
-        if (plan.workspace_bytes) {
+        {
             std::lock_guard<std::mutex> lock(g_mutex);
             if (d->workspace_bytes < plan.workspace_bytes) return AWQ_ERR_NO_WORKSPACE;
             ws = d->workspace;
         }
-        return note_cuda(launch_gemv(x, qweight, scales, zeros, y, M, N, K, group, plan, ws, st));
+        return note_cuda(launch_gemv(x, qweight, scales, zeros, y, M, N, K, group, ws, d->status_word,
+                                     d->sms, st));
     }
     return note_cuda(launch_gemm(x, qweight, scales, zeros, y, M, N, K, group, d->status_word, st));
 }
@@ -215,7 +219,7 @@ const char* awq_status_string(int status) {
 }
 
 const char* awq_last_cuda_error(void) { return t_cuda_error; }
-int awq_layout_version(void) { return 1; }
+int awq_layout_version(void) { return 2; }
 unsigned long long awq_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
 }  // extern "C"

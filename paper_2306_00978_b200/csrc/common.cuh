@@ -34,15 +34,16 @@ cudaError_t launch_unpack(const uint32_t* qweight, const __half* scales, const u
                           int N, int K, int group, uint8_t* codes, uint16_t* scales_nk,
                           uint8_t* zeros_nk, cudaStream_t st);
 
+constexpr int kGemvMaxBlocks = 256;      // upper bound on the matrix-vector kernel's grid
+
 struct GemvPlan {
-    int splits;          // thread blocks along K per 128-row slab
-    int ktiles_per_split;
-    size_t workspace_bytes;
+    int max_blocks;
+    size_t workspace_bytes;   // arrival counters + two fp32 partial-sum slots per block
 };
 GemvPlan gemv_plan(int M, int N, int K, int group);
 cudaError_t launch_gemv(const void* x, const void* qweight, const void* scales, const void* zeros,
-                        void* y, int M, int N, int K, int group, const GemvPlan& plan,
-                        void* workspace, cudaStream_t st);
+                        void* y, int M, int N, int K, int group, void* workspace,
+                        unsigned int* status_word, int sms, cudaStream_t st);
 
 cudaError_t launch_gemm(const void* x, const void* qweight, const void* scales, const void* zeros,
                         void* y, int M, int N, int K, int group, unsigned int* status_word,

@@ -26,6 +26,7 @@
 
 #include <mutex>
 
+#include "async_copy.cuh"
 #include "common.cuh"
 
 namespace awq {
@@ -36,8 +37,6 @@ constexpr int kGemmThreads = 512;
 constexpr int kBK = 64;
 constexpr int kATileBytes = 128 * kBK * 2;            // dequantized fp16 weight tile
 constexpr int kMetaBytes = 1024;                      // 256 B scales + 64 B zeros, padded to keep stages 1024-aligned
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;
-constexpr unsigned int kTimeoutCode = 0x57A17u;
 
 template <int BN> struct GemmCfg {
     static constexpr int kXTileBytes = BN * kBK * 2;
@@ -50,67 +49,10 @@ template <int BN> struct GemmCfg {
 };
 
 // ------------------------------------------------------------------ small PTX wrappers
-__device__ __forceinline__ uint32_t smem_u32(const void* p) {
-    return (uint32_t)__cvta_generic_to_shared(p);
-}
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok != 0;
-}
-__device__ __forceinline__ unsigned long long global_ns() {
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    return t;
-}
-
-struct WaitCtl {
-    unsigned int* status;            // device status word (global)
-    volatile unsigned int* abort;    // block-wide flag (shared)
-};
-
-// Bounded wait on an mbarrier phase.  Returns false if the block is giving up.
-__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, const WaitCtl& ctl) {
-    const unsigned long long t0 = global_ns();
-    for (unsigned int i = 1;; ++i) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if ((i & 63u) == 0u) {
-            if (*ctl.abort) return false;
-            if (global_ns() - t0 > kWaitLimitNs) {
-                *ctl.abort = 1u;
-                atomicExch(ctl.status, kTimeoutCode);
-                return false;
-            }
-        }
-    }
-}
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const WaitCtl& ctl) {
-    if (mbar_try_wait(bar, parity)) return true;
-    return mbar_wait_slow(bar, parity, ctl);
-}
-
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
     asm volatile(
         "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
         ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar) : "memory");
-}
-__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
-    asm volatile(
-        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-        ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
 __device__ __forceinline__ void fence_proxy_async_smem() {
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -205,7 +147,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const unsigned char* __re
         s_abort = 0u;
         for (int s = 0; s < S; ++s) { mbar_init(raw_full(s), 1); mbar_init(a_full(s), 8); mbar_init(empty(s), 1); }
         for (int b = 0; b < 2; ++b) { mbar_init(acc_full(b), 1); mbar_init(acc_empty(b), 4); }
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        mbar_fence_init();
     }
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
@@ -235,8 +177,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const unsigned char* __re
                     tma_load_2d(x_addr(stage), &x_map, kb * kBK, mt * BN, bar);
                     const uint32_t raw = a_addr(stage) + kATileBytes;
                     bulk_load(raw, wsrc + (size_t)kb * kTileBytes, kTileBytes, bar);
-                    bulk_load(raw + kTileBytes, scales + (size_t)gi * N + slab * 128, 256, bar);
-                    bulk_load(raw + kTileBytes + 256, zeros + (size_t)gi * (N / 2) + slab * 64, 64, bar);
+                    const size_t sg = (size_t)slab * (K / G) + gi;
+                    bulk_load(raw + kTileBytes, scales + sg * 128, 256, bar);
+                    bulk_load(raw + kTileBytes + 256, zeros + sg * 64, 64, bar);
                     ++issued;
                     if (++stage == S) { stage = 0; phase ^= 1u; }
                 }

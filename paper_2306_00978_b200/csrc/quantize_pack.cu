@@ -123,7 +123,6 @@ quantize_pack_kernel(const __half* __restrict__ W, const float* __restrict__ a, 
                 mx[ti][h] = fmaxf(mx[ti][h], __shfl_xor_sync(0xFFFFFFFFu, mx[ti][h], off));
             }
 
-    const int band = slab * 8 + warp;
 #pragma unroll
     for (int ti = 0; ti < 2; ++ti) {
         __half d16[2]; float d[2], z[2];
@@ -146,10 +145,12 @@ quantize_pack_kernel(const __half* __restrict__ W, const float* __restrict__ a, 
         *dst = make_uint4(words[0], words[1], words[2], words[3]);
 
         if (t == 0 && (G == 64 || ti == 0)) {
+            // parameters are stored slab by slab, group by group: 128 scales, 64 zero bytes
             const int gi = (G == 64) ? kblk * 2 + ti : kblk;
-            scales[(size_t)gi * N + n0] = d16[0];
-            scales[(size_t)gi * N + n0 + 8] = d16[1];
-            zeros[(size_t)gi * (N / 2) + band * 8 + g] = (uint8_t)((uint32_t)z[0] | ((uint32_t)z[1] << 4));
+            const size_t sg = (size_t)slab * (K / G) + gi;
+            scales[sg * 128 + warp * 16 + g] = d16[0];
+            scales[sg * 128 + warp * 16 + g + 8] = d16[1];
+            zeros[sg * 64 + warp * 8 + g] = (uint8_t)((uint32_t)z[0] | ((uint32_t)z[1] << 4));
         }
     }
 }
@@ -173,8 +174,9 @@ __global__ void unpack_kernel(const uint32_t* __restrict__ qweight, const __half
     codes[idx] = (uint8_t)((w >> (4 * nib)) & 0xFu);
     if (k % group == 0) {
         const int gi = k / group, ng = K / group;
-        scales_nk[(size_t)n * ng + gi] = __half_as_ushort(scales[(size_t)gi * N + n]);
-        const uint8_t zb = zeros[(size_t)gi * (N / 2) + (n / 16) * 8 + g];
+        const size_t sg = (size_t)(n / 128) * ng + gi;
+        scales_nk[(size_t)n * ng + gi] = __half_as_ushort(scales[sg * 128 + r]);
+        const uint8_t zb = zeros[sg * 64 + band * 8 + g];
         zeros_nk[(size_t)n * ng + gi] = (uint8_t)((zb >> (4 * h)) & 0xFu);
     }
 }

@@ -32,7 +32,7 @@ def test_header_symbols_are_exported(lib):
 
 
 def test_sizes_and_layout_version(lib):
-    assert lib.awq_layout_version() == 1
+    assert lib.awq_layout_version() == 2
     assert lib.awq_qweight_bytes(4096, 4096) == 4096 * 4096 // 2
     assert lib.awq_scales_bytes(4096, 4096, 128) == 32 * 4096 * 2
     assert lib.awq_zeros_bytes(4096, 11008, 64) == 172 * 4096 // 2
@@ -40,6 +40,7 @@ def test_sizes_and_layout_version(lib):
     assert lib.awq_scales_bytes(4096, 4096, 32) == 0
     assert lib.awq_workspace_bytes(1, 4096, 4096, 128) > 4096
     assert lib.awq_workspace_bytes(64, 4096, 4096, 128) == 0
+    assert lib.awq_workspace_bytes(8, 4096, 4096, 128) == 4096 + 256 * 2 * 8 * 128 * 4
 
 
 def test_argument_errors_need_no_gpu(lib):

@@ -73,8 +73,9 @@ def test_auto_dispatch_and_special_values():
         ref = orc.linear(x, orc.dequantize(codes, zeros, scales, G))
         mask = np.ones(N, bool)
         mask[200] = False
-        assert not y[:, mask].any()
-        assert np.allclose(y[:, 200], ref[:, 200], rtol=2e-3, atol=0)
+        # zero up to fp32 rounding of (sum q x) - z (sum x): far below one fp16 ulp of a typical output
+        assert np.abs(y[:, mask]).max() <= 1e-5
+        assert np.allclose(y[:, 200], ref[:, 200], rtol=2e-3, atol=1e-5)
 
 
 def test_end_to_end_quantize_then_linear():

@@ -201,15 +201,26 @@ def test_zero_and_scale_packing():
     N, ng = 256, 3
     zeros = rng.integers(0, 16, size=(N, ng), dtype=np.uint8)
     packed = orc.pack_zeros(zeros)
-    assert packed.shape == (ng, N // 2)
+    assert packed.shape == (N // 128, ng, 64)
     flat = packed.reshape(-1)
+    seen = set()
     for n in range(N):
         for gi in range(ng):
-            b, nib = orc.zeros_location(n, gi, N)
+            b, nib = orc.zeros_location(n, gi, ng)
+            assert (b, nib) not in seen
+            seen.add((b, nib))
             assert (int(flat[b]) >> (4 * nib)) & 0xF == int(zeros[n, gi])
     assert np.array_equal(orc.unpack_zeros(packed, N, ng), zeros)
     sc = rng.standard_normal((N, ng)).astype(np.float16)
-    assert np.array_equal(orc.pack_scales(sc)[2], sc[:, 2])
+    ps = orc.pack_scales(sc)
+    assert ps.shape == (N // 128, ng, 128)
+    for n in (0, 5, 127, 128, 255):
+        for gi in range(ng):
+            assert ps.reshape(-1)[orc.scales_location(n, gi, ng)] == sc[n, gi]
+    assert np.array_equal(orc.unpack_scales(ps, N, ng), sc)
+    # one slab's parameters of consecutive groups are contiguous: 256 and 64 bytes per group
+    assert orc.scales_location(0, 1, ng) - orc.scales_location(0, 0, ng) == 128
+    assert orc.zeros_location(0, 1, ng)[0] - orc.zeros_location(0, 0, ng)[0] == 64
 
 
 # ------------------------------------------------------- dequantize-then-multiply, exactly

@@ -20,12 +20,12 @@ def _gpu_quantize(case, a_override="case"):
 
 
 def _assert_bit_exact(case, qw, sc, zp):
-    got_q = qw.cpu().numpy().view(np.uint32)
-    got_s = sc.cpu().numpy().view(np.uint16)
-    got_z = zp.cpu().numpy()
-    bad_s = int((got_s != case.scales_gn.view(np.uint16)).sum())
-    bad_z = int((got_z != case.zeros_packed).sum())
-    bad_q = int((got_q != case.qweight).sum())
+    got_q = qw.cpu().numpy().view(np.uint32).reshape(-1)
+    got_s = sc.cpu().numpy().view(np.uint16).reshape(-1)
+    got_z = zp.cpu().numpy().reshape(-1)
+    bad_s = int((got_s != case.scales_gn.view(np.uint16).reshape(-1)).sum())
+    bad_z = int((got_z != case.zeros_packed.reshape(-1)).sum())
+    bad_q = int((got_q != case.qweight.reshape(-1)).sum())
     assert (bad_s, bad_z, bad_q) == (0, 0, 0), f"mismatching scales/zeros/words: {bad_s}/{bad_z}/{bad_q}"
 
 
