@@ -53,7 +53,8 @@ typedef enum AwqStatus {
     AWQ_ERR_WRONG_DEVICE = 7,   /* current device is not compute capability 10.x */
     AWQ_ERR_CUDA = 8,           /* a CUDA runtime / driver call failed */
     AWQ_ERR_TIMEOUT = 9,        /* a bounded device-side wait ran out (see awq_poll_status) */
-    AWQ_ERR_BAD_ARGUMENT = 10
+    AWQ_ERR_BAD_ARGUMENT = 10,
+    AWQ_ERR_STATIC_LIMIT = 11   /* awq_linear_gemv_static: problem larger than its built-in scratch */
 } AwqStatus;
 
 /* Which kernel awq_linear_path runs. */
@@ -109,6 +110,31 @@ int awq_linear(const void* x, const void* qweight, const void* scales, const voi
  * AWQ_PATH_GEMV with M > 16 returns AWQ_ERR_BAD_SHAPE. */
 int awq_linear_path(const void* x, const void* qweight, const void* scales, const void* zeros,
                     void* y, int M, int N, int K, int group, int path, void* stream);
+
+/*
+ * The matrix-vector kernel of awq_linear for callers that cannot allocate device memory.
+ * (The paper has no counterpart: this is a deployment variant of the same computation.)
+ *
+ * Some hosts of this library may not call cudaMalloc at all - for example an inference
+ * server whose memory pool owns the whole device and forbids allocations after start-up, or
+ * code running where an allocation would synchronize the device or fail.  Such callers
+ * cannot provide the workspace awq_set_workspace expects.  This entry point needs none: the
+ * kernel's scratch (arrival counters and fp32 partial sums) lives in an array that is part
+ * of the library's device image, about 2 MB, held by every GPU that loads the library until
+ * the process exits.  The call itself allocates nothing: no cudaMalloc, no cudaFree, no
+ * allocating library routine.
+ *
+ * Arguments, layouts and result are those of awq_linear with the matrix-vector kernel; the
+ * output is bit-identical to awq_linear_path(..., AWQ_PATH_GEMV, ...).
+ * Limits: M <= 8 and K <= 65536; anything larger returns AWQ_ERR_STATIC_LIMIT and does nothing.
+ * The first call on a device looks up the scratch array's device address (this can load the
+ * library's device code), so make that first call before any stream capture begins.
+ * All calls on a device share the one array, and each call re-zeroes its counters on `stream`
+ * before the kernel: two calls that overlap on the GPU (different streams, or one stream with
+ * work that is allowed to overlap) race and give undefined output.  Issue them on one stream.
+ */
+int awq_linear_gemv_static(const void* x, const void* qweight, const void* scales, const void* zeros,
+                            void* y, int M, int N, int K, int group, void* stream);
 
 /* Workspace (scratch for split-K partial sums and arrival counters).
  * awq_workspace_bytes: bytes awq_linear needs for this problem (0 if none).

@@ -21,7 +21,7 @@ EXPORTS = (
     "awq_qweight_bytes", "awq_scales_bytes", "awq_zeros_bytes", "awq_quantize_pack",
     "awq_channel_scale", "awq_linear", "awq_linear_path", "awq_workspace_bytes",
     "awq_set_workspace", "awq_unpack_canonical", "awq_poll_status", "awq_status_string",
-    "awq_last_cuda_error", "awq_layout_version", "awq_launch_count",
+    "awq_last_cuda_error", "awq_layout_version", "awq_launch_count", "awq_linear_gemv_static",
 )
 
 _lib = None
@@ -48,6 +48,7 @@ def lib() -> ctypes.CDLL:
     L.awq_channel_scale.restype, L.awq_channel_scale.argtypes = i, [vp, f, vp, i, vp]
     L.awq_linear.restype, L.awq_linear.argtypes = i, [vp, vp, vp, vp, vp, i, i, i, i, vp]
     L.awq_linear_path.restype, L.awq_linear_path.argtypes = i, [vp, vp, vp, vp, vp, i, i, i, i, i, vp]
+    L.awq_linear_gemv_static.restype, L.awq_linear_gemv_static.argtypes = i, [vp, vp, vp, vp, vp, i, i, i, i, vp]
     L.awq_workspace_bytes.restype, L.awq_workspace_bytes.argtypes = sz, [i, i, i, i]
     L.awq_set_workspace.restype, L.awq_set_workspace.argtypes = i, [vp, sz]
     L.awq_unpack_canonical.restype, L.awq_unpack_canonical.argtypes = i, [vp, vp, vp, i, i, i, vp, vp, vp, vp]
@@ -151,6 +152,23 @@ def linear(x: torch.Tensor, qweight: torch.Tensor, scales: torch.Tensor, zeros: 
         rc = lib().awq_linear_path(*args, int(path), _stream())
     _check(rc, "awq_linear")
     return y
+
+
+def linear_gemv_static(x: torch.Tensor, qweight: torch.Tensor, scales: torch.Tensor, zeros: torch.Tensor,
+                       N: int, K: int, group: int, out: torch.Tensor) -> torch.Tensor:
+    """awq_linear_gemv_static: the matrix-vector kernel on the library's built-in scratch.
+
+    For callers that must not allocate device memory: nothing is allocated here either,
+    so the output tensor `out` (fp16 [M][N]) has to be passed in.  M <= 8."""
+    M = x.shape[0]
+    if x.shape[1] != K or tuple(out.shape) != (M, N):
+        raise AwqError("x must be [M][K] and out [M][N]")
+    rc = lib().awq_linear_gemv_static(
+        _dev(x, torch.float16, "x"), _dev(qweight, torch.uint8, "qweight"),
+        _dev(scales, torch.float16, "scales"), _dev(zeros, torch.uint8, "zeros"),
+        _dev(out, torch.float16, "out"), M, N, K, int(group), _stream())
+    _check(rc, "awq_linear_gemv_static")
+    return out
 
 
 def unpack_canonical(qweight, scales, zeros, N: int, K: int, group: int):

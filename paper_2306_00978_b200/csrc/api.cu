@@ -170,6 +170,25 @@ int awq_linear_path(const void* x, const void* qweight, const void* scales, cons
     return note_cuda(launch_gemm(x, qweight, scales, zeros, y, M, N, K, group, d->status_word, st));
 }
 
+int awq_linear_gemv_static(const void* x, const void* qweight, const void* scales, const void* zeros,
+                            void* y, int M, int N, int K, int group, void* stream) {
+    if (int rc = check_shape(N, K, group)) return rc;
+    if (M < 1) return AWQ_ERR_BAD_SHAPE;
+    if (M > gemv_static_max_m() || K > 65536) return AWQ_ERR_STATIC_LIMIT;
+    if (!x || !qweight || !scales || !zeros || !y) return AWQ_ERR_NULL_POINTER;
+    if (!aligned16(x) || !aligned16(qweight) || !aligned16(scales) || !aligned16(zeros) || !aligned16(y))
+        return AWQ_ERR_MISALIGNED;
+    DeviceState* d;
+    if (int rc = device_state(&d)) return rc;
+    void* scratch = nullptr;
+    if (int rc = note_cuda(gemv_static_scratch(&scratch))) return rc;
+    const cudaStream_t st = (cudaStream_t)stream;
+    // the arrival counters must start at zero whatever an earlier call left behind
+    if (int rc = note_cuda(cudaMemsetAsync(scratch, 0, kCounterBytes, st))) return rc;
+    return note_cuda(launch_gemv(x, qweight, scales, zeros, y, M, N, K, group, scratch, d->status_word,
+                                 d->sms, st));
+}
+
 int awq_linear(const void* x, const void* qweight, const void* scales, const void* zeros,
                void* y, int M, int N, int K, int group, void* stream) {
     return awq_linear_path(x, qweight, scales, zeros, y, M, N, K, group, AWQ_PATH_AUTO, stream);
@@ -214,6 +233,7 @@ const char* awq_status_string(int status) {
         case AWQ_ERR_CUDA: return "CUDA call failed (see awq_last_cuda_error)";
         case AWQ_ERR_TIMEOUT: return "a device-side wait ran out";
         case AWQ_ERR_BAD_ARGUMENT: return "bad argument";
+        case AWQ_ERR_STATIC_LIMIT: return "problem exceeds the built-in scratch of awq_linear_gemv_static (M <= 8, K <= 65536)";
         default: return "unknown status";
     }
 }

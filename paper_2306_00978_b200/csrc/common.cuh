@@ -45,6 +45,10 @@ cudaError_t launch_gemv(const void* x, const void* qweight, const void* scales, 
                         void* y, int M, int N, int K, int group, void* workspace,
                         unsigned int* status_word, int sms, cudaStream_t st);
 
+// the matrix-vector kernel's built-in scratch (no allocation): address on the current device
+cudaError_t gemv_static_scratch(void** out);
+int gemv_static_max_m();
+
 cudaError_t launch_gemm(const void* x, const void* qweight, const void* scales, const void* zeros,
                         void* y, int M, int N, int K, int group, unsigned int* status_word,
                         cudaStream_t st);

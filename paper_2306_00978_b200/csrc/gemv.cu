@@ -28,6 +28,8 @@
 // All mbarrier waits are bounded; a wait that runs out records a time-out in the status
 // word, after which every wait of the block returns at once and the block runs to its end
 // (its output is then undefined, the status word says so).
+#include <mutex>
+
 #include "async_copy.cuh"
 #include "common.cuh"
 
@@ -464,6 +466,34 @@ GemvPlan gemv_plan(int M, int N, int K, int group) {
     p.max_blocks = kGemvMaxBlocks;
     p.workspace_bytes = kCounterBytes + (size_t)kGemvMaxBlocks * 2 * M * 128 * sizeof(float);
     return p;
+}
+
+// Built-in scratch of awq_linear_gemv_static: arrival counters followed by the partial-sum
+// slots of up to kStaticMaxM tokens.  Every GPU that loads the library holds it until exit.
+constexpr int kStaticMaxM = 8;
+constexpr size_t kStaticScratchBytes = kCounterBytes + (size_t)kGemvMaxBlocks * 2 * kStaticMaxM * 128 * sizeof(float);
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+int gemv_static_max_m() { return kStaticMaxM; }
+
+// Device address of the built-in scratch on the current device, looked up once per device
+// (in host code the array's name is only a handle; kernels need the address from the runtime).
+cudaError_t gemv_static_scratch(void** out) {
+    static void* s_ptr[64] = {};
+    static std::mutex s_mutex;
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(s_mutex);
+    if (!s_ptr[dev]) {
+        void* p = nullptr;
+        e = cudaGetSymbolAddress(&p, g_static_scratch);
+        if (e != cudaSuccess) return e;
+        s_ptr[dev] = p;
+    }
+    *out = s_ptr[dev];
+    return cudaSuccess;
 }
 
 cudaError_t launch_gemv(const void* x, const void* qweight, const void* scales, const void* zeros,
