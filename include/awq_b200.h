@@ -18,19 +18,20 @@
  *    group 64 or 128, M >= 1.  W is fp16 [N][K] row-major, x fp16 [M][K] row-major,
  *    y fp16 [M][N] row-major.
  *
- * Packed layout (layout version 2)
- *  qweight: N*K/2 bytes.  Tiles of 128 rows x 64 columns are stored whole (4096 bytes),
- *    tile index (n/128)*(K/64) + k/64.  A tile is 8 bands of 16 rows; a band is 32 pieces
- *    of 16 bytes, piece index 4*g + t (g = 0..7, t = 0..3) holding rows g and g+8 of the
- *    band and columns 16t..16t+15 of the tile.  32-bit word j of a piece holds columns
- *    c = 16t+4j .. +3 of both rows as eight 4-bit slots
+ * Packed layout (layout version 3, "band-major": all data of 16 consecutive output rows - a
+ * band - is contiguous along K)
+ *  qweight: N*K/2 bytes.  Block (band, kt) = rows 16*band..+15, columns 64*kt..+63 is 512
+ *    bytes at ((n/16)*(K/64) + k/64) * 512.  A block is 32 pieces of 16 bytes, piece index
+ *    4*g + t (g = 0..7, t = 0..3) holding rows g and g+8 of the band and columns 16t..16t+15 of
+ *    the block.  32-bit word j of a piece holds columns c = 16t+4j .. +3 of both rows as eight
+ *    4-bit slots
  *      (g,c) (g,c+1) (g+8,c) (g+8,c+1) (g,c+2) (g,c+3) (g+8,c+2) (g+8,c+3),
  *    slot e stored at bits 4p..4p+3 with p = {0,4,1,5,2,6,3,7}[e]  (read from the low
  *    nibble up, the slots appear in the order 0,2,4,6,1,3,5,7 - the GPU order of Sec. 4.2).
- *  scales: fp16 [N/128][K/group][128] (slab, group, row in slab): the parameters one slab
- *    needs for consecutive groups are contiguous.
- *  zeros:  bytes [N/128][K/group][64]; byte (n%128)/16*8 + n%8 of a (slab, group) block holds
- *    the zero point of row n (n%16 < 8) in its low nibble and of row n+8 in its high nibble.
+ *  scales: fp16 [N/16][K/group][16] (band, group, row in band).
+ *  zeros:  bytes [N/32][K/group][16]: per pair of bands and group, bytes 0-7 belong to the even
+ *    band, 8-15 to the odd one; byte n%8 of a band holds the zero point of row n (n%16 < 8)
+ *    in its low nibble and of row n+8 in its high nibble.
  */
 #ifndef AWQ_B200_H_
 #define AWQ_B200_H_
@@ -60,8 +61,10 @@ typedef enum AwqStatus {
 /* Which kernel awq_linear_path runs. */
 typedef enum AwqPath {
     AWQ_PATH_AUTO = 0,          /* what awq_linear does: chosen from M */
-    AWQ_PATH_GEMV = 1,          /* fused dequant matrix-vector kernel, M <= 16 */
-    AWQ_PATH_GEMM = 2           /* tcgen05 tensor-core kernel, any M >= 1 */
+    AWQ_PATH_GEMV = 1,          /* fused dequant matrix-vector kernel, M <= 16: band kernel when
+                                   M <= 4 and N/16 is not much below the SM count, else split-K */
+    AWQ_PATH_GEMM = 2,          /* tcgen05 tensor-core kernel, any M >= 1 */
+    AWQ_PATH_GEMV_SPLITK = 3    /* the split-K matrix-vector kernel, M <= 16 */
 } AwqPath;
 
 /* Sizes of the packed arrays, in bytes (0 if the shape is not accepted). */
@@ -94,20 +97,21 @@ int awq_channel_scale(const float* act_mean_abs, float alpha, float* s, int K, v
  *   y[m][n] = sum_g Delta[g][n] * sum_{k in g} (q[n][k] - z[g][n]) * x[m][k],  stored as fp16.
  * x must already be divided by s (the paper folds diag(s)^-1 into the previous operator).
  * x: in, fp16 [M][K].  y: out, fp16 [M][N], fully overwritten; must not alias an input.
- * M <= 8 runs the matrix-vector kernel (HBM-bound; exact integer (q - z) in fp16 into
- * fp32 tensor-core accumulation, Delta applied in fp32 per group), larger M the tcgen05
- * kernel ((q - z) * Delta rounded once to fp16, fp32 accumulation in tensor memory).
- * The matrix-vector kernel splits K across thread blocks and combines the partial sums in a
- * fixed order through the registered workspace: results are bit-reproducible.  Calls that
- * use the workspace must not overlap on the GPU (issue them on one stream).
- * Errors: AWQ_ERR_NO_WORKSPACE if awq_workspace_bytes(M,N,K,group) exceeds the registered
- * size; shape / pointer errors as listed in AwqStatus.
+ * M <= 8 runs a matrix-vector kernel (HBM-bound; the 4-bit codes enter warp-level tensor-core
+ * products exactly, accumulation, zero point and Delta in fp32, one rounding to fp16 at the
+ * end), larger M the tcgen05 kernel ((q - z) * Delta rounded once to fp16, fp32 accumulation
+ * in tensor memory).  Results are bit-reproducible.
+ * The split-K matrix-vector kernel (used when N is small or M > 4) combines partial sums in a
+ * fixed order through the registered workspace; calls that use the workspace must not
+ * overlap on the GPU (issue them on one stream).
+ * Errors: AWQ_ERR_NO_WORKSPACE if that kernel is chosen and awq_workspace_bytes(M,N,K,group)
+ * exceeds the registered size; shape / pointer errors as listed in AwqStatus.
  */
 int awq_linear(const void* x, const void* qweight, const void* scales, const void* zeros,
                void* y, int M, int N, int K, int group, void* stream);
 
 /* Same as awq_linear with the kernel forced (for the small-batch crossover measurement).
- * AWQ_PATH_GEMV with M > 16 returns AWQ_ERR_BAD_SHAPE. */
+ * A matrix-vector path with M > 16 or K > 65536 returns AWQ_ERR_BAD_SHAPE. */
 int awq_linear_path(const void* x, const void* qweight, const void* scales, const void* zeros,
                     void* y, int M, int N, int K, int group, int path, void* stream);
 
@@ -124,8 +128,8 @@ int awq_linear_path(const void* x, const void* qweight, const void* scales, cons
  * the process exits.  The call itself allocates nothing: no cudaMalloc, no cudaFree, no
  * allocating library routine.
  *
- * Arguments, layouts and result are those of awq_linear with the matrix-vector kernel; the
- * output is bit-identical to awq_linear_path(..., AWQ_PATH_GEMV, ...).
+ * Arguments, layouts and result are those of awq_linear with the split-K matrix-vector
+ * kernel; the output is bit-identical to awq_linear_path(..., AWQ_PATH_GEMV_SPLITK, ...).
  * Limits: M <= 8 and K <= 65536; anything larger returns AWQ_ERR_STATIC_LIMIT and does nothing.
  * The first call on a device looks up the scratch array's device address (this can load the
  * library's device code), so make that first call before any stream capture begins.
@@ -137,7 +141,7 @@ int awq_linear_gemv_static(const void* x, const void* qweight, const void* scale
                             void* y, int M, int N, int K, int group, void* stream);
 
 /* Workspace (scratch for split-K partial sums and arrival counters).
- * awq_workspace_bytes: bytes awq_linear needs for this problem (0 if none).
+ * awq_workspace_bytes: bytes awq_linear may need for this problem (0 if none).
  * awq_set_workspace: registers caller-owned device memory for the current device; the first
  * 4096 bytes are cleared with a synchronous cudaMemset.  Pass (NULL, 0) to unregister.
  * The memory must stay valid until it is unregistered or replaced. */

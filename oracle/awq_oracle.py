@@ -17,8 +17,8 @@ What is computed, and where it comes from
                      represented in FP16").
 * pack_* / unpack_*  eight 4-bit codes per 32-bit word in the order
                      w{0,2,4,6,1,3,5,7} (Sec. 4.2, SIMD-aware weight packing), inside
-                     a 128-row x 64-column tile whose 16-byte pieces are ordered for a
-                     warp-wide register fragment; see `qweight_location`.
+                     512-byte blocks (16 rows x 64 columns) whose 16-byte pieces are ordered
+                     for a warp-wide register fragment; see `qweight_location`.
 * dequantize         (q - z) * Delta, exact in fp64.
 * linear             y = x . dequant(Wq)^T in fp64 (Sec. 4.2, on-the-fly weight
                      dequantization followed by the matrix product; here unfused).
@@ -39,9 +39,9 @@ from __future__ import annotations
 
 import numpy as np
 
-TILE_ROWS = 128          # output channels per packed tile
-TILE_COLS = 64           # input channels per packed tile
-WORDS_PER_TILE = TILE_ROWS * TILE_COLS // 8
+BAND_ROWS = 16           # output channels per band (one packed block holds a band x 64 columns)
+TILE_COLS = 64           # input channels per packed block
+WORDS_PER_BLOCK = BAND_ROWS * TILE_COLS // 8
 # Nibble position (bits 4p..4p+3) of element slot e inside a word: slot order read from
 # the low nibble upwards is {0,2,4,6,1,3,5,7} (Sec. 4.2).
 NIBBLE_OF_SLOT = (0, 4, 1, 5, 2, 6, 3, 7)
@@ -116,19 +116,19 @@ def quantize(W, s, group: int):
 def qweight_location(n: int, k: int, K: int):
     """(word index, nibble position) of code (n, k) in the packed weight array.
 
-    Tiles of 128 output rows x 64 input columns are stored whole (1024 words), row-slab
-    major: tile = (n // 128) * (K // 64) + k // 64.  A tile is 8 bands of 16 rows; a band
-    is 32 pieces of 16 bytes; piece (g, t) holds rows g and g+8 of the band and columns
-    16t .. 16t+15 of the tile.  Word j of a piece holds columns 16t+4j .. 16t+4j+3 of both
+    Rows are taken in bands of 16; everything a band needs is contiguous along K.  Block
+    (band, k // 64) is 512 bytes (128 words) at word (band * (K // 64) + k // 64) * 128.  A
+    block is 32 pieces of 16 bytes; piece (g, t) holds rows g and g+8 of the band and columns
+    16t .. 16t+15 of the block.  Word j of a piece holds columns 16t+4j .. 16t+4j+3 of both
     rows in the slot order (g,c0) (g,c1) (g+8,c0) (g+8,c1) (g,c2) (g,c3) (g+8,c2) (g+8,c3),
     and slot e sits at nibble NIBBLE_OF_SLOT[e].
     """
-    tile = (n // TILE_ROWS) * (K // TILE_COLS) + k // TILE_COLS
-    r, c = n % TILE_ROWS, k % TILE_COLS
-    band, rr = r // 16, r % 16
+    band, rr = n // BAND_ROWS, n % BAND_ROWS
+    block = band * (K // TILE_COLS) + k // TILE_COLS
+    c = k % TILE_COLS
     g, h = rr % 8, rr // 8
     t, j, i = c // 16, (c % 16) // 4, c % 4
-    word = tile * WORDS_PER_TILE + band * 128 + (g * 4 + t) * 4 + j
+    word = block * WORDS_PER_BLOCK + (g * 4 + t) * 4 + j
     slot = (i // 2) * 4 + h * 2 + (i % 2)
     return word, NIBBLE_OF_SLOT[slot]
 
@@ -136,29 +136,28 @@ def qweight_location(n: int, k: int, K: int):
 def zeros_location(n: int, gi: int, ng: int):
     """(byte index, nibble position) of the zero point of row n, group gi (ng groups per row).
 
-    Zero points are stored slab by slab (128 rows), group by group: 64 bytes per (slab,
-    group).  One byte holds the zero points of rows g (low nibble) and g+8 (high nibble) of
-    a 16-row band.
+    Two bands (32 rows) share a 16-byte block per group: [N/32][ng][16].  Bytes 0-7 belong to
+    the even band, 8-15 to the odd band; byte g of a band holds the zero points of its rows g
+    (low nibble) and g+8 (high nibble).
     """
-    slab, r = n // TILE_ROWS, n % TILE_ROWS
-    band, rr = r // 16, r % 16
-    return (slab * ng + gi) * 64 + band * 8 + rr % 8, rr // 8
+    band, rr = n // BAND_ROWS, n % BAND_ROWS
+    return ((band // 2) * ng + gi) * 16 + (band % 2) * 8 + rr % 8, rr // 8
 
 
 def scales_location(n: int, gi: int, ng: int) -> int:
-    """Element index of Delta of row n, group gi: fp16 [N/128][ng][128] (slab, group, row)."""
-    return ((n // TILE_ROWS) * ng + gi) * TILE_ROWS + n % TILE_ROWS
+    """Element index of Delta of row n, group gi: fp16 [N/16][ng][16] (band, group, row)."""
+    return ((n // BAND_ROWS) * ng + gi) * BAND_ROWS + n % BAND_ROWS
 
 
 def pack_qweight(codes) -> np.ndarray:
     """codes u8 [N][K] -> uint32 [N*K/8] in the layout of `qweight_location`."""
     codes = np.asarray(codes, dtype=np.uint8)
     N, K = codes.shape
-    assert N % TILE_ROWS == 0 and K % TILE_COLS == 0
-    # axes: R, band, h, g, C, t, j, ihi, ilo
-    a = codes.reshape(N // 128, 8, 2, 8, K // 64, 4, 4, 2, 2)
-    # -> R, C, band, g, t, j, ihi, h, ilo   (the last three are the slot bits, high to low)
-    a = a.transpose(0, 4, 1, 3, 5, 6, 7, 2, 8).reshape(-1, 8).astype(np.uint32)
+    assert N % BAND_ROWS == 0 and K % TILE_COLS == 0
+    # axes: band, h, g, C, t, j, ihi, ilo
+    a = codes.reshape(N // 16, 2, 8, K // 64, 4, 4, 2, 2)
+    # -> band, C, g, t, j, ihi, h, ilo   (the last three are the slot bits, high to low)
+    a = a.transpose(0, 3, 2, 4, 5, 6, 1, 7).reshape(-1, 8).astype(np.uint32)
     words = np.zeros(a.shape[0], dtype=np.uint32)
     for slot in range(8):
         words |= a[:, slot] << np.uint32(4 * NIBBLE_OF_SLOT[slot])
@@ -172,39 +171,40 @@ def unpack_qweight(words, N: int, K: int) -> np.ndarray:
     a = np.empty((words.size, 8), dtype=np.uint8)
     for slot in range(8):
         a[:, slot] = (words >> np.uint32(4 * NIBBLE_OF_SLOT[slot])) & np.uint32(0xF)
-    a = a.reshape(N // 128, K // 64, 8, 8, 4, 4, 2, 2, 2)
-    return a.transpose(0, 2, 7, 3, 1, 4, 5, 6, 8).reshape(N, K)
+    a = a.reshape(N // 16, K // 64, 8, 4, 4, 2, 2, 2)   # band, C, g, t, j, ihi, h, ilo
+    return a.transpose(0, 6, 2, 1, 3, 4, 5, 7).reshape(N, K)
 
 
 def pack_zeros(zeros) -> np.ndarray:
-    """zeros u8 [N][ng] -> u8 [N/128][ng][64] in the layout of `zeros_location`."""
+    """zeros u8 [N][ng] -> u8 [N/32][ng][16] in the layout of `zeros_location`."""
     zeros = np.asarray(zeros, dtype=np.uint8)
     N, ng = zeros.shape
-    a = zeros.reshape(N // 128, 8, 2, 8, ng)            # slab, band, h, g, gi
-    a = a.transpose(0, 4, 1, 3, 2)                      # slab, gi, band, g, h
-    return (a[..., 0] | (a[..., 1] << 4)).reshape(N // 128, ng, 64).astype(np.uint8)
+    assert N % 32 == 0
+    a = zeros.reshape(N // 32, 2, 2, 8, ng)             # pair, band-in-pair, h, g, gi
+    a = a.transpose(0, 4, 1, 3, 2)                      # pair, gi, band-in-pair, g, h
+    return (a[..., 0] | (a[..., 1] << 4)).reshape(N // 32, ng, 16).astype(np.uint8)
 
 
 def unpack_zeros(packed, N: int, ng: int) -> np.ndarray:
-    p = np.asarray(packed, dtype=np.uint8).reshape(N // 128, ng, 8, 8)   # slab, gi, band, g
-    a = np.stack([p & 0xF, p >> 4], axis=-1)            # slab, gi, band, g, h
+    p = np.asarray(packed, dtype=np.uint8).reshape(N // 32, ng, 2, 8)    # pair, gi, band-in-pair, g
+    a = np.stack([p & 0xF, p >> 4], axis=-1)            # pair, gi, band-in-pair, g, h
     return a.transpose(0, 2, 4, 3, 1).reshape(N, ng).copy()
 
 
 def pack_scales(scales) -> np.ndarray:
-    """scales fp16 [N][ng] -> fp16 [N/128][ng][128] (slab, group, row)."""
+    """scales fp16 [N][ng] -> fp16 [N/16][ng][16] (band, group, row)."""
     sc = np.asarray(scales, dtype=np.float16)
     N, ng = sc.shape
-    return np.ascontiguousarray(sc.reshape(N // 128, 128, ng).transpose(0, 2, 1))
+    return np.ascontiguousarray(sc.reshape(N // 16, 16, ng).transpose(0, 2, 1))
 
 
 def unpack_scales(packed, N: int, ng: int) -> np.ndarray:
-    p = np.asarray(packed, dtype=np.float16).reshape(N // 128, ng, 128)
+    p = np.asarray(packed, dtype=np.float16).reshape(N // 16, ng, 16)
     return np.ascontiguousarray(p.transpose(0, 2, 1).reshape(N, ng))
 
 
 def quantize_pack(W, act_mean_abs, alpha: float, group: int):
-    """The whole offline step: returns (qweight u32, scales fp16 [N/128][ng][128], zeros u8 [N/128][ng][64])."""
+    """The whole offline step: returns (qweight u32, scales fp16 [N/16][ng][16], zeros u8 [N/32][ng][16])."""
     K = W.shape[1]
     a = np.ones(K, np.float32) if act_mean_abs is None else act_mean_abs
     codes, zeros, scales = quantize(W, channel_scale(a, alpha), group)

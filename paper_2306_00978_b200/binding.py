@@ -15,7 +15,7 @@ import torch
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libawq_b200.so")
 
-PATH_AUTO, PATH_GEMV, PATH_GEMM = 0, 1, 2
+PATH_AUTO, PATH_GEMV, PATH_GEMM, PATH_GEMV_SPLITK = 0, 1, 2, 3
 
 EXPORTS = (
     "awq_qweight_bytes", "awq_scales_bytes", "awq_zeros_bytes", "awq_quantize_pack",
@@ -100,14 +100,14 @@ def channel_scale(act_mean_abs: Optional[torch.Tensor], alpha: float, K: int) ->
 
 
 def quantize_pack(W: torch.Tensor, act_mean_abs: Optional[torch.Tensor], alpha: float, group: int):
-    """awq_quantize_pack: returns (qweight u8 [N*K/2], scales fp16 [N/128][K/group][128],
-    zeros u8 [N/128][K/group][64])."""
+    """awq_quantize_pack: returns (qweight u8 [N*K/2], scales fp16 [N/16][K/group][16],
+    zeros u8 [N/32][K/group][16])."""
     N, K = W.shape
     qb, sb, zb = packed_sizes(N, K, group)
     dev = W.device
     qweight = torch.empty(qb, dtype=torch.uint8, device=dev)
-    scales = torch.empty((N // 128, K // group, 128), dtype=torch.float16, device=dev)
-    zeros = torch.empty((N // 128, K // group, 64), dtype=torch.uint8, device=dev)
+    scales = torch.empty((N // 16, K // group, 16), dtype=torch.float16, device=dev)
+    zeros = torch.empty((N // 32, K // group, 16), dtype=torch.uint8, device=dev)
     a = 0 if act_mean_abs is None else _dev(act_mean_abs, torch.float32, "act_mean_abs")
     rc = lib().awq_quantize_pack(_dev(W, torch.float16, "W"), a, float(alpha), int(group),
                                  qweight.data_ptr(), scales.data_ptr(), zeros.data_ptr(), N, K, _stream())

@@ -125,7 +125,7 @@ static int resolve_path(int M, int K, int path) {
 size_t awq_workspace_bytes(int M, int N, int K, int group) {
     if (check_shape(N, K, group) != AWQ_OK || M < 1) return 0;
     if (M > 16) return 0;
-    return gemv_plan(M, N, K, group).workspace_bytes;
+    return gemv_workspace_bytes(M);
 }
 
 int awq_set_workspace(void* dev_ptr, size_t bytes) {
@@ -150,22 +150,25 @@ int awq_linear_path(const void* x, const void* qweight, const void* scales, cons
     if (!x || !qweight || !scales || !zeros || !y) return AWQ_ERR_NULL_POINTER;
     if (!aligned16(x) || !aligned16(qweight) || !aligned16(scales) || !aligned16(zeros) || !aligned16(y))
         return AWQ_ERR_MISALIGNED;
-    if (path != AWQ_PATH_AUTO && path != AWQ_PATH_GEMV && path != AWQ_PATH_GEMM) return AWQ_ERR_BAD_ARGUMENT;
+    if (path != AWQ_PATH_AUTO && path != AWQ_PATH_GEMV && path != AWQ_PATH_GEMM && path != AWQ_PATH_GEMV_SPLITK)
+        return AWQ_ERR_BAD_ARGUMENT;
     path = resolve_path(M, K, path);
-    if (path == AWQ_PATH_GEMV && (M > 16 || K > 65536)) return AWQ_ERR_BAD_SHAPE;
+    if (path != AWQ_PATH_GEMM && (M > 16 || K > 65536)) return AWQ_ERR_BAD_SHAPE;
     DeviceState* d;
     if (int rc = device_state(&d)) return rc;
     const cudaStream_t st = (cudaStream_t)stream;
-    if (path == AWQ_PATH_GEMV) {
-        const GemvPlan plan = gemv_plan(M, N, K, group);
+    if (path == AWQ_PATH_GEMV && gemv_uses_band_kernel(M, N, d->sms))
+        return note_cuda(launch_gemv_band(x, qweight, scales, zeros, y, M, N, K, group, d->status_word,
+                                          d->sms, st));
+    if (path == AWQ_PATH_GEMV || path == AWQ_PATH_GEMV_SPLITK) {
         void* ws = nullptr;
         {
             std::lock_guard<std::mutex> lock(g_mutex);
-            if (d->workspace_bytes < plan.workspace_bytes) return AWQ_ERR_NO_WORKSPACE;
+            if (d->workspace_bytes < gemv_workspace_bytes(M)) return AWQ_ERR_NO_WORKSPACE;
             ws = d->workspace;
         }
-        return note_cuda(launch_gemv(x, qweight, scales, zeros, y, M, N, K, group, ws, d->status_word,
-                                     d->sms, st));
+        return note_cuda(launch_gemv_splitk(x, qweight, scales, zeros, y, M, N, K, group, ws, d->status_word,
+                                            d->sms, st));
     }
     return note_cuda(launch_gemm(x, qweight, scales, zeros, y, M, N, K, group, d->status_word, st));
 }
@@ -185,8 +188,8 @@ int awq_linear_gemv_static(const void* x, const void* qweight, const void* scale
     const cudaStream_t st = (cudaStream_t)stream;
     // the arrival counters must start at zero whatever an earlier call left behind
     if (int rc = note_cuda(cudaMemsetAsync(scratch, 0, kCounterBytes, st))) return rc;
-    return note_cuda(launch_gemv(x, qweight, scales, zeros, y, M, N, K, group, scratch, d->status_word,
-                                 d->sms, st));
+    return note_cuda(launch_gemv_splitk(x, qweight, scales, zeros, y, M, N, K, group, scratch,
+                                        d->status_word, d->sms, st));
 }
 
 int awq_linear(const void* x, const void* qweight, const void* scales, const void* zeros,
@@ -239,7 +242,7 @@ const char* awq_status_string(int status) {
 }
 
 const char* awq_last_cuda_error(void) { return t_cuda_error; }
-int awq_layout_version(void) { return 2; }
+int awq_layout_version(void) { return 3; }
 unsigned long long awq_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
 }  // extern "C"

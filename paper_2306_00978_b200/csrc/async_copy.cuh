@@ -66,6 +66,23 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const W
     return mbar_wait_slow(bar, parity, ctl);
 }
 
+// The same for warps whose wait may be long and is not latency-critical (copy and flush
+// warps): sleep between polls so that the spinning does not take issue slots from the math warps.
+__device__ __forceinline__ bool mbar_wait_relaxed(uint32_t bar, uint32_t parity, const WaitCtl& ctl) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const unsigned long long t0 = global_ns();
+    for (;;) {
+        __nanosleep(128);
+        if (mbar_try_wait(bar, parity)) return true;
+        if (*ctl.abort) return false;
+        if (global_ns() - t0 > kWaitLimitNs) {
+            *ctl.abort = 1u;
+            atomicExch(ctl.status, kTimeoutCode);
+            return false;
+        }
+    }
+}
+
 // global -> shared bulk copy (sizes and both addresses multiples of 16 bytes), completion
 // counted in bytes on an mbarrier of this block
 __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {

@@ -9,7 +9,7 @@ namespace awq {
 
 constexpr int kTileRows = 128;           // output channels per packed tile
 constexpr int kTileCols = 64;            // input channels per packed tile
-constexpr int kTileBytes = kTileRows * kTileCols / 2;
+constexpr int kTileBytes = kTileRows * kTileCols / 2;   // 8 bands x 512 bytes
 constexpr size_t kCounterBytes = 4096;   // head of the workspace: split-K arrival counters
 constexpr int kMaxSlabs = int(kCounterBytes / sizeof(unsigned int));
 
@@ -34,16 +34,18 @@ cudaError_t launch_unpack(const uint32_t* qweight, const __half* scales, const u
                           int N, int K, int group, uint8_t* codes, uint16_t* scales_nk,
                           uint8_t* zeros_nk, cudaStream_t st);
 
-constexpr int kGemvMaxBlocks = 256;      // upper bound on the matrix-vector kernel's grid
+constexpr int kGemvMaxBlocks = 256;      // upper bound on the split-K matrix-vector kernel's grid
 
-struct GemvPlan {
-    int max_blocks;
-    size_t workspace_bytes;   // arrival counters + two fp32 partial-sum slots per block
-};
-GemvPlan gemv_plan(int M, int N, int K, int group);
-cudaError_t launch_gemv(const void* x, const void* qweight, const void* scales, const void* zeros,
-                        void* y, int M, int N, int K, int group, void* workspace,
-                        unsigned int* status_word, int sms, cudaStream_t st);
+// Matrix-vector kernels.  The band kernel needs no workspace; the split-K kernel needs
+// gemv_workspace_bytes(M): arrival counters + two fp32 partial-sum slots per block.
+bool gemv_uses_band_kernel(int M, int N, int sms);
+size_t gemv_workspace_bytes(int M);
+cudaError_t launch_gemv_band(const void* x, const void* qweight, const void* scales, const void* zeros,
+                             void* y, int M, int N, int K, int group, unsigned int* status_word, int sms,
+                             cudaStream_t st);
+cudaError_t launch_gemv_splitk(const void* x, const void* qweight, const void* scales, const void* zeros,
+                               void* y, int M, int N, int K, int group, void* workspace,
+                               unsigned int* status_word, int sms, cudaStream_t st);
 
 // the matrix-vector kernel's built-in scratch (no allocation): address on the current device
 cudaError_t gemv_static_scratch(void** out);

@@ -5,14 +5,16 @@
 // D[n][m] = sum_k dequant(Wq)[n][k] * x[m][k] and the epilogue writes y[m][n] = D[n][m].
 //
 // One persistent thread block per SM, warp-specialised:
-//   warp 0      producer: per 64-wide k-block one TMA tensor copy of the x tile
-//               (BN x 64 fp16, 128-byte swizzle) and three bulk copies (4 KB packed weight
-//               tile, 256 B of fp16 scales, 64 B of zero points) into a ring of stages,
+//   warp 0      producer: per 64-wide k-block two TMA tensor copies into a ring of stages -
+//               the x tile (BN x 64 fp16, 128-byte swizzle) and the packed weights of the
+//               slab's 8 bands (8 x 512 bytes, one box of the band-major weight array) -
 //               completion counted on an mbarrier.
-//   warps 8-15  dequantizers: each lane takes its 16-byte packed piece (rows g, g+8 of its
-//               band, 16 columns), converts two codes at a time to exact fp16 (q - z),
-//               multiplies by Delta (one fp16 rounding) and stores four 16-byte pieces into
-//               the stage's A tile in the K-major 128-byte-swizzled layout the MMA reads.
+//   warps 8-15  dequantizers, one per band: each lane takes its 16-byte packed piece (rows
+//               g, g+8 of the band, 16 columns), converts two codes at a time to exact fp16
+//               (q - z), multiplies by Delta (one fp16 rounding) and stores four 16-byte
+//               pieces into the stage's A tile in the K-major 128-byte-swizzled layout the
+//               MMA reads.  Scales and zero points (32 + 8 bytes per band and group) are read
+//               straight from global memory two groups ahead.
 //   warp 1      one thread issues tcgen05.mma (kind::f16, M = 128, N = BN, K = 16, four per
 //               k-block), commits to the stage's "empty" barrier and, after the last
 //               k-block, to the accumulator's "full" barrier.
@@ -36,16 +38,15 @@ namespace {
 constexpr int kGemmThreads = 512;
 constexpr int kBK = 64;
 constexpr int kATileBytes = 128 * kBK * 2;            // dequantized fp16 weight tile
-constexpr int kMetaBytes = 1024;                      // 256 B scales + 64 B zeros, padded to keep stages 1024-aligned
 
 template <int BN> struct GemmCfg {
     static constexpr int kXTileBytes = BN * kBK * 2;
-    static constexpr int kStageBytes = kXTileBytes + kATileBytes + kTileBytes + kMetaBytes;
+    static constexpr int kStageBytes = kXTileBytes + kATileBytes + kTileBytes;
     static constexpr int kStagesRaw = (216 * 1024) / kStageBytes;
     static constexpr int kStages = kStagesRaw > 8 ? 8 : kStagesRaw;
     static constexpr int kTmemCols = 2 * BN < 32 ? 32 : 2 * BN;   // two accumulator buffers
     static constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*align*/ + 256 /*barriers*/;
-    static constexpr uint32_t kTxBytes = kXTileBytes + kTileBytes + 256 + 64;
+    static constexpr uint32_t kTxBytes = kXTileBytes + kTileBytes;
 };
 
 // ------------------------------------------------------------------ small PTX wrappers
@@ -115,7 +116,7 @@ __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.
 // ------------------------------------------------------------------------- the kernel
 template <int G, int BN>
 __global__ void __launch_bounds__(kGemmThreads, 1)
-gemm_kernel(const __grid_constant__ CUtensorMap x_map, const unsigned char* __restrict__ qweight,
+gemm_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ CUtensorMap w_map,
             const __half* __restrict__ scales, const unsigned char* __restrict__ zeros,
             __half* __restrict__ y, int M, int N, int K, unsigned int* status_word) {
     using Cfg = GemmCfg<BN>;
@@ -127,7 +128,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const unsigned char* __re
     const uint32_t dyn = smem_u32(smem_dyn);
     const uint32_t base = (dyn + 1023u) & ~1023u;                    // 1024-byte aligned stage ring
     unsigned char* base_ptr = smem_dyn + (base - dyn);
-    // stage layout: [X tile | A tile | packed tile | scales(256) zeros(64) pad]
+    // stage layout: [X tile | A tile | packed tile]
     auto x_addr = [&](int s) { return base + (uint32_t)s * Cfg::kStageBytes; };
     auto a_addr = [&](int s) { return x_addr(s) + Cfg::kXTileBytes; };
     auto stage_ptr = [&](int s) { return base_ptr + (size_t)s * Cfg::kStageBytes; };
@@ -168,18 +169,13 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const unsigned char* __re
             bool ok = true;
             for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
                 const int slab = tile / m_tiles, mt = tile % m_tiles;
-                const unsigned char* wsrc = qweight + (size_t)slab * nkb * kTileBytes;
                 for (int kb = 0; kb < nkb; ++kb) {
                     if (!mbar_wait(empty(stage), phase ^ 1u, ctl)) { ok = false; break; }
-                    const int gi = kb * kBK / G;
                     const uint32_t bar = raw_full(stage);
                     mbar_arrive_expect_tx(bar, Cfg::kTxBytes);
                     tma_load_2d(x_addr(stage), &x_map, kb * kBK, mt * BN, bar);
-                    const uint32_t raw = a_addr(stage) + kATileBytes;
-                    bulk_load(raw, wsrc + (size_t)kb * kTileBytes, kTileBytes, bar);
-                    const size_t sg = (size_t)slab * (K / G) + gi;
-                    bulk_load(raw + kTileBytes, scales + sg * 128, 256, bar);
-                    bulk_load(raw + kTileBytes + 256, zeros + sg * 64, 64, bar);
+                    // weights: box of 8 bands x 512 bytes (128 words) at (k-block, first band)
+                    tma_load_2d(a_addr(stage) + kATileBytes, &w_map, kb * 128, slab * 8, bar);
                     ++issued;
                     if (++stage == S) { stage = 0; phase ^= 1u; }
                 }
@@ -235,18 +231,34 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const unsigned char* __re
         const uint32_t row_up = (uint32_t)(2 * band) * 1024u + (uint32_t)g * 128u;
         const uint32_t row_lo = row_up + 1024u;
         const uint32_t c0 = (uint32_t)((2 * t) ^ g) * 16u, c1 = (uint32_t)((2 * t + 1) ^ g) * 16u;
+        constexpr int KPG = G / kBK;                    // k-blocks per group
+        const int ng = K / G;
         for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+            const int slab = tile / m_tiles;
+            // this lane's rows' parameters: scales [band][group][16], zero bytes [band pair][group][16]
+            const unsigned short* sc_g = reinterpret_cast<const unsigned short*>(scales) +
+                                         (size_t)(slab * 8 + band) * ng * 16 + g;
+            const unsigned char* z_g = zeros + (size_t)(slab * 4 + (band >> 1)) * ng * 16 + (band & 1) * 8 + g;
+            // parameters of the current group and of the next two (fetched ahead of use)
+            uint32_t du = 0, dl = 0, zb = 0, du1, dl1, zb1, du2, dl2, zb2;
+            {
+                const int g1 = min(1, ng - 1);
+                du1 = __ldg(sc_g); dl1 = __ldg(sc_g + 8); zb1 = __ldg(z_g);
+                du2 = __ldg(sc_g + g1 * 16); dl2 = __ldg(sc_g + g1 * 16 + 8); zb2 = __ldg(z_g + g1 * 16);
+            }
             for (int kb = 0; kb < nkb; ++kb) {
+                if (kb % KPG == 0) {
+                    du = du1; dl = dl1; zb = zb1;
+                    du1 = du2; dl1 = dl2; zb1 = zb2;
+                    const int g2 = min(kb / KPG + 2, ng - 1);
+                    du2 = __ldg(sc_g + g2 * 16); dl2 = __ldg(sc_g + g2 * 16 + 8); zb2 = __ldg(z_g + g2 * 16);
+                }
                 ok = mbar_wait(raw_full(stage), phase, ctl);
                 ok = __all_sync(0xFFFFFFFFu, ok);
                 if (!ok) break;
                 const unsigned char* sp = stage_ptr(stage) + Cfg::kXTileBytes;
                 const unsigned char* raw = sp + kATileBytes;
                 const uint4 pk = *reinterpret_cast<const uint4*>(raw + band * 512 + lane * 16);
-                const __half* sc = reinterpret_cast<const __half*>(raw + kTileBytes);
-                const uint32_t du = __half_as_ushort(sc[band * 16 + g]);
-                const uint32_t dl = __half_as_ushort(sc[band * 16 + g + 8]);
-                const uint32_t zb = raw[kTileBytes + 256 + band * 8 + g];
                 const uint32_t d_up = du | (du << 16), d_lo = dl | (dl << 16);
                 const uint32_t zu = 0x6400u + (zb & 0xFu), zl = 0xD400u + ((zb >> 4) << 4);
                 const uint32_t zlo = zu | (zu << 16), zhi = zl | (zl << 16);
@@ -335,7 +347,7 @@ EncodeTiledFn encode_fn() {
 }
 
 template <int G, int BN>
-cudaError_t launch_one(const CUtensorMap& map, const void* qweight, const void* scales, const void* zeros,
+cudaError_t launch_one(const CUtensorMap& map, const CUtensorMap& wmap, const void* scales, const void* zeros,
                        void* y, int M, int N, int K, unsigned int* status_word, int sms, cudaStream_t st) {
     using Cfg = GemmCfg<BN>;
     static bool attr_done[64] = {};
@@ -350,7 +362,7 @@ cudaError_t launch_one(const CUtensorMap& map, const void* qweight, const void* 
     const int tiles = (N / 128) * ((M + BN - 1) / BN);
     const int grid = tiles < sms ? tiles : sms;
     gemm_kernel<G, BN><<<grid, kGemmThreads, Cfg::kSmemBytes, st>>>(
-        map, reinterpret_cast<const unsigned char*>(qweight), reinterpret_cast<const __half*>(scales),
+        map, wmap, reinterpret_cast<const __half*>(scales),
         reinterpret_cast<const unsigned char*>(zeros), reinterpret_cast<__half*>(y), M, N, K, status_word);
     count_launch();
     return cudaGetLastError();
@@ -373,13 +385,22 @@ cudaError_t launch_gemm(const void* x, const void* qweight, const void* scales, 
                            estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
+    // packed weights as a 2-D array of 32-bit words: one row per 16-row band (K * 8 bytes)
+    CUtensorMap wmap;
+    const cuuint64_t wdims[2] = {(cuuint64_t)K * 2, (cuuint64_t)(N / 16)};
+    const cuuint64_t wstrides[1] = {(cuuint64_t)K * 8};
+    const cuuint32_t wbox[2] = {128, 8};
+    const CUresult rw = enc(&wmap, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<void*>(qweight), wdims,
+                            wstrides, wbox, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+                            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (rw != CUDA_SUCCESS) return cudaErrorInvalidValue;
     int dev = 0, sms = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
     e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     if (e != cudaSuccess) return e;
 #define AWQ_GEMM_CASE(GG, BNN) \
-    return launch_one<GG, BNN>(map, qweight, scales, zeros, y, M, N, K, status_word, sms, st)
+    return launch_one<GG, BNN>(map, wmap, scales, zeros, y, M, N, K, status_word, sms, st)
     if (group == 128) {
         switch (bn) { case 256: AWQ_GEMM_CASE(128, 256); case 128: AWQ_GEMM_CASE(128, 128);
                       case 64: AWQ_GEMM_CASE(128, 64); default: AWQ_GEMM_CASE(128, 32); }

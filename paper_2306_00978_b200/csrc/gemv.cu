@@ -1,33 +1,40 @@
 // Decode path of the layer (Sec. 4.2: fused dequantize + matrix-vector product), M <= 16.
 //
-// HBM-bound: the packed weights (0.5 byte per weight) are streamed exactly once.  One
-// persistent thread block per SM takes a contiguous range of the (128-row slab, 512-column)
-// work units.  A copy warp keeps a ring of shared-memory stages full with bulk asynchronous
-// copies - 32 KB of packed weight tiles, the units' fp16 scales and zero points, and the
-// matching slice of x - so that well over 100 KB per SM is always in flight, independent of
-// registers and of what the math warps are doing.
+// HBM-bound: the packed weights (0.5 byte per weight) are streamed exactly once by persistent
+// thread blocks, one per SM.  A copy warp keeps a ring of shared-memory stages full with bulk
+// asynchronous copies (packed weights, fp16 scales, zero points and the matching slice of x,
+// completion counted in bytes on an mbarrier), so that well over 100 KB per SM is always in
+// flight, independent of registers and of what the math warps are doing.
 //
-// Sixteen math warps each own one 16-row band of four 64-column tiles per stage.  The 16
-// bytes a lane reads from the stage are already the A fragments of four warp-level m16n8k16
-// tensor-core products: thanks to the w{0,2,4,6,1,3,5,7} nibble order, masking a packed word
-// with 0x000F000F / 0x00F000F0 (before and after one shift by 8) leaves two codes in the
-// mantissa bits of an fp16x2 register, i.e. the exact values q * 2^-24 (upper row) and
-// q * 2^-20 (lower row) as fp16 subnormals.  Five logic operations and one MMA per eight
-// weights - the paper counts a shift, an AND and an FMA per single weight.  x (up to 8 tokens
-// per product) is the B operand, accumulation is fp32.  The zero point is applied once per
-// group in fp32:  sum (q - z) x = 2^24 * D - z * X,  X = sum of x over the group (the same
-// for every output row: each block sums it once, in fp32, while its first weight stages are
-// in flight); Delta is applied in the same step.  Nothing is rounded to fp16 before the output.
+// Math (both kernels).  Sixteen math warps.  The 16 bytes a lane reads from a stage are already
+// the A fragments of four warp-level m16n8k16 tensor-core products: thanks to the
+// w{0,2,4,6,1,3,5,7} nibble order, masking a packed word with 0x000F000F / 0x00F000F0 (before
+// and after one shift by 8) leaves two codes in the mantissa bits of an fp16x2 register, i.e.
+// the exact values q * 2^-24 (upper row) and q * 2^-20 (lower row) as fp16 subnormals.  Five
+// logic operations and one MMA per eight weights - the paper counts a shift, an AND and an FMA
+// per single weight.  x (up to 8 tokens per product) is the B operand, accumulation is fp32.
+// Zero point and scale are applied once per 64 columns in fp32:
+//   sum (q - z) x = 2^24 * D - z * X,   X = sum of x over those columns,
+// where X is the same for every output row, so each block sums it once, in fp32, while its
+// first weight stages are in flight.  Nothing is rounded to fp16 before the output.
 //
-// A block's range may begin or end inside a slab.  At the end of each slab segment the math
-// warps hand their fp32 sums to two flush warps through shared memory and go on streaming;
-// the flush warps write y, or publish a partial sum in an fp32 workspace slot owned by the
-// block, and the last block to arrive for that slab (an atomic counter; nobody waits) adds
-// the slots in block order: deterministic, no float atomics.
+// Two work decompositions:
+//   gemv_band_kernel    M <= 4, N/16 not much smaller than the SM count.  A task is one 16-row
+//                       band over all of K (contiguous in the band-major weight layout); the 16
+//                       math warps split the columns of each stage and their sums meet in
+//                       shared memory - no traffic between blocks, no workspace.
+//   gemv_splitk_kernel  everything else (M <= 16, small N).  Work units are (128-row slab,
+//                       512 columns); each block takes a contiguous range of units, so a slab
+//                       can be shared by several blocks: such partial sums go to an fp32
+//                       workspace slot owned by the block, and the last block to arrive for the
+//                       slab (an atomic counter; nobody waits) adds the slots in block order:
+//                       deterministic, no float atomics.
+// In both, finished sums are handed through shared memory to separate flush warps, so the math
+// warps go straight on to the next stage.
 //
-// All mbarrier waits are bounded; a wait that runs out records a time-out in the status
-// word, after which every wait of the block returns at once and the block runs to its end
-// (its output is then undefined, the status word says so).
+// All mbarrier waits are bounded; a wait that runs out records a time-out in the status word,
+// after which every wait of the block returns at once and the block runs to its end (its
+// output is then undefined, the status word says so).
 #include <mutex>
 
 #include "async_copy.cuh"
@@ -39,30 +46,326 @@ namespace {
 
 constexpr int kMathWarps = 16;
 constexpr int kMathThreads = kMathWarps * 32;
+constexpr int kZeroRowBytes = 1024;                    // a row of zeros read by lanes without a token
+constexpr int kSmemBudget = 216 * 1024;
+
+__device__ __forceinline__ void mma_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2,
+                                          uint32_t a3, uint32_t b0, uint32_t b1) {
+    asm("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+// the same product starting a new accumulation (C = 0)
+__device__ __forceinline__ void mma_16816_first(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2,
+                                                uint32_t a3, uint32_t b0, uint32_t b1) {
+    asm("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
+        : "=f"(c[0]), "=f"(c[1]), "=f"(c[2]), "=f"(c[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "f"(0.0f));
+}
+
+// One 16-row x 64-column packed block (this lane's 16 bytes `pk`) times the matching 64
+// activations of MT*8 tokens (this lane's 32 bytes per token tile, `xa` / `xb`):
+// c[mt][chain] receive D = sum q * 2^-24 x (rows g) and sum q * 2^-20 x (rows g+8).
+template <int MT, int NCH, bool FIRST = true>
+__device__ __forceinline__ void block_mma(const uint4& pk, const uint4 (&xa)[MT], const uint4 (&xb)[MT],
+                                          float (&c)[MT][NCH][4]) {
+    const uint32_t wds[4] = {pk.x, pk.y, pk.z, pk.w};
+#pragma unroll
+    for (int jw = 0; jw < 4; ++jw) {
+        const uint32_t w = wds[jw], w8 = w >> 8;
+        const uint32_t a0 = w & 0x000F000Fu, a1 = w & 0x00F000F0u;
+        const uint32_t a2 = w8 & 0x000F000Fu, a3 = w8 & 0x00F000F0u;
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt) {
+            const uint32_t b0 = (jw == 0) ? xa[mt].x : (jw == 1) ? xa[mt].z : (jw == 2) ? xb[mt].x : xb[mt].z;
+            const uint32_t b1 = (jw == 0) ? xa[mt].y : (jw == 1) ? xa[mt].w : (jw == 2) ? xb[mt].y : xb[mt].w;
+            if (FIRST && jw < NCH) mma_16816_first(c[mt][jw % NCH], a0, a1, a2, a3, b0, b1);
+            else mma_16816(c[mt][jw % NCH], a0, a1, a2, a3, b0, b1);
+        }
+    }
+}
+
+// X[k-tile][token] = sum of x over the 64 columns of the k-tile, in fp32.  A warp takes 256
+// consecutive activations of one token per item (8 halfs per lane, 8 lanes per k-tile) and
+// keeps four items' loads in flight.  Called by `nwarps` warps (index w) of the block.
+__device__ __forceinline__ void tile_sums_of_x(const __half* __restrict__ x, float* xsum, int M, int K,
+                                               int mtok, int w, int nwarps, int lane) {
+    const int cpr = K / 256;                       // whole 256-column chunks per token row
+    const int items = M * cpr;
+    for (int i0 = w; i0 < items; i0 += 4 * nwarps) {
+        uint4 h[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const int it = i0 + q * nwarps;
+            h[q] = make_uint4(0u, 0u, 0u, 0u);
+            if (it < items) {
+                const int m = it / cpr, c = it - m * cpr;
+                h[q] = __ldg(reinterpret_cast<const uint4*>(x + (size_t)m * K + (size_t)c * 256) + lane);
+            }
+        }
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const int it = i0 + q * nwarps;
+            const uint32_t u[4] = {h[q].x, h[q].y, h[q].z, h[q].w};
+            float v = 0.0f;
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&u[e]));
+                v += f.x + f.y;
+            }
+#pragma unroll
+            for (int off = 4; off >= 1; off >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, off);
+            if ((lane & 7) == 0 && it < items) {
+                const int m = it / cpr, c = it - m * cpr;
+                xsum[(c * 4 + (lane >> 3)) * mtok + m] = v;
+            }
+        }
+    }
+    // K is a multiple of 128: a last half chunk of 128 columns (2 k-tiles) may remain
+    if ((K & 255) != 0) {
+        for (int m = w; m < M; m += nwarps) {
+            const uint2 h2 = __ldg(reinterpret_cast<const uint2*>(x + (size_t)m * K + (size_t)cpr * 256) + lane);
+            const float2 f0 = __half22float2(*reinterpret_cast<const __half2*>(&h2.x));
+            const float2 f1 = __half22float2(*reinterpret_cast<const __half2*>(&h2.y));
+            float v = (f0.x + f0.y) + (f1.x + f1.y);
+#pragma unroll
+            for (int off = 8; off >= 1; off >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, off);
+            if ((lane & 15) == 0) xsum[(cpr * 4 + (lane >> 4)) * mtok + m] = v;
+        }
+    }
+}
+
+// =========================================================================== band kernel
+constexpr int kBandThreads = kMathThreads + 64;        // + copy warp + flush warp
+
+// Stage layout of the band kernel, fixed at compile time by TPW (k-tiles per math warp and
+// stage) and the group size, so that every shared-memory read is base + immediate.
+template <int G, int TPW> struct BandStage {
+    static constexpr int kUT = 16 * TPW;                // k-tiles per stage
+    static constexpr int kGroups = kUT * 64 / G;
+    static constexpr int kScOff = kUT * 512;            // [group][16] fp16
+    static constexpr int kZOff = kScOff + kGroups * 32; // [group][16] bytes (a pair of bands)
+    static constexpr int kXOff = kZOff + kGroups * 16;  // [token][kXRow]
+    static constexpr int kXRow = kUT * 128 + 16;        // padded against bank conflicts
+};
+
+struct BandLayout {
+    int stage_bytes, stages, xsum_off, red_off, bar_off, total;
+};
+template <int G, int TPW>
+inline BandLayout band_layout(int M, int K) {
+    using St = BandStage<G, TPW>;
+    BandLayout l;
+    l.stage_bytes = ((St::kXOff + M * St::kXRow + 127) / 128) * 128;
+    const int xsum = (K / 64 + St::kUT) * 8 * 4;        // + one stage of slack for ragged reads
+    const int red = 2 * kMathWarps * 8 * 16 * 4;        // two buffers of [warp][token][row] fp32
+    int s = (kSmemBudget - xsum - red - 256) / l.stage_bytes;
+    l.stages = s > 6 ? 6 : s;
+    l.xsum_off = l.stages * l.stage_bytes;
+    l.red_off = l.xsum_off + xsum;
+    l.bar_off = l.red_off + red;
+    l.total = l.bar_off + 256;
+    return l;
+}
+
+// TPW = k-tiles per math warp and stage (stage = 16 * TPW k-tiles).  M <= 8 tokens (one token tile).
+template <int G, int TPW>
+__global__ void __launch_bounds__(kBandThreads, 1)
+gemv_band_kernel(const unsigned char* __restrict__ qweight, const __half* __restrict__ scales,
+                 const unsigned char* __restrict__ zeros, const __half* __restrict__ x,
+                 __half* __restrict__ y, int M, int N, int K, const BandLayout lay,
+                 unsigned int* status_word) {
+    extern __shared__ __align__(128) unsigned char smem[];
+    __shared__ unsigned int s_abort;
+    using St = BandStage<G, TPW>;
+    constexpr int UT = St::kUT;
+    constexpr int TPG = G / 64;                         // k-tiles per group
+    constexpr int GPW = (TPW + TPG - 1) / TPG;          // groups touched by one warp in a stage
+    static_assert(TPW % TPG == 0, "a warp's tiles must cover whole groups");
+    const int S = lay.stages;
+    const uint32_t sbase = smem_u32(smem);
+    // barriers: full[s] at 8s, empty[s] at 64 + 8s, flush_req[b] at 128 + 8b, red_free[b] at 144 + 8b
+    const uint32_t bars = sbase + (uint32_t)lay.bar_off;
+
+    const int ktiles = K / 64, ng = K / G;
+    const int upb = (ktiles + UT - 1) / UT;                           // units per band
+    const int nbands = N / 16;
+    const int b0 = (int)(((unsigned)nbands * blockIdx.x) / gridDim.x);
+    const int b1 = (int)(((unsigned)nbands * (blockIdx.x + 1)) / gridDim.x);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (threadIdx.x < (unsigned)S) {
+        mbar_init(bars + 8u * threadIdx.x, 1);
+        mbar_init(bars + 64u + 8u * threadIdx.x, kMathWarps);
+        mbar_fence_init();
+    } else if (threadIdx.x >= 32 && threadIdx.x < 34) {
+        mbar_init(bars + 128u + 8u * (threadIdx.x - 32), kMathWarps);
+        mbar_init(bars + 144u + 8u * (threadIdx.x - 32), 1);
+        mbar_fence_init();
+        if (threadIdx.x == 32) s_abort = 0u;
+    }
+    __syncthreads();
+    const WaitCtl ctl{status_word, &s_abort};
+
+    if (warp == kMathWarps) {
+        // ------------------------------------------------------------------ copy warp
+        // lane 0 posts the byte count; lanes 0, 1, 2 and 3 .. 3+M-1 each issue one bulk copy
+        uint32_t stage = 0, phase = 0;
+        for (int band = b0; band < b1; ++band) {
+            for (int j = 0; j < upb; ++j) {
+                const int kt = j * UT;
+                const int nt = min(UT, ktiles - kt);
+                const int ngr = nt * 64 / G;
+                const uint32_t dst = sbase + stage * (uint32_t)lay.stage_bytes;
+                const uint32_t bar = bars + 8u * stage;
+                if (lane == 0) {
+                    mbar_wait_relaxed(bars + 64u + 8u * stage, phase ^ 1u, ctl);
+                    mbar_arrive_expect_tx(bar, (uint32_t)(nt * 512 + ngr * 48 + M * nt * 128));
+                }
+                __syncwarp();
+                const int gi0 = kt * 64 / G;
+                if (lane == 0)
+                    bulk_load(dst, qweight + ((size_t)band * ktiles + kt) * 512, (uint32_t)(nt * 512), bar);
+                else if (lane == 1)
+                    bulk_load(dst + St::kScOff, scales + ((size_t)band * ng + gi0) * 16, (uint32_t)(ngr * 32), bar);
+                else if (lane == 2)
+                    bulk_load(dst + St::kZOff, zeros + ((size_t)(band >> 1) * ng + gi0) * 16, (uint32_t)(ngr * 16), bar);
+                else if (lane - 3 < M)
+                    bulk_load(dst + St::kXOff + (lane - 3) * St::kXRow, x + (size_t)(lane - 3) * K + (size_t)kt * 64,
+                              (uint32_t)(nt * 128), bar);
+                if (++stage == (uint32_t)S) { stage = 0; phase ^= 1u; }
+            }
+        }
+        if (lane != 0) return;
+        // every copy issued above must have landed before the block may exit
+        const int issued = (b1 - b0) * upb;
+        const int pending = issued < S ? issued : S;
+        for (int i = 0; i < pending; ++i) {
+            if (stage == 0) { stage = S - 1; phase ^= 1u; } else { --stage; }
+            const unsigned long long t0 = global_ns();
+            while (!mbar_try_wait(bars + 8u * stage, phase) && global_ns() - t0 < 200000000ull) {}
+        }
+        return;
+    }
+
+    // x sums per k-tile (math warps and the flush warp), while the first stages are in flight
+    float* xsum = reinterpret_cast<float*>(smem + lay.xsum_off);
+    tile_sums_of_x(x, xsum, M, K, 8, warp < kMathWarps ? warp : warp - 1, kMathWarps + 1, lane);
+    named_barrier_sync(3, kBandThreads - 32);
+
+    float* red = reinterpret_cast<float*>(smem + lay.red_off);
+    if (warp == kMathWarps + 1) {
+        // ------------------------------------------------------------------ flush warp
+        int nflush = 0;
+        for (int band = b0; band < b1; ++band, ++nflush) {
+            const uint32_t b = (uint32_t)nflush & 1u, use = ((uint32_t)nflush >> 1) & 1u;
+            mbar_wait_relaxed(bars + 128u + 8u * b, use, ctl);
+            const float* rb = red + b * (kMathWarps * 8 * 16);
+            for (int idx = lane; idx < M * 16; idx += 32) {          // idx = token * 16 + row
+                float sum = 0.0f;
+#pragma unroll
+                for (int w = 0; w < kMathWarps; ++w) sum += rb[w * 128 + idx];
+                y[(size_t)(idx >> 4) * N + band * 16 + (idx & 15)] = __float2half_rn(sum);
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bars + 144u + 8u * b);
+        }
+        return;
+    }
+
+    // -------------------------------------------------------------------- math warps
+    // warp w owns k-tiles w*TPW .. w*TPW+TPW-1 of every stage, i.e. GPW whole groups
+    const int g = lane >> 2, t = lane & 3;
+    const bool tok_ok = g < M;
+    // this lane's fixed byte offsets inside a stage
+    const int o_w = warp * (TPW * 512) + lane * 16;
+    const int o_sc = St::kScOff + warp * (GPW * 32) + g * 2;
+    const int o_x = St::kXOff + g * St::kXRow + warp * (TPW * 128) + t * 32;
+    const float* xs_lane = xsum + warp * (TPW * 8) + 2 * t;
+
+    uint32_t stage = 0, phase = 0;
+    int nflush = 0;
+    for (int band = b0; band < b1; ++band, ++nflush) {
+        float acc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+        const int o_z = St::kZOff + warp * (GPW * 16) + (band & 1) * 8 + g;
+        for (int j = 0; j < upb; ++j) {
+            const int nt = min(UT, ktiles - j * UT) - warp * TPW;     // this warp's tiles: <= 0 .. TPW
+            mbar_wait(bars + 8u * stage, phase, ctl);
+            const unsigned char* st = smem + stage * (uint32_t)lay.stage_bytes;
+            if (nt > 0) {
+                const float* xs = xs_lane + j * (UT * 8);
+#pragma unroll
+                for (int q = 0; q < GPW; ++q) {
+                    if (q * TPG < nt) {                               // whole groups only (K % G == 0)
+                        float c[1][2][4];
+                        float Xx = 0.0f, Xy = 0.0f;
+#pragma unroll
+                        for (int v = 0; v < TPG; ++v) {
+                            const int tile = q * TPG + v;
+                            const uint4 pk = *reinterpret_cast<const uint4*>(st + o_w + tile * 512);
+                            // lanes without a token must not touch shared memory: even a
+                            // broadcast read costs wavefronts on the shared-memory pipe
+                            uint4 xa[1] = {make_uint4(0u, 0u, 0u, 0u)}, xb[1] = {make_uint4(0u, 0u, 0u, 0u)};
+                            if (tok_ok) {
+                                xa[0] = *reinterpret_cast<const uint4*>(st + o_x + tile * 128);
+                                xb[0] = *reinterpret_cast<const uint4*>(st + o_x + tile * 128 + 16);
+                            }
+                            const float2 X = *reinterpret_cast<const float2*>(xs + tile * 8);
+                            Xx += X.x;
+                            Xy += X.y;
+                            if (v == 0) block_mma<1, 2, true>(pk, xa, xb, c);
+                            else block_mma<1, 2, false>(pk, xa, xb, c);
+                        }
+                        const float d_up = __half2float(*reinterpret_cast<const __half*>(st + o_sc + q * 32));
+                        const float d_lo = __half2float(*reinterpret_cast<const __half*>(st + o_sc + q * 32 + 16));
+                        const uint32_t zb = st[o_z + q * 16];
+                        const float su = d_up * 16777216.0f, sl = d_lo * 1048576.0f;
+                        const float zu = d_up * (float)(zb & 0xFu), zl = d_lo * (float)(zb >> 4);
+                        acc[0] = fmaf(su, c[0][0][0] + c[0][1][0], fmaf(-zu, Xx, acc[0]));
+                        acc[1] = fmaf(su, c[0][0][1] + c[0][1][1], fmaf(-zu, Xy, acc[1]));
+                        acc[2] = fmaf(sl, c[0][0][2] + c[0][1][2], fmaf(-zl, Xx, acc[2]));
+                        acc[3] = fmaf(sl, c[0][0][3] + c[0][1][3], fmaf(-zl, Xy, acc[3]));
+                    }
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bars + 64u + 8u * stage);
+            if (++stage == (uint32_t)S) { stage = 0; phase ^= 1u; }
+        }
+        // hand this band's sums to the flush warp: red[buffer][warp][token][row]
+        const uint32_t b = (uint32_t)nflush & 1u, use = ((uint32_t)nflush >> 1) & 1u;
+        mbar_wait(bars + 144u + 8u * b, use ^ 1u, ctl);
+        float* rb = red + b * (kMathWarps * 8 * 16) + warp * 128;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) rb[(2 * t + (i & 1)) * 16 + g + (i >> 1) * 8] = acc[i];
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bars + 128u + 8u * b);
+    }
+}
+
+// ======================================================================== split-K kernel
 constexpr int kFlushThreads = 64;
-constexpr int kGemvThreads = kMathThreads + 32 + kFlushThreads;   // + copy warp, two flush warps
+constexpr int kSplitkThreads = kMathThreads + 32 + kFlushThreads;   // + copy warp, two flush warps
 constexpr int kUT = 8;                                 // k-tiles per work unit (512 input channels)
 constexpr int kWT = kUT / 2;                           // k-tiles per math warp and stage
-constexpr int kWBytes = kUT * kTileBytes;              // 32 KB of packed weights per stage
-constexpr int kScaleBytes = kUT * 256;                 // up to kUT groups x 128 rows x fp16
-constexpr int kZeroBytes = kUT * 64;                   // up to kUT groups x 64 bytes
+constexpr int kWBytes = kUT * kTileBytes;              // 32 KB of packed weights per stage: [band][k-tile][512]
+constexpr int kScaleBytes = 8 * kUT * 32;              // [band][group][16] fp16
+constexpr int kZeroBytes = 4 * kUT * 16;               // [band pair][group][16]
 constexpr int kXRowBytes = kUT * 128 + 16;             // one token's slice, padded against bank conflicts
 constexpr int kXOff = kWBytes + kScaleBytes + kZeroBytes;
-constexpr int kZeroRowBytes = 1024;                    // a row of zeros read by lanes without a token
-constexpr int kSmemBudget = 200 * 1024;
 
 // Shared-memory layout, computed once on the host and passed to the kernel.
-struct GemvLayout {
+struct SplitkLayout {
     int stage_bytes, stages, zero_off, xsum_off, red_off, bar_off, total;
 };
-inline GemvLayout gemv_layout(int M, int K, int group) {
-    GemvLayout l;
+inline SplitkLayout splitk_layout(int M, int K) {
+    SplitkLayout l;
     const int mtok = M <= 8 ? 8 : 16;
     l.stage_bytes = kXOff + ((M * kXRowBytes + 127) / 128) * 128;
     const int red = 2 * (2 * mtok * 128 * 4);            // two buffers of [k-half][token][row] fp32
-    const int xsum = (K / group) * mtok * 4;             // [group][token] fp32 sums of x
+    const int xsum = (K / 64) * mtok * 4;                // [k-tile][token] fp32 sums of x
     int s = (kSmemBudget - red - xsum - kZeroRowBytes - 256) / l.stage_bytes;
-    l.stages = s > 8 ? 8 : s;
+    l.stages = s > 6 ? 6 : s;
     l.zero_off = l.stages * l.stage_bytes;
     l.xsum_off = l.zero_off + kZeroRowBytes;
     l.red_off = l.xsum_off + xsum;
@@ -71,22 +374,7 @@ inline GemvLayout gemv_layout(int M, int K, int group) {
     return l;
 }
 
-__device__ __forceinline__ void mma_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2,
-                                          uint32_t a3, uint32_t b0, uint32_t b1) {
-    asm(
-        "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
-}
-// the same product starting a new accumulation (C = 0)
-__device__ __forceinline__ void mma_16816_first(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2,
-                                                uint32_t a3, uint32_t b0, uint32_t b1) {
-    asm(
-        "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
-        : "=f"(c[0]), "=f"(c[1]), "=f"(c[2]), "=f"(c[3])
-        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "f"(0.0f));
-}
-// Work decomposition shared by the producer and the math warps.
+// Work decomposition shared by the copy, math and flush warps.
 struct Range {
     int ups;        // units per slab
     int U;          // units in total
@@ -98,114 +386,24 @@ struct Range {
     }
 };
 
-// One math warp's share of one stage: NT tiles (4, or 2 for a ragged last unit of a slab).
-// The accumulation chains are independent (one or two per tile), and the activations are
-// fetched 8 bytes at a time right before the product that uses them.
-template <int G, int MT, int NT>
-__device__ __forceinline__ void math_stage(const unsigned char* st, const unsigned char* const (&xp)[MT],
-                                           int w_off, int sc_off, int z_off, const float* xs,
-                                           float (&acc)[MT][4]) {
-    constexpr int TPG = G / 64, NG = NT / TPG, NCH = (MT == 1) ? 2 : 1;
-    // all shared-memory reads of the stage first, then one straight run of logic + MMA work
-    uint4 pk[NT];
-    uint4 xv[MT][NT][2];
-#pragma unroll
-    for (int tile = 0; tile < NT; ++tile)
-        pk[tile] = *reinterpret_cast<const uint4*>(st + w_off + tile * kTileBytes);
-#pragma unroll
-    for (int mt = 0; mt < MT; ++mt)
-#pragma unroll
-        for (int tile = 0; tile < NT; ++tile) {
-            xv[mt][tile][0] = *reinterpret_cast<const uint4*>(xp[mt] + tile * 128);
-            xv[mt][tile][1] = *reinterpret_cast<const uint4*>(xp[mt] + tile * 128 + 16);
-        }
-    // group parameters, folded with the power-of-two scales of the subnormal codes
-    float su[NG], sl[NG], zu[NG], zl[NG];
-#pragma unroll
-    for (int q = 0; q < NG; ++q) {
-        const float d_up = __half2float(*reinterpret_cast<const __half*>(st + sc_off + q * 256));
-        const float d_lo = __half2float(*reinterpret_cast<const __half*>(st + sc_off + q * 256 + 16));
-        const uint32_t zb = st[z_off + q * 64];
-        su[q] = d_up * 16777216.0f;
-        sl[q] = d_lo * 1048576.0f;
-        zu[q] = -d_up * (float)(zb & 0xFu);
-        zl[q] = -d_lo * (float)(zb >> 4);
-    }
-    float c[NT][MT][NCH][4];
-#pragma unroll
-    for (int jw = 0; jw < 4; ++jw) {
-#pragma unroll
-        for (int tile = 0; tile < NT; ++tile) {
-            // codes as fp16 subnormals: q * 2^-24 (upper row), q * 2^-20 (lower row)
-            const uint32_t w = (jw == 0) ? pk[tile].x : (jw == 1) ? pk[tile].y : (jw == 2) ? pk[tile].z : pk[tile].w;
-            const uint32_t w8 = w >> 8;
-            const uint32_t a0 = w & 0x000F000Fu, a1 = w & 0x00F000F0u;
-            const uint32_t a2 = w8 & 0x000F000Fu, a3 = w8 & 0x00F000F0u;
-#pragma unroll
-            for (int mt = 0; mt < MT; ++mt) {
-                const uint4 xq = xv[mt][tile][jw >> 1];
-                const uint32_t b0 = (jw & 1) ? xq.z : xq.x, b1 = (jw & 1) ? xq.w : xq.y;
-                if (jw < NCH) mma_16816_first(c[tile][mt][jw % NCH], a0, a1, a2, a3, b0, b1);
-                else mma_16816(c[tile][mt][jw % NCH], a0, a1, a2, a3, b0, b1);
-            }
-        }
-    }
-    // per group: sum (q - z) x = 2^24 * D - z * X (upper row; 2^20 for the lower row), times Delta
-#pragma unroll
-    for (int q = 0; q < NG; ++q) {
-#pragma unroll
-        for (int mt = 0; mt < MT; ++mt) {
-            const float2 X = *reinterpret_cast<const float2*>(xs + q * (MT * 8) + mt * 8);
-            float d[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-#pragma unroll
-            for (int v = 0; v < TPG; ++v)
-#pragma unroll
-                for (int ch = 0; ch < NCH; ++ch)
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) d[i] += c[q * TPG + v][mt][ch][i];
-            acc[mt][0] = fmaf(su[q], d[0], fmaf(zu[q], X.x, acc[mt][0]));
-            acc[mt][1] = fmaf(su[q], d[1], fmaf(zu[q], X.y, acc[mt][1]));
-            acc[mt][2] = fmaf(sl[q], d[2], fmaf(zl[q], X.x, acc[mt][2]));
-            acc[mt][3] = fmaf(sl[q], d[3], fmaf(zl[q], X.y, acc[mt][3]));
-        }
-    }
-}
-
-#ifdef AWQ_DBG_TS
-__device__ unsigned long long g_dbg_ts[256 * 16];
-#define DBG_TS(i) do { if (threadIdx.x == 0) g_dbg_ts[blockIdx.x * 16 + (i)] = global_ns(); } while (0)
-#define DBG_TS_ANY(i) do { g_dbg_ts[blockIdx.x * 16 + (i)] = global_ns(); } while (0)
-#define DBG_CLK(v) const long long v = clock64()
-#define DBG_ACC(i, a, b) do { dbg_acc[i] += (b) - (a); } while (0)
-#define DBG_ACC_DECL long long dbg_acc[4] = {0, 0, 0, 0}
-#define DBG_ACC_STORE(base) do { for (int _i = 0; _i < 4; ++_i) g_dbg_ts[blockIdx.x * 16 + (base) + _i] = (unsigned long long)dbg_acc[_i]; } while (0)
-#else
-#define DBG_CLK(v) do {} while (0)
-#define DBG_ACC(i, a, b) do {} while (0)
-#define DBG_ACC_DECL do {} while (0)
-#define DBG_ACC_STORE(base) do {} while (0)
-#define DBG_TS(i) do {} while (0)
-#define DBG_TS_ANY(i) do {} while (0)
-#endif
-
 // MT = number of 8-token column tiles (1: M <= 8, 2: M <= 16).
 template <int G, int MT>
-__global__ void __launch_bounds__(kGemvThreads, 1)
-gemv_kernel(const unsigned char* __restrict__ qweight, const __half* __restrict__ scales,
-            const unsigned char* __restrict__ zeros, const __half* __restrict__ x,
-            __half* __restrict__ y, float* __restrict__ partial, unsigned int* __restrict__ counters,
-            int M, int N, int K, const GemvLayout lay, unsigned int* status_word) {
+__global__ void __launch_bounds__(kSplitkThreads, 1)
+gemv_splitk_kernel(const unsigned char* __restrict__ qweight, const __half* __restrict__ scales,
+                   const unsigned char* __restrict__ zeros, const __half* __restrict__ x,
+                   __half* __restrict__ y, float* __restrict__ partial, unsigned int* __restrict__ counters,
+                   int M, int N, int K, const SplitkLayout lay, unsigned int* status_word) {
     extern __shared__ __align__(128) unsigned char smem[];
     __shared__ unsigned int s_abort;
     __shared__ unsigned int s_last;
 
-    DBG_TS(0);
     const int S = lay.stages;
     const uint32_t sbase = smem_u32(smem);
-    // barriers: full[s] at 8s (copies landed), empty[s] at 64 + 8s (math warps done)
+    // barriers: full[s] at 8s (copies landed), empty[s] at 64 + 8s (math warps done),
+    // flush_req[b] at 192 + 8b (math warps handed over buffer b), red_free[b] at 208 + 8b
     const uint32_t bars = sbase + (uint32_t)lay.bar_off;
 
-    const int ktiles = K / 64;
+    const int ktiles = K / 64, ng = K / G;
     Range rg;
     rg.ups = (ktiles + kUT - 1) / kUT;
     rg.U = (N / 128) * rg.ups;
@@ -221,8 +419,6 @@ gemv_kernel(const unsigned char* __restrict__ qweight, const __half* __restrict_
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int g = lane >> 2, t = lane & 3;
-    // barriers also at 192 + 8b: flush_req[b] (math warps handed over buffer b) and
-    // 208 + 8b: red_free[b] (flush warps are done with buffer b)
     if (threadIdx.x < (unsigned)S) {
         mbar_init(bars + 8u * threadIdx.x, 1);
         mbar_init(bars + 64u + 8u * threadIdx.x, kMathWarps);
@@ -235,92 +431,62 @@ gemv_kernel(const unsigned char* __restrict__ qweight, const __half* __restrict_
     }
     if (threadIdx.x < kZeroRowBytes / 4) reinterpret_cast<uint32_t*>(smem + lay.zero_off)[threadIdx.x] = 0u;
     __syncthreads();
-    DBG_TS(1);
     const WaitCtl ctl{status_word, &s_abort};
     const unsigned char* zero_row = smem + lay.zero_off;
+    constexpr int MTOK = MT * 8;
 
     if (warp == kMathWarps) {
         // ------------------------------------------------------------------ copy warp
-        // lane 0 posts the byte count, then lanes 0 .. 2+M-1 each issue one bulk copy
-        // (weights, scales, zero points, one x row per token)
-        {
-            DBG_ACC_DECL;
-            uint32_t stage = 0, phase = 0;
-            const int ng = K / G;
-            for (int p = 0; p < nu; ++p) {
-                const int u = (p < nl) ? ul + p : u0 + (p - nl);
-                const int slab = u / rg.ups, j = u - slab * rg.ups;
-                const int kt = j * kUT;
-                const int nt = min(kUT, ktiles - kt);
-                const int ngr = nt * 64 / G;
-                const uint32_t dst = sbase + stage * (uint32_t)lay.stage_bytes;
-                const uint32_t bar = bars + 8u * stage;
-                if (lane == 0) {
-                    DBG_CLK(tc0);
-                    mbar_wait(bars + 64u + 8u * stage, phase ^ 1u, ctl);
-                    DBG_CLK(tc1);
-                    DBG_ACC(0, tc0, tc1);
-                    mbar_arrive_expect_tx(bar, (uint32_t)(nt * kTileBytes + ngr * (256 + 64) + M * nt * 128));
-                }
-                __syncwarp();
-                const size_t sg = (size_t)slab * ng + (size_t)(kt * 64 / G);
-                if (lane == 0)
-                    bulk_load(dst, qweight + ((size_t)slab * ktiles + kt) * kTileBytes, (uint32_t)(nt * kTileBytes), bar);
-                else if (lane == 1)
-                    bulk_load(dst + kWBytes, scales + sg * 128, (uint32_t)(ngr * 256), bar);
-                else if (lane == 2)
-                    bulk_load(dst + kWBytes + kScaleBytes, zeros + sg * 64, (uint32_t)(ngr * 64), bar);
-                else if (lane - 3 < M)
-                    bulk_load(dst + kXOff + (lane - 3) * kXRowBytes, x + (size_t)(lane - 3) * K + (size_t)kt * 64,
+        // lane 0 posts the byte count; then lanes 0-7 copy the 8 bands' weights, 8-15 their
+        // scales, 16-19 the 4 band pairs' zero points, 20-31 the x rows
+        uint32_t stage = 0, phase = 0;
+        for (int p = 0; p < nu; ++p) {
+            const int u = (p < nl) ? ul + p : u0 + (p - nl);
+            const int slab = u / rg.ups, j = u - slab * rg.ups;
+            const int kt = j * kUT;
+            const int nt = min(kUT, ktiles - kt);
+            const int ngr = nt * 64 / G;
+            const uint32_t dst = sbase + stage * (uint32_t)lay.stage_bytes;
+            const uint32_t bar = bars + 8u * stage;
+            if (lane == 0) {
+                mbar_wait(bars + 64u + 8u * stage, phase ^ 1u, ctl);
+                mbar_arrive_expect_tx(bar, (uint32_t)(nt * kTileBytes + ngr * (256 + 64) + M * nt * 128));
+            }
+            __syncwarp();
+            const int gi0 = kt * 64 / G;
+            if (lane < 8) {
+                bulk_load(dst + lane * (kUT * 512), qweight + ((size_t)(slab * 8 + lane) * ktiles + kt) * 512,
+                          (uint32_t)(nt * 512), bar);
+            } else if (lane < 16) {
+                const int b = lane - 8;
+                bulk_load(dst + kWBytes + b * (kUT * 32), scales + ((size_t)(slab * 8 + b) * ng + gi0) * 16,
+                          (uint32_t)(ngr * 32), bar);
+            } else if (lane < 20) {
+                const int pr = lane - 16;
+                bulk_load(dst + kWBytes + kScaleBytes + pr * (kUT * 16),
+                          zeros + ((size_t)(slab * 4 + pr) * ng + gi0) * 16, (uint32_t)(ngr * 16), bar);
+            } else {
+                for (int m = lane - 20; m < M; m += 12)
+                    bulk_load(dst + kXOff + m * kXRowBytes, x + (size_t)m * K + (size_t)kt * 64,
                               (uint32_t)(nt * 128), bar);
-                if (++stage == (uint32_t)S) { stage = 0; phase ^= 1u; }
             }
-            if (lane != 0) return;
-            DBG_ACC_STORE(9);   // [9] = copy warp cycles waiting for an empty stage
-            // every copy issued above must have landed before the block may exit
-            const int issued = nu;
-            const int pending = issued < S ? issued : S;
-            for (int i = 0; i < pending; ++i) {
-                if (stage == 0) { stage = S - 1; phase ^= 1u; } else { --stage; }
-                const unsigned long long t0 = global_ns();
-                while (!mbar_try_wait(bars + 8u * stage, phase) && global_ns() - t0 < 200000000ull) {}
-            }
+            if (++stage == (uint32_t)S) { stage = 0; phase ^= 1u; }
+        }
+        if (lane != 0) return;
+        // every copy issued above must have landed before the block may exit
+        const int pending = nu < S ? nu : S;
+        for (int i = 0; i < pending; ++i) {
+            if (stage == 0) { stage = S - 1; phase ^= 1u; } else { --stage; }
+            const unsigned long long t0 = global_ns();
+            while (!mbar_try_wait(bars + 8u * stage, phase) && global_ns() - t0 < 200000000ull) {}
         }
         return;
     }
 
-    constexpr int MTOK = MT * 8;
-    constexpr int TPG = G / 64;                        // tiles per group
-
-    // ---------------------------------------------------------- x sums (all but the copy warp)
-    // X[group][token] = sum of x over the group's input channels, in fp32, one warp per sum.
-    {
-        float* xsum = reinterpret_cast<float*>(smem + lay.xsum_off);
-        const int w = warp < kMathWarps ? warp : warp - 1;          // 0 .. 17
-        constexpr int NW = kMathWarps + kFlushThreads / 32;
-        constexpr int LPS = G / 4;                                  // lanes per sum, 4 halfs each
-        constexpr int SPW = 32 / LPS;                               // sums per warp and pass
-        const int nsum = (K / G) * M;
-        const int sub = lane / LPS, l = lane % LPS;
-        for (int s0 = w * SPW; s0 < nsum; s0 += NW * SPW) {
-            const int sidx = s0 + sub;
-            float v = 0.0f;
-            if (sidx < nsum) {
-                const int gi = sidx / M, m = sidx - gi * M;
-                const uint2 h = __ldg(reinterpret_cast<const uint2*>(x + (size_t)m * K + (size_t)gi * G) + l);
-                const float2 f0 = __half22float2(*reinterpret_cast<const __half2*>(&h.x));
-                const float2 f1 = __half22float2(*reinterpret_cast<const __half2*>(&h.y));
-                v = (f0.x + f0.y) + (f1.x + f1.y);
-            }
-#pragma unroll
-            for (int off = LPS / 2; off >= 1; off >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, off);
-            if (l == 0 && sidx < nsum) {
-                const int gi = sidx / M, m = sidx - gi * M;
-                xsum[gi * MTOK + m] = v;
-            }
-        }
-        named_barrier_sync(3, kGemvThreads - 32);
-    }
+    // x sums per k-tile (all but the copy warp), while the first stages are in flight
+    float* xsum = reinterpret_cast<float*>(smem + lay.xsum_off);
+    tile_sums_of_x(x, xsum, M, K, MTOK, warp < kMathWarps ? warp : warp - 1, kMathWarps + 2, lane);
+    named_barrier_sync(3, kSplitkThreads - 32);
 
     if (warp >= kMathWarps + 1) {
         // --------------------------------------------------------------- flush warps
@@ -333,7 +499,6 @@ gemv_kernel(const unsigned char* __restrict__ qweight, const __half* __restrict_
             if (j == rg.ups - 1 || u == u1 - 1) {
                 const bool whole = (u - j >= u0) && (j == rg.ups - 1);
                 const uint32_t b = (uint32_t)nflush & 1u, use = ((uint32_t)nflush >> 1) & 1u;
-                if (ft == 0) DBG_TS_ANY(3 + 2 * min(nflush, 5));
                 mbar_wait(bars + 192u + 8u * b, use, ctl);
                 const float* rb = red + b * (2 * MTOK * 128);
                 const int slot = (slab == slab0) ? 0 : 1;
@@ -356,38 +521,44 @@ gemv_kernel(const unsigned char* __restrict__ qweight, const __half* __restrict_
                     named_barrier_sync(2, kFlushThreads);
                     if (s_last != 0u) {
                         __threadfence();
-                        for (int idx = ft; idx < M * 128; idx += kFlushThreads) {
-                            const int m = idx >> 7, r = idx & 127;
-                            float sum = 0.0f;
+                        for (int i0 = ft; i0 < M * 128; i0 += 4 * kFlushThreads) {
+                            float sum[4] = {0.0f, 0.0f, 0.0f, 0.0f};
                             for (int c = c_first; c <= c_last; ++c) {
                                 const int cslot = (rg.start(c) / rg.ups == slab) ? 0 : 1;
-                                sum += __ldcg(partial + (size_t)(c * 2 + cslot) * M * 128 + idx);
+                                const float* src = partial + (size_t)(c * 2 + cslot) * M * 128;
+#pragma unroll
+                                for (int q = 0; q < 4; ++q) {
+                                    const int idx = i0 + q * kFlushThreads;
+                                    if (idx < M * 128) sum[q] += __ldcg(src + idx);
+                                }
                             }
-                            y[(size_t)m * N + slab * 128 + r] = __float2half_rn(sum);
+#pragma unroll
+                            for (int q = 0; q < 4; ++q) {
+                                const int idx = i0 + q * kFlushThreads;
+                                if (idx < M * 128)
+                                    y[(size_t)(idx >> 7) * N + slab * 128 + (idx & 127)] = __float2half_rn(sum[q]);
+                            }
                         }
                         if (ft == 0) counters[slab] = 0u;           // ready for the next call
                     }
                     named_barrier_sync(2, kFlushThreads);           // s_last may be rewritten
                 }
-                if (ft == 0) DBG_TS_ANY(4 + 2 * min(nflush, 5));
                 ++nflush;
             }
         }
-        if (ft == 0) DBG_TS_ANY(15);
         return;
     }
 
     // -------------------------------------------------------------------- math warps
-    // warp = (half, band): tiles kWT*half .. +kWT-1 of each stage, rows 16*band .. +15
+    // warp = (half, band): k-tiles kWT*half .. +kWT-1 of each stage, rows 16*band .. +15
     const int half = warp >> 3, band = warp & 7;
-    constexpr int GPW = kWT * 64 / G;                  // groups per warp and stage
+    constexpr int TPG = G / 64;
     float* red = reinterpret_cast<float*>(smem + lay.red_off);
 
     // stage-relative byte offsets of this lane's pieces
-    const int w_off = (kWT * half) * kTileBytes + band * 512 + lane * 16;
-    const int sc_off = kWBytes + ((GPW * half) * 128 + band * 16 + g) * 2;
-    const int z_off = kWBytes + kScaleBytes + (GPW * half) * 64 + band * 8 + g;
-    const float* xsum = reinterpret_cast<const float*>(smem + lay.xsum_off);
+    const int w_off = band * (kUT * 512) + (kWT * half) * 512 + lane * 16;
+    const int sc_off = kWBytes + band * (kUT * 32) + g * 2;
+    const int z_off = kWBytes + kScaleBytes + (band >> 1) * (kUT * 16) + (band & 1) * 8 + g;
     int x_off[MT];
     bool tok_ok[MT];
 #pragma unroll
@@ -404,31 +575,59 @@ gemv_kernel(const unsigned char* __restrict__ qweight, const __half* __restrict_
 
     uint32_t stage = 0, phase = 0;
     int nflush = 0;
-    DBG_ACC_DECL;
     for (int p = 0; p < nu; ++p) {
         const int u = (p < nl) ? ul + p : u0 + (p - nl);
         const int slab = u / rg.ups, j = u - slab * rg.ups;
         const int ntw = min(kUT, ktiles - j * kUT) - kWT * half;      // tiles of this warp: <= 0, 2 or 4
-        DBG_CLK(tm0);
         mbar_wait(bars + 8u * stage, phase, ctl);
-        DBG_CLK(tm1);
-        DBG_ACC(0, tm0, tm1);
-        if (p == 0) DBG_TS(2);
         const unsigned char* st = smem + (size_t)stage * lay.stage_bytes;
-        const unsigned char* xp[MT];
+        if (ntw > 0) {
+            const unsigned char* xp[MT];
 #pragma unroll
-        for (int mt = 0; mt < MT; ++mt) xp[mt] = tok_ok[mt] ? st + x_off[mt] : zero_row;
-        // this warp's first group of the unit, and its tokens 2t, 2t+1 (+ 8 per column tile)
-        const float* xs = xsum + ((j * kUT + kWT * half) * 64 / G) * MTOK + 2 * t;
-        if (ntw >= kWT) math_stage<G, MT, kWT>(st, xp, w_off, sc_off, z_off, xs, acc);
-        else if (ntw >= 2) math_stage<G, MT, 2>(st, xp, w_off, sc_off, z_off, xs, acc);
-        DBG_CLK(tm3);
-        DBG_ACC(1, tm1, tm3);
+            for (int mt = 0; mt < MT; ++mt) xp[mt] = st + x_off[mt];
+            constexpr int NCH = (MT == 1) ? 2 : 1;
+#pragma unroll
+            for (int v = 0; v < kWT; ++v) {
+                if (v < ntw) {
+                    const int tile = kWT * half + v;                   // k-tile inside the stage
+                    const uint4 pk = *reinterpret_cast<const uint4*>(st + w_off + v * 512);
+                    uint4 xa[MT], xb[MT];
+#pragma unroll
+                    for (int mt = 0; mt < MT; ++mt) {
+                        // lanes without a token must not touch shared memory (see the band kernel)
+                        xa[mt] = make_uint4(0u, 0u, 0u, 0u);
+                        xb[mt] = make_uint4(0u, 0u, 0u, 0u);
+                        if (tok_ok[mt]) {
+                            xa[mt] = *reinterpret_cast<const uint4*>(xp[mt] + v * 128);
+                            xb[mt] = *reinterpret_cast<const uint4*>(xp[mt] + v * 128 + 16);
+                        }
+                    }
+                    const int q = tile / TPG;
+                    const float d_up = __half2float(*reinterpret_cast<const __half*>(st + sc_off + q * 32));
+                    const float d_lo = __half2float(*reinterpret_cast<const __half*>(st + sc_off + q * 32 + 16));
+                    const uint32_t zb = st[z_off + q * 16];
+                    const float su = d_up * 16777216.0f, sl = d_lo * 1048576.0f;
+                    const float zu = -d_up * (float)(zb & 0xFu), zl = -d_lo * (float)(zb >> 4);
+                    float c[MT][NCH][4];
+                    block_mma<MT, NCH>(pk, xa, xb, c);
+#pragma unroll
+                    for (int mt = 0; mt < MT; ++mt) {
+                        const float2 X = *reinterpret_cast<const float2*>(
+                            xsum + (j * kUT + tile) * MTOK + mt * 8 + 2 * t);
+                        float d[4];
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) d[i] = (NCH == 2) ? c[mt][0][i] + c[mt][NCH - 1][i] : c[mt][0][i];
+                        acc[mt][0] = fmaf(su, d[0], fmaf(zu, X.x, acc[mt][0]));
+                        acc[mt][1] = fmaf(su, d[1], fmaf(zu, X.y, acc[mt][1]));
+                        acc[mt][2] = fmaf(sl, d[2], fmaf(zl, X.x, acc[mt][2]));
+                        acc[mt][3] = fmaf(sl, d[3], fmaf(zl, X.y, acc[mt][3]));
+                    }
+                }
+            }
+        }
         __syncwarp();
         if (lane == 0) mbar_arrive(bars + 64u + 8u * stage);
         if (++stage == (uint32_t)S) { stage = 0; phase ^= 1u; }
-        DBG_CLK(tm4);
-        DBG_ACC(3, tm3, tm4);
 
         if (j == rg.ups - 1 || u == u1 - 1) {
             // end of this block's segment of the slab: hand the sums to the flush warps
@@ -447,25 +646,33 @@ gemv_kernel(const unsigned char* __restrict__ qweight, const __half* __restrict_
             if (lane == 0) mbar_arrive(bars + 192u + 8u * b);
             ++nflush;
         }
+        (void)slab;
     }
-    DBG_TS(14);
-    if (threadIdx.x == 0) DBG_ACC_STORE(10);   // [10..13] math warp 0: full wait, mma, ready wait, finalize
+}
+
+template <typename Kernel>
+cudaError_t allow_big_smem(Kernel kernel, bool (&done)[64]) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (!done[dev & 63]) {
+        e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
+        if (e != cudaSuccess) return e;
+        done[dev & 63] = true;
+    }
+    return cudaSuccess;
 }
 
 }  // namespace
 
-#ifdef AWQ_DBG_TS
-extern "C" __attribute__((visibility("default"))) int awq_dbg_read_ts(unsigned long long* dst) {
-    return (int)cudaMemcpyFromSymbol(dst, g_dbg_ts, sizeof(g_dbg_ts));
+bool gemv_uses_band_kernel(int M, int N, int sms) {
+    // one 16-row band per task: needs enough bands to occupy the SMs, and few tokens (every
+    // band re-reads its slice of x from L2)
+    return M <= 4 && (N / 16) * 4 >= sms * 3;
 }
-#endif
 
-GemvPlan gemv_plan(int M, int N, int K, int group) {
-    (void)group; (void)N; (void)K;
-    GemvPlan p;
-    p.max_blocks = kGemvMaxBlocks;
-    p.workspace_bytes = kCounterBytes + (size_t)kGemvMaxBlocks * 2 * M * 128 * sizeof(float);
-    return p;
+size_t gemv_workspace_bytes(int M) {
+    return kCounterBytes + (size_t)kGemvMaxBlocks * 2 * M * 128 * sizeof(float);
 }
 
 // Built-in scratch of awq_linear_gemv_static: arrival counters followed by the partial-sum
@@ -496,47 +703,65 @@ cudaError_t gemv_static_scratch(void** out) {
     return cudaSuccess;
 }
 
-cudaError_t launch_gemv(const void* x, const void* qweight, const void* scales, const void* zeros,
-                        void* y, int M, int N, int K, int group, void* workspace,
-                        unsigned int* status_word, int sms, cudaStream_t st) {
+cudaError_t launch_gemv_band(const void* x, const void* qweight, const void* scales, const void* zeros,
+                             void* y, int M, int N, int K, int group, unsigned int* status_word, int sms,
+                             cudaStream_t st) {
+    const int bands = N / 16;
+    const int blocks = bands < sms ? bands : sms;
+    const int tpw = M <= 2 ? 4 : 2;                            // 64 or 32 k-tiles per stage
+    cudaError_t e = cudaSuccess;
+#define AWQ_BAND_LAUNCH(GG, TT)                                                                      \
+    do {                                                                                             \
+        const BandLayout lay = band_layout<GG, TT>(M, K);                                            \
+        if (lay.stages < 2) return cudaErrorInvalidValue;      /* K too large for the x-sum table */ \
+        static bool done[64] = {};                                                                   \
+        e = allow_big_smem(gemv_band_kernel<GG, TT>, done);                                          \
+        if (e != cudaSuccess) return e;                                                              \
+        gemv_band_kernel<GG, TT><<<blocks, kBandThreads, lay.total, st>>>(                           \
+            reinterpret_cast<const unsigned char*>(qweight), reinterpret_cast<const __half*>(scales), \
+            reinterpret_cast<const unsigned char*>(zeros), reinterpret_cast<const __half*>(x),       \
+            reinterpret_cast<__half*>(y), M, N, K, lay, status_word);                                \
+    } while (0)
+    if (group == 128) { if (tpw == 4) AWQ_BAND_LAUNCH(128, 4); else AWQ_BAND_LAUNCH(128, 2); }
+    else              { if (tpw == 4) AWQ_BAND_LAUNCH(64, 4);  else AWQ_BAND_LAUNCH(64, 2); }
+#undef AWQ_BAND_LAUNCH
+    count_launch();
+    return cudaGetLastError();
+}
+
+cudaError_t launch_gemv_splitk(const void* x, const void* qweight, const void* scales, const void* zeros,
+                               void* y, int M, int N, int K, int group, void* workspace,
+                               unsigned int* status_word, int sms, cudaStream_t st) {
     const int ktiles = K / 64;
-    const int units = (N / 128) * ((ktiles + kUT - 1) / kUT);
+    const int ups = (ktiles + kUT - 1) / kUT;
+    const int units = (N / 128) * ups;
     int blocks = sms < kGemvMaxBlocks ? sms : kGemvMaxBlocks;
     if (units < blocks) blocks = units;
-    {
-        // Prefer a slightly smaller grid whose equal shares line up with slab boundaries
-        // (every block then ends exactly one segment, and fewer partial sums are exchanged).
-        const int ups = (ktiles + kUT - 1) / kUT;
-        for (int b = blocks; b * 20 >= blocks * 17; --b) {
-            if (units % b != 0) continue;
-            const int share = units / b;
-            if (share % ups == 0 || ups % share == 0) { blocks = b; break; }
-        }
+    // Prefer a slightly smaller grid whose equal shares line up with slab boundaries (every
+    // block then ends exactly one segment, and fewer partial sums are exchanged).
+    for (int b = blocks; b * 20 >= blocks * 17; --b) {
+        if (units % b != 0) continue;
+        const int share = units / b;
+        if (share % ups == 0 || ups % share == 0) { blocks = b; break; }
     }
     unsigned int* counters = reinterpret_cast<unsigned int*>(workspace);
     float* partial = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(workspace) + kCounterBytes);
-    const GemvLayout lay = gemv_layout(M, K, group);
-    if (lay.stages < 2) return cudaErrorInvalidValue;      // K too large for the x-sum table
+    const SplitkLayout lay = splitk_layout(M, K);
+    if (lay.stages < 2) return cudaErrorInvalidValue;          // K too large for the x-sum table
     cudaError_t e = cudaSuccess;
-#define AWQ_GEMV_LAUNCH(GG, MTT)                                                                     \
+#define AWQ_SPLITK_LAUNCH(GG, MTT)                                                                   \
     do {                                                                                             \
-        static bool attr_done[64] = {};                                                              \
-        int dev = 0;                                                                                 \
-        cudaGetDevice(&dev);                                                                         \
-        if (!attr_done[dev & 63]) {                                                                  \
-            e = cudaFuncSetAttribute(gemv_kernel<GG, MTT>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
-                                     kSmemBudget);                                                   \
-            if (e != cudaSuccess) return e;                                                          \
-            attr_done[dev & 63] = true;                                                              \
-        }                                                                                            \
-        gemv_kernel<GG, MTT><<<blocks, kGemvThreads, lay.total, st>>>(                               \
+        static bool done[64] = {};                                                                   \
+        e = allow_big_smem(gemv_splitk_kernel<GG, MTT>, done);                                       \
+        if (e != cudaSuccess) return e;                                                              \
+        gemv_splitk_kernel<GG, MTT><<<blocks, kSplitkThreads, lay.total, st>>>(                      \
             reinterpret_cast<const unsigned char*>(qweight), reinterpret_cast<const __half*>(scales), \
             reinterpret_cast<const unsigned char*>(zeros), reinterpret_cast<const __half*>(x),       \
-            reinterpret_cast<__half*>(y), partial, counters, M, N, K, lay, status_word);                  \
+            reinterpret_cast<__half*>(y), partial, counters, M, N, K, lay, status_word);             \
     } while (0)
-    if (group == 128) { if (M <= 8) AWQ_GEMV_LAUNCH(128, 1); else AWQ_GEMV_LAUNCH(128, 2); }
-    else              { if (M <= 8) AWQ_GEMV_LAUNCH(64, 1);  else AWQ_GEMV_LAUNCH(64, 2); }
-#undef AWQ_GEMV_LAUNCH
+    if (group == 128) { if (M <= 8) AWQ_SPLITK_LAUNCH(128, 1); else AWQ_SPLITK_LAUNCH(128, 2); }
+    else              { if (M <= 8) AWQ_SPLITK_LAUNCH(64, 1);  else AWQ_SPLITK_LAUNCH(64, 2); }
+#undef AWQ_SPLITK_LAUNCH
     count_launch();
     return cudaGetLastError();
 }

@@ -140,17 +140,20 @@ quantize_pack_kernel(const __half* __restrict__ W, const float* __restrict__ a, 
                        (code_of(wp[ti][0][c + 2], d[0], z[0]) << 8) | (code_of(wp[ti][0][c + 3], d[0], z[0]) << 24) |
                        (code_of(wp[ti][1][c + 2], d[1], z[1]) << 12) | (code_of(wp[ti][1][c + 3], d[1], z[1]) << 28);
         }
-        const size_t tile = (size_t)slab * (K / 64) + (size_t)kblk * 2 + ti;
-        uint4* dst = reinterpret_cast<uint4*>(qweight) + tile * 256 + warp * 32 + lane;
+        // band-major: block (band, k-tile) is 512 bytes, a band's blocks are contiguous along K
+        const size_t band = (size_t)slab * 8 + warp;
+        const size_t block = band * (K / 64) + (size_t)kblk * 2 + ti;
+        uint4* dst = reinterpret_cast<uint4*>(qweight) + block * 32 + lane;
         *dst = make_uint4(words[0], words[1], words[2], words[3]);
 
         if (t == 0 && (G == 64 || ti == 0)) {
-            // parameters are stored slab by slab, group by group: 128 scales, 64 zero bytes
+            // scales: [band][group][16]; zero bytes: [band pair][group][16], 8 per band
             const int gi = (G == 64) ? kblk * 2 + ti : kblk;
-            const size_t sg = (size_t)slab * (K / G) + gi;
-            scales[sg * 128 + warp * 16 + g] = d16[0];
-            scales[sg * 128 + warp * 16 + g + 8] = d16[1];
-            zeros[sg * 64 + warp * 8 + g] = (uint8_t)((uint32_t)z[0] | ((uint32_t)z[1] << 4));
+            const size_t ng = K / G;
+            scales[(band * ng + gi) * 16 + g] = d16[0];
+            scales[(band * ng + gi) * 16 + g + 8] = d16[1];
+            zeros[((band >> 1) * ng + gi) * 16 + (band & 1) * 8 + g] =
+                (uint8_t)((uint32_t)z[0] | ((uint32_t)z[1] << 4));
         }
     }
 }
@@ -164,19 +167,18 @@ __global__ void unpack_kernel(const uint32_t* __restrict__ qweight, const __half
     const size_t total = (size_t)N * K;
     if (idx >= total) return;
     const int n = (int)(idx / K), k = (int)(idx % K);
-    const size_t tile = (size_t)(n / 128) * (K / 64) + k / 64;
-    const int r = n % 128, c = k % 64;
-    const int band = r / 16, rr = r % 16, g = rr % 8, h = rr / 8;
+    const int band = n / 16, rr = n % 16, g = rr % 8, h = rr / 8;
+    const size_t block = (size_t)band * (K / 64) + k / 64;
+    const int c = k % 64;
     const int t = c / 16, j = (c % 16) / 4, i = c % 4;
-    const uint32_t w = qweight[tile * 1024 + band * 128 + (g * 4 + t) * 4 + j];
+    const uint32_t w = qweight[block * 128 + (g * 4 + t) * 4 + j];
     const int slot = (i / 2) * 4 + h * 2 + (i % 2);
     const int nib = (slot % 2) * 4 + slot / 2;
     codes[idx] = (uint8_t)((w >> (4 * nib)) & 0xFu);
     if (k % group == 0) {
         const int gi = k / group, ng = K / group;
-        const size_t sg = (size_t)(n / 128) * ng + gi;
-        scales_nk[(size_t)n * ng + gi] = __half_as_ushort(scales[sg * 128 + r]);
-        const uint8_t zb = zeros[sg * 64 + band * 8 + g];
+        scales_nk[(size_t)n * ng + gi] = __half_as_ushort(scales[((size_t)band * ng + gi) * 16 + rr]);
+        const uint8_t zb = zeros[((size_t)(band >> 1) * ng + gi) * 16 + (band & 1) * 8 + g];
         zeros_nk[(size_t)n * ng + gi] = (uint8_t)((zb >> (4 * h)) & 0xFu);
     }
 }

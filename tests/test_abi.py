@@ -32,7 +32,7 @@ def test_header_symbols_are_exported(lib):
 
 
 def test_sizes_and_layout_version(lib):
-    assert lib.awq_layout_version() == 2
+    assert lib.awq_layout_version() == 3
     assert lib.awq_qweight_bytes(4096, 4096) == 4096 * 4096 // 2
     assert lib.awq_scales_bytes(4096, 4096, 128) == 32 * 4096 * 2
     assert lib.awq_zeros_bytes(4096, 11008, 64) == 172 * 4096 // 2
@@ -57,6 +57,7 @@ def test_argument_errors_need_no_gpu(lib):
     assert lib.awq_linear(one, one, one, one, one, 1, 128, 192, 128, None) == 2
     assert lib.awq_linear_path(one, one, one, one, one, 17, 128, 128, 128, 1, None) == 2
     assert lib.awq_linear_path(one, one, one, one, one, 1, 128, 128, 128, 7, None) == 10
+    assert lib.awq_linear_path(one, one, one, one, one, 17, 128, 128, 128, 3, None) == 2
     assert b"group" in lib.awq_status_string(3)
     assert lib.awq_launch_count() == 0
 

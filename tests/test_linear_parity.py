@@ -18,20 +18,25 @@ def _run(case, path, packed=None):
 
 
 GEMV_CASES = [
-    # N, K, M, G, alpha  - several tiles, ragged k-tile counts, both groups, all token counts
+    # N, K, M, G, alpha  - several tiles, ragged k-tile counts, both groups, all token counts.
+    # PATH_GEMV picks the band kernel for the large-N, M <= 4 cases and the split-K kernel for
+    # the others; PATH_GEMV_SPLITK forces the split-K kernel on all of them.
     (128, 128, 1, 128, 0.5), (128, 384, 1, 64, 0.5), (256, 640, 3, 128, 0.0), (384, 1152, 8, 64, 1.0),
     (1024, 1408, 5, 128, 0.5), (512, 2048, 16, 128, 0.5), (256, 896, 9, 64, 0.5),
     (4096, 4096, 1, 128, 0.5), (4096, 4096, 2, 64, 0.5), (4096, 4096, 4, 128, 0.0),
+    (2048, 1152, 3, 64, 0.5), (2432, 8320, 1, 128, 0.5), (11008, 4096, 1, 128, 0.5),
 ]
 
 
+@pytest.mark.parametrize("forced", [False, True])
 @pytest.mark.parametrize("N,K,M,G,alpha", GEMV_CASES)
-def test_gemv_parity(N, K, M, G, alpha):
+def test_gemv_parity(N, K, M, G, alpha, forced):
     from paper_2306_00978_b200 import binding
+    path = binding.PATH_GEMV_SPLITK if forced else binding.PATH_GEMV
     case = Case(2000 + N + K + M, N, K, M, G, alpha)
-    y = _run(case, binding.PATH_GEMV)
-    assert_parity(y, case.y_ref(), f"gemv N={N} K={K} M={M} G={G}")
-    y2 = _run(case, binding.PATH_GEMV)
+    y = _run(case, path)
+    assert_parity(y, case.y_ref(), f"gemv N={N} K={K} M={M} G={G} path={path}")
+    y2 = _run(case, path)
     assert np.array_equal(y.view(np.uint16), y2.view(np.uint16))       # bit-reproducible
 
 

@@ -161,7 +161,7 @@ def test_pack_order_worked_example(golden_dir):
     # the slot stored at nibble p is order[p]
     assert [orc.NIBBLE_OF_SLOT.index(p) for p in range(8)] == order
     codes = np.zeros((128, 64), np.uint8)
-    # the eight slots of word 0 are rows 0 and 8, columns 0..3 of the first piece
+    # the eight slots of word 0 are rows 0 and 8, columns 0..3 of the first piece of band 0
     slots = [(0, 0), (0, 1), (8, 0), (8, 1), (0, 2), (0, 3), (8, 2), (8, 3)]
     for v, (n, k) in enumerate(slots):
         codes[n, k] = v
@@ -190,10 +190,10 @@ def test_pack_matches_location_formula_and_round_trips():
                 ref[wi] |= int(codes[n, k]) << (4 * p)
         assert words.tolist() == ref
         assert np.array_equal(orc.unpack_qweight(words, N, K), codes)
-    # a tile is 4096 contiguous bytes and tiles of one 128-row slab follow each other along K
-    assert orc.qweight_location(127, 63, 192)[0] == 1023
-    assert orc.qweight_location(0, 64, 192)[0] == 1024
-    assert orc.qweight_location(128, 0, 192)[0] == 3 * 1024
+    # a block is 512 contiguous bytes and the blocks of one 16-row band follow each other along K
+    assert orc.qweight_location(15, 63, 192)[0] == 127
+    assert orc.qweight_location(0, 64, 192)[0] == 128
+    assert orc.qweight_location(16, 0, 192)[0] == 3 * 128
 
 
 def test_zero_and_scale_packing():
@@ -201,7 +201,7 @@ def test_zero_and_scale_packing():
     N, ng = 256, 3
     zeros = rng.integers(0, 16, size=(N, ng), dtype=np.uint8)
     packed = orc.pack_zeros(zeros)
-    assert packed.shape == (N // 128, ng, 64)
+    assert packed.shape == (N // 32, ng, 16)
     flat = packed.reshape(-1)
     seen = set()
     for n in range(N):
@@ -213,14 +213,16 @@ def test_zero_and_scale_packing():
     assert np.array_equal(orc.unpack_zeros(packed, N, ng), zeros)
     sc = rng.standard_normal((N, ng)).astype(np.float16)
     ps = orc.pack_scales(sc)
-    assert ps.shape == (N // 128, ng, 128)
-    for n in (0, 5, 127, 128, 255):
+    assert ps.shape == (N // 16, ng, 16)
+    for n in (0, 5, 15, 16, 127, 128, 255):
         for gi in range(ng):
             assert ps.reshape(-1)[orc.scales_location(n, gi, ng)] == sc[n, gi]
     assert np.array_equal(orc.unpack_scales(ps, N, ng), sc)
-    # one slab's parameters of consecutive groups are contiguous: 256 and 64 bytes per group
-    assert orc.scales_location(0, 1, ng) - orc.scales_location(0, 0, ng) == 128
-    assert orc.zeros_location(0, 1, ng)[0] - orc.zeros_location(0, 0, ng)[0] == 64
+    # parameters of consecutive groups are contiguous: 32 bytes of scales per band, 16 bytes of
+    # zero points per pair of bands
+    assert orc.scales_location(0, 1, ng) - orc.scales_location(0, 0, ng) == 16
+    assert orc.zeros_location(0, 1, ng)[0] - orc.zeros_location(0, 0, ng)[0] == 16
+    assert orc.zeros_location(16, 0, ng)[0] - orc.zeros_location(0, 0, ng)[0] == 8
 
 
 # ------------------------------------------------------- dequantize-then-multiply, exactly

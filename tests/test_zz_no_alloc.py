@@ -26,7 +26,7 @@ def test_static_scratch_matches_regular_entry_point(N, K, M, G):
     case = Case(7000 + N + K + M, N, K, M, G, 0.5)
     qw, sc, zp = oracle_packed_to_cuda(case)
     x = to_cuda(case.x)
-    want = binding.linear(x, qw, sc, zp, N, K, G, path=binding.PATH_GEMV)
+    want = binding.linear(x, qw, sc, zp, N, K, G, path=binding.PATH_GEMV_SPLITK)
     binding.poll_status()
     want = want.cpu().numpy().astype(np.float64)
 
