@@ -283,6 +283,12 @@ gemv_band_kernel(const unsigned char* __restrict__ qweight, const __half* __rest
     const int o_x = St::kXOff + g * St::kXRow + warp * (TPW * 128) + t * 32;
     const float* xs_lane = xsum + warp * (TPW * 8) + 2 * t;
 
+    // B fragments: lanes without a token keep zeros for the whole kernel and never touch
+    // shared memory (even a broadcast read costs wavefronts on the shared-memory pipe)
+    uint4 xr[TPW][2];
+#pragma unroll
+    for (int v = 0; v < TPW; ++v) xr[v][0] = xr[v][1] = make_uint4(0u, 0u, 0u, 0u);
+
     uint32_t stage = 0, phase = 0;
     int nflush = 0;
     for (int band = b0; band < b1; ++band, ++nflush) {
@@ -292,19 +298,69 @@ gemv_band_kernel(const unsigned char* __restrict__ qweight, const __half* __rest
             const int nt = min(UT, ktiles - j * UT) - warp * TPW;     // this warp's tiles: <= 0 .. TPW
             mbar_wait(bars + 8u * stage, phase, ctl);
             const unsigned char* st = smem + stage * (uint32_t)lay.stage_bytes;
-            if (nt > 0) {
-                const float* xs = xs_lane + j * (UT * 8);
+            const float* xs = xs_lane + j * (UT * 8);
+            if (nt >= TPW) {
+                // ---- full stage: straight-line code, one accumulation chain per group, the
+                // groups' products interleaved word by word so that no MMA waits for the last
+                uint4 pk[TPW];
+#pragma unroll
+                for (int v = 0; v < TPW; ++v) pk[v] = *reinterpret_cast<const uint4*>(st + o_w + v * 512);
+                if (tok_ok) {
+#pragma unroll
+                    for (int v = 0; v < TPW; ++v) {
+                        xr[v][0] = *reinterpret_cast<const uint4*>(st + o_x + v * 128);
+                        xr[v][1] = *reinterpret_cast<const uint4*>(st + o_x + v * 128 + 16);
+                    }
+                }
+                float c[GPW][4];
+#pragma unroll
+                for (int v = 0; v < TPG; ++v)
+#pragma unroll
+                    for (int jw = 0; jw < 4; ++jw)
+#pragma unroll
+                        for (int q = 0; q < GPW; ++q) {
+                            const int tile = q * TPG + v;
+                            const uint32_t w = (jw == 0) ? pk[tile].x : (jw == 1) ? pk[tile].y : (jw == 2) ? pk[tile].z : pk[tile].w;
+                            const uint32_t w8 = w >> 8;
+                            const uint4 xq = xr[tile][jw >> 1];
+                            const uint32_t bb0 = (jw & 1) ? xq.z : xq.x, bb1 = (jw & 1) ? xq.w : xq.y;
+                            if (v == 0 && jw == 0)
+                                mma_16816_first(c[q], w & 0x000F000Fu, w & 0x00F000F0u, w8 & 0x000F000Fu,
+                                                w8 & 0x00F000F0u, bb0, bb1);
+                            else
+                                mma_16816(c[q], w & 0x000F000Fu, w & 0x00F000F0u, w8 & 0x000F000Fu,
+                                          w8 & 0x00F000F0u, bb0, bb1);
+                        }
 #pragma unroll
                 for (int q = 0; q < GPW; ++q) {
-                    if (q * TPG < nt) {                               // whole groups only (K % G == 0)
+                    float Xx = 0.0f, Xy = 0.0f;
+#pragma unroll
+                    for (int v = 0; v < TPG; ++v) {
+                        const float2 X = *reinterpret_cast<const float2*>(xs + (q * TPG + v) * 8);
+                        Xx += X.x;
+                        Xy += X.y;
+                    }
+                    const float d_up = __half2float(*reinterpret_cast<const __half*>(st + o_sc + q * 32));
+                    const float d_lo = __half2float(*reinterpret_cast<const __half*>(st + o_sc + q * 32 + 16));
+                    const uint32_t zb = st[o_z + q * 16];
+                    const float su = d_up * 16777216.0f, sl = d_lo * 1048576.0f;
+                    const float zu = d_up * (float)(zb & 0xFu), zl = d_lo * (float)(zb >> 4);
+                    acc[0] = fmaf(su, c[q][0], fmaf(-zu, Xx, acc[0]));
+                    acc[1] = fmaf(su, c[q][1], fmaf(-zu, Xy, acc[1]));
+                    acc[2] = fmaf(sl, c[q][2], fmaf(-zl, Xx, acc[2]));
+                    acc[3] = fmaf(sl, c[q][3], fmaf(-zl, Xy, acc[3]));
+                }
+            } else if (nt > 0) {
+                // ---- ragged last stage of a band: whole groups only (K % G == 0), one at a time
+#pragma unroll
+                for (int q = 0; q < GPW; ++q) {
+                    if (q * TPG < nt) {
                         float c[1][2][4];
                         float Xx = 0.0f, Xy = 0.0f;
 #pragma unroll
                         for (int v = 0; v < TPG; ++v) {
                             const int tile = q * TPG + v;
                             const uint4 pk = *reinterpret_cast<const uint4*>(st + o_w + tile * 512);
-                            // lanes without a token must not touch shared memory: even a
-                            // broadcast read costs wavefronts on the shared-memory pipe
                             uint4 xa[1] = {make_uint4(0u, 0u, 0u, 0u)}, xb[1] = {make_uint4(0u, 0u, 0u, 0u)};
                             if (tok_ok) {
                                 xa[0] = *reinterpret_cast<const uint4*>(st + o_x + tile * 128);
@@ -432,7 +488,6 @@ gemv_splitk_kernel(const unsigned char* __restrict__ qweight, const __half* __re
     if (threadIdx.x < kZeroRowBytes / 4) reinterpret_cast<uint32_t*>(smem + lay.zero_off)[threadIdx.x] = 0u;
     __syncthreads();
     const WaitCtl ctl{status_word, &s_abort};
-    const unsigned char* zero_row = smem + lay.zero_off;
     constexpr int MTOK = MT * 8;
 
     if (warp == kMathWarps) {
@@ -449,7 +504,7 @@ gemv_splitk_kernel(const unsigned char* __restrict__ qweight, const __half* __re
             const uint32_t dst = sbase + stage * (uint32_t)lay.stage_bytes;
             const uint32_t bar = bars + 8u * stage;
             if (lane == 0) {
-                mbar_wait(bars + 64u + 8u * stage, phase ^ 1u, ctl);
+                mbar_wait_relaxed(bars + 64u + 8u * stage, phase ^ 1u, ctl);
                 mbar_arrive_expect_tx(bar, (uint32_t)(nt * kTileBytes + ngr * (256 + 64) + M * nt * 128));
             }
             __syncwarp();
@@ -499,7 +554,7 @@ gemv_splitk_kernel(const unsigned char* __restrict__ qweight, const __half* __re
             if (j == rg.ups - 1 || u == u1 - 1) {
                 const bool whole = (u - j >= u0) && (j == rg.ups - 1);
                 const uint32_t b = (uint32_t)nflush & 1u, use = ((uint32_t)nflush >> 1) & 1u;
-                mbar_wait(bars + 192u + 8u * b, use, ctl);
+                mbar_wait_relaxed(bars + 192u + 8u * b, use, ctl);
                 const float* rb = red + b * (2 * MTOK * 128);
                 const int slot = (slab == slab0) ? 0 : 1;
                 float* mine = partial + (size_t)(blockIdx.x * 2 + slot) * M * 128;
