@@ -44,7 +44,7 @@ NOMINAL_HBM_GBS = 8000.0
 NOMINAL_FP16_TFLOPS = 2250.0
 # DRAM bytes per launch of the dominant kernel from the ncu capture summarised under
 # profiles/ (None until a capture of the current kernel exists).
-NCU_TRAFFIC_BYTES_PER_LAUNCH = None
+NCU_TRAFFIC_BYTES_PER_LAUNCH = {(11008, 4096): 23470000, (4096, 4096): 8760000}
 
 
 def algorithmic_bytes(N: int, K: int, M: int, group: int = GROUP) -> int:
@@ -362,6 +362,35 @@ def reference_arm(args):
     return 0
 
 
+def one_shape(args):
+    """A small, self-contained run of one shape for ncu captures (random packed bytes: the
+    kernels' work does not depend on the values)."""
+    import torch
+    from paper_2306_00978_b200 import binding
+    N, K, M = args.one
+    copies = []
+    for _ in range(3):
+        qw = torch.randint(0, 256, (N * K // 2,), dtype=torch.uint8, device="cuda")
+        sc = (torch.rand((N // 16, K // GROUP, 16), device="cuda") * 0.01 + 0.001).half()
+        zp = torch.randint(0, 256, (N // 32, K // GROUP, 16), dtype=torch.uint8, device="cuda")
+        copies.append((qw, sc, zp))
+    x = torch.randn((M, K), device="cuda").half()
+    y = torch.empty((M, N), device="cuda", dtype=torch.float16)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for r in range(args.reps):
+        if r == args.reps - 1:
+            e0.record()
+        for (qw, sc, zp) in copies:
+            binding.linear(x, qw, sc, zp, N, K, GROUP, out=y, path=args.path)
+    e1.record()
+    torch.cuda.synchronize()
+    binding.poll_status()
+    us = e0.elapsed_time(e1) * 1e3 / len(copies)
+    print(json.dumps({"one": [N, K, M], "path": args.path, "us_per_launch_last_pass": us,
+                      "algorithmic_bytes": algorithmic_bytes(N, K, M), "flops": 2 * M * N * K}))
+    return 0
+
+
 # --------------------------------------------------------------------------------- main
 def main():
     ap = argparse.ArgumentParser()
@@ -371,7 +400,14 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--layers", type=int, default=4, help="independently seeded layers to rotate over")
     ap.add_argument("--skip-extras", action="store_true", help="only the headline step (for profiling)")
+    ap.add_argument("--one", nargs=3, type=int, metavar=("N", "K", "M"),
+                    help="profiling aid: a few awq_linear launches of one shape on random packed "
+                         "weights (three rotating copies), then exit")
+    ap.add_argument("--path", type=int, default=0, help="with --one: 0 auto, 1 GEMV, 2 GEMM, 3 split-K GEMV")
+    ap.add_argument("--reps", type=int, default=3, help="with --one: passes over the three copies")
     args = ap.parse_args()
+    if args.one:
+        return one_shape(args)
 
     if args.impl == "reference":
         return reference_arm(args)
@@ -437,10 +473,15 @@ def main():
                                 f"({args.layers * packed_bytes / 1e6:.0f} MB > 2 x 126 MB L2)",
                    "algorithmic_bytes_per_step": step_bytes, "parallelism": f"replicas x{world}",
                    "launch": "each step is one CUDA-graph replay of its 7 awq_linear calls"},
-        "roofline": {"bound": "hbm", "kernel": "gemv_kernel<128,1>", "achieved": achieved,
+        "roofline": {"bound": "hbm", "kernel": "gemv_band_kernel<128,4>", "achieved": achieved,
                      "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
                      "peak_source": peaks["source"], "frac_of_nominal_8000": achieved / NOMINAL_HBM_GBS,
-                     "avg_launch_us": per_launch_s * 1e6, "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH},
+                     "avg_launch_us": per_launch_s * 1e6,
+                     # per launch, averaged over the step's 7 launches (4x 4096^2, 3x 4096x11008),
+                     # from the captures in profiles/gemv_band_kernel_llama2_7b_M1.md
+                     "traffic": (4 * NCU_TRAFFIC_BYTES_PER_LAUNCH[(4096, 4096)] +
+                                 3 * NCU_TRAFFIC_BYTES_PER_LAUNCH[(11008, 4096)]) / 7,
+                     "algorithmic_bytes_per_launch": step_bytes / 7},
         "e2e": {"value": e2e_value, "unit": UNIT,
                 "h2d_bytes_per_step": sum(2 * l["K"] for l in layers[0]),
                 "d2h_bytes_per_step": sum(2 * l["N"] for l in layers[0])},
