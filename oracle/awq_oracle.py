@@ -118,16 +118,17 @@ def qweight_location(n: int, k: int, K: int):
 
     Rows are taken in bands of 16; everything a band needs is contiguous along K.  Block
     (band, k // 64) is 512 bytes (128 words) at word (band * (K // 64) + k // 64) * 128.  A
-    block is 32 pieces of 16 bytes; piece (g, t) holds rows g and g+8 of the band and columns
-    16t .. 16t+15 of the block.  Word j of a piece holds columns 16t+4j .. 16t+4j+3 of both
-    rows in the slot order (g,c0) (g,c1) (g+8,c0) (g+8,c1) (g,c2) (g,c3) (g+8,c2) (g+8,c3),
-    and slot e sits at nibble NIBBLE_OF_SLOT[e].
+    block is 32 pieces of 16 bytes; piece (g, t), g = 0..7, t = 0..3, holds rows g and g+8 of
+    the band.  Word j of a piece holds columns 16j+4t .. 16j+4t+3 of the block for both rows
+    (so the four pieces of a row pair interleave along K in runs of four columns), in the
+    slot order (g,c0) (g,c1) (g+8,c0) (g+8,c1) (g,c2) (g,c3) (g+8,c2) (g+8,c3), and slot e
+    sits at nibble NIBBLE_OF_SLOT[e].
     """
     band, rr = n // BAND_ROWS, n % BAND_ROWS
     block = band * (K // TILE_COLS) + k // TILE_COLS
     c = k % TILE_COLS
     g, h = rr % 8, rr // 8
-    t, j, i = c // 16, (c % 16) // 4, c % 4
+    j, t, i = c // 16, (c % 16) // 4, c % 4
     word = block * WORDS_PER_BLOCK + (g * 4 + t) * 4 + j
     slot = (i // 2) * 4 + h * 2 + (i % 2)
     return word, NIBBLE_OF_SLOT[slot]
@@ -154,10 +155,10 @@ def pack_qweight(codes) -> np.ndarray:
     codes = np.asarray(codes, dtype=np.uint8)
     N, K = codes.shape
     assert N % BAND_ROWS == 0 and K % TILE_COLS == 0
-    # axes: band, h, g, C, t, j, ihi, ilo
+    # axes: band, h, g, C, j, t, ihi, ilo      (column in block = 16 j + 4 t + 2 ihi + ilo)
     a = codes.reshape(N // 16, 2, 8, K // 64, 4, 4, 2, 2)
     # -> band, C, g, t, j, ihi, h, ilo   (the last three are the slot bits, high to low)
-    a = a.transpose(0, 3, 2, 4, 5, 6, 1, 7).reshape(-1, 8).astype(np.uint32)
+    a = a.transpose(0, 3, 2, 5, 4, 6, 1, 7).reshape(-1, 8).astype(np.uint32)
     words = np.zeros(a.shape[0], dtype=np.uint32)
     for slot in range(8):
         words |= a[:, slot] << np.uint32(4 * NIBBLE_OF_SLOT[slot])
@@ -172,7 +173,7 @@ def unpack_qweight(words, N: int, K: int) -> np.ndarray:
     for slot in range(8):
         a[:, slot] = (words >> np.uint32(4 * NIBBLE_OF_SLOT[slot])) & np.uint32(0xF)
     a = a.reshape(N // 16, K // 64, 8, 4, 4, 2, 2, 2)   # band, C, g, t, j, ihi, h, ilo
-    return a.transpose(0, 6, 2, 1, 3, 4, 5, 7).reshape(N, K)
+    return a.transpose(0, 6, 2, 1, 4, 3, 5, 7).reshape(N, K)
 
 
 def pack_zeros(zeros) -> np.ndarray:

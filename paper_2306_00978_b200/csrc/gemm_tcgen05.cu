@@ -4,23 +4,32 @@
 // its N side (BN = 32..256 columns of the fp32 accumulator in tensor memory), so
 // D[n][m] = sum_k dequant(Wq)[n][k] * x[m][k] and the epilogue writes y[m][n] = D[n][m].
 //
-// One persistent thread block per SM, warp-specialised:
-//   warp 0      producer: per 64-wide k-block two TMA tensor copies into a ring of stages -
-//               the x tile (BN x 64 fp16, 128-byte swizzle) and the packed weights of the
-//               slab's 8 bands (8 x 512 bytes, one box of the band-major weight array) -
-//               completion counted on an mbarrier.
-//   warps 8-15  dequantizers, one per band: each lane takes its 16-byte packed piece (rows
-//               g, g+8 of the band, 16 columns), converts two codes at a time to exact fp16
-//               (q - z), multiplies by Delta (one fp16 rounding) and stores four 16-byte
-//               pieces into the stage's A tile in the K-major 128-byte-swizzled layout the
-//               MMA reads.  Scales and zero points (32 + 8 bytes per band and group) are read
-//               straight from global memory two groups ahead.
-//   warp 1      one thread issues tcgen05.mma (kind::f16, M = 128, N = BN, K = 16, four per
-//               k-block), commits to the stage's "empty" barrier and, after the last
-//               k-block, to the accumulator's "full" barrier.
-//   warps 4-7   epilogue: tcgen05.ld 32 columns at a time, convert to fp16, store to y.
-//               Two accumulator buffers let the epilogue of one tile overlap the next main loop.
+// Shared-memory bandwidth, not the tensor pipe, is what a dequantizing GEMM runs out of first
+// (per 64-wide k-block the x tile is written once and read once, 64 KB at BN = 256).  So the
+// dequantized weights never touch shared memory: they go from registers straight into tensor
+// memory (tcgen05.st) and the MMA takes its A operand from there.
 //
+// One persistent thread block per SM, warp-specialised:
+//   warp 0       producer: per k-block two TMA tensor copies into a ring of stages - the x tile
+//                (BN x 64 fp16, 128-byte swizzle) and the packed weights of the slab's 8 bands
+//                (8 x 512 bytes, one box of the band-major weight array) - completion counted
+//                on an mbarrier.
+//   warps 8-15   dequantizers, one per 16-row band.  Lane (g, t) reads its 16-byte packed piece
+//                (rows g, g+8; columns 16j+4t..+3), converts two codes at a time to exact fp16
+//                (q - z) with the magic-number trick that the w{0,2,4,6,1,3,5,7} nibble order
+//                allows, multiplies by Delta (one fp16 rounding) and stores its 16 registers
+//                with one tcgen05.st: the piece layout is exactly the 16x256b register layout,
+//                so the band's 16 lanes x 32 columns of A land in the stage's slot of tensor
+//                memory without any shuffle.  Scales and zero points (32 + 8 bytes per band
+//                and group) are read straight from global memory two groups ahead.
+//   warp 1       one thread issues tcgen05.mma (kind::f16, M = 128, N = BN, K = 16, four per
+//                k-block, A from tensor memory, B through a shared-memory descriptor), commits
+//                to the stage's "empty" barrier and, after the last k-block, to the
+//                accumulator's "full" barrier.
+//   warps 4-7    epilogue: tcgen05.ld 32 columns at a time, convert to fp16, store to y.
+//                BN <= 128 keeps two accumulators so that the epilogue overlaps the next tile.
+//
+// Tensor-memory columns: accumulators first (BN or 2 BN), then 32 columns per stage for A.
 // Every wait is bounded (about two seconds of wall clock): a wait that runs out writes a code to
 // the status word, raises a block-wide flag, and every role leaves its loop; the block
 // then waits (bounded) for its own copies in flight, frees its tensor memory and returns.
@@ -37,14 +46,17 @@ namespace {
 
 constexpr int kGemmThreads = 512;
 constexpr int kBK = 64;
-constexpr int kATileBytes = 128 * kBK * 2;            // dequantized fp16 weight tile
 
 template <int BN> struct GemmCfg {
     static constexpr int kXTileBytes = BN * kBK * 2;
-    static constexpr int kStageBytes = kXTileBytes + kATileBytes + kTileBytes;
-    static constexpr int kStagesRaw = (216 * 1024) / kStageBytes;
-    static constexpr int kStages = kStagesRaw > 8 ? 8 : kStagesRaw;
-    static constexpr int kTmemCols = 2 * BN < 32 ? 32 : 2 * BN;   // two accumulator buffers
+    static constexpr int kStageBytes = kXTileBytes + kTileBytes;          // x tile + packed weights
+    static constexpr int kNumAcc = BN <= 128 ? 2 : 1;                      // accumulators in TMEM
+    static constexpr int kStagesSmem = (216 * 1024) / kStageBytes;
+    static constexpr int kStagesTmem = (512 - kNumAcc * BN) / 32;          // 32 columns of A per stage
+    static constexpr int kStagesMin = kStagesSmem < kStagesTmem ? kStagesSmem : kStagesTmem;
+    static constexpr int kStages = kStagesMin > 8 ? 8 : kStagesMin;
+    static constexpr int kAColumn0 = kNumAcc * BN;                         // first A column
+    static constexpr int kTmemCols = 512;
     static constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*align*/ + 256 /*barriers*/;
     static constexpr uint32_t kTxBytes = kXTileBytes + kTileBytes;
 };
@@ -69,6 +81,27 @@ __device__ __forceinline__ void umma_f16(uint32_t d_tmem, uint64_t a_desc, uint6
         "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
         ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
 }
+// the same with the A operand in tensor memory (128 lanes x 8 columns of fp16 pairs per K = 16)
+__device__ __forceinline__ void umma_f16_a_tmem(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
+                                                uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// A warp stores 16 lanes x 32 columns: four blocks of 8 columns, each in the 16x256b register
+// layout (lane-group g = lane / 4 holds rows g and g+8; t = lane % 4 holds columns 2t, 2t+1 of
+// the block; registers 4i .. 4i+3 of block i = (g, 2t) (g, 2t+1) (g+8, 2t) (g+8, 2t+1)).
+__device__ __forceinline__ void tmem_st_16x32cols(uint32_t taddr, const uint32_t (&v)[16]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.16x256b.x4.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, "
+        "%14, %15, %16};"
+        ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]),
+          "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15])
+        : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
@@ -121,6 +154,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ C
             __half* __restrict__ y, int M, int N, int K, unsigned int* status_word) {
     using Cfg = GemmCfg<BN>;
     constexpr int S = Cfg::kStages;
+    constexpr int NACC = Cfg::kNumAcc;
     extern __shared__ unsigned char smem_dyn[];
     __shared__ unsigned int s_abort;
     __shared__ uint32_t s_tmem_base;
@@ -128,10 +162,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ C
     const uint32_t dyn = smem_u32(smem_dyn);
     const uint32_t base = (dyn + 1023u) & ~1023u;                    // 1024-byte aligned stage ring
     unsigned char* base_ptr = smem_dyn + (base - dyn);
-    // stage layout: [X tile | A tile | packed tile]
+    // stage layout: [x tile | packed weights (8 bands x 512 bytes)]
     auto x_addr = [&](int s) { return base + (uint32_t)s * Cfg::kStageBytes; };
-    auto a_addr = [&](int s) { return x_addr(s) + Cfg::kXTileBytes; };
-    auto stage_ptr = [&](int s) { return base_ptr + (size_t)s * Cfg::kStageBytes; };
+    auto w_ptr = [&](int s) { return base_ptr + (size_t)s * Cfg::kStageBytes + Cfg::kXTileBytes; };
     const uint32_t bars = base + (uint32_t)S * Cfg::kStageBytes;       // 8-byte barriers follow the ring
     auto raw_full = [&](int s) { return bars + 8u * (uint32_t)s; };
     auto a_full = [&](int s) { return bars + 8u * (uint32_t)(S + s); };
@@ -175,7 +208,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ C
                     mbar_arrive_expect_tx(bar, Cfg::kTxBytes);
                     tma_load_2d(x_addr(stage), &x_map, kb * kBK, mt * BN, bar);
                     // weights: box of 8 bands x 512 bytes (128 words) at (k-block, first band)
-                    tma_load_2d(a_addr(stage) + kATileBytes, &w_map, kb * 128, slab * 8, bar);
+                    tma_load_2d(x_addr(stage) + Cfg::kXTileBytes, &w_map, kb * 128, slab * 8, bar);
                     ++issued;
                     if (++stage == S) { stage = 0; phase ^= 1u; }
                 }
@@ -199,8 +232,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ C
             int local = 0;
             bool ok = true;
             for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++local) {
-                const int b = local & 1;
-                const uint32_t use = (uint32_t)(local >> 1) & 1u;
+                const int b = local % NACC;
+                const uint32_t use = (uint32_t)(local / NACC) & 1u;
                 if (!mbar_wait(acc_empty(b), use ^ 1u, ctl)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(b * BN);
@@ -209,12 +242,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ C
                         ok = false; break;
                     }
                     tc_fence_after();
-                    const uint64_t adesc = smem_desc_sw128(a_addr(stage));
+                    const uint32_t a_tmem = tmem_base + (uint32_t)(Cfg::kAColumn0 + stage * 32);
                     const uint64_t bdesc = smem_desc_sw128(x_addr(stage));
 #pragma unroll
-                    for (int k = 0; k < kBK / 16; ++k)       // +32 bytes per K = 16 step, 16-byte units
-                        umma_f16(d_tmem, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), idesc,
-                                 (kb | k) != 0 ? 1u : 0u);
+                    for (int k = 0; k < kBK / 16; ++k)       // A: +8 columns, B: +32 bytes per K = 16 step
+                        umma_f16_a_tmem(d_tmem, a_tmem + (uint32_t)(8 * k), bdesc + (uint64_t)(2 * k), idesc,
+                                        (kb | k) != 0 ? 1u : 0u);
                     umma_commit(empty(stage));
                     if (++stage == S) { stage = 0; phase ^= 1u; }
                 }
@@ -223,16 +256,17 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ C
         }
     } else if (warp >= 8) {
         // -------------------------------------------------------------- dequantizers
-        const int band = warp - 8;
-        const int g = lane >> 2, t = lane & 3;
+        // one warp per 16-row band; lane (g, t) holds the band's piece (rows g and g+8, columns
+        // 16j + 4t .. +3 for j = 0..3), which is exactly its share of a 16-lane x 32-column
+        // tensor-memory store in the 16x256b register layout (four columns blocks of 8)
+        const int wi = warp - 8, quad = wi & 3, hsel = wi >> 2;
+        const int band = 2 * quad + hsel;               // bands 0..7 <-> TMEM lanes 16*band .. +15
+        const int g = lane >> 2;
+        const int ng = K / G;
+        constexpr int KPG = G / kBK;                    // k-blocks per group
+        const uint32_t taddr_band = tmem_base + ((uint32_t)(quad * 32 + hsel * 16) << 16) + (uint32_t)Cfg::kAColumn0;
         uint32_t stage = 0, phase = 0;
         bool ok = true;
-        // destination of this lane's four 16-byte pieces inside the swizzled A tile
-        const uint32_t row_up = (uint32_t)(2 * band) * 1024u + (uint32_t)g * 128u;
-        const uint32_t row_lo = row_up + 1024u;
-        const uint32_t c0 = (uint32_t)((2 * t) ^ g) * 16u, c1 = (uint32_t)((2 * t + 1) ^ g) * 16u;
-        constexpr int KPG = G / kBK;                    // k-blocks per group
-        const int ng = K / G;
         for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
             const int slab = tile / m_tiles;
             // this lane's rows' parameters: scales [band][group][16], zero bytes [band pair][group][16]
@@ -256,29 +290,25 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ C
                 ok = mbar_wait(raw_full(stage), phase, ctl);
                 ok = __all_sync(0xFFFFFFFFu, ok);
                 if (!ok) break;
-                const unsigned char* sp = stage_ptr(stage) + Cfg::kXTileBytes;
-                const unsigned char* raw = sp + kATileBytes;
-                const uint4 pk = *reinterpret_cast<const uint4*>(raw + band * 512 + lane * 16);
+                const uint4 pk = *reinterpret_cast<const uint4*>(w_ptr(stage) + band * 512 + lane * 16);
                 const uint32_t d_up = du | (du << 16), d_lo = dl | (dl << 16);
                 const uint32_t zu = 0x6400u + (zb & 0xFu), zl = 0xD400u + ((zb >> 4) << 4);
                 const uint32_t zlo = zu | (zu << 16), zhi = zl | (zl << 16);
                 const uint32_t wds[4] = {pk.x, pk.y, pk.z, pk.w};
-                uint32_t up[8], lo[8];                 // rows g / g+8: columns 16t .. 16t+15 as fp16x2
+                // per word j: (row g: c, c+1) (row g: c+2, c+3) (row g+8: c, c+1) (row g+8: c+2, c+3)
+                uint32_t v[16];
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
                     constexpr uint32_t kMagic = 0x64006400u, kSixteenth = 0x2C002C00u;
                     const uint32_t w = wds[j], w8 = w >> 8;
-                    up[2 * j] = hmul2_u32(hsub2_u32((w & 0x000F000Fu) | kMagic, zlo), d_up);
-                    lo[2 * j] = hmul2_u32(hfma2_u32((w & 0x00F000F0u) | kMagic, kSixteenth, zhi), d_lo);
-                    up[2 * j + 1] = hmul2_u32(hsub2_u32((w8 & 0x000F000Fu) | kMagic, zlo), d_up);
-                    lo[2 * j + 1] = hmul2_u32(hfma2_u32((w8 & 0x00F000F0u) | kMagic, kSixteenth, zhi), d_lo);
+                    v[4 * j + 0] = hmul2_u32(hsub2_u32((w & 0x000F000Fu) | kMagic, zlo), d_up);
+                    v[4 * j + 1] = hmul2_u32(hsub2_u32((w8 & 0x000F000Fu) | kMagic, zlo), d_up);
+                    v[4 * j + 2] = hmul2_u32(hfma2_u32((w & 0x00F000F0u) | kMagic, kSixteenth, zhi), d_lo);
+                    v[4 * j + 3] = hmul2_u32(hfma2_u32((w8 & 0x00F000F0u) | kMagic, kSixteenth, zhi), d_lo);
                 }
-                unsigned char* a_tile = const_cast<unsigned char*>(sp);
-                *reinterpret_cast<uint4*>(a_tile + row_up + c0) = make_uint4(up[0], up[1], up[2], up[3]);
-                *reinterpret_cast<uint4*>(a_tile + row_up + c1) = make_uint4(up[4], up[5], up[6], up[7]);
-                *reinterpret_cast<uint4*>(a_tile + row_lo + c0) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
-                *reinterpret_cast<uint4*>(a_tile + row_lo + c1) = make_uint4(lo[4], lo[5], lo[6], lo[7]);
-                fence_proxy_async_smem();
+                tmem_st_16x32cols(taddr_band + stage * 32u, v);
+                tmem_st_wait();
+                tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(a_full(stage));
                 if (++stage == S) { stage = 0; phase ^= 1u; }
@@ -291,8 +321,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ C
         bool ok = true;
         for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++local) {
             const int slab = tile / m_tiles, mt = tile % m_tiles;
-            const int b = local & 1;
-            const uint32_t use = (uint32_t)(local >> 1) & 1u;
+            const int b = local % NACC;
+            const uint32_t use = (uint32_t)(local / NACC) & 1u;
             ok = mbar_wait(acc_full(b), use, ctl);
             ok = __all_sync(0xFFFFFFFFu, ok);
             if (!ok) break;

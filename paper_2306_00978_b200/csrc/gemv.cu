@@ -64,10 +64,11 @@ __device__ __forceinline__ void mma_16816_first(float (&c)[4], uint32_t a0, uint
 }
 
 // One 16-row x 64-column packed block (this lane's 16 bytes `pk`) times the matching 64
-// activations of MT*8 tokens (this lane's 32 bytes per token tile, `xa` / `xb`):
+// activations of MT*8 tokens (this lane's 4 x 8 bytes per token tile: word j of the piece
+// multiplies x[16j + 4t .. +3]):
 // c[mt][chain] receive D = sum q * 2^-24 x (rows g) and sum q * 2^-20 x (rows g+8).
 template <int MT, int NCH, bool FIRST = true>
-__device__ __forceinline__ void block_mma(const uint4& pk, const uint4 (&xa)[MT], const uint4 (&xb)[MT],
+__device__ __forceinline__ void block_mma(const uint4& pk, const uint2 (&xq)[MT][4],
                                           float (&c)[MT][NCH][4]) {
     const uint32_t wds[4] = {pk.x, pk.y, pk.z, pk.w};
 #pragma unroll
@@ -77,8 +78,7 @@ __device__ __forceinline__ void block_mma(const uint4& pk, const uint4 (&xa)[MT]
         const uint32_t a2 = w8 & 0x000F000Fu, a3 = w8 & 0x00F000F0u;
 #pragma unroll
         for (int mt = 0; mt < MT; ++mt) {
-            const uint32_t b0 = (jw == 0) ? xa[mt].x : (jw == 1) ? xa[mt].z : (jw == 2) ? xb[mt].x : xb[mt].z;
-            const uint32_t b1 = (jw == 0) ? xa[mt].y : (jw == 1) ? xa[mt].w : (jw == 2) ? xb[mt].y : xb[mt].w;
+            const uint32_t b0 = xq[mt][jw].x, b1 = xq[mt][jw].y;
             if (FIRST && jw < NCH) mma_16816_first(c[mt][jw % NCH], a0, a1, a2, a3, b0, b1);
             else mma_16816(c[mt][jw % NCH], a0, a1, a2, a3, b0, b1);
         }
@@ -280,14 +280,16 @@ gemv_band_kernel(const unsigned char* __restrict__ qweight, const __half* __rest
     // this lane's fixed byte offsets inside a stage
     const int o_w = warp * (TPW * 512) + lane * 16;
     const int o_sc = St::kScOff + warp * (GPW * 32) + g * 2;
-    const int o_x = St::kXOff + g * St::kXRow + warp * (TPW * 128) + t * 32;
+    const int o_x = St::kXOff + g * St::kXRow + warp * (TPW * 128) + t * 8;
     const float* xs_lane = xsum + warp * (TPW * 8) + 2 * t;
 
     // B fragments: lanes without a token keep zeros for the whole kernel and never touch
     // shared memory (even a broadcast read costs wavefronts on the shared-memory pipe)
-    uint4 xr[TPW][2];
+    uint2 xr[TPW][4];
 #pragma unroll
-    for (int v = 0; v < TPW; ++v) xr[v][0] = xr[v][1] = make_uint4(0u, 0u, 0u, 0u);
+    for (int v = 0; v < TPW; ++v)
+#pragma unroll
+        for (int jw = 0; jw < 4; ++jw) xr[v][jw] = make_uint2(0u, 0u);
 
     uint32_t stage = 0, phase = 0;
     int nflush = 0;
@@ -307,10 +309,10 @@ gemv_band_kernel(const unsigned char* __restrict__ qweight, const __half* __rest
                 for (int v = 0; v < TPW; ++v) pk[v] = *reinterpret_cast<const uint4*>(st + o_w + v * 512);
                 if (tok_ok) {
 #pragma unroll
-                    for (int v = 0; v < TPW; ++v) {
-                        xr[v][0] = *reinterpret_cast<const uint4*>(st + o_x + v * 128);
-                        xr[v][1] = *reinterpret_cast<const uint4*>(st + o_x + v * 128 + 16);
-                    }
+                    for (int v = 0; v < TPW; ++v)
+#pragma unroll
+                        for (int jw = 0; jw < 4; ++jw)
+                            xr[v][jw] = *reinterpret_cast<const uint2*>(st + o_x + v * 128 + jw * 32);
                 }
                 float c[GPW][4];
 #pragma unroll
@@ -322,8 +324,7 @@ gemv_band_kernel(const unsigned char* __restrict__ qweight, const __half* __rest
                             const int tile = q * TPG + v;
                             const uint32_t w = (jw == 0) ? pk[tile].x : (jw == 1) ? pk[tile].y : (jw == 2) ? pk[tile].z : pk[tile].w;
                             const uint32_t w8 = w >> 8;
-                            const uint4 xq = xr[tile][jw >> 1];
-                            const uint32_t bb0 = (jw & 1) ? xq.z : xq.x, bb1 = (jw & 1) ? xq.w : xq.y;
+                            const uint32_t bb0 = xr[tile][jw].x, bb1 = xr[tile][jw].y;
                             if (v == 0 && jw == 0)
                                 mma_16816_first(c[q], w & 0x000F000Fu, w & 0x00F000F0u, w8 & 0x000F000Fu,
                                                 w8 & 0x00F000F0u, bb0, bb1);
@@ -361,16 +362,17 @@ gemv_band_kernel(const unsigned char* __restrict__ qweight, const __half* __rest
                         for (int v = 0; v < TPG; ++v) {
                             const int tile = q * TPG + v;
                             const uint4 pk = *reinterpret_cast<const uint4*>(st + o_w + tile * 512);
-                            uint4 xa[1] = {make_uint4(0u, 0u, 0u, 0u)}, xb[1] = {make_uint4(0u, 0u, 0u, 0u)};
+                            uint2 xq[1][4] = {{make_uint2(0u, 0u), make_uint2(0u, 0u), make_uint2(0u, 0u), make_uint2(0u, 0u)}};
                             if (tok_ok) {
-                                xa[0] = *reinterpret_cast<const uint4*>(st + o_x + tile * 128);
-                                xb[0] = *reinterpret_cast<const uint4*>(st + o_x + tile * 128 + 16);
+#pragma unroll
+                                for (int jw = 0; jw < 4; ++jw)
+                                    xq[0][jw] = *reinterpret_cast<const uint2*>(st + o_x + tile * 128 + jw * 32);
                             }
                             const float2 X = *reinterpret_cast<const float2*>(xs + tile * 8);
                             Xx += X.x;
                             Xy += X.y;
-                            if (v == 0) block_mma<1, 2, true>(pk, xa, xb, c);
-                            else block_mma<1, 2, false>(pk, xa, xb, c);
+                            if (v == 0) block_mma<1, 2, true>(pk, xq, c);
+                            else block_mma<1, 2, false>(pk, xq, c);
                         }
                         const float d_up = __half2float(*reinterpret_cast<const __half*>(st + o_sc + q * 32));
                         const float d_lo = __half2float(*reinterpret_cast<const __half*>(st + o_sc + q * 32 + 16));
@@ -619,7 +621,7 @@ gemv_splitk_kernel(const unsigned char* __restrict__ qweight, const __half* __re
 #pragma unroll
     for (int mt = 0; mt < MT; ++mt) {
         tok_ok[mt] = (mt * 8 + g) < M;
-        x_off[mt] = kXOff + (mt * 8 + g) * kXRowBytes + (kWT * half) * 128 + t * 32;
+        x_off[mt] = kXOff + (mt * 8 + g) * kXRowBytes + (kWT * half) * 128 + t * 8;
     }
 
     float acc[MT][4];
@@ -646,17 +648,15 @@ gemv_splitk_kernel(const unsigned char* __restrict__ qweight, const __half* __re
                 if (v < ntw) {
                     const int tile = kWT * half + v;                   // k-tile inside the stage
                     const uint4 pk = *reinterpret_cast<const uint4*>(st + w_off + v * 512);
-                    uint4 xa[MT], xb[MT];
+                    uint2 xq[MT][4];
 #pragma unroll
-                    for (int mt = 0; mt < MT; ++mt) {
-                        // lanes without a token must not touch shared memory (see the band kernel)
-                        xa[mt] = make_uint4(0u, 0u, 0u, 0u);
-                        xb[mt] = make_uint4(0u, 0u, 0u, 0u);
-                        if (tok_ok[mt]) {
-                            xa[mt] = *reinterpret_cast<const uint4*>(xp[mt] + v * 128);
-                            xb[mt] = *reinterpret_cast<const uint4*>(xp[mt] + v * 128 + 16);
+                    for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+                        for (int jw = 0; jw < 4; ++jw) {
+                            // lanes without a token must not touch shared memory (see the band kernel)
+                            xq[mt][jw] = make_uint2(0u, 0u);
+                            if (tok_ok[mt]) xq[mt][jw] = *reinterpret_cast<const uint2*>(xp[mt] + v * 128 + jw * 32);
                         }
-                    }
                     const int q = tile / TPG;
                     const float d_up = __half2float(*reinterpret_cast<const __half*>(st + sc_off + q * 32));
                     const float d_lo = __half2float(*reinterpret_cast<const __half*>(st + sc_off + q * 32 + 16));
@@ -664,7 +664,7 @@ gemv_splitk_kernel(const unsigned char* __restrict__ qweight, const __half* __re
                     const float su = d_up * 16777216.0f, sl = d_lo * 1048576.0f;
                     const float zu = -d_up * (float)(zb & 0xFu), zl = -d_lo * (float)(zb >> 4);
                     float c[MT][NCH][4];
-                    block_mma<MT, NCH>(pk, xa, xb, c);
+                    block_mma<MT, NCH>(pk, xq, c);
 #pragma unroll
                     for (int mt = 0; mt < MT; ++mt) {
                         const float2 X = *reinterpret_cast<const float2*>(

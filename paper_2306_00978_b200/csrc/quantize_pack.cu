@@ -2,9 +2,10 @@
 // asymmetric 4-bit round-to-nearest (Eq. 2) and the packed tile layout (Sec. 4.2).
 //
 // HBM-bound: 2 bytes read and ~0.52 bytes written per weight.  One warp owns a band of 16
-// rows x 128 columns; lane (g, t) loads rows g and g+8, columns 16t..16t+15 of both
-// 64-column tiles (eight 16-byte loads in flight per thread), which is exactly the data of
-// the two 16-byte packed pieces it writes, so no shared-memory transpose is needed.  Every
+// rows x 128 columns; lane (g, t) loads rows g and g+8, columns 16j+4t..+3 (j = 0..3) of both
+// 64-column tiles (sixteen 8-byte loads in flight per thread; the four lanes of a row read 32
+// contiguous bytes), which is exactly the data of the two 16-byte packed pieces it writes, so
+// no shared-memory transpose is needed.  Every
 // rounding point is an explicit IEEE operation (no contraction, no reciprocal).
 #include "common.cuh"
 
@@ -25,10 +26,9 @@ __global__ void channel_scale_kernel(const float* __restrict__ a, float alpha, i
     if (k < K) s[k] = channel_scale_one(mode == kAlphaZero ? 1.0f : a[k], alpha, mode);
 }
 
-__device__ __forceinline__ uint4 ldg_stream(const uint4* p) {
-    uint4 v;
-    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+__device__ __forceinline__ uint2 ldg_stream(const uint2* p) {
+    uint2 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "l"(p));
     return v;
 }
 
@@ -59,38 +59,37 @@ quantize_pack_kernel(const __half* __restrict__ W, const float* __restrict__ a, 
     const int n0 = slab * 128 + warp * 16 + g;            // this lane's upper row; lower = n0 + 8
     const int kbase = kblk * 128;
 
-    // issue the weight loads first: [tile][row h][2 x 16 bytes]
-    uint4 raw[2][2][2];
+    // issue the weight loads first: [tile][row h][word j] = columns 16j + 4t .. +3 of the tile
+    uint2 raw[2][2][4];
 #pragma unroll
     for (int ti = 0; ti < 2; ++ti)
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {
-            const uint4* p = reinterpret_cast<const uint4*>(
-                W + (size_t)(n0 + 8 * h) * K + kbase + ti * 64 + 16 * t);
-            raw[ti][h][0] = ldg_stream(p);
-            raw[ti][h][1] = ldg_stream(p + 1);
-        }
+        for (int h = 0; h < 2; ++h)
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                raw[ti][h][j] = ldg_stream(reinterpret_cast<const uint2*>(
+                    W + (size_t)(n0 + 8 * h) * K + kbase + ti * 64 + 16 * j + 4 * t));
     if (threadIdx.x < 128) {
         const int k = kbase + threadIdx.x;
         s_sm[threadIdx.x] = channel_scale_one(mode == kAlphaZero ? 1.0f : a[k], alpha, mode);
     }
     __syncthreads();
 
-    // w' = fp32(w) * s  (Eq. 3), kept in registers: [tile][row][16 columns]
+    // w' = fp32(w) * s  (Eq. 3), kept in registers: [tile][row][4 words x 4 columns]
     float wp[2][2][16];
 #pragma unroll
     for (int ti = 0; ti < 2; ++ti)
 #pragma unroll
         for (int h = 0; h < 2; ++h)
 #pragma unroll
-            for (int v = 0; v < 2; ++v) {
-                const uint32_t u[4] = {raw[ti][h][v].x, raw[ti][h][v].y, raw[ti][h][v].z, raw[ti][h][v].w};
+            for (int j = 0; j < 4; ++j) {
+                const uint32_t u[2] = {raw[ti][h][j].x, raw[ti][h][j].y};
 #pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    const int c = v * 8 + e * 2;
-                    const float s0 = s_sm[ti * 64 + 16 * t + c], s1 = s_sm[ti * 64 + 16 * t + c + 1];
-                    wp[ti][h][c] = __fmul_rn(__half2float(__ushort_as_half((unsigned short)(u[e] & 0xFFFFu))), s0);
-                    wp[ti][h][c + 1] = __fmul_rn(__half2float(__ushort_as_half((unsigned short)(u[e] >> 16))), s1);
+                for (int e = 0; e < 2; ++e) {
+                    const int c = 4 * j + 2 * e;                      // position among this lane's 16 columns
+                    const int col = ti * 64 + 16 * j + 4 * t + 2 * e; // column in the 128-column block
+                    wp[ti][h][c] = __fmul_rn(__half2float(__ushort_as_half((unsigned short)(u[e] & 0xFFFFu))), s_sm[col]);
+                    wp[ti][h][c + 1] = __fmul_rn(__half2float(__ushort_as_half((unsigned short)(u[e] >> 16))), s_sm[col + 1]);
                 }
             }
 
@@ -170,7 +169,7 @@ __global__ void unpack_kernel(const uint32_t* __restrict__ qweight, const __half
     const int band = n / 16, rr = n % 16, g = rr % 8, h = rr / 8;
     const size_t block = (size_t)band * (K / 64) + k / 64;
     const int c = k % 64;
-    const int t = c / 16, j = (c % 16) / 4, i = c % 4;
+    const int j = c / 16, t = (c % 16) / 4, i = c % 4;
     const uint32_t w = qweight[block * 128 + (g * 4 + t) * 4 + j];
     const int slot = (i / 2) * 4 + h * 2 + (i % 2);
     const int nib = (slot % 2) * 4 + slot / 2;
