@@ -26,7 +26,9 @@
 //                k-block, A from tensor memory, B through a shared-memory descriptor), commits
 //                to the stage's "empty" barrier and, after the last k-block, to the
 //                accumulator's "full" barrier.
-//   warps 4-7    epilogue: tcgen05.ld 32 columns at a time, convert to fp16, store to y.
+//   warps 4-7    epilogue: tcgen05.ld 32 columns at a time, convert to fp16, transpose through a
+//                2 KB shared-memory block to [token][channel] and store it with one TMA tensor
+//                store (two-byte global stores were an order of magnitude slower).
 //                BN <= 128 keeps two accumulators so that the epilogue overlaps the next tile.
 //
 // Tensor-memory columns: accumulators first (BN or 2 BN), then 32 columns per stage for A.
@@ -51,13 +53,14 @@ template <int BN> struct GemmCfg {
     static constexpr int kXTileBytes = BN * kBK * 2;
     static constexpr int kStageBytes = kXTileBytes + kTileBytes;          // x tile + packed weights
     static constexpr int kNumAcc = BN <= 128 ? 2 : 1;                      // accumulators in TMEM
-    static constexpr int kStagesSmem = (216 * 1024) / kStageBytes;
+    static constexpr int kOutBytes = 4 * 2 * 2048;                         // 4 epilogue warps x 2 staging buffers
+    static constexpr int kStagesSmem = (216 * 1024 - kOutBytes) / kStageBytes;
     static constexpr int kStagesTmem = (512 - kNumAcc * BN) / 32;          // 32 columns of A per stage
     static constexpr int kStagesMin = kStagesSmem < kStagesTmem ? kStagesSmem : kStagesTmem;
     static constexpr int kStages = kStagesMin > 8 ? 8 : kStagesMin;
     static constexpr int kAColumn0 = kNumAcc * BN;                         // first A column
     static constexpr int kTmemCols = 512;
-    static constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*align*/ + 256 /*barriers*/;
+    static constexpr int kSmemBytes = kStages * kStageBytes + kOutBytes + 1024 /*align*/ + 256 /*barriers*/;
     static constexpr uint32_t kTxBytes = kXTileBytes + kTileBytes;
 };
 
@@ -67,6 +70,15 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
         "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
         ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar) : "memory");
 }
+// shared -> global tensor store of one box (bulk async-group completion)
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, int c0, int c1, uint32_t src) {
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%1, %2}], [%3];"
+                 ::"l"(map), "r"(c0), "r"(c1), "r"(src) : "memory");
+}
+__device__ __forceinline__ void bulk_commit_group() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// wait until at most one / none of this thread's store groups still reads shared memory
+__device__ __forceinline__ void bulk_wait_read_1() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 __device__ __forceinline__ void fence_proxy_async_smem() {
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 }
@@ -146,12 +158,17 @@ __device__ __forceinline__ void tmem_ld_32cols(uint32_t taddr, uint32_t (&r)[32]
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
+#ifdef AWQ_DBG_TS
+__device__ unsigned long long g_dbg_ts[256 * 16];
+#endif
+
 // ------------------------------------------------------------------------- the kernel
 template <int G, int BN>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ CUtensorMap w_map,
+            const __grid_constant__ CUtensorMap y_map,
             const __half* __restrict__ scales, const unsigned char* __restrict__ zeros,
-            __half* __restrict__ y, int M, int N, int K, unsigned int* status_word) {
+            int M, int N, int K, unsigned int* status_word) {
     using Cfg = GemmCfg<BN>;
     constexpr int S = Cfg::kStages;
     constexpr int NACC = Cfg::kNumAcc;
@@ -165,7 +182,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ C
     // stage layout: [x tile | packed weights (8 bands x 512 bytes)]
     auto x_addr = [&](int s) { return base + (uint32_t)s * Cfg::kStageBytes; };
     auto w_ptr = [&](int s) { return base_ptr + (size_t)s * Cfg::kStageBytes + Cfg::kXTileBytes; };
-    const uint32_t bars = base + (uint32_t)S * Cfg::kStageBytes;       // 8-byte barriers follow the ring
+    const uint32_t out_base = base + (uint32_t)S * Cfg::kStageBytes;   // epilogue staging, then 8-byte barriers
+    const uint32_t bars = out_base + (uint32_t)Cfg::kOutBytes;
     auto raw_full = [&](int s) { return bars + 8u * (uint32_t)s; };
     auto a_full = [&](int s) { return bars + 8u * (uint32_t)(S + s); };
     auto empty = [&](int s) { return bars + 8u * (uint32_t)(2 * S + s); };
@@ -231,16 +249,34 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ C
             uint32_t stage = 0, phase = 0;
             int local = 0;
             bool ok = true;
+#ifdef AWQ_DBG_TS
+            long long w_acc = 0, w_raw = 0, w_a = 0, t_begin = clock64();
+#endif
             for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++local) {
                 const int b = local % NACC;
                 const uint32_t use = (uint32_t)(local / NACC) & 1u;
+#ifdef AWQ_DBG_TS
+                const long long q0 = clock64();
+#endif
                 if (!mbar_wait(acc_empty(b), use ^ 1u, ctl)) { ok = false; break; }
+#ifdef AWQ_DBG_TS
+                w_acc += clock64() - q0;
+#endif
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(b * BN);
                 for (int kb = 0; kb < nkb; ++kb) {
+#ifdef AWQ_DBG_TS
+                    const long long q1 = clock64();
+                    const bool okr = mbar_wait(raw_full(stage), phase, ctl);
+                    const long long q2 = clock64();
+                    const bool oka = mbar_wait(a_full(stage), phase, ctl);
+                    w_raw += q2 - q1; w_a += clock64() - q2;
+                    if (!okr || !oka) { ok = false; break; }
+#else
                     if (!mbar_wait(raw_full(stage), phase, ctl) || !mbar_wait(a_full(stage), phase, ctl)) {
                         ok = false; break;
                     }
+#endif
                     tc_fence_after();
                     const uint32_t a_tmem = tmem_base + (uint32_t)(Cfg::kAColumn0 + stage * 32);
                     const uint64_t bdesc = smem_desc_sw128(x_addr(stage));
@@ -253,6 +289,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ C
                 }
                 if (ok) umma_commit(acc_full(b));
             }
+#ifdef AWQ_DBG_TS
+            g_dbg_ts[blockIdx.x * 16 + 0] = w_acc; g_dbg_ts[blockIdx.x * 16 + 1] = w_raw;
+            g_dbg_ts[blockIdx.x * 16 + 2] = w_a; g_dbg_ts[blockIdx.x * 16 + 3] = clock64() - t_begin;
+#endif
         }
     } else if (warp >= 8) {
         // -------------------------------------------------------------- dequantizers
@@ -318,6 +358,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ C
         // ------------------------------------------------------------------ epilogue
         const int quad = warp & 3;                     // TMEM lanes 32*quad .. +31
         int local = 0;
+        int obuf = 0;
         bool ok = true;
         for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++local) {
             const int slab = tile / m_tiles, mt = tile % m_tiles;
@@ -327,7 +368,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ C
             ok = __all_sync(0xFFFFFFFFu, ok);
             if (!ok) break;
             tc_fence_after();
-            const int n = slab * 128 + quad * 32 + lane;
+            const int n0 = slab * 128 + quad * 32;
             const int m0 = mt * BN;
             const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(b * BN);
 #pragma unroll 1
@@ -335,16 +376,32 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ C
                 uint32_t r[32];
                 tmem_ld_32cols(taddr + (uint32_t)c, r);
                 tmem_ld_wait();
-#pragma unroll
-                for (int i = 0; i < 32; ++i) {
-                    const int m = m0 + c + i;
-                    if (m < M) y[(size_t)m * N + n] = __float2half_rn(__uint_as_float(r[i]));
+                if (c + 32 >= BN) {
+                    // the accumulator is in registers: the MMA thread may start the next tile
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(acc_empty(b));
                 }
+                // stage the 32 x 32 block as [token][channel] fp16 and hand it to the copy engine:
+                // one tensor store per block instead of 32 two-byte stores per thread (rows past
+                // M are clipped by the tensor map)
+                if (lane == 0) bulk_wait_read_1();                  // the store that last used this buffer
+                __syncwarp();
+                const uint32_t tb = out_base + (uint32_t)((quad * 2 + obuf) * 2048);
+                unsigned char* tp = base_ptr + (tb - base);
+#pragma unroll
+                for (int i = 0; i < 32; ++i)
+                    *reinterpret_cast<__half*>(tp + i * 64 + lane * 2) = __float2half_rn(__uint_as_float(r[i]));
+                fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) {
+                    tma_store_2d(&y_map, n0, m0 + c, tb);
+                    bulk_commit_group();
+                }
+                obuf ^= 1;
             }
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(acc_empty(b));
         }
+        if (lane == 0) bulk_wait_all();                             // all of y written before exit
     }
 
     __syncwarp();
@@ -377,8 +434,9 @@ EncodeTiledFn encode_fn() {
 }
 
 template <int G, int BN>
-cudaError_t launch_one(const CUtensorMap& map, const CUtensorMap& wmap, const void* scales, const void* zeros,
-                       void* y, int M, int N, int K, unsigned int* status_word, int sms, cudaStream_t st) {
+cudaError_t launch_one(const CUtensorMap& map, const CUtensorMap& wmap, const CUtensorMap& ymap,
+                       const void* scales, const void* zeros,
+                       int M, int N, int K, unsigned int* status_word, int sms, cudaStream_t st) {
     using Cfg = GemmCfg<BN>;
     static bool attr_done[64] = {};
     int dev = 0;
@@ -392,13 +450,19 @@ cudaError_t launch_one(const CUtensorMap& map, const CUtensorMap& wmap, const vo
     const int tiles = (N / 128) * ((M + BN - 1) / BN);
     const int grid = tiles < sms ? tiles : sms;
     gemm_kernel<G, BN><<<grid, kGemmThreads, Cfg::kSmemBytes, st>>>(
-        map, wmap, reinterpret_cast<const __half*>(scales),
-        reinterpret_cast<const unsigned char*>(zeros), reinterpret_cast<__half*>(y), M, N, K, status_word);
+        map, wmap, ymap, reinterpret_cast<const __half*>(scales),
+        reinterpret_cast<const unsigned char*>(zeros), M, N, K, status_word);
     count_launch();
     return cudaGetLastError();
 }
 
 }  // namespace
+
+#ifdef AWQ_DBG_TS
+extern "C" __attribute__((visibility("default"))) int awq_dbg_read_ts(unsigned long long* dst) {
+    return (int)cudaMemcpyFromSymbol(dst, g_dbg_ts, sizeof(g_dbg_ts));
+}
+#endif
 
 cudaError_t launch_gemm(const void* x, const void* qweight, const void* scales, const void* zeros,
                         void* y, int M, int N, int K, int group, unsigned int* status_word,
@@ -424,13 +488,22 @@ cudaError_t launch_gemm(const void* x, const void* qweight, const void* scales, 
                             wstrides, wbox, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
                             CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (rw != CUDA_SUCCESS) return cudaErrorInvalidValue;
+    // y as [M][N] fp16, stored in boxes of 32 tokens x 32 channels
+    CUtensorMap ymap;
+    const cuuint64_t ydims[2] = {(cuuint64_t)N, (cuuint64_t)M};
+    const cuuint64_t ystrides[1] = {(cuuint64_t)N * 2};
+    const cuuint32_t ybox[2] = {32, 32};
+    const CUresult ry = enc(&ymap, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, y, ydims, ystrides, ybox, estr,
+                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+                            CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (ry != CUDA_SUCCESS) return cudaErrorInvalidValue;
     int dev = 0, sms = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
     e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     if (e != cudaSuccess) return e;
 #define AWQ_GEMM_CASE(GG, BNN) \
-    return launch_one<GG, BNN>(map, wmap, scales, zeros, y, M, N, K, status_word, sms, st)
+    return launch_one<GG, BNN>(map, wmap, ymap, scales, zeros, M, N, K, status_word, sms, st)
     if (group == 128) {
         switch (bn) { case 256: AWQ_GEMM_CASE(128, 256); case 128: AWQ_GEMM_CASE(128, 128);
                       case 64: AWQ_GEMM_CASE(128, 64); default: AWQ_GEMM_CASE(128, 32); }
