@@ -110,6 +110,26 @@ int awq_channel_scale(const float* act_mean_abs, float alpha, float* s, int K, v
 int awq_linear(const void* x, const void* qweight, const void* scales, const void* zeros,
                void* y, int M, int N, int K, int group, void* stream);
 
+/*
+ * Several layers that read the same x in one call (Sec. 4.2, kernel fusion: the paper fuses the
+ * Q, K and V projections into a single kernel because at batch 1 a kernel's run time is
+ * comparable to its launch overhead).  y_i = x . dequant(Wq_i)^T for i < count, count <= 4; all
+ * matrices share K and `group`, each has its own N.  `problems` is a HOST array read during the
+ * call.  For M <= 4 with enough output rows in total the matrices are served by ONE launch of
+ * the matrix-vector band kernel; otherwise this is the same as `count` awq_linear calls.  Each
+ * output is what awq_linear would give with the band kernel (bit-identical when awq_linear picks
+ * that kernel for the matrix on its own, within the usual tolerance otherwise).
+ */
+typedef struct AwqLinearProblem {
+    const void* qweight;   /* packed weights of matrix i (device) */
+    const void* scales;
+    const void* zeros;
+    void* y;               /* out, fp16 [M][N] (device) */
+    int N;
+} AwqLinearProblem;
+int awq_linear_multi(const void* x, const AwqLinearProblem* problems, int count,
+                     int M, int K, int group, void* stream);
+
 /* Same as awq_linear with the kernel forced (for the small-batch crossover measurement).
  * A matrix-vector path with M > 16 or K > 65536 returns AWQ_ERR_BAD_SHAPE. */
 int awq_linear_path(const void* x, const void* qweight, const void* scales, const void* zeros,

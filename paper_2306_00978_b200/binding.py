@@ -22,7 +22,13 @@ EXPORTS = (
     "awq_channel_scale", "awq_linear", "awq_linear_path", "awq_workspace_bytes",
     "awq_set_workspace", "awq_unpack_canonical", "awq_poll_status", "awq_status_string",
     "awq_last_cuda_error", "awq_layout_version", "awq_launch_count", "awq_linear_gemv_static",
+    "awq_linear_multi",
 )
+
+
+class _Problem(ctypes.Structure):
+    _fields_ = [("qweight", ctypes.c_void_p), ("scales", ctypes.c_void_p), ("zeros", ctypes.c_void_p),
+                ("y", ctypes.c_void_p), ("N", ctypes.c_int)]
 
 _lib = None
 _workspace: dict = {}          # device index -> torch tensor registered with the library
@@ -49,6 +55,7 @@ def lib() -> ctypes.CDLL:
     L.awq_linear.restype, L.awq_linear.argtypes = i, [vp, vp, vp, vp, vp, i, i, i, i, vp]
     L.awq_linear_path.restype, L.awq_linear_path.argtypes = i, [vp, vp, vp, vp, vp, i, i, i, i, i, vp]
     L.awq_linear_gemv_static.restype, L.awq_linear_gemv_static.argtypes = i, [vp, vp, vp, vp, vp, i, i, i, i, vp]
+    L.awq_linear_multi.restype, L.awq_linear_multi.argtypes = i, [vp, vp, i, i, i, i, vp]
     L.awq_workspace_bytes.restype, L.awq_workspace_bytes.argtypes = sz, [i, i, i, i]
     L.awq_set_workspace.restype, L.awq_set_workspace.argtypes = i, [vp, sz]
     L.awq_unpack_canonical.restype, L.awq_unpack_canonical.argtypes = i, [vp, vp, vp, i, i, i, vp, vp, vp, vp]
@@ -152,6 +159,26 @@ def linear(x: torch.Tensor, qweight: torch.Tensor, scales: torch.Tensor, zeros: 
         rc = lib().awq_linear_path(*args, int(path), _stream())
     _check(rc, "awq_linear")
     return y
+
+
+def linear_multi(x: torch.Tensor, mats, K: int, group: int, outs=None):
+    """awq_linear_multi: several packed matrices that read the same x (fused q/k/v or gate/up), one
+    call.  `mats` is a list of (qweight, scales, zeros, N); returns the list of outputs."""
+    M = x.shape[0]
+    if x.shape[1] != K:
+        raise AwqError("x must be [M][K]")
+    if outs is None:
+        outs = [torch.empty((M, m[3]), dtype=torch.float16, device=x.device) for m in mats]
+    if M <= 16:
+        ensure_workspace(max(workspace_bytes(M, m[3], K, group) for m in mats))
+    arr = (_Problem * len(mats))()
+    for k, ((qw, sc, zp, N), y) in enumerate(zip(mats, outs)):
+        arr[k] = _Problem(_dev(qw, torch.uint8, "qweight"), _dev(sc, torch.float16, "scales"),
+                          _dev(zp, torch.uint8, "zeros"), _dev(y, torch.float16, "y"), int(N))
+    rc = lib().awq_linear_multi(_dev(x, torch.float16, "x"), ctypes.byref(arr), len(mats), M, K, int(group),
+                                _stream())
+    _check(rc, "awq_linear_multi")
+    return outs
 
 
 def linear_gemv_static(x: torch.Tensor, qweight: torch.Tensor, scales: torch.Tensor, zeros: torch.Tensor,

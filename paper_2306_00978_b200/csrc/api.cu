@@ -157,9 +157,10 @@ int awq_linear_path(const void* x, const void* qweight, const void* scales, cons
     DeviceState* d;
     if (int rc = device_state(&d)) return rc;
     const cudaStream_t st = (cudaStream_t)stream;
-    if (path == AWQ_PATH_GEMV && gemv_uses_band_kernel(M, N, d->sms))
-        return note_cuda(launch_gemv_band(x, qweight, scales, zeros, y, M, N, K, group, d->status_word,
-                                          d->sms, st));
+    if (path == AWQ_PATH_GEMV && gemv_uses_band_kernel(M, N, d->sms)) {
+        const GemvMatrix one = {qweight, scales, zeros, y, N};
+        return note_cuda(launch_gemv_band(x, &one, 1, M, K, group, d->status_word, d->sms, st));
+    }
     if (path == AWQ_PATH_GEMV || path == AWQ_PATH_GEMV_SPLITK) {
         void* ws = nullptr;
         {
@@ -190,6 +191,39 @@ int awq_linear_gemv_static(const void* x, const void* qweight, const void* scale
     if (int rc = note_cuda(cudaMemsetAsync(scratch, 0, kCounterBytes, st))) return rc;
     return note_cuda(launch_gemv_splitk(x, qweight, scales, zeros, y, M, N, K, group, scratch,
                                         d->status_word, d->sms, st));
+}
+
+int awq_linear_multi(const void* x, const AwqLinearProblem* problems, int count,
+                     int M, int K, int group, void* stream) {
+    if (!problems || !x) return AWQ_ERR_NULL_POINTER;
+    if (count < 1 || count > kMaxMulti) return AWQ_ERR_BAD_ARGUMENT;
+    int total_n = 0;
+    for (int i = 0; i < count; ++i) {
+        const AwqLinearProblem& p = problems[i];
+        if (int rc = check_shape(p.N, K, group)) return rc;
+        if (!p.qweight || !p.scales || !p.zeros || !p.y) return AWQ_ERR_NULL_POINTER;
+        if (!aligned16(p.qweight) || !aligned16(p.scales) || !aligned16(p.zeros) || !aligned16(p.y))
+            return AWQ_ERR_MISALIGNED;
+        total_n += p.N;
+    }
+    if (M < 1) return AWQ_ERR_BAD_SHAPE;
+    if (!aligned16(x)) return AWQ_ERR_MISALIGNED;
+    DeviceState* d;
+    if (int rc = device_state(&d)) return rc;
+    if (M <= 8 && K <= 65536 && gemv_uses_band_kernel(M, total_n, d->sms)) {
+        GemvMatrix mats[kMaxMulti];
+        for (int i = 0; i < count; ++i)
+            mats[i] = GemvMatrix{problems[i].qweight, problems[i].scales, problems[i].zeros, problems[i].y,
+                                 problems[i].N};
+        return note_cuda(launch_gemv_band(x, mats, count, M, K, group, d->status_word, d->sms,
+                                          (cudaStream_t)stream));
+    }
+    // otherwise one call per matrix, as awq_linear would run it
+    for (int i = 0; i < count; ++i) {
+        const AwqLinearProblem& p = problems[i];
+        if (int rc = awq_linear(x, p.qweight, p.scales, p.zeros, p.y, M, p.N, K, group, stream)) return rc;
+    }
+    return AWQ_OK;
 }
 
 int awq_linear(const void* x, const void* qweight, const void* scales, const void* zeros,

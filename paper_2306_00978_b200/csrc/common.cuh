@@ -38,11 +38,19 @@ constexpr int kGemvMaxBlocks = 256;      // upper bound on the split-K matrix-ve
 
 // Matrix-vector kernels.  The band kernel needs no workspace; the split-K kernel needs
 // gemv_workspace_bytes(M): arrival counters + two fp32 partial-sum slots per block.
+constexpr int kMaxMulti = 4;             // matrices that one band-kernel launch can serve
+struct GemvMatrix {                      // one packed weight matrix and its output
+    const void* qweight;
+    const void* scales;
+    const void* zeros;
+    void* y;
+    int n;
+};
 bool gemv_uses_band_kernel(int M, int N, int sms);
 size_t gemv_workspace_bytes(int M);
-cudaError_t launch_gemv_band(const void* x, const void* qweight, const void* scales, const void* zeros,
-                             void* y, int M, int N, int K, int group, unsigned int* status_word, int sms,
-                             cudaStream_t st);
+// `count` matrices (1..kMaxMulti) sharing x, K and the group size, in one launch
+cudaError_t launch_gemv_band(const void* x, const GemvMatrix* mats, int count, int M, int K, int group,
+                             unsigned int* status_word, int sms, cudaStream_t st);
 cudaError_t launch_gemv_splitk(const void* x, const void* qweight, const void* scales, const void* zeros,
                                void* y, int M, int N, int K, int group, void* workspace,
                                unsigned int* status_word, int sms, cudaStream_t st);

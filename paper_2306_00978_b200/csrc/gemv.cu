@@ -152,6 +152,38 @@ template <int G, int TPW> struct BandStage {
 struct BandLayout {
     int stage_bytes, stages, xsum_off, red_off, bar_off, total;
 };
+
+// Up to four weight matrices that share x, K and the group size (fused q/k/v or gate/up
+// projections): their 16-row bands form one task list for one launch.
+struct BandProblems {
+    const unsigned char* qweight[kMaxMulti];
+    const __half* scales[kMaxMulti];
+    const unsigned char* zeros[kMaxMulti];
+    __half* y[kMaxMulti];
+    int n[kMaxMulti];            // output channels of each matrix
+    int first_band[kMaxMulti + 1];
+    int count;
+};
+struct BandRef {                 // one task: matrix, band inside it
+    const unsigned char* qweight;
+    const __half* scales;
+    const unsigned char* zeros;
+    __half* y;
+    int n, band;
+};
+__device__ __forceinline__ BandRef band_ref(const BandProblems& pr, int task) {
+    int p = 0;
+#pragma unroll
+    for (int i = 1; i < kMaxMulti; ++i)
+        if (i < pr.count && task >= pr.first_band[i]) p = i;
+    BandRef r;
+    r.qweight = pr.qweight[0]; r.scales = pr.scales[0]; r.zeros = pr.zeros[0]; r.y = pr.y[0]; r.n = pr.n[0];
+#pragma unroll
+    for (int i = 1; i < kMaxMulti; ++i)
+        if (p == i) { r.qweight = pr.qweight[i]; r.scales = pr.scales[i]; r.zeros = pr.zeros[i]; r.y = pr.y[i]; r.n = pr.n[i]; }
+    r.band = task - pr.first_band[p];
+    return r;
+}
 template <int G, int TPW>
 inline BandLayout band_layout(int M, int K) {
     using St = BandStage<G, TPW>;
@@ -171,10 +203,8 @@ inline BandLayout band_layout(int M, int K) {
 // TPW = k-tiles per math warp and stage (stage = 16 * TPW k-tiles).  M <= 8 tokens (one token tile).
 template <int G, int TPW>
 __global__ void __launch_bounds__(kBandThreads, 1)
-gemv_band_kernel(const unsigned char* __restrict__ qweight, const __half* __restrict__ scales,
-                 const unsigned char* __restrict__ zeros, const __half* __restrict__ x,
-                 __half* __restrict__ y, int M, int N, int K, const BandLayout lay,
-                 unsigned int* status_word) {
+gemv_band_kernel(const BandProblems probs, const __half* __restrict__ x, int M, int K,
+                 const BandLayout lay, unsigned int* status_word) {
     extern __shared__ __align__(128) unsigned char smem[];
     __shared__ unsigned int s_abort;
     using St = BandStage<G, TPW>;
@@ -189,7 +219,7 @@ gemv_band_kernel(const unsigned char* __restrict__ qweight, const __half* __rest
 
     const int ktiles = K / 64, ng = K / G;
     const int upb = (ktiles + UT - 1) / UT;                           // units per band
-    const int nbands = N / 16;
+    const int nbands = probs.first_band[probs.count];
     const int b0 = (int)(((unsigned)nbands * blockIdx.x) / gridDim.x);
     const int b1 = (int)(((unsigned)nbands * (blockIdx.x + 1)) / gridDim.x);
 
@@ -211,7 +241,9 @@ gemv_band_kernel(const unsigned char* __restrict__ qweight, const __half* __rest
         // ------------------------------------------------------------------ copy warp
         // lane 0 posts the byte count; lanes 0, 1, 2 and 3 .. 3+M-1 each issue one bulk copy
         uint32_t stage = 0, phase = 0;
-        for (int band = b0; band < b1; ++band) {
+        for (int task = b0; task < b1; ++task) {
+            const BandRef br = band_ref(probs, task);
+            const int band = br.band;
             for (int j = 0; j < upb; ++j) {
                 const int kt = j * UT;
                 const int nt = min(UT, ktiles - kt);
@@ -225,11 +257,11 @@ gemv_band_kernel(const unsigned char* __restrict__ qweight, const __half* __rest
                 __syncwarp();
                 const int gi0 = kt * 64 / G;
                 if (lane == 0)
-                    bulk_load(dst, qweight + ((size_t)band * ktiles + kt) * 512, (uint32_t)(nt * 512), bar);
+                    bulk_load(dst, br.qweight + ((size_t)band * ktiles + kt) * 512, (uint32_t)(nt * 512), bar);
                 else if (lane == 1)
-                    bulk_load(dst + St::kScOff, scales + ((size_t)band * ng + gi0) * 16, (uint32_t)(ngr * 32), bar);
+                    bulk_load(dst + St::kScOff, br.scales + ((size_t)band * ng + gi0) * 16, (uint32_t)(ngr * 32), bar);
                 else if (lane == 2)
-                    bulk_load(dst + St::kZOff, zeros + ((size_t)(band >> 1) * ng + gi0) * 16, (uint32_t)(ngr * 16), bar);
+                    bulk_load(dst + St::kZOff, br.zeros + ((size_t)(band >> 1) * ng + gi0) * 16, (uint32_t)(ngr * 16), bar);
                 else if (lane - 3 < M)
                     bulk_load(dst + St::kXOff + (lane - 3) * St::kXRow, x + (size_t)(lane - 3) * K + (size_t)kt * 64,
                               (uint32_t)(nt * 128), bar);
@@ -257,7 +289,8 @@ gemv_band_kernel(const unsigned char* __restrict__ qweight, const __half* __rest
     if (warp == kMathWarps + 1) {
         // ------------------------------------------------------------------ flush warp
         int nflush = 0;
-        for (int band = b0; band < b1; ++band, ++nflush) {
+        for (int task = b0; task < b1; ++task, ++nflush) {
+            const BandRef br = band_ref(probs, task);
             const uint32_t b = (uint32_t)nflush & 1u, use = ((uint32_t)nflush >> 1) & 1u;
             mbar_wait_relaxed(bars + 128u + 8u * b, use, ctl);
             const float* rb = red + b * (kMathWarps * 8 * 16);
@@ -265,7 +298,7 @@ gemv_band_kernel(const unsigned char* __restrict__ qweight, const __half* __rest
                 float sum = 0.0f;
 #pragma unroll
                 for (int w = 0; w < kMathWarps; ++w) sum += rb[w * 128 + idx];
-                y[(size_t)(idx >> 4) * N + band * 16 + (idx & 15)] = __float2half_rn(sum);
+                br.y[(size_t)(idx >> 4) * br.n + br.band * 16 + (idx & 15)] = __float2half_rn(sum);
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(bars + 144u + 8u * b);
@@ -293,9 +326,10 @@ gemv_band_kernel(const unsigned char* __restrict__ qweight, const __half* __rest
 
     uint32_t stage = 0, phase = 0;
     int nflush = 0;
-    for (int band = b0; band < b1; ++band, ++nflush) {
+    for (int task = b0; task < b1; ++task, ++nflush) {
         float acc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-        const int o_z = St::kZOff + warp * (GPW * 16) + (band & 1) * 8 + g;
+        // odd bands of a matrix use the upper 8 bytes of the pair's zero-point block
+        const int o_z = St::kZOff + warp * (GPW * 16) + (band_ref(probs, task).band & 1) * 8 + g;
         for (int j = 0; j < upb; ++j) {
             const int nt = min(UT, ktiles - j * UT) - warp * TPW;     // this warp's tiles: <= 0 .. TPW
             mbar_wait(bars + 8u * stage, phase, ctl);
@@ -758,10 +792,23 @@ cudaError_t gemv_static_scratch(void** out) {
     return cudaSuccess;
 }
 
-cudaError_t launch_gemv_band(const void* x, const void* qweight, const void* scales, const void* zeros,
-                             void* y, int M, int N, int K, int group, unsigned int* status_word, int sms,
-                             cudaStream_t st) {
-    const int bands = N / 16;
+cudaError_t launch_gemv_band(const void* x, const GemvMatrix* mats, int count, int M, int K, int group,
+                             unsigned int* status_word, int sms, cudaStream_t st) {
+    BandProblems pr;
+    pr.count = count;
+    int bands = 0;
+    for (int i = 0; i < kMaxMulti; ++i) {
+        const GemvMatrix& m = mats[i < count ? i : 0];
+        pr.qweight[i] = reinterpret_cast<const unsigned char*>(m.qweight);
+        pr.scales[i] = reinterpret_cast<const __half*>(m.scales);
+        pr.zeros[i] = reinterpret_cast<const unsigned char*>(m.zeros);
+        pr.y[i] = reinterpret_cast<__half*>(m.y);
+        pr.n[i] = m.n;
+        pr.first_band[i] = bands;
+        if (i < count) bands += m.n / 16;
+    }
+    pr.first_band[kMaxMulti] = bands;
+    for (int i = count; i <= kMaxMulti; ++i) pr.first_band[i] = bands;
     const int blocks = bands < sms ? bands : sms;
     const int tpw = M <= 2 ? 4 : 2;                            // 64 or 32 k-tiles per stage
     cudaError_t e = cudaSuccess;
@@ -773,9 +820,7 @@ cudaError_t launch_gemv_band(const void* x, const void* qweight, const void* sca
         e = allow_big_smem(gemv_band_kernel<GG, TT>, done);                                          \
         if (e != cudaSuccess) return e;                                                              \
         gemv_band_kernel<GG, TT><<<blocks, kBandThreads, lay.total, st>>>(                           \
-            reinterpret_cast<const unsigned char*>(qweight), reinterpret_cast<const __half*>(scales), \
-            reinterpret_cast<const unsigned char*>(zeros), reinterpret_cast<const __half*>(x),       \
-            reinterpret_cast<__half*>(y), M, N, K, lay, status_word);                                \
+            pr, reinterpret_cast<const __half*>(x), M, K, lay, status_word);                         \
     } while (0)
     if (group == 128) { if (tpw == 4) AWQ_BAND_LAUNCH(128, 4); else AWQ_BAND_LAUNCH(128, 2); }
     else              { if (tpw == 4) AWQ_BAND_LAUNCH(64, 4);  else AWQ_BAND_LAUNCH(64, 2); }

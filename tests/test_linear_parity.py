@@ -83,6 +83,29 @@ def test_auto_dispatch_and_special_values():
         assert np.allclose(y[:, 200], ref[:, 200], rtol=2e-3, atol=1e-5)
 
 
+@pytest.mark.parametrize("M,G", [(1, 128), (3, 64)])
+def test_multi_matrix_call(M, G):
+    """awq_linear_multi: three matrices reading the same x in one launch; each output against
+    the oracle, and bit-equal to the single call where that also runs the band kernel."""
+    import torch
+    from paper_2306_00978_b200 import binding
+    K = 1152
+    cases = [Case(6000 + i, N, K, M, G, 0.5) for i, N in enumerate((1024, 2432, 1280))]
+    x = cases[0].x                                    # one shared activation
+    mats = []
+    for c in cases:
+        qw, sc, zp = oracle_packed_to_cuda(c)
+        mats.append((qw, sc, zp, c.N))
+    ys = binding.linear_multi(to_cuda(x), mats, K, G)
+    binding.poll_status()
+    from oracle import awq_oracle as orc
+    for c, y, m in zip(cases, ys, mats):
+        ref = orc.linear(x, orc.dequantize(c.codes, c.zeros, c.scales, G))
+        assert_parity(y.cpu().numpy(), ref, f"multi N={c.N}")
+    single = binding.linear(to_cuda(x), *mats[1][:3], mats[1][3], K, G, path=binding.PATH_GEMV)
+    assert torch.equal(single, ys[1])                 # N = 2432 runs the band kernel on its own too
+
+
 def test_end_to_end_quantize_then_linear():
     """The product path end to end: GPU quantize+pack feeding the GPU linear layer."""
     from paper_2306_00978_b200 import binding
