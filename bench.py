@@ -3,8 +3,9 @@
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
 
-One step = the seven linear layers of one Llama-2-7B-shaped decoder layer at M = 1 (decode),
-each a single awq_linear call on packed INT4 weights resident in HBM; the step's weights
+One step = the seven linear layers of one Llama-2-7B-shaped decoder layer at M = 1 (decode)
+on packed INT4 weights resident in HBM, issued as four C-ABI calls (fused q/k/v, o, fused
+gate/up, down) and replayed as a CUDA graph; the step's weights
 rotate over several independently seeded layers so that consecutive steps never find their
 weights in L2.  The headline value is the algorithmic GB/s of that step (packed codes +
 scales + zero points + activations in and out, each moved once).  The same JSON line also
