@@ -85,15 +85,7 @@ __device__ __forceinline__ void fence_proxy_async_smem() {
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
-__device__ __forceinline__ void umma_f16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
-                                         uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
-}
-// the same with the A operand in tensor memory (128 lanes x 8 columns of fp16 pairs per K = 16)
+// D (tensor memory) += A (tensor memory: 128 lanes x 8 columns of fp16 pairs per K = 16) * B (smem)
 __device__ __forceinline__ void umma_f16_a_tmem(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
                                                 uint32_t accumulate) {
     asm volatile(
@@ -157,10 +149,6 @@ __device__ __forceinline__ void tmem_ld_32cols(uint32_t taddr, uint32_t (&r)[32]
         : "r"(taddr) : "memory");
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-
-#ifdef AWQ_DBG_TS
-__device__ unsigned long long g_dbg_ts[256 * 16];
-#endif
 
 // ------------------------------------------------------------------------- the kernel
 template <int G, int BN>
@@ -249,34 +237,16 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ C
             uint32_t stage = 0, phase = 0;
             int local = 0;
             bool ok = true;
-#ifdef AWQ_DBG_TS
-            long long w_acc = 0, w_raw = 0, w_a = 0, t_begin = clock64();
-#endif
             for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++local) {
                 const int b = local % NACC;
                 const uint32_t use = (uint32_t)(local / NACC) & 1u;
-#ifdef AWQ_DBG_TS
-                const long long q0 = clock64();
-#endif
                 if (!mbar_wait(acc_empty(b), use ^ 1u, ctl)) { ok = false; break; }
-#ifdef AWQ_DBG_TS
-                w_acc += clock64() - q0;
-#endif
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(b * BN);
                 for (int kb = 0; kb < nkb; ++kb) {
-#ifdef AWQ_DBG_TS
-                    const long long q1 = clock64();
-                    const bool okr = mbar_wait(raw_full(stage), phase, ctl);
-                    const long long q2 = clock64();
-                    const bool oka = mbar_wait(a_full(stage), phase, ctl);
-                    w_raw += q2 - q1; w_a += clock64() - q2;
-                    if (!okr || !oka) { ok = false; break; }
-#else
                     if (!mbar_wait(raw_full(stage), phase, ctl) || !mbar_wait(a_full(stage), phase, ctl)) {
                         ok = false; break;
                     }
-#endif
                     tc_fence_after();
                     const uint32_t a_tmem = tmem_base + (uint32_t)(Cfg::kAColumn0 + stage * 32);
                     const uint64_t bdesc = smem_desc_sw128(x_addr(stage));
@@ -289,10 +259,6 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ C
                 }
                 if (ok) umma_commit(acc_full(b));
             }
-#ifdef AWQ_DBG_TS
-            g_dbg_ts[blockIdx.x * 16 + 0] = w_acc; g_dbg_ts[blockIdx.x * 16 + 1] = w_raw;
-            g_dbg_ts[blockIdx.x * 16 + 2] = w_a; g_dbg_ts[blockIdx.x * 16 + 3] = clock64() - t_begin;
-#endif
         }
     } else if (warp >= 8) {
         // -------------------------------------------------------------- dequantizers
@@ -457,12 +423,6 @@ cudaError_t launch_one(const CUtensorMap& map, const CUtensorMap& wmap, const CU
 }
 
 }  // namespace
-
-#ifdef AWQ_DBG_TS
-extern "C" __attribute__((visibility("default"))) int awq_dbg_read_ts(unsigned long long* dst) {
-    return (int)cudaMemcpyFromSymbol(dst, g_dbg_ts, sizeof(g_dbg_ts));
-}
-#endif
 
 cudaError_t launch_gemm(const void* x, const void* qweight, const void* scales, const void* zeros,
                         void* y, int M, int N, int K, int group, unsigned int* status_word,
