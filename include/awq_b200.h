@@ -63,8 +63,11 @@ typedef enum AwqPath {
     AWQ_PATH_AUTO = 0,          /* what awq_linear does: chosen from M */
     AWQ_PATH_GEMV = 1,          /* fused dequant matrix-vector kernel, M <= 16: band kernel when
                                    M <= 4 and N/16 is not much below the SM count, else split-K */
-    AWQ_PATH_GEMM = 2,          /* tcgen05 tensor-core kernel, any M >= 1 */
-    AWQ_PATH_GEMV_SPLITK = 3    /* the split-K matrix-vector kernel, M <= 16 */
+    AWQ_PATH_GEMM = 2,          /* tcgen05 tensor-core kernel, any M >= 1: pairs of SMs
+                                   (cta_group::2, 256 channels x 256 tokens per tile) when
+                                   M > 128 and N is a multiple of 256, else one SM per tile */
+    AWQ_PATH_GEMV_SPLITK = 3,   /* the split-K matrix-vector kernel, M <= 16 */
+    AWQ_PATH_GEMM_1SM = 4       /* the tensor-core kernel with one SM per tile, any M >= 1 */
 } AwqPath;
 
 /* Sizes of the packed arrays, in bytes (0 if the shape is not accepted). */

@@ -15,7 +15,7 @@ import torch
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libawq_b200.so")
 
-PATH_AUTO, PATH_GEMV, PATH_GEMM, PATH_GEMV_SPLITK = 0, 1, 2, 3
+PATH_AUTO, PATH_GEMV, PATH_GEMM, PATH_GEMV_SPLITK, PATH_GEMM_1SM = 0, 1, 2, 3, 4
 
 EXPORTS = (
     "awq_qweight_bytes", "awq_scales_bytes", "awq_zeros_bytes", "awq_quantize_pack",
@@ -148,7 +148,7 @@ def linear(x: torch.Tensor, qweight: torch.Tensor, scales: torch.Tensor, zeros: 
     if x.shape[1] != K:
         raise AwqError("x must be [M][K]")
     y = out if out is not None else torch.empty((M, N), dtype=torch.float16, device=x.device)
-    if M <= 16 and path != PATH_GEMM:
+    if M <= 16 and path not in (PATH_GEMM, PATH_GEMM_1SM):
         ensure_workspace(workspace_bytes(M, N, K, group))
     args = (_dev(x, torch.float16, "x"), _dev(qweight, torch.uint8, "qweight"),
             _dev(scales, torch.float16, "scales"), _dev(zeros, torch.uint8, "zeros"),

@@ -150,10 +150,12 @@ int awq_linear_path(const void* x, const void* qweight, const void* scales, cons
     if (!x || !qweight || !scales || !zeros || !y) return AWQ_ERR_NULL_POINTER;
     if (!aligned16(x) || !aligned16(qweight) || !aligned16(scales) || !aligned16(zeros) || !aligned16(y))
         return AWQ_ERR_MISALIGNED;
-    if (path != AWQ_PATH_AUTO && path != AWQ_PATH_GEMV && path != AWQ_PATH_GEMM && path != AWQ_PATH_GEMV_SPLITK)
+    if (path != AWQ_PATH_AUTO && path != AWQ_PATH_GEMV && path != AWQ_PATH_GEMM && path != AWQ_PATH_GEMV_SPLITK &&
+        path != AWQ_PATH_GEMM_1SM)
         return AWQ_ERR_BAD_ARGUMENT;
     path = resolve_path(M, K, path);
-    if (path != AWQ_PATH_GEMM && (M > 16 || K > 65536)) return AWQ_ERR_BAD_SHAPE;
+    const bool tensor_path = path == AWQ_PATH_GEMM || path == AWQ_PATH_GEMM_1SM;
+    if (!tensor_path && (M > 16 || K > 65536)) return AWQ_ERR_BAD_SHAPE;
     DeviceState* d;
     if (int rc = device_state(&d)) return rc;
     const cudaStream_t st = (cudaStream_t)stream;
@@ -171,7 +173,8 @@ int awq_linear_path(const void* x, const void* qweight, const void* scales, cons
         return note_cuda(launch_gemv_splitk(x, qweight, scales, zeros, y, M, N, K, group, ws, d->status_word,
                                             d->sms, st));
     }
-    return note_cuda(launch_gemm(x, qweight, scales, zeros, y, M, N, K, group, d->status_word, st));
+    return note_cuda(launch_gemm(x, qweight, scales, zeros, y, M, N, K, group, path != AWQ_PATH_GEMM_1SM,
+                                 d->status_word, st));
 }
 
 int awq_linear_gemv_static(const void* x, const void* qweight, const void* scales, const void* zeros,

@@ -60,7 +60,7 @@ cudaError_t gemv_static_scratch(void** out);
 int gemv_static_max_m();
 
 cudaError_t launch_gemm(const void* x, const void* qweight, const void* scales, const void* zeros,
-                        void* y, int M, int N, int K, int group, unsigned int* status_word,
-                        cudaStream_t st);
+                        void* y, int M, int N, int K, int group, bool path_pair_allowed,
+                        unsigned int* status_word, cudaStream_t st);
 
 }  // namespace awq

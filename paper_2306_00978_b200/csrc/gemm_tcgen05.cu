@@ -35,19 +35,13 @@
 // Every wait is bounded (about two seconds of wall clock): a wait that runs out writes a code to
 // the status word, raises a block-wide flag, and every role leaves its loop; the block
 // then waits (bounded) for its own copies in flight, frees its tensor memory and returns.
-#include <cuda.h>
-
-#include <mutex>
-
-#include "async_copy.cuh"
-#include "common.cuh"
+#include "tcgen05.cuh"
 
 namespace awq {
 
 namespace {
 
 constexpr int kGemmThreads = 512;
-constexpr int kBK = 64;
 
 template <int BN> struct GemmCfg {
     static constexpr int kXTileBytes = BN * kBK * 2;
@@ -63,92 +57,6 @@ template <int BN> struct GemmCfg {
     static constexpr int kSmemBytes = kStages * kStageBytes + kOutBytes + 1024 /*align*/ + 256 /*barriers*/;
     static constexpr uint32_t kTxBytes = kXTileBytes + kTileBytes;
 };
-
-// ------------------------------------------------------------------ small PTX wrappers
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar) : "memory");
-}
-// shared -> global tensor store of one box (bulk async-group completion)
-__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, int c0, int c1, uint32_t src) {
-    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%1, %2}], [%3];"
-                 ::"l"(map), "r"(c0), "r"(c1), "r"(src) : "memory");
-}
-__device__ __forceinline__ void bulk_commit_group() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
-// wait until at most one / none of this thread's store groups still reads shared memory
-__device__ __forceinline__ void bulk_wait_read_1() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
-__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
-__device__ __forceinline__ void fence_proxy_async_smem() {
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-}
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-
-// D (tensor memory) += A (tensor memory: 128 lanes x 8 columns of fp16 pairs per K = 16) * B (smem)
-__device__ __forceinline__ void umma_f16_a_tmem(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
-                                                uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
-}
-// A warp stores 16 lanes x 32 columns: four blocks of 8 columns, each in the 16x256b register
-// layout (lane-group g = lane / 4 holds rows g and g+8; t = lane % 4 holds columns 2t, 2t+1 of
-// the block; registers 4i .. 4i+3 of block i = (g, 2t) (g, 2t+1) (g+8, 2t) (g+8, 2t+1)).
-__device__ __forceinline__ void tmem_st_16x32cols(uint32_t taddr, const uint32_t (&v)[16]) {
-    asm volatile(
-        "tcgen05.st.sync.aligned.16x256b.x4.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, "
-        "%14, %15, %16};"
-        ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]),
-          "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15])
-        : "memory");
-}
-__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
-__device__ __forceinline__ void umma_commit(uint32_t bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-
-// Shared-memory matrix descriptor: K-major operand, 128-byte swizzle, rows of 128 bytes,
-// 8-row atoms 1024 bytes apart.
-__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
-    uint64_t d = 0;
-    d |= (uint64_t)((addr & 0x3FFFFu) >> 4);          // start address, 16-byte units
-    d |= (uint64_t)1 << 16;                           // leading byte offset (unused for swizzled K-major)
-    d |= (uint64_t)(1024 >> 4) << 32;                 // stride byte offset between 8-row atoms
-    d |= (uint64_t)1 << 46;                           // descriptor version (sm_100)
-    d |= (uint64_t)2 << 61;                           // layout: 128-byte swizzle
-    return d;
-}
-
-// Instruction descriptor: D fp32, A and B fp16, both K-major, M = 128, N = BN.
-__host__ __device__ constexpr uint32_t instr_desc(int bn) {
-    return (1u << 4) | (0u << 7) | (0u << 10) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
-}
-
-__device__ __forceinline__ uint32_t hsub2_u32(uint32_t a, uint32_t b) {
-    uint32_t d; asm("sub.rn.f16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b)); return d;
-}
-__device__ __forceinline__ uint32_t hfma2_u32(uint32_t a, uint32_t b, uint32_t c) {
-    uint32_t d; asm("fma.rn.f16x2 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c)); return d;
-}
-__device__ __forceinline__ uint32_t hmul2_u32(uint32_t a, uint32_t b) {
-    uint32_t d; asm("mul.rn.f16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b)); return d;
-}
-
-__device__ __forceinline__ void tmem_ld_32cols(uint32_t taddr, uint32_t (&r)[32]) {
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
-          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
-          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-        : "r"(taddr) : "memory");
-}
-__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 // ------------------------------------------------------------------------- the kernel
 template <int G, int BN>
@@ -381,24 +289,6 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ C
 }
 
 // ------------------------------------------------------------------------------ host
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
-                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
-                                  CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn() {
-    static EncodeTiledFn fn = nullptr;
-    static std::once_flag once;
-    std::call_once(once, [] {
-        void* p = nullptr;
-        cudaDriverEntryPointQueryResult q;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
-            q == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<EncodeTiledFn>(p);
-    });
-    return fn;
-}
-
 template <int G, int BN>
 cudaError_t launch_one(const CUtensorMap& map, const CUtensorMap& wmap, const CUtensorMap& ymap,
                        const void* scales, const void* zeros,
@@ -425,29 +315,31 @@ cudaError_t launch_one(const CUtensorMap& map, const CUtensorMap& wmap, const CU
 }  // namespace
 
 cudaError_t launch_gemm(const void* x, const void* qweight, const void* scales, const void* zeros,
-                        void* y, int M, int N, int K, int group, unsigned int* status_word,
-                        cudaStream_t st) {
+                        void* y, int M, int N, int K, int group, bool path_pair_allowed,
+                        unsigned int* status_word, cudaStream_t st) {
     EncodeTiledFn enc = encode_fn();
     if (!enc) return cudaErrorNotSupported;
     const int bn = M > 128 ? 256 : M > 64 ? 128 : M > 32 ? 64 : 32;
-    CUtensorMap map;
-    const cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)M};
-    const cuuint64_t strides[1] = {(cuuint64_t)K * 2};
-    const cuuint32_t box[2] = {(cuuint32_t)kBK, (cuuint32_t)bn};
     const cuuint32_t estr[2] = {1, 1};
-    const CUresult r = enc(&map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void*>(x), dims, strides, box,
-                           estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                           CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
-    // packed weights as a 2-D array of 32-bit words: one row per 16-row band (K * 8 bytes)
-    CUtensorMap wmap;
-    const cuuint64_t wdims[2] = {(cuuint64_t)K * 2, (cuuint64_t)(N / 16)};
-    const cuuint64_t wstrides[1] = {(cuuint64_t)K * 8};
-    const cuuint32_t wbox[2] = {128, 8};
-    const CUresult rw = enc(&wmap, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<void*>(qweight), wdims,
-                            wstrides, wbox, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
-                            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    if (rw != CUDA_SUCCESS) return cudaErrorInvalidValue;
+    // x as [M][K] fp16 in boxes of `tokens` rows x one k-block, 128-byte swizzle
+    auto make_x_map = [&](CUtensorMap* map, int tokens) {
+        const cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)M};
+        const cuuint64_t strides[1] = {(cuuint64_t)K * 2};
+        const cuuint32_t box[2] = {(cuuint32_t)kBK, (cuuint32_t)tokens};
+        return enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void*>(x), dims, strides, box, estr,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                   CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    };
+    // packed weights as a 2-D array of 32-bit words, one row per 16-row band (K * 8 bytes):
+    // boxes of 8 bands x `words` (128 words = one 64-wide k-tile of a band)
+    auto make_w_map = [&](CUtensorMap* map, int words) {
+        const cuuint64_t wdims[2] = {(cuuint64_t)K * 2, (cuuint64_t)(N / 16)};
+        const cuuint64_t wstrides[1] = {(cuuint64_t)K * 8};
+        const cuuint32_t wbox[2] = {(cuuint32_t)words, 8};
+        return enc(map, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<void*>(qweight), wdims, wstrides, wbox,
+                   estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+                   CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    };
     // y as [M][N] fp16, stored in boxes of 32 tokens x 32 channels
     CUtensorMap ymap;
     const cuuint64_t ydims[2] = {(cuuint64_t)N, (cuuint64_t)M};
@@ -462,6 +354,14 @@ cudaError_t launch_gemm(const void* x, const void* qweight, const void* scales, 
     if (e != cudaSuccess) return e;
     e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     if (e != cudaSuccess) return e;
+    CUtensorMap map, wmap;
+    if (path_pair_allowed && gemm_pair_applies(M, N)) {
+        if (!make_x_map(&map, 128) || !make_w_map(&wmap, 256)) return cudaErrorInvalidValue;
+        bool launched = false;
+        e = launch_gemm_pair(map, wmap, ymap, scales, zeros, M, N, K, group, status_word, sms, st, &launched);
+        if (e != cudaSuccess || launched) return e;
+    }
+    if (!make_x_map(&map, bn) || !make_w_map(&wmap, 128)) return cudaErrorInvalidValue;
 #define AWQ_GEMM_CASE(GG, BNN) \
     return launch_one<GG, BNN>(map, wmap, ymap, scales, zeros, M, N, K, status_word, sms, st)
     if (group == 128) {

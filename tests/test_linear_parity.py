@@ -44,16 +44,22 @@ GEMM_CASES = [
     (128, 128, 16, 128, 0.5), (128, 256, 32, 64, 0.5), (256, 384, 17, 128, 0.0), (384, 640, 100, 64, 1.0),
     (256, 1024, 128, 128, 0.5), (512, 512, 300, 128, 0.5), (1024, 1408, 257, 64, 0.5),
     (2048, 2048, 1000, 128, 0.5), (128, 128, 1, 128, 0.5),
+    # more tiles than SM pairs (each pair takes a second tile), ragged last token tile
+    (2560, 256, 2100, 128, 0.5), (2560, 384, 2100, 64, 0.5),
 ]
 
 
+@pytest.mark.parametrize("one_sm", [False, True], ids=["auto", "one-sm"])
 @pytest.mark.parametrize("N,K,M,G,alpha", GEMM_CASES)
-def test_gemm_parity(N, K, M, G, alpha):
+def test_gemm_parity(N, K, M, G, alpha, one_sm):
+    """PATH_GEMM runs SM pairs when M > 128 and N % 256 == 0 and one SM per tile otherwise;
+    PATH_GEMM_1SM forces the latter on every case."""
     from paper_2306_00978_b200 import binding
+    path = binding.PATH_GEMM_1SM if one_sm else binding.PATH_GEMM
     case = Case(3000 + N + K + M, N, K, M, G, alpha)
-    y = _run(case, binding.PATH_GEMM)
+    y = _run(case, path)
     assert_parity(y, case.y_ref(), f"gemm N={N} K={K} M={M} G={G}")
-    y2 = _run(case, binding.PATH_GEMM)
+    y2 = _run(case, path)
     assert np.array_equal(y.view(np.uint16), y2.view(np.uint16))
 
 
