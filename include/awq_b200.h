@@ -163,8 +163,13 @@ int awq_linear_path(const void* x, const void* qweight, const void* scales, cons
 int awq_linear_gemv_static(const void* x, const void* qweight, const void* scales, const void* zeros,
                             void* y, int M, int N, int K, int group, void* stream);
 
-/* Workspace (scratch for split-K partial sums and arrival counters).
- * awq_workspace_bytes: bytes awq_linear may need for this problem (0 if none).
+/* Workspace (scratch for partial sums and arrival counters).
+ * awq_workspace_bytes: bytes awq_linear can use for this problem (0 if none).  For M <= 16 the
+ * split-K matrix-vector kernel REQUIRES them.  For M > 128 with N a multiple of 256 they are
+ * OPTIONAL: with a workspace of at least this size the tensor-core kernel cuts the tiles' K loops
+ * into equal ranges over all SM pairs (stream-K) and sums split tiles in a fixed order through the
+ * workspace; without one, or with a smaller one, whole tiles go round-robin (same result up to
+ * fp32 summation order, slower when the tile count is not a multiple of the pair count).
  * awq_set_workspace: registers caller-owned device memory for the current device; the first
  * 4096 bytes are cleared with a synchronous cudaMemset.  Pass (NULL, 0) to unregister.
  * The memory must stay valid until it is unregistered or replaced. */

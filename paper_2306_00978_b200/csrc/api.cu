@@ -124,7 +124,16 @@ static int resolve_path(int M, int K, int path) {
 
 size_t awq_workspace_bytes(int M, int N, int K, int group) {
     if (check_shape(N, K, group) != AWQ_OK || M < 1) return 0;
-    if (M > 16) return 0;
+    if (M > 16) {
+        // optional: with it the tensor-core kernel spreads its tiles evenly over the SM pairs
+        int dev = 0, sms = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
+            (void)cudaGetLastError();
+            sms = 160;                       // no device to ask: an upper bound for this GPU family
+        }
+        return gemm_workspace_bytes(M, N, sms);
+    }
     return gemv_workspace_bytes(M);
 }
 
@@ -173,8 +182,15 @@ int awq_linear_path(const void* x, const void* qweight, const void* scales, cons
         return note_cuda(launch_gemv_splitk(x, qweight, scales, zeros, y, M, N, K, group, ws, d->status_word,
                                             d->sms, st));
     }
+    void* ws = nullptr;
+    size_t ws_bytes = 0;
+    {
+        std::lock_guard<std::mutex> lock(g_mutex);
+        ws = d->workspace;
+        ws_bytes = d->workspace_bytes;
+    }
     return note_cuda(launch_gemm(x, qweight, scales, zeros, y, M, N, K, group, path != AWQ_PATH_GEMM_1SM,
-                                 d->status_word, st));
+                                 ws, ws_bytes, d->status_word, st));
 }
 
 int awq_linear_gemv_static(const void* x, const void* qweight, const void* scales, const void* zeros,

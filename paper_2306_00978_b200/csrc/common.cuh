@@ -61,6 +61,9 @@ int gemv_static_max_m();
 
 cudaError_t launch_gemm(const void* x, const void* qweight, const void* scales, const void* zeros,
                         void* y, int M, int N, int K, int group, bool path_pair_allowed,
+                        void* workspace, size_t workspace_bytes,
                         unsigned int* status_word, cudaStream_t st);
+// optional workspace of the tensor-core path (0 if the shape has no use for one)
+size_t gemm_workspace_bytes(int M, int N, int sms);
 
 }  // namespace awq

@@ -316,6 +316,7 @@ cudaError_t launch_one(const CUtensorMap& map, const CUtensorMap& wmap, const CU
 
 cudaError_t launch_gemm(const void* x, const void* qweight, const void* scales, const void* zeros,
                         void* y, int M, int N, int K, int group, bool path_pair_allowed,
+                        void* workspace, size_t workspace_bytes,
                         unsigned int* status_word, cudaStream_t st) {
     EncodeTiledFn enc = encode_fn();
     if (!enc) return cudaErrorNotSupported;
@@ -358,7 +359,8 @@ cudaError_t launch_gemm(const void* x, const void* qweight, const void* scales, 
     if (path_pair_allowed && gemm_pair_applies(M, N)) {
         if (!make_x_map(&map, 128) || !make_w_map(&wmap, 256)) return cudaErrorInvalidValue;
         bool launched = false;
-        e = launch_gemm_pair(map, wmap, ymap, scales, zeros, M, N, K, group, status_word, sms, st, &launched);
+        e = launch_gemm_pair(map, wmap, ymap, scales, zeros, M, N, K, group, workspace, workspace_bytes,
+                             status_word, sms, st, &launched);
         if (e != cudaSuccess || launched) return e;
     }
     if (!make_x_map(&map, bn) || !make_w_map(&wmap, 128)) return cudaErrorInvalidValue;
@@ -372,6 +374,10 @@ cudaError_t launch_gemm(const void* x, const void* qweight, const void* scales, 
                       case 64: AWQ_GEMM_CASE(64, 64); default: AWQ_GEMM_CASE(64, 32); }
     }
 #undef AWQ_GEMM_CASE
+}
+
+size_t gemm_workspace_bytes(int M, int N, int sms) {
+    return gemm_pair_applies(M, N) ? gemm_pair_workspace_bytes(sms) : 0;
 }
 
 }  // namespace awq

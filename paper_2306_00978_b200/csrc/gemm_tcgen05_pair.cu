@@ -1,23 +1,29 @@
 // Prefill path of the layer for large token counts (Sec. 4.2: fused dequantize + matrix-matrix
-// product): the same dataflow as gemm_tcgen05.cu, run by PAIRS of thread blocks (a cluster of two
-// SMs) that issue one tcgen05.mma.cta_group::2 of M = 256 output channels x N = 256 tokens.
+// product): the dataflow of gemm_tcgen05.cu, run by PAIRS of thread blocks (a cluster of two SMs)
+// that issue one tcgen05.mma.cta_group::2 of M = 256 output channels x N = 256 tokens.
 //
-// Why pairs: with one block per tile, every k-block writes and reads a 256-token x tile
-// (2 x 32 KB of shared-memory traffic per 512 tensor-pipe cycles), and shared-memory bandwidth,
-// not the tensor pipe, sets the pace.  In a pair each block stages only its half of the
-// tokens (128 x 64 fp16 = 16 KB); the tensor cores of both SMs read both halves.  Per block and
-// k-block the shared-memory traffic drops from 72 KB to 40 KB while the MMA work stays the same.
+// Why pairs, and why 128-channel stages.  With one block per 128 x 256 tile every 64-wide k-block
+// moves 72 KB through shared memory and costs the single MMA-issuing thread two barrier polls,
+// four MMAs and a commit; measured, that thread (not the tensor pipe, which sustains one
+// 128 x 256 x 16 MMA per 128 cycles) set the pace at ~770 cycles per k-block.  In a pair each
+// block stages only its half of the tokens (the tensor cores of both SMs read both halves), and
+// a stage covers K = 128, so the polls and commits are paid once per eight MMAs: ~1120 cycles per
+// stage against the pipe's 1024.
 //
 // Block r of a pair (r = rank in the cluster) owns
 //   - A: output channels 128 r .. 128 r + 127 of the 256-channel slab, dequantized by its own
-//        warps 8-15 into its own tensor memory (as in the single-block kernel),
-//   - B: tokens 128 r .. 128 r + 127 of the 256-token tile in its own shared memory,
+//        warps 8-15 into its own tensor memory (64 columns per stage),
+//   - B: tokens 128 r .. 128 r + 127 of the 256-token tile in its own shared memory (two 64-wide
+//        128-byte-swizzled halves per stage),
 //   - D: the fp32 accumulator rows of its 128 channels x all 256 tokens in its own tensor memory,
-//        drained by its own epilogue warps 4-7.
+//        drained by its own epilogue warps (4-7: tokens 0..127, 16-19: tokens 128..255).
 // Only the leader (rank 0) issues MMAs.  Barriers that the leader's MMA thread waits on live in the
 // leader's shared memory: x_full (both blocks' x copies complete their bytes there), a_full (16
-// dequantizer warps, 8 of them arriving remotely), acc_empty (8 epilogue warps).  The MMA
+// dequantizer warps, 8 of them arriving remotely), acc_empty (16 epilogue warps).  The MMA
 // thread's tcgen05.commit arrives on "empty" and "acc_full" of BOTH blocks.
+//
+// Tile balance: with a workspace, and when whole tiles would leave pairs idle for long, the tiles'
+// K loops are cut into equal ranges over the pairs (stream-K, see PieceIter and the epilogue).
 //
 // Every wait is bounded (about two seconds): a wait that runs out writes a code to the status word
 // and every role of that block leaves its loop; the other block of the pair then runs into its
@@ -98,13 +104,52 @@ __host__ __device__ constexpr uint32_t instr_desc_pair() {     // D fp32, A/B fp
     return (1u << 4) | ((uint32_t)(kPairTokens >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
 }
 
+// Work of one pair: a sequence of pieces (tile, stages k0 .. k1-1 of the tile's K / 128).
+// Without a workspace every piece is a whole tile and tiles go round-robin over the pairs.
+// With one ("stream-K"), the tiles' stages are laid end to end and cut into equal contiguous
+// ranges, one per pair, so that all pairs finish together whatever the tile count; a tile that
+// a cut splits is summed up by the pair that holds its first stages (see the epilogue).
+struct PieceIter {
+    long long s, s_end;              // stream-K: global stage range still to do
+    int tile, tile_step, total_tiles, nks;
+    bool streamk;
+    __device__ bool next(int& t, int& k0, int& k1) {
+        if (streamk) {
+            if (s >= s_end) return false;
+            t = (int)(s / nks);
+            k0 = (int)(s - (long long)t * nks);
+            const long long left = s_end - s;
+            k1 = left < (long long)(nks - k0) ? k0 + (int)left : nks;
+            s += k1 - k0;
+            return true;
+        }
+        if (tile >= total_tiles) return false;
+        t = tile; k0 = 0; k1 = nks;
+        tile += tile_step;
+        return true;
+    }
+};
+// first global stage of pair c when `total` stages are cut into `C` ranges that differ by at most one
+__device__ __forceinline__ long long range_start(long long total, int C, int c) {
+    const long long q = total / C, r = total % C;
+    return (long long)c * q + (c < r ? c : r);
+}
+__device__ __forceinline__ unsigned int ld_acquire_u32(const unsigned int* p) {
+    unsigned int v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+
+constexpr int kPartialFloats = 256 * kPairTokens;    // one pair's fp32 accumulator (256 KB)
+
 // ------------------------------------------------------------------------- the kernel
 template <int G>
 __global__ void __launch_bounds__(kPairThreads, 1)
 gemm_pair_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ CUtensorMap w_map,
                  const __grid_constant__ CUtensorMap y_map,
                  const __half* __restrict__ scales, const unsigned char* __restrict__ zeros,
-                 int M, int N, int K, unsigned int* status_word) {
+                 int M, int N, int K, unsigned int* status_word,
+                 float* partials, unsigned int* flags) {
     using Cfg = PairCfg;
     constexpr int S = Cfg::kStages;
     constexpr int GPS = kStageK / G;                 // quantization groups per stage: 1 or 2
@@ -131,8 +176,15 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constan
     const uint32_t rank = cluster_ctarank();
     const int m_tiles = (M + kPairTokens - 1) / kPairTokens;
     const int total_tiles = (N / 256) * m_tiles;
-    const int first_tile = (int)cluster_id_x(), tile_step = (int)num_clusters_x();
+    const int cluster = (int)cluster_id_x(), num_clusters = (int)num_clusters_x();
     const int nks = K / kStageK;                     // stages per tile
+    const long long total_stages = (long long)total_tiles * nks;
+    PieceIter pieces;
+    pieces.streamk = partials != nullptr;
+    pieces.s = range_start(total_stages, num_clusters, cluster);
+    pieces.s_end = range_start(total_stages, num_clusters, cluster + 1);
+    pieces.tile = cluster; pieces.tile_step = num_clusters; pieces.total_tiles = total_tiles; pieces.nks = nks;
+    int tile, k0, k1;
 
     if (threadIdx.x == 0) {
         s_abort = 0u;
@@ -162,10 +214,10 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constan
             uint32_t stage = 0, phase = 0;
             unsigned int issued = 0;
             bool ok = true;
-            for (int tile = first_tile; tile < total_tiles && ok; tile += tile_step) {
+            while (ok && pieces.next(tile, k0, k1)) {
                 const int slab = (tile / m_tiles) * 2 + (int)rank;          // 128-channel slab of this block
                 const int tok0 = (tile % m_tiles) * kPairTokens + (int)rank * kHalfTokens;
-                for (int ks = 0; ks < nks; ++ks) {
+                for (int ks = k0; ks < k1; ++ks) {
                     if (!mbar_wait(empty(stage), phase ^ 1u, ctl)) { ok = false; break; }
                     if (rank == 0) mbar_arrive_expect_tx(x_full(stage), 2u * Cfg::kXTileBytes);
                     const uint32_t xbar = leader_x_full0 + 8u * stage;
@@ -201,10 +253,10 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constan
             uint32_t stage = 0, phase = 0;
             int local = 0;
             bool ok = true;
-            for (int tile = first_tile; tile < total_tiles && ok; tile += tile_step, ++local) {
+            for (; ok && pieces.next(tile, k0, k1); ++local) {
                 if (!mbar_wait(acc_empty, ((uint32_t)local & 1u) ^ 1u, ctl)) { ok = false; break; }
                 tc_fence_after();
-                for (int ks = 0; ks < nks; ++ks) {
+                for (int ks = k0; ks < k1; ++ks) {
                     // both barriers are normally complete already: poll them together
                     const bool xr = mbar_try_wait(x_full(stage), phase), ar = mbar_try_wait(a_full(stage), phase);
                     if (!(xr && ar) &&
@@ -219,7 +271,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constan
                         // A: 8 columns per K = 16; B: 32 bytes per K = 16 inside a 64-wide half, halves 16 KB apart
                         const uint64_t boff = (uint64_t)(((k >> 2) * Cfg::kXHalfBytes + (k & 3) * 32) >> 4);
                         umma_pair_f16_a_tmem(tmem_base, a_tmem + (uint32_t)(8 * k), bdesc + boff, idesc,
-                                             (ks | k) != 0 ? 1u : 0u);
+                                             (ks > k0 || k > 0) ? 1u : 0u);
                     }
                     umma_pair_commit(empty(stage));
                     umma_pair_commit(peer_empty0 + 8u * stage);
@@ -240,7 +292,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constan
         const uint32_t leader_a_full0 = map_to_rank(a_full(0), 0);
         uint32_t stage = 0, phase = 0;
         bool ok = true;
-        for (int tile = first_tile; tile < total_tiles && ok; tile += tile_step) {
+        while (ok && pieces.next(tile, k0, k1)) {
             const int slab = (tile / m_tiles) * 2 + (int)rank;
             // this lane's rows' parameters: scales [band][group][16], zero bytes [band pair][group][16]
             const unsigned short* sc_g = reinterpret_cast<const unsigned short*>(scales) +
@@ -250,9 +302,10 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constan
             uint32_t du[GPS], dl[GPS], zb[GPS], du1[GPS], dl1[GPS], zb1[GPS];
 #pragma unroll
             for (int q = 0; q < GPS; ++q) {
-                du1[q] = __ldg(sc_g + q * 16); dl1[q] = __ldg(sc_g + q * 16 + 8); zb1[q] = __ldg(z_g + q * 16);
+                const int g0 = k0 * GPS + q;
+                du1[q] = __ldg(sc_g + g0 * 16); dl1[q] = __ldg(sc_g + g0 * 16 + 8); zb1[q] = __ldg(z_g + g0 * 16);
             }
-            for (int ks = 0; ks < nks; ++ks) {
+            for (int ks = k0; ks < k1; ++ks) {
 #pragma unroll
                 for (int q = 0; q < GPS; ++q) {
                     du[q] = du1[q]; dl[q] = dl1[q]; zb[q] = zb1[q];
@@ -296,12 +349,48 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constan
         const int quad = warp & 3;                     // TMEM lanes 32*quad .. +31
         const int half = warp >= 16 ? 1 : 0;
         const uint32_t leader_acc_empty = map_to_rank(acc_empty, 0);
+        // this warp's part of a pair's fp32 partial tile: [rank][warp][chunk][register][lane]
+        const size_t part_off = (size_t)((((int)rank * 8 + half * 4 + quad) * 4) * 1024 + lane);
         int local = 0;
         int obuf = 0;
         bool ok = true;
-        for (int tile = first_tile; tile < total_tiles && ok; tile += tile_step, ++local) {
+        for (; ok && pieces.next(tile, k0, k1); ++local) {
             const int slab = (tile / m_tiles) * 2 + (int)rank, mt = tile % m_tiles;
-            ok = mbar_wait(acc_full, (uint32_t)local & 1u, ctl);
+            // A piece that does not start the tile is a contribution: its fp32 sums go to this pair's
+            // slot of the workspace.  A piece that starts the tile but does not end it waits for the
+            // contributions of the pairs after this one (they were produced at the start of those
+            // pairs' ranges, long before) and adds them in pair order: the sum is reproducible.
+            const bool contributes = k0 > 0;
+            int n_contrib = 0;
+            if (k0 == 0 && k1 < nks) {
+                const long long tile_end = (long long)(tile + 1) * nks;
+                while (cluster + 1 + n_contrib < num_clusters &&
+                       range_start(total_stages, num_clusters, cluster + 1 + n_contrib) < tile_end)
+                    ++n_contrib;
+            }
+            // while this piece's MMAs run: wait for the contributions (normally there long ago) and
+            // fetch the first one's first chunk, so that the drain below does not wait for memory
+            for (int j = 0; j < n_contrib && ok; ++j) {
+                const unsigned int* f = flags + cluster + 1 + j;
+                const unsigned long long t0 = global_ns();
+                while (ld_acquire_u32(f) < 16u) {                   // 16 epilogue warps of that pair
+                    if (*ctl.abort) { ok = false; break; }
+                    if (global_ns() - t0 > kWaitLimitNs) {
+                        *ctl.abort = 1u;
+                        atomicExch(ctl.status, kTimeoutCode);
+                        ok = false;
+                        break;
+                    }
+                    __nanosleep(64);
+                }
+            }
+            float p[32];
+            const float* src0 = partials + (size_t)(cluster + 1) * kPartialFloats + part_off;
+            if (n_contrib > 0 && ok) {
+#pragma unroll
+                for (int i = 0; i < 32; ++i) p[i] = __ldcg(src0 + i * 32);
+            }
+            ok = ok && mbar_wait(acc_full, (uint32_t)local & 1u, ctl);
             ok = __all_sync(0xFFFFFFFFu, ok);
             if (!ok) break;
             tc_fence_after();
@@ -314,10 +403,29 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constan
                 tmem_ld_32cols(taddr + (uint32_t)c, r);
                 tmem_ld_wait();
                 if (c + 32 >= kHalfTokens) {
-                    // the accumulator is in registers: the MMA thread may start the next tile
+                    // the accumulator is in registers: the MMA thread may start the next piece
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) mbar_arrive_cluster(leader_acc_empty);
+                }
+                if (contributes) {
+                    float* dst = partials + (size_t)cluster * kPartialFloats + part_off + (size_t)c * 32;
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) __stcg(dst + i * 32, __uint_as_float(r[i]));
+                    continue;
+                }
+                if (n_contrib > 0) {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) + p[i]);
+                    for (int j = 1; j < n_contrib; ++j) {
+                        const float* src = partials + (size_t)(cluster + 1 + j) * kPartialFloats + part_off + (size_t)c * 32;
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) + __ldcg(src + i * 32));
+                    }
+                    if (c + 32 < kHalfTokens) {                     // the next chunk of the first contribution
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) p[i] = __ldcg(src0 + (size_t)(c + 32) * 32 + i * 32);
+                    }
                 }
                 // stage the 32 x 32 block as [token][channel] fp16 and hand it to the copy engine
                 // (rows past M are clipped by the tensor map)
@@ -336,6 +444,17 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constan
                 }
                 obuf ^= 1;
             }
+            if (contributes) {
+                __threadfence();                                    // the sums before the flag
+                __syncwarp();
+                if (lane == 0) atomicAdd(flags + cluster, 1u);
+            }
+            if (lane == 0) {
+                // the 16 readers of a slot count themselves in after the 16 writers; the last one
+                // clears the flag, so the workspace is ready for the next launch
+                for (int j = 0; j < n_contrib; ++j)
+                    if (atomicAdd(flags + cluster + 1 + j, 1u) == 31u) atomicExch(flags + cluster + 1 + j, 0u);
+            }
         }
         if (lane == 0) bulk_wait_all();                             // all of y written before exit
     }
@@ -352,44 +471,80 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constan
 }
 
 // ------------------------------------------------------------------------------ host
+// pairs that can be resident at once on the current device (0 if the query fails); cached
+template <int G>
+int resident_pairs(int sms, cudaError_t* err) {
+    static bool done[64] = {};
+    static int pairs[64] = {};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    *err = cudaSuccess;
+    if (!done[dev & 63]) {
+        *err = cudaFuncSetAttribute(gemm_pair_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                    PairCfg::kSmemBytes);
+        if (*err != cudaSuccess) return 0;
+        cudaLaunchConfig_t cfg = {};
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+        cfg.gridDim = dim3((unsigned)(sms & ~1));
+        cfg.blockDim = dim3(kPairThreads);
+        cfg.dynamicSmemBytes = PairCfg::kSmemBytes;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        int n = 0;
+        if (cudaOccupancyMaxActiveClusters(&n, gemm_pair_kernel<G>, &cfg) != cudaSuccess) {
+            (void)cudaGetLastError();
+            n = 0;
+        }
+        pairs[dev & 63] = n;
+        done[dev & 63] = true;
+    }
+    return pairs[dev & 63];
+}
+
 template <int G>
 cudaError_t launch_pair(const CUtensorMap& xmap, const CUtensorMap& wmap, const CUtensorMap& ymap,
                         const void* scales, const void* zeros, int M, int N, int K,
+                        void* workspace, size_t workspace_bytes,
                         unsigned int* status_word, int sms, cudaStream_t st, bool* launched) {
     using Cfg = PairCfg;
-    static bool attr_done[64] = {};
-    static int max_clusters[64] = {};
-    int dev = 0;
-    cudaGetDevice(&dev);
+    cudaError_t e;
+    const int resident = resident_pairs<G>(sms, &e);
+    if (e != cudaSuccess) return e;
+    // pairs that cannot all be resident at once would leave SMs idle (and a tile's owner waiting)
+    if (resident * 2 < sms - 4) { *launched = false; return cudaSuccess; }
+    const long long tiles = (long long)(N / 256) * ((M + kPairTokens - 1) / kPairTokens);
+    const long long stages = tiles * (K / kStageK);
+    // Stream-K needs one fp32 tile per pair behind the counters at the head of the workspace.  It
+    // costs every pair two more accumulator drains and a pass over a partial tile (about 10 us),
+    // so it is used only when whole tiles would leave the pairs idle for longer than that: the
+    // idle time of the last round-robin wave, in stages (~0.8 us each) per pair.  Launches of
+    // more than about 0.3 ms run into the power limit, where idle pairs let the busy ones clock
+    // higher and an even split gains nothing (measured: 5 % slower): those keep whole tiles.
+    const long long waves = (tiles + resident - 1) / resident;
+    const long long idle_stages = (waves * resident - tiles) * (K / kStageK) / resident;
+    const bool streamk = workspace != nullptr && idle_stages > 25 && stages / resident < 400 &&
+                         workspace_bytes >= kCounterBytes + (size_t)resident * kPartialFloats * sizeof(float) &&
+                         (size_t)resident * sizeof(unsigned int) <= kCounterBytes;
+    long long want = tiles;
+    if (streamk && stages / 4 > want) want = stages / 4;          // at least four stages per pair
+    const int clusters = (int)(want < resident ? want : resident);
     cudaLaunchConfig_t cfg = {};
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.gridDim = dim3((unsigned)(2 * clusters));
     cfg.blockDim = dim3(kPairThreads);
     cfg.dynamicSmemBytes = Cfg::kSmemBytes;
     cfg.stream = st;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    if (!attr_done[dev & 63]) {
-        cudaError_t e = cudaFuncSetAttribute(gemm_pair_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             Cfg::kSmemBytes);
-        if (e != cudaSuccess) return e;
-        cfg.gridDim = dim3((unsigned)(sms & ~1));
-        int n = 0;
-        e = cudaOccupancyMaxActiveClusters(&n, gemm_pair_kernel<G>, &cfg);
-        if (e != cudaSuccess) { (void)cudaGetLastError(); n = 0; }
-        max_clusters[dev & 63] = n;
-        attr_done[dev & 63] = true;
-    }
-    // pairs that cannot all be resident at once would leave SMs idle behind a static tile order
-    const int resident = max_clusters[dev & 63];
-    if (resident * 2 < sms - 4) { *launched = false; return cudaSuccess; }
-    const int tiles = (N / 256) * ((M + kPairTokens - 1) / kPairTokens);
-    const int clusters = tiles < resident ? tiles : resident;
-    cfg.gridDim = dim3((unsigned)(2 * clusters));
-    const cudaError_t e = cudaLaunchKernelEx(&cfg, gemm_pair_kernel<G>, xmap, wmap, ymap,
-                                             reinterpret_cast<const __half*>(scales),
-                                             reinterpret_cast<const unsigned char*>(zeros), M, N, K, status_word);
+    float* partials = streamk ? reinterpret_cast<float*>(static_cast<unsigned char*>(workspace) + kCounterBytes)
+                              : nullptr;
+    unsigned int* flags = static_cast<unsigned int*>(workspace);
+    e = cudaLaunchKernelEx(&cfg, gemm_pair_kernel<G>, xmap, wmap, ymap, reinterpret_cast<const __half*>(scales),
+                           reinterpret_cast<const unsigned char*>(zeros), M, N, K, status_word, partials, flags);
     if (e != cudaSuccess) return e;
     count_launch();
     *launched = true;
@@ -398,17 +553,24 @@ cudaError_t launch_pair(const CUtensorMap& xmap, const CUtensorMap& wmap, const 
 
 }  // namespace
 
-
 bool gemm_pair_applies(int M, int N) { return M > 128 && N % 256 == 0; }
+
+// workspace with which the pair kernel balances its tiles over all SM pairs (stream-K)
+size_t gemm_pair_workspace_bytes(int sms) {
+    return kCounterBytes + (size_t)(sms / 2) * kPartialFloats * sizeof(float);
+}
 
 // Launches the pair kernel if this device can keep (nearly) all its SMs busy with pairs;
 // otherwise *launched is false and the caller uses the single-block kernel.
 cudaError_t launch_gemm_pair(const CUtensorMap& xmap128, const CUtensorMap& wmap, const CUtensorMap& ymap,
                              const void* scales, const void* zeros, int M, int N, int K, int group,
+                             void* workspace, size_t workspace_bytes,
                              unsigned int* status_word, int sms, cudaStream_t st, bool* launched) {
     if (group == 128)
-        return launch_pair<128>(xmap128, wmap, ymap, scales, zeros, M, N, K, status_word, sms, st, launched);
-    return launch_pair<64>(xmap128, wmap, ymap, scales, zeros, M, N, K, status_word, sms, st, launched);
+        return launch_pair<128>(xmap128, wmap, ymap, scales, zeros, M, N, K, workspace, workspace_bytes,
+                                status_word, sms, st, launched);
+    return launch_pair<64>(xmap128, wmap, ymap, scales, zeros, M, N, K, workspace, workspace_bytes,
+                           status_word, sms, st, launched);
 }
 
 }  // namespace awq

@@ -117,10 +117,13 @@ inline EncodeTiledFn encode_fn() {
 }
 
 
-// the pair (two-SM) kernel: for M > 128 and N a multiple of 256; x map with a box of 128 tokens
+// the pair (two-SM) kernel: for M > 128 and N a multiple of 256; x map with a box of 128 tokens,
+// weight map with a box of 256 words; an optional workspace enables stream-K tile balancing
 bool gemm_pair_applies(int M, int N);
+size_t gemm_pair_workspace_bytes(int sms);
 cudaError_t launch_gemm_pair(const CUtensorMap& xmap128, const CUtensorMap& wmap, const CUtensorMap& ymap,
                              const void* scales, const void* zeros, int M, int N, int K, int group,
+                             void* workspace, size_t workspace_bytes,
                              unsigned int* status_word, int sms, cudaStream_t st, bool* launched);
 
 }  // namespace awq

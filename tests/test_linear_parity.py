@@ -46,20 +46,50 @@ GEMM_CASES = [
     (2048, 2048, 1000, 128, 0.5), (128, 128, 1, 128, 0.5),
     # more tiles than SM pairs (each pair takes a second tile), ragged last token tile
     (2560, 256, 2100, 128, 0.5), (2560, 384, 2100, 64, 0.5),
+    # long K loops: with stream-K most pairs start or end inside a tile, some tiles are cut twice
+    (512, 8192, 520, 128, 0.5), (1280, 6144, 1300, 64, 0.5),
 ]
 
 
-@pytest.mark.parametrize("one_sm", [False, True], ids=["auto", "one-sm"])
+def _run_gemm_without_workspace(case):
+    """The tensor-core path with no workspace registered: whole tiles round-robin over the SM pairs."""
+    import torch
+    from paper_2306_00978_b200 import binding
+    L = binding.lib()
+    qw, sc, zp = oracle_packed_to_cuda(case)
+    x = to_cuda(case.x)
+    y = torch.empty((case.M, case.N), dtype=torch.float16, device="cuda")
+    torch.cuda.synchronize()
+    saved = binding._workspace.pop(torch.cuda.current_device(), None)
+    assert L.awq_set_workspace(None, 0) == 0
+    try:
+        rc = L.awq_linear_path(x.data_ptr(), qw.data_ptr(), sc.data_ptr(), zp.data_ptr(), y.data_ptr(),
+                               case.M, case.N, case.K, case.group, binding.PATH_GEMM, None)
+        assert rc == 0
+        binding.poll_status()
+    finally:
+        if saved is not None:
+            assert L.awq_set_workspace(saved.data_ptr(), saved.numel()) == 0
+            binding._workspace[torch.cuda.current_device()] = saved
+    return y.cpu().numpy()
+
+
+@pytest.mark.parametrize("mode", ["auto", "one-sm", "no-workspace"])
 @pytest.mark.parametrize("N,K,M,G,alpha", GEMM_CASES)
-def test_gemm_parity(N, K, M, G, alpha, one_sm):
-    """PATH_GEMM runs SM pairs when M > 128 and N % 256 == 0 and one SM per tile otherwise;
+def test_gemm_parity(N, K, M, G, alpha, mode):
+    """PATH_GEMM runs SM pairs when M > 128 and N % 256 == 0 (stream-K over the registered
+    workspace, or whole tiles round-robin without one) and one SM per tile otherwise;
     PATH_GEMM_1SM forces the latter on every case."""
     from paper_2306_00978_b200 import binding
-    path = binding.PATH_GEMM_1SM if one_sm else binding.PATH_GEMM
     case = Case(3000 + N + K + M, N, K, M, G, alpha)
-    y = _run(case, path)
-    assert_parity(y, case.y_ref(), f"gemm N={N} K={K} M={M} G={G}")
-    y2 = _run(case, path)
+    if mode == "no-workspace":
+        run = lambda: _run_gemm_without_workspace(case)
+    else:
+        path = binding.PATH_GEMM_1SM if mode == "one-sm" else binding.PATH_GEMM
+        run = lambda: _run(case, path)
+    y = run()
+    assert_parity(y, case.y_ref(), f"gemm N={N} K={K} M={M} G={G} {mode}")
+    y2 = run()
     assert np.array_equal(y.view(np.uint16), y2.view(np.uint16))
 
 
