@@ -136,7 +136,7 @@ __device__ __forceinline__ void tile_sums_of_x(const __half* __restrict__ x, flo
 }
 
 // =========================================================================== band kernel
-constexpr int kBandThreads = kMathThreads + 64;        // + copy warp + flush warp
+constexpr int kBandThreads = kMathThreads + 96;        // + weight-copy warp + flush warp + x-copy warp
 
 // Stage layout of the band kernel, fixed at compile time by TPW (k-tiles per math warp and
 // stage) and the group size, so that every shared-memory read is base + immediate.
@@ -236,10 +236,35 @@ gemv_band_kernel(const BandProblems probs, const __half* __restrict__ x, int M, 
     }
     __syncthreads();
     const WaitCtl ctl{status_word, &s_abort};
+    // Programmatic dependent launch: the next kernel of the stream may be scheduled onto an SM as
+    // soon as this block has left it, and this kernel may itself have started before the one in
+    // front of it finished.  Weights, scales and zero points are constants of the layer, so the
+    // weight-copy warp starts filling the ring at once; everything that touches x or y first
+    // waits for the preceding kernel to complete (griddepcontrol.wait).
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
+    if (warp == kMathWarps + 2) {
+        // ---------------------------------------------------------------- x-copy warp
+        // lane m < M copies token m's slice of x for each stage (counted on the stage's barrier)
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+        uint32_t stage = 0, phase = 0;
+        for (int task = b0; task < b1; ++task) {
+            for (int j = 0; j < upb; ++j) {
+                const int kt = j * UT;
+                const int nt = min(UT, ktiles - kt);
+                if (lane == 0) mbar_wait_relaxed(bars + 64u + 8u * stage, phase ^ 1u, ctl);
+                __syncwarp();
+                if (lane < M)
+                    bulk_load(sbase + stage * (uint32_t)lay.stage_bytes + St::kXOff + lane * St::kXRow,
+                              x + (size_t)lane * K + (size_t)kt * 64, (uint32_t)(nt * 128), bars + 8u * stage);
+                if (++stage == (uint32_t)S) { stage = 0; phase ^= 1u; }
+            }
+        }
+        return;
+    }
     if (warp == kMathWarps) {
-        // ------------------------------------------------------------------ copy warp
-        // lane 0 posts the byte count; lanes 0, 1, 2 and 3 .. 3+M-1 each issue one bulk copy
+        // ------------------------------------------------------------- weight-copy warp
+        // lane 0 posts the stage's byte count (x included); lanes 0, 1, 2 each issue one bulk copy
         uint32_t stage = 0, phase = 0;
         for (int task = b0; task < b1; ++task) {
             const BandRef br = band_ref(probs, task);
@@ -262,9 +287,6 @@ gemv_band_kernel(const BandProblems probs, const __half* __restrict__ x, int M, 
                     bulk_load(dst + St::kScOff, br.scales + ((size_t)band * ng + gi0) * 16, (uint32_t)(ngr * 32), bar);
                 else if (lane == 2)
                     bulk_load(dst + St::kZOff, br.zeros + ((size_t)(band >> 1) * ng + gi0) * 16, (uint32_t)(ngr * 16), bar);
-                else if (lane - 3 < M)
-                    bulk_load(dst + St::kXOff + (lane - 3) * St::kXRow, x + (size_t)(lane - 3) * K + (size_t)kt * 64,
-                              (uint32_t)(nt * 128), bar);
                 if (++stage == (uint32_t)S) { stage = 0; phase ^= 1u; }
             }
         }
@@ -281,9 +303,10 @@ gemv_band_kernel(const BandProblems probs, const __half* __restrict__ x, int M, 
     }
 
     // x sums per k-tile (math warps and the flush warp), while the first stages are in flight
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     float* xsum = reinterpret_cast<float*>(smem + lay.xsum_off);
     tile_sums_of_x(x, xsum, M, K, 8, warp < kMathWarps ? warp : warp - 1, kMathWarps + 1, lane);
-    named_barrier_sync(3, kBandThreads - 32);
+    named_barrier_sync(3, kMathThreads + 32);
 
     float* red = reinterpret_cast<float*>(smem + lay.red_off);
     if (warp == kMathWarps + 1) {
@@ -812,6 +835,17 @@ cudaError_t launch_gemv_band(const void* x, const GemvMatrix* mats, int count, i
     const int blocks = bands < sms ? bands : sms;
     const int tpw = M <= 2 ? 4 : 2;                            // 64 or 32 k-tiles per stage
     cudaError_t e = cudaSuccess;
+    // programmatic stream serialization: this launch may begin while the kernel in front of it in
+    // the stream is still finishing (see the kernel: it waits before it touches x or y)
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.gridDim = dim3((unsigned)blocks);
+    cfg.blockDim = dim3(kBandThreads);
+    cfg.stream = st;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
 #define AWQ_BAND_LAUNCH(GG, TT)                                                                      \
     do {                                                                                             \
         const BandLayout lay = band_layout<GG, TT>(M, K);                                            \
@@ -819,8 +853,10 @@ cudaError_t launch_gemv_band(const void* x, const GemvMatrix* mats, int count, i
         static bool done[64] = {};                                                                   \
         e = allow_big_smem(gemv_band_kernel<GG, TT>, done);                                          \
         if (e != cudaSuccess) return e;                                                              \
-        gemv_band_kernel<GG, TT><<<blocks, kBandThreads, lay.total, st>>>(                           \
-            pr, reinterpret_cast<const __half*>(x), M, K, lay, status_word);                         \
+        cfg.dynamicSmemBytes = lay.total;                                                            \
+        e = cudaLaunchKernelEx(&cfg, gemv_band_kernel<GG, TT>, pr, reinterpret_cast<const __half*>(x), M, K, \
+                               lay, status_word);                                                    \
+        if (e != cudaSuccess) return e;                                                              \
     } while (0)
     if (group == 128) { if (tpw == 4) AWQ_BAND_LAUNCH(128, 4); else AWQ_BAND_LAUNCH(128, 2); }
     else              { if (tpw == 4) AWQ_BAND_LAUNCH(64, 4);  else AWQ_BAND_LAUNCH(64, 2); }
