@@ -201,7 +201,8 @@ inline BandLayout band_layout(int M, int K) {
 }
 
 // TPW = k-tiles per math warp and stage (stage = 16 * TPW k-tiles).  M <= 8 tokens (one token tile).
-template <int G, int TPW>
+// ONE: M == 1, the sums of the second token column of each accumulator fragment are not formed.
+template <int G, int TPW, bool ONE>
 __global__ void __launch_bounds__(kBandThreads, 1)
 gemv_band_kernel(const BandProblems probs, const __half* __restrict__ x, int M, int K,
                  const BandLayout lay, unsigned int* status_word) {
@@ -302,11 +303,8 @@ gemv_band_kernel(const BandProblems probs, const __half* __restrict__ x, int M, 
         return;
     }
 
-    // x sums per k-tile (math warps and the flush warp), while the first stages are in flight
     asm volatile("griddepcontrol.wait;" ::: "memory");
     float* xsum = reinterpret_cast<float*>(smem + lay.xsum_off);
-    tile_sums_of_x(x, xsum, M, K, 8, warp < kMathWarps ? warp : warp - 1, kMathWarps + 1, lane);
-    named_barrier_sync(3, kMathThreads + 32);
 
     float* red = reinterpret_cast<float*>(smem + lay.red_off);
     if (warp == kMathWarps + 1) {
@@ -347,6 +345,12 @@ gemv_band_kernel(const BandProblems probs, const __half* __restrict__ x, int M, 
 #pragma unroll
         for (int jw = 0; jw < 4; ++jw) xr[v][jw] = make_uint2(0u, 0u);
 
+    // x sums per k-tile for the zero-point term (the 16 math warps), while the first stages are in
+    // flight.  (Deferring them behind the first stage's products, and polling barriers ahead of
+    // use, were both measured slower.)
+    tile_sums_of_x(x, xsum, M, K, 8, warp, kMathWarps, lane);
+    named_barrier_sync(3, kMathThreads);
+
     uint32_t stage = 0, phase = 0;
     int nflush = 0;
     for (int task = b0; task < b1; ++task, ++nflush) {
@@ -358,10 +362,13 @@ gemv_band_kernel(const BandProblems probs, const __half* __restrict__ x, int M, 
             mbar_wait(bars + 8u * stage, phase, ctl);
             const unsigned char* st = smem + stage * (uint32_t)lay.stage_bytes;
             const float* xs = xs_lane + j * (UT * 8);
-            if (nt >= TPW) {
+            const bool full_stage = nt >= TPW;
+            float c[GPW][4];
+            float zu[GPW], zl[GPW];
+            uint4 pk[TPW];
+            if (full_stage) {
                 // ---- full stage: straight-line code, one accumulation chain per group, the
                 // groups' products interleaved word by word so that no MMA waits for the last
-                uint4 pk[TPW];
 #pragma unroll
                 for (int v = 0; v < TPW; ++v) pk[v] = *reinterpret_cast<const uint4*>(st + o_w + v * 512);
                 if (tok_ok) {
@@ -371,7 +378,6 @@ gemv_band_kernel(const BandProblems probs, const __half* __restrict__ x, int M, 
                         for (int jw = 0; jw < 4; ++jw)
                             xr[v][jw] = *reinterpret_cast<const uint2*>(st + o_x + v * 128 + jw * 32);
                 }
-                float c[GPW][4];
 #pragma unroll
                 for (int v = 0; v < TPG; ++v)
 #pragma unroll
@@ -389,6 +395,25 @@ gemv_band_kernel(const BandProblems probs, const __half* __restrict__ x, int M, 
                                 mma_16816(c[q], w & 0x000F000Fu, w & 0x00F000F0u, w8 & 0x000F000Fu,
                                           w8 & 0x00F000F0u, bb0, bb1);
                         }
+                // per group: scale term, then zero-point term (integers below 2^23 become floats
+                // without a conversion instruction)
+#pragma unroll
+                for (int q = 0; q < GPW; ++q) {
+                    const float d_up = __half2float(*reinterpret_cast<const __half*>(st + o_sc + q * 32));
+                    const float d_lo = __half2float(*reinterpret_cast<const __half*>(st + o_sc + q * 32 + 16));
+                    const uint32_t zb = st[o_z + q * 16];
+                    const float z_up = __uint_as_float(0x4B000000u | (zb & 0xFu)) - 8388608.0f;
+                    const float z_lo16 = __uint_as_float(0x4B000000u | (zb & 0xF0u)) - 8388608.0f;   // 16 * z
+                    zu[q] = d_up * z_up;
+                    zl[q] = (d_lo * 0.0625f) * z_lo16;
+                    const float su = d_up * 16777216.0f, sl = d_lo * 1048576.0f;
+                    acc[0] = fmaf(su, c[q][0], acc[0]);
+                    acc[2] = fmaf(sl, c[q][2], acc[2]);
+                    if (!ONE) {
+                        acc[1] = fmaf(su, c[q][1], acc[1]);
+                        acc[3] = fmaf(sl, c[q][3], acc[3]);
+                    }
+                }
 #pragma unroll
                 for (int q = 0; q < GPW; ++q) {
                     float Xx = 0.0f, Xy = 0.0f;
@@ -398,15 +423,12 @@ gemv_band_kernel(const BandProblems probs, const __half* __restrict__ x, int M, 
                         Xx += X.x;
                         Xy += X.y;
                     }
-                    const float d_up = __half2float(*reinterpret_cast<const __half*>(st + o_sc + q * 32));
-                    const float d_lo = __half2float(*reinterpret_cast<const __half*>(st + o_sc + q * 32 + 16));
-                    const uint32_t zb = st[o_z + q * 16];
-                    const float su = d_up * 16777216.0f, sl = d_lo * 1048576.0f;
-                    const float zu = d_up * (float)(zb & 0xFu), zl = d_lo * (float)(zb >> 4);
-                    acc[0] = fmaf(su, c[q][0], fmaf(-zu, Xx, acc[0]));
-                    acc[1] = fmaf(su, c[q][1], fmaf(-zu, Xy, acc[1]));
-                    acc[2] = fmaf(sl, c[q][2], fmaf(-zl, Xx, acc[2]));
-                    acc[3] = fmaf(sl, c[q][3], fmaf(-zl, Xy, acc[3]));
+                    acc[0] = fmaf(-zu[q], Xx, acc[0]);
+                    acc[2] = fmaf(-zl[q], Xx, acc[2]);
+                    if (!ONE) {
+                        acc[1] = fmaf(-zu[q], Xy, acc[1]);
+                        acc[3] = fmaf(-zl[q], Xy, acc[3]);
+                    }
                 }
             } else if (nt > 0) {
                 // ---- ragged last stage of a band: whole groups only (K % G == 0), one at a time
@@ -846,20 +868,27 @@ cudaError_t launch_gemv_band(const void* x, const GemvMatrix* mats, int count, i
     cfg.stream = st;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-#define AWQ_BAND_LAUNCH(GG, TT)                                                                      \
+#define AWQ_BAND_LAUNCH(GG, TT, ONE1)                                                                      \
     do {                                                                                             \
         const BandLayout lay = band_layout<GG, TT>(M, K);                                            \
         if (lay.stages < 2) return cudaErrorInvalidValue;      /* K too large for the x-sum table */ \
         static bool done[64] = {};                                                                   \
-        e = allow_big_smem(gemv_band_kernel<GG, TT>, done);                                          \
+        e = allow_big_smem(gemv_band_kernel<GG, TT, ONE1>, done);                                          \
         if (e != cudaSuccess) return e;                                                              \
         cfg.dynamicSmemBytes = lay.total;                                                            \
-        e = cudaLaunchKernelEx(&cfg, gemv_band_kernel<GG, TT>, pr, reinterpret_cast<const __half*>(x), M, K, \
+        e = cudaLaunchKernelEx(&cfg, gemv_band_kernel<GG, TT, ONE1>, pr, reinterpret_cast<const __half*>(x), M, K, \
                                lay, status_word);                                                    \
         if (e != cudaSuccess) return e;                                                              \
     } while (0)
-    if (group == 128) { if (tpw == 4) AWQ_BAND_LAUNCH(128, 4); else AWQ_BAND_LAUNCH(128, 2); }
-    else              { if (tpw == 4) AWQ_BAND_LAUNCH(64, 4);  else AWQ_BAND_LAUNCH(64, 2); }
+    if (group == 128) {
+        if (M == 1) AWQ_BAND_LAUNCH(128, 4, true);
+        else if (tpw == 4) AWQ_BAND_LAUNCH(128, 4, false);
+        else AWQ_BAND_LAUNCH(128, 2, false);
+    } else {
+        if (M == 1) AWQ_BAND_LAUNCH(64, 4, true);
+        else if (tpw == 4) AWQ_BAND_LAUNCH(64, 4, false);
+        else AWQ_BAND_LAUNCH(64, 2, false);
+    }
 #undef AWQ_BAND_LAUNCH
     count_launch();
     return cudaGetLastError();
