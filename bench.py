@@ -497,7 +497,7 @@ def main():
                    "algorithmic_bytes_per_step": step_bytes, "parallelism": f"replicas x{world}",
                    "launch": "each step is one CUDA-graph replay of 4 C-ABI calls: awq_linear_multi(q,k,v), "
                              "awq_linear(o), awq_linear_multi(gate,up), awq_linear(down)"},
-        "roofline": {"bound": "hbm", "kernel": "gemv_band_kernel<128,4,true>", "achieved": achieved,
+        "roofline": {"bound": "hbm", "kernel": "gemv_band_kernel<128,4,true,true>", "achieved": achieved,
                      "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
                      "peak_source": peaks["source"], "frac_of_nominal_8000": achieved / NOMINAL_HBM_GBS,
                      "avg_launch_us": per_launch_s * 1e6,

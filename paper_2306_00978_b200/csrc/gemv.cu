@@ -185,10 +185,10 @@ __device__ __forceinline__ BandRef band_ref(const BandProblems& pr, int task) {
     return r;
 }
 template <int G, int TPW>
-inline BandLayout band_layout(int M, int K) {
+inline BandLayout band_layout(int M, int K, bool x_in_registers) {
     using St = BandStage<G, TPW>;
     BandLayout l;
-    l.stage_bytes = ((St::kXOff + M * St::kXRow + 127) / 128) * 128;
+    l.stage_bytes = ((St::kXOff + (x_in_registers ? 0 : M * St::kXRow) + 127) / 128) * 128;
     const int xsum = (K / 64 + St::kUT) * 8 * 4;        // + one stage of slack for ragged reads
     const int red = 2 * kMathWarps * 8 * 16 * 4;        // two buffers of [warp][token][row] fp32
     int s = (kSmemBudget - xsum - red - 256) / l.stage_bytes;
@@ -202,7 +202,10 @@ inline BandLayout band_layout(int M, int K) {
 
 // TPW = k-tiles per math warp and stage (stage = 16 * TPW k-tiles).  M <= 8 tokens (one token tile).
 // ONE: M == 1, the sums of the second token column of each accumulator fragment are not formed.
-template <int G, int TPW, bool ONE>
+// XREG: K == 64 * 16 * TPW, i.e. a band is exactly one stage and a math warp meets the same
+// k-tiles in every stage: its B fragments of x and its per-group sums of x are loaded once, from
+// global memory, and stay in registers; no x travels through the stages.
+template <int G, int TPW, bool ONE, bool XREG>
 __global__ void __launch_bounds__(kBandThreads, 1)
 gemv_band_kernel(const BandProblems probs, const __half* __restrict__ x, int M, int K,
                  const BandLayout lay, unsigned int* status_word) {
@@ -247,6 +250,7 @@ gemv_band_kernel(const BandProblems probs, const __half* __restrict__ x, int M, 
     if (warp == kMathWarps + 2) {
         // ---------------------------------------------------------------- x-copy warp
         // lane m < M copies token m's slice of x for each stage (counted on the stage's barrier)
+        if (XREG) return;
         asm volatile("griddepcontrol.wait;" ::: "memory");
         uint32_t stage = 0, phase = 0;
         for (int task = b0; task < b1; ++task) {
@@ -278,7 +282,7 @@ gemv_band_kernel(const BandProblems probs, const __half* __restrict__ x, int M, 
                 const uint32_t bar = bars + 8u * stage;
                 if (lane == 0) {
                     mbar_wait_relaxed(bars + 64u + 8u * stage, phase ^ 1u, ctl);
-                    mbar_arrive_expect_tx(bar, (uint32_t)(nt * 512 + ngr * 48 + M * nt * 128));
+                    mbar_arrive_expect_tx(bar, (uint32_t)(nt * 512 + ngr * 48 + (XREG ? 0 : M * nt * 128)));
                 }
                 __syncwarp();
                 const int gi0 = kt * 64 / G;
@@ -345,11 +349,32 @@ gemv_band_kernel(const BandProblems probs, const __half* __restrict__ x, int M, 
 #pragma unroll
         for (int jw = 0; jw < 4; ++jw) xr[v][jw] = make_uint2(0u, 0u);
 
+    if (XREG && tok_ok) {
+        const __half* xg = x + (size_t)g * K + (size_t)warp * (TPW * 64) + t * 4;
+#pragma unroll
+        for (int v = 0; v < TPW; ++v)
+#pragma unroll
+            for (int jw = 0; jw < 4; ++jw)
+                xr[v][jw] = __ldg(reinterpret_cast<const uint2*>(xg + v * 64 + jw * 16));
+    }
     // x sums per k-tile for the zero-point term (the 16 math warps), while the first stages are in
     // flight.  (Deferring them behind the first stage's products, and polling barriers ahead of
     // use, were both measured slower.)
     tile_sums_of_x(x, xsum, M, K, 8, warp, kMathWarps, lane);
     named_barrier_sync(3, kMathThreads);
+    float XxR[GPW], XyR[GPW];                            // XREG: this warp's group sums of x
+#pragma unroll
+    for (int q = 0; q < GPW; ++q) {
+        XxR[q] = 0.0f; XyR[q] = 0.0f;
+        if (XREG) {
+#pragma unroll
+            for (int v = 0; v < TPG; ++v) {
+                const float2 X = *reinterpret_cast<const float2*>(xs_lane + (q * TPG + v) * 8);
+                XxR[q] += X.x;
+                XyR[q] += X.y;
+            }
+        }
+    }
 
     uint32_t stage = 0, phase = 0;
     int nflush = 0;
@@ -362,7 +387,7 @@ gemv_band_kernel(const BandProblems probs, const __half* __restrict__ x, int M, 
             mbar_wait(bars + 8u * stage, phase, ctl);
             const unsigned char* st = smem + stage * (uint32_t)lay.stage_bytes;
             const float* xs = xs_lane + j * (UT * 8);
-            const bool full_stage = nt >= TPW;
+            const bool full_stage = XREG || nt >= TPW;
             float c[GPW][4];
             float zu[GPW], zl[GPW];
             uint4 pk[TPW];
@@ -371,7 +396,7 @@ gemv_band_kernel(const BandProblems probs, const __half* __restrict__ x, int M, 
                 // groups' products interleaved word by word so that no MMA waits for the last
 #pragma unroll
                 for (int v = 0; v < TPW; ++v) pk[v] = *reinterpret_cast<const uint4*>(st + o_w + v * 512);
-                if (tok_ok) {
+                if (!XREG && tok_ok) {
 #pragma unroll
                     for (int v = 0; v < TPW; ++v)
 #pragma unroll
@@ -416,12 +441,14 @@ gemv_band_kernel(const BandProblems probs, const __half* __restrict__ x, int M, 
                 }
 #pragma unroll
                 for (int q = 0; q < GPW; ++q) {
-                    float Xx = 0.0f, Xy = 0.0f;
+                    float Xx = XxR[q], Xy = XyR[q];
+                    if (!XREG) {
 #pragma unroll
-                    for (int v = 0; v < TPG; ++v) {
-                        const float2 X = *reinterpret_cast<const float2*>(xs + (q * TPG + v) * 8);
-                        Xx += X.x;
-                        Xy += X.y;
+                        for (int v = 0; v < TPG; ++v) {
+                            const float2 X = *reinterpret_cast<const float2*>(xs + (q * TPG + v) * 8);
+                            Xx += X.x;
+                            Xy += X.y;
+                        }
                     }
                     acc[0] = fmaf(-zu[q], Xx, acc[0]);
                     acc[2] = fmaf(-zl[q], Xx, acc[2]);
@@ -430,7 +457,7 @@ gemv_band_kernel(const BandProblems probs, const __half* __restrict__ x, int M, 
                         acc[3] = fmaf(-zl[q], Xy, acc[3]);
                     }
                 }
-            } else if (nt > 0) {
+            } else if (!XREG && nt > 0) {
                 // ---- ragged last stage of a band: whole groups only (K % G == 0), one at a time
 #pragma unroll
                 for (int q = 0; q < GPW; ++q) {
@@ -868,27 +895,29 @@ cudaError_t launch_gemv_band(const void* x, const GemvMatrix* mats, int count, i
     cfg.stream = st;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-#define AWQ_BAND_LAUNCH(GG, TT, ONE1)                                                                      \
+#define AWQ_BAND_LAUNCH(GG, TT, ONE1, XR)                                                            \
     do {                                                                                             \
-        const BandLayout lay = band_layout<GG, TT>(M, K);                                            \
+        const BandLayout lay = band_layout<GG, TT>(M, K, XR);                                        \
         if (lay.stages < 2) return cudaErrorInvalidValue;      /* K too large for the x-sum table */ \
         static bool done[64] = {};                                                                   \
-        e = allow_big_smem(gemv_band_kernel<GG, TT, ONE1>, done);                                          \
+        e = allow_big_smem(gemv_band_kernel<GG, TT, ONE1, XR>, done);                                \
         if (e != cudaSuccess) return e;                                                              \
         cfg.dynamicSmemBytes = lay.total;                                                            \
-        e = cudaLaunchKernelEx(&cfg, gemv_band_kernel<GG, TT, ONE1>, pr, reinterpret_cast<const __half*>(x), M, K, \
-                               lay, status_word);                                                    \
+        e = cudaLaunchKernelEx(&cfg, gemv_band_kernel<GG, TT, ONE1, XR>, pr,                         \
+                               reinterpret_cast<const __half*>(x), M, K, lay, status_word);          \
         if (e != cudaSuccess) return e;                                                              \
     } while (0)
-    if (group == 128) {
-        if (M == 1) AWQ_BAND_LAUNCH(128, 4, true);
-        else if (tpw == 4) AWQ_BAND_LAUNCH(128, 4, false);
-        else AWQ_BAND_LAUNCH(128, 2, false);
-    } else {
-        if (M == 1) AWQ_BAND_LAUNCH(64, 4, true);
-        else if (tpw == 4) AWQ_BAND_LAUNCH(64, 4, false);
-        else AWQ_BAND_LAUNCH(64, 2, false);
-    }
+    const bool xreg = tpw == 4 && K == 64 * 16 * 4;            // a band is exactly one stage
+#define AWQ_BAND_PICK(GG)                                                                            \
+    do {                                                                                             \
+        if (tpw != 4) AWQ_BAND_LAUNCH(GG, 2, false, false);                                          \
+        else if (M == 1 && xreg) AWQ_BAND_LAUNCH(GG, 4, true, true);                                 \
+        else if (M == 1) AWQ_BAND_LAUNCH(GG, 4, true, false);                                        \
+        else if (xreg) AWQ_BAND_LAUNCH(GG, 4, false, true);                                          \
+        else AWQ_BAND_LAUNCH(GG, 4, false, false);                                                   \
+    } while (0)
+    if (group == 128) AWQ_BAND_PICK(128); else AWQ_BAND_PICK(64);
+#undef AWQ_BAND_PICK
 #undef AWQ_BAND_LAUNCH
     count_launch();
     return cudaGetLastError();
