@@ -246,6 +246,12 @@ gemv_band_kernel(const BandProblems probs, const __half* __restrict__ x, int M, 
     // weight-copy warp starts filling the ring at once; everything that touches x or y first
     // waits for the preceding kernel to complete (griddepcontrol.wait).
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    // x may still be unwritten, but its lines can already be pulled into L2 (a hint; L2 stays
+    // coherent), so that the loads after the wait below do not go to HBM
+    if (warp == kMathWarps + 1) {
+        const int lines = (M * K * 2 + 127) / 128;
+        for (int i = lane; i < lines; i += 32) prefetch_l2(reinterpret_cast<const unsigned char*>(x) + (size_t)i * 128);
+    }
 
     if (warp == kMathWarps + 2) {
         // ---------------------------------------------------------------- x-copy warp
@@ -271,6 +277,7 @@ gemv_band_kernel(const BandProblems probs, const __half* __restrict__ x, int M, 
         // ------------------------------------------------------------- weight-copy warp
         // lane 0 posts the stage's byte count (x included); lanes 0, 1, 2 each issue one bulk copy
         uint32_t stage = 0, phase = 0;
+        const uint64_t once = l2_policy_evict_first();     // every packed byte is read exactly once
         for (int task = b0; task < b1; ++task) {
             const BandRef br = band_ref(probs, task);
             const int band = br.band;
@@ -287,9 +294,9 @@ gemv_band_kernel(const BandProblems probs, const __half* __restrict__ x, int M, 
                 __syncwarp();
                 const int gi0 = kt * 64 / G;
                 if (lane == 0)
-                    bulk_load(dst, br.qweight + ((size_t)band * ktiles + kt) * 512, (uint32_t)(nt * 512), bar);
+                    bulk_load_hint(dst, br.qweight + ((size_t)band * ktiles + kt) * 512, (uint32_t)(nt * 512), bar, once);
                 else if (lane == 1)
-                    bulk_load(dst + St::kScOff, br.scales + ((size_t)band * ng + gi0) * 16, (uint32_t)(ngr * 32), bar);
+                    bulk_load_hint(dst + St::kScOff, br.scales + ((size_t)band * ng + gi0) * 16, (uint32_t)(ngr * 32), bar, once);
                 else if (lane == 2)
                     bulk_load(dst + St::kZOff, br.zeros + ((size_t)(band >> 1) * ng + gi0) * 16, (uint32_t)(ngr * 16), bar);
                 if (++stage == (uint32_t)S) { stage = 0; phase ^= 1u; }
