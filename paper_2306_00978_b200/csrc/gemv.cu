@@ -92,6 +92,7 @@ __device__ __forceinline__ void tile_sums_of_x(const __half* __restrict__ x, flo
                                                int mtok, int w, int nwarps, int lane) {
     const int cpr = K / 256;                       // whole 256-column chunks per token row
     const int items = M * cpr;
+    const float inv_cpr = 1.0f / (float)cpr;
     for (int i0 = w; i0 < items; i0 += 4 * nwarps) {
         uint4 h[4];
 #pragma unroll
@@ -99,7 +100,7 @@ __device__ __forceinline__ void tile_sums_of_x(const __half* __restrict__ x, flo
             const int it = i0 + q * nwarps;
             h[q] = make_uint4(0u, 0u, 0u, 0u);
             if (it < items) {
-                const int m = it / cpr, c = it - m * cpr;
+                const int m = (int)(((float)it + 0.5f) * inv_cpr), c = it - m * cpr;   // items <= 4096: exact
                 h[q] = __ldg(reinterpret_cast<const uint4*>(x + (size_t)m * K + (size_t)c * 256) + lane);
             }
         }
@@ -116,7 +117,7 @@ __device__ __forceinline__ void tile_sums_of_x(const __half* __restrict__ x, flo
 #pragma unroll
             for (int off = 4; off >= 1; off >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, off);
             if ((lane & 7) == 0 && it < items) {
-                const int m = it / cpr, c = it - m * cpr;
+                const int m = (int)(((float)it + 0.5f) * inv_cpr), c = it - m * cpr;
                 xsum[(c * 4 + (lane >> 3)) * mtok + m] = v;
             }
         }
@@ -364,23 +365,35 @@ gemv_band_kernel(const BandProblems probs, const __half* __restrict__ x, int M, 
             for (int jw = 0; jw < 4; ++jw)
                 xr[v][jw] = __ldg(reinterpret_cast<const uint2*>(xg + v * 64 + jw * 16));
     }
-    // x sums per k-tile for the zero-point term (the 16 math warps), while the first stages are in
-    // flight.  (Deferring them behind the first stage's products, and polling barriers ahead of
-    // use, were both measured slower.)
-    tile_sums_of_x(x, xsum, M, K, 8, warp, kMathWarps, lane);
-    named_barrier_sync(3, kMathThreads);
     float XxR[GPW], XyR[GPW];                            // XREG: this warp's group sums of x
+    if (XREG) {
+        // the sums of x over this warp's groups (for the zero-point term) come straight from the
+        // fragments: 16 values per lane and k-tile, the four lanes of a token, then each lane
+        // fetches the two tokens of its accumulator columns
 #pragma unroll
-    for (int q = 0; q < GPW; ++q) {
-        XxR[q] = 0.0f; XyR[q] = 0.0f;
-        if (XREG) {
+        for (int q = 0; q < GPW; ++q) {
+            float part = 0.0f;
 #pragma unroll
-            for (int v = 0; v < TPG; ++v) {
-                const float2 X = *reinterpret_cast<const float2*>(xs_lane + (q * TPG + v) * 8);
-                XxR[q] += X.x;
-                XyR[q] += X.y;
-            }
+            for (int v = 0; v < TPG; ++v)
+#pragma unroll
+                for (int jw = 0; jw < 4; ++jw) {
+                    const float2 f0 = __half22float2(*reinterpret_cast<const __half2*>(&xr[q * TPG + v][jw].x));
+                    const float2 f1 = __half22float2(*reinterpret_cast<const __half2*>(&xr[q * TPG + v][jw].y));
+                    part += (f0.x + f0.y) + (f1.x + f1.y);
+                }
+            part += __shfl_xor_sync(0xFFFFFFFFu, part, 1);
+            part += __shfl_xor_sync(0xFFFFFFFFu, part, 2);
+            XxR[q] = __shfl_sync(0xFFFFFFFFu, part, 8 * t);
+            XyR[q] = __shfl_sync(0xFFFFFFFFu, part, 8 * t + 4);
         }
+    } else {
+        // x sums per k-tile (the 16 math warps), while the first stages are in flight.  (Deferring
+        // them behind the first stage's products, and polling barriers ahead of use, were both
+        // measured slower.)
+        tile_sums_of_x(x, xsum, M, K, 8, warp, kMathWarps, lane);
+        named_barrier_sync(3, kMathThreads);
+#pragma unroll
+        for (int q = 0; q < GPW; ++q) { XxR[q] = 0.0f; XyR[q] = 0.0f; }
     }
 
     uint32_t stage = 0, phase = 0;
