@@ -401,7 +401,9 @@ gemv_band_kernel(const BandProblems probs, const __half* __restrict__ x, int M, 
     for (int task = b0; task < b1; ++task, ++nflush) {
         float acc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
         // odd bands of a matrix use the upper 8 bytes of the pair's zero-point block
-        const int o_z = St::kZOff + warp * (GPW * 16) + (band_ref(probs, task).band & 1) * 8 + g;
+        // (every matrix has an even number of bands - N is a multiple of 128 - so a band's parity
+        // inside its matrix is the task's parity)
+        const int o_z = St::kZOff + warp * (GPW * 16) + (task & 1) * 8 + g;
         for (int j = 0; j < upb; ++j) {
             const int nt = min(UT, ktiles - j * UT) - warp * TPW;     // this warp's tiles: <= 0 .. TPW
             mbar_wait(bars + 8u * stage, phase, ctl);
