@@ -191,7 +191,7 @@ inline BandLayout band_layout(int M, int K, bool x_in_registers) {
     BandLayout l;
     l.stage_bytes = ((St::kXOff + (x_in_registers ? 0 : M * St::kXRow) + 127) / 128) * 128;
     const int xsum = (K / 64 + St::kUT) * 8 * 4;        // + one stage of slack for ragged reads
-    const int red = 2 * kMathWarps * 8 * 16 * 4;        // two buffers of [warp][token][row] fp32
+    const int red = 6 * kMathWarps * 4 * 16 * 4;        // one buffer per stage of [warp][token < 4][row] fp32
     int s = (kSmemBudget - xsum - red - 256) / l.stage_bytes;
     l.stages = s > 6 ? 6 : s;
     l.xsum_off = l.stages * l.stage_bytes;
@@ -219,7 +219,7 @@ gemv_band_kernel(const BandProblems probs, const __half* __restrict__ x, int M, 
     static_assert(TPW % TPG == 0, "a warp's tiles must cover whole groups");
     const int S = lay.stages;
     const uint32_t sbase = smem_u32(smem);
-    // barriers: full[s] at 8s, empty[s] at 64 + 8s, flush_req[b] at 128 + 8b, red_free[b] at 144 + 8b
+    // barriers: full[s] at 8s, empty[s] at 64 + 8s, flush_req[s] at 128 + 8s
     const uint32_t bars = sbase + (uint32_t)lay.bar_off;
 
     const int ktiles = K / 64, ng = K / G;
@@ -230,14 +230,12 @@ gemv_band_kernel(const BandProblems probs, const __half* __restrict__ x, int M, 
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x < (unsigned)S) {
-        mbar_init(bars + 8u * threadIdx.x, 1);
-        mbar_init(bars + 64u + 8u * threadIdx.x, kMathWarps);
+        mbar_init(bars + 8u * threadIdx.x, 1);                      // full: the copy warp's byte count
+        mbar_init(bars + 64u + 8u * threadIdx.x, kMathWarps + 1);   // empty: math warps and the flush warp
+        mbar_init(bars + 128u + 8u * threadIdx.x, kMathWarps);      // flush_req: a band's sums are in red[stage]
         mbar_fence_init();
-    } else if (threadIdx.x >= 32 && threadIdx.x < 34) {
-        mbar_init(bars + 128u + 8u * (threadIdx.x - 32), kMathWarps);
-        mbar_init(bars + 144u + 8u * (threadIdx.x - 32), 1);
-        mbar_fence_init();
-        if (threadIdx.x == 32) s_abort = 0u;
+    } else if (threadIdx.x == 32) {
+        s_abort = 0u;
     }
     __syncthreads();
     const WaitCtl ctl{status_word, &s_abort};
@@ -321,20 +319,33 @@ gemv_band_kernel(const BandProblems probs, const __half* __restrict__ x, int M, 
     float* red = reinterpret_cast<float*>(smem + lay.red_off);
     if (warp == kMathWarps + 1) {
         // ------------------------------------------------------------------ flush warp
-        int nflush = 0;
-        for (int task = b0; task < b1; ++task, ++nflush) {
+        // Walks the stages like a math warp.  The sums of a band wait in the reduction buffer of
+        // the band's last stage; the flush warp is one of the arrivals on that stage's "empty"
+        // barrier, so the buffer cannot be overwritten before it has been read and the math
+        // warps never wait for the flush warp.
+        uint32_t stage = 0, phase = 0, req_phase = 0;               // req_phase: one parity bit per stage
+        for (int task = b0; task < b1; ++task) {
             const BandRef br = band_ref(probs, task);
-            const uint32_t b = (uint32_t)nflush & 1u, use = ((uint32_t)nflush >> 1) & 1u;
-            mbar_wait_relaxed(bars + 128u + 8u * b, use, ctl);
-            const float* rb = red + b * (kMathWarps * 8 * 16);
-            for (int idx = lane; idx < M * 16; idx += 32) {          // idx = token * 16 + row
-                float sum = 0.0f;
+            for (int j = 0; j < upb; ++j) {
+                if (!mbar_wait_relaxed(bars + 8u * stage, phase, ctl)) return;
+                if (j == upb - 1) {
+                    if (!mbar_wait_relaxed(bars + 128u + 8u * stage, (req_phase >> stage) & 1u, ctl)) return;
+                    req_phase ^= 1u << stage;
+                    const float* rb = red + stage * (kMathWarps * 4 * 16);
+                    for (int idx = lane; idx < M * 16; idx += 32) {  // idx = token * 16 + row
+                        float s0 = 0.0f, s1 = 0.0f, s2 = 0.0f, s3 = 0.0f;
 #pragma unroll
-                for (int w = 0; w < kMathWarps; ++w) sum += rb[w * 128 + idx];
-                br.y[(size_t)(idx >> 4) * br.n + br.band * 16 + (idx & 15)] = __float2half_rn(sum);
+                        for (int w = 0; w < kMathWarps; w += 4) {
+                            s0 += rb[w * 64 + idx]; s1 += rb[(w + 1) * 64 + idx];
+                            s2 += rb[(w + 2) * 64 + idx]; s3 += rb[(w + 3) * 64 + idx];
+                        }
+                        br.y[(size_t)(idx >> 4) * br.n + br.band * 16 + (idx & 15)] = __float2half_rn((s0 + s1) + (s2 + s3));
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bars + 64u + 8u * stage);
+                if (++stage == (uint32_t)S) { stage = 0; phase ^= 1u; }
             }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bars + 144u + 8u * b);
         }
         return;
     }
@@ -397,8 +408,7 @@ gemv_band_kernel(const BandProblems probs, const __half* __restrict__ x, int M, 
     }
 
     uint32_t stage = 0, phase = 0;
-    int nflush = 0;
-    for (int task = b0; task < b1; ++task, ++nflush) {
+    for (int task = b0; task < b1; ++task) {
         float acc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
         // odd bands of a matrix use the upper 8 bytes of the pair's zero-point block
         // (every matrix has an even number of bands - N is a multiple of 128 - so a band's parity
@@ -514,18 +524,25 @@ gemv_band_kernel(const BandProblems probs, const __half* __restrict__ x, int M, 
                     }
                 }
             }
+            if (j == upb - 1) {
+                // the band's sums go to the reduction buffer of its last stage: red[stage][warp][token][row]
+                // (tokens 4..7 of the fragment do not exist in this kernel: M <= 4)
+                float* rb = red + stage * (kMathWarps * 4 * 16) + warp * 64;
+                if (t < 2) {
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        if (ONE && (i & 1)) continue;
+                        rb[(2 * t + (i & 1)) * 16 + g + (i >> 1) * 8] = acc[i];
+                    }
+                }
+            }
             __syncwarp();
-            if (lane == 0) mbar_arrive(bars + 64u + 8u * stage);
+            if (lane == 0) {
+                if (j == upb - 1) mbar_arrive(bars + 128u + 8u * stage);
+                mbar_arrive(bars + 64u + 8u * stage);
+            }
             if (++stage == (uint32_t)S) { stage = 0; phase ^= 1u; }
         }
-        // hand this band's sums to the flush warp: red[buffer][warp][token][row]
-        const uint32_t b = (uint32_t)nflush & 1u, use = ((uint32_t)nflush >> 1) & 1u;
-        mbar_wait(bars + 144u + 8u * b, use ^ 1u, ctl);
-        float* rb = red + b * (kMathWarps * 8 * 16) + warp * 128;
-#pragma unroll
-        for (int i = 0; i < 4; ++i) rb[(2 * t + (i & 1)) * 16 + g + (i >> 1) * 8] = acc[i];
-        __syncwarp();
-        if (lane == 0) mbar_arrive(bars + 128u + 8u * b);
     }
 }
 
