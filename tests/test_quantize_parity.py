@@ -92,3 +92,35 @@ def test_degenerate_and_grid_aligned_groups():
     assert float(scales[5, 0]) == 1.0 and not codes[5, :G].any() and zeros[5, 0] == 0
     back = orc.dequantize(codes, zeros, scales, G)
     assert np.array_equal(back, W.astype(np.float64))
+
+
+def test_rounding_boundaries_bit_exact():
+    """Weights whose quotient w / Delta sits exactly on, one fp16 step below and one above a
+    half-integer (where round-to-nearest-even decides the code), and groups whose range is tiny
+    against their magnitude (quotients in the thousands): the kernel replaces the per-weight
+    division by a multiplication only away from such points, so these exercise its exact path."""
+    import torch
+    from paper_2306_00978_b200 import binding
+    N, K, G = 128, 256, 128
+    rng = np.random.default_rng(11)
+    W = np.zeros((N, K), dtype=np.float16)
+    delta = np.float16(2.0 ** -6)
+    for n in range(N):
+        for gi in range(K // G):
+            k = rng.integers(0, 15, size=G).astype(np.float32)
+            base = (k + 0.5) * np.float32(delta)                   # exact in fp16: quotient k + 0.5
+            w = base.astype(np.float16)
+            step = np.spacing(w)                                   # one fp16 step at each value
+            choice = rng.integers(0, 3, size=G)
+            w = np.where(choice == 1, w - step, np.where(choice == 2, w + step, w)).astype(np.float16)
+            w[0], w[1] = np.float16(0.0), np.float16(15.0 * float(delta))   # min and max fix Delta = 2^-6
+            if n % 4 == 3:                                         # tiny range on a large offset
+                w = (np.float16(8.0) + (k * np.float32(2.0 ** -7)).astype(np.float16)).astype(np.float16)
+            W[n, gi * G:(gi + 1) * G] = w
+    s = np.ones(K, dtype=np.float32)                               # alpha = 0
+    codes, zeros, scales = orc.quantize(W, s, G)
+    qw, sc, zp = binding.quantize_pack(to_cuda(W), None, 0.0, G)
+    torch.cuda.synchronize()
+    assert np.array_equal(qw.cpu().numpy().view(np.uint32).reshape(-1), orc.pack_qweight(codes).reshape(-1))
+    assert np.array_equal(sc.cpu().numpy().view(np.uint16).reshape(-1), orc.pack_scales(scales).view(np.uint16).reshape(-1))
+    assert np.array_equal(zp.cpu().numpy().reshape(-1), orc.pack_zeros(zeros).reshape(-1))
