@@ -22,6 +22,9 @@ What is computed, and where it comes from
 * dequantize         (q - z) * Delta, exact in fp64.
 * linear             y = x . dequant(Wq)^T in fp64 (Sec. 4.2, on-the-fly weight
                      dequantization followed by the matrix product; here unfused).
+* search_alpha       the scale search of Sec. 3.2: L(s) = || Q(W diag(s)) (diag(s)^-1 X) - W X ||
+                     (Eq. 4) evaluated for s = s_X ** alpha over a given list of alpha (Eq. 5),
+                     and the first alpha of least loss.
 
 Readings adopted where the paper is silent
 ------------------------------------------
@@ -31,6 +34,10 @@ q = clamp(Round(w'/Delta) + z, 0, 15).  Round is round-half-to-even in fp32; Del
 rounded to fp16 *before* it is used, so that quantize and dequantize use the same grid; the
 group's raw min and max are used (the range is not widened to contain 0); a degenerate
 group (Delta rounds to 0 or is not finite) takes Delta = 1.  w * s stays in fp32.
+The search's norm is not named in the paper: the mean of the squared differences is used (any
+monotone function of the Frobenius norm has the same minimizer); diag(s)^-1 X is rounded to fp16
+once, because that is what the layer is given; the grid of alpha is an argument (the paper says
+"a grid size of 20" over [0, 1] without saying whether 1 is a grid point).
 Parity for these asymmetric details is unpinned by the paper (it prints no worked numeric
 example of Q); they are pinned by closed-form invariants, grid-aligned round trips and
 brute-force enumeration in tests/test_oracle_pins.py.
@@ -242,6 +249,26 @@ def linear_from_packed(x, qweight, scales_gn, zeros_packed, N: int, K: int, grou
     if rows is not None:
         codes, zeros, scales = codes[rows], zeros[rows], scales[rows]
     return linear(x, dequantize(codes, zeros, scales, group))
+
+
+def search_alpha(W, act_mean_abs, X, group: int, alphas):
+    """Eq. 4 and Eq. 5: for every alpha, s = s_X ** alpha, quantize W diag(s), and measure the
+    layer-output error on the calibration activations X (fp16 [M][K]) against the fp16 layer:
+        loss(alpha) = mean over (m, n) of ( sum_k dequant(Q(W s))[n][k] * fp16(X[m][k] / s[k])
+                                            - sum_k W[n][k] * X[m][k] ) ** 2,        all in fp64.
+    Returns (losses fp64 [len(alphas)], index of the first least loss)."""
+    W = np.asarray(W)
+    X = np.asarray(X)
+    assert W.dtype == np.float16 and X.dtype == np.float16
+    y_ref = X.astype(np.float64) @ W.astype(np.float64).T
+    losses = np.zeros(len(alphas), dtype=np.float64)
+    for i, alpha in enumerate(alphas):
+        s = channel_scale(act_mean_abs, float(np.float32(alpha)))      # alpha is an fp32 argument
+        codes, zeros, scales = quantize(W, s, group)
+        xs = (X.astype(np.float32) / s[None, :]).astype(np.float16)
+        y = linear(xs, dequantize(codes, zeros, scales, group))
+        losses[i] = np.mean((y - y_ref) ** 2)
+    return losses, int(np.argmin(losses))
 
 
 def parity_errors(y, y_ref):

@@ -419,3 +419,76 @@ def test_parity_error_helper():
     y_ref = np.array([[3.0, 4.0]])
     rel, mx = orc.parity_errors(np.array([[3.0, 4.5]]), y_ref)
     assert abs(rel - 0.1) < 1e-12 and abs(mx - 0.125) < 1e-12
+
+
+# ----------------------------------------------------------------- scale search (Eq. 4, Eq. 5)
+def _search_inputs(seed, N=64, K=256, M=48, outliers=True):
+    rng = np.random.default_rng(seed)
+    W = (rng.standard_normal((N, K)) * 0.05).astype(np.float16)
+    X = rng.standard_normal((M, K)).astype(np.float32)
+    if outliers:                      # a few input channels carry activations ~30x larger (Sec. 3.1)
+        X[:, rng.choice(K, size=4, replace=False)] *= 30.0
+    X = X.astype(np.float16)
+    a = np.abs(X.astype(np.float32)).mean(axis=0).astype(np.float32)
+    return W, a, X
+
+
+def test_search_alpha_zero_is_plain_rtn_loss():
+    """alpha = 0 is "do not scale" (Sec. 3.2): its loss is the round-to-nearest layer's output
+    error, written out here without the search routine."""
+    W, a, X = _search_inputs(1)
+    losses, _ = orc.search_alpha(W, a, X, 128, [0.0])
+    codes, zeros, scales = orc.quantize(W, np.ones(W.shape[1], dtype=np.float32), 128)
+    Wd = orc.dequantize(codes, zeros, scales, 128)
+    direct = np.mean((X.astype(np.float64) @ (Wd - W.astype(np.float64)).T) ** 2)
+    assert np.isclose(losses[0], direct, rtol=1e-12)
+
+
+def test_search_alpha_brute_force_tiny():
+    """A tiny case evaluated element by element with Python loops (Eq. 4 as printed)."""
+    rng = np.random.default_rng(2)
+    N, K, M, G = 2, 64, 3, 64
+    W = (rng.standard_normal((N, K)) * 0.1).astype(np.float16)
+    X = rng.standard_normal((M, K)).astype(np.float16)
+    a = np.abs(X.astype(np.float32)).mean(axis=0).astype(np.float32)
+    alphas = [0.0, 0.5, 1.0]
+    losses, best = orc.search_alpha(W, a, X, G, alphas)
+    for i, alpha in enumerate(alphas):
+        s = orc.channel_scale(a, alpha)
+        codes, zeros, scales = orc.quantize(W, s, G)
+        total = 0.0
+        for m in range(M):
+            for n in range(N):
+                yq = 0.0
+                yr = 0.0
+                for k in range(K):
+                    wq = (float(codes[n, k]) - float(zeros[n, k // G])) * float(scales[n, k // G])
+                    xs = float(np.float16(np.float32(X[m, k]) / s[k]))
+                    yq += wq * xs
+                    yr += float(W[n, k]) * float(X[m, k])
+                total += (yq - yr) ** 2
+        assert np.isclose(losses[i], total / (M * N), rtol=1e-9)
+    assert best == int(np.argmin(losses))
+
+
+def test_search_alpha_loss_scales_with_the_square_of_x():
+    """Multiplying the calibration activations by 2 (exact in fp16) with the statistic s_X held
+    fixed multiplies every output difference by 2, hence the loss by 4."""
+    W, a, X = _search_inputs(3)
+    alphas = [0.0, 0.25, 0.5, 1.0]
+    l1, b1 = orc.search_alpha(W, a, X, 128, alphas)
+    l2, b2 = orc.search_alpha(W, a, (X.astype(np.float32) * 2).astype(np.float16), 128, alphas)
+    assert np.allclose(l2, 4.0 * l1, rtol=1e-12) and b1 == b2
+
+
+def test_search_alpha_prefers_scaling_when_activations_have_outliers():
+    """Sec. 3.1-3.2: protecting the weight channels that meet large activations lowers the
+    output error, so with outlier channels some alpha > 0 beats alpha = 0; without outliers and
+    with a flat statistic every alpha gives s = 1 and the same loss."""
+    W, a, X = _search_inputs(4, outliers=True)
+    alphas = [i / 20 for i in range(20)]
+    losses, best = orc.search_alpha(W, a, X, 128, alphas)
+    assert best > 0 and losses[best] < 0.9 * losses[0]
+    flat = np.ones_like(a)
+    lf, _ = orc.search_alpha(W, flat, X, 128, [0.0, 0.5, 1.0])
+    assert lf[0] == lf[1] == lf[2]
