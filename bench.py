@@ -297,6 +297,26 @@ def quantize_section(peaks, reps: int = 10):
             "note": "includes the output allocation of the Python binding"}
 
 
+def search_section():
+    """Scale search (Sec. 3.2) on one 4096 -> 4096 layer: 20 grid points, 512 synthetic calibration
+    tokens with outlier channels; wall-clock of the call (it returns its result on the host)."""
+    import time
+    import torch
+    from paper_2306_00978_b200 import binding
+    N, K, M = 4096, 4096, 512
+    W = torch.from_numpy(synth.weight(2000, N, K)).cuda()
+    X = torch.from_numpy(synth.calibration(2000, K, M)).cuda()
+    a = X.float().abs().mean(dim=0).contiguous()
+    alphas = [i / 20 for i in range(20)]
+    binding.search_alpha(W, a, X, GROUP, alphas)
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    losses, best = binding.search_alpha(W, a, X, GROUP, alphas)
+    dt = time.perf_counter() - t0
+    return {"shape": f"{K}->{N}", "calibration_tokens": M, "grid": len(alphas), "ms": dt * 1e3,
+            "best_alpha": alphas[best], "loss_best_over_loss_alpha0": losses[best] / losses[0]}
+
+
 # ------------------------------------------------------------------- oracle (CPU) arm
 def _oracle_layer_inputs(max_rows=None):
     """Quantizes one decoder layer's matrices with the oracle; optionally only the first
@@ -515,6 +535,7 @@ def main():
     if rank == 0 and not args.skip_extras:
         line["gemm_m2048"] = gemm_section(peaks)
         line["quantize_pack"] = quantize_section(peaks)
+        line["alpha_search"] = search_section()
         if world == 1:
             del graphs, e2e_graphs, layers
             torch.cuda.empty_cache()

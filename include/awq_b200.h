@@ -163,6 +163,29 @@ int awq_linear_path(const void* x, const void* qweight, const void* scales, cons
 int awq_linear_gemv_static(const void* x, const void* qweight, const void* scales, const void* zeros,
                             void* y, int M, int N, int K, int group, void* stream);
 
+/*
+ * Scale search (Sec. 3.2).  For each alpha_i of `alphas`: s = s_X^alpha_i (Eq. 5, s_X = act_mean_abs),
+ * Wq = awq_quantize_pack(W, s), and
+ *   loss_i = mean over (m, n) of ( awq_linear(fp16(X / s), Wq)[m][n] - sum_k X[m][k] W[n][k] )^2   (Eq. 4;
+ * the paper does not name its norm: the mean squared difference has the same minimizer as any other
+ * monotone function of the Frobenius norm).  The quantizer and the layer are the library's own
+ * kernels, so the search scores exactly what deployment runs; the fp16 reference product is a cuBLAS
+ * GEMM with fp32 accumulation.  The paper uses 20 grid points over [0, 1]; the grid is the caller's.
+ * W: in, fp16 [N][K] (device).  act_mean_abs: in, fp32 [K] (device).  X: in, fp16 [M][K] calibration
+ * activations (device), M >= 1.  alphas: in, HOST array of n_alphas <= 64 values in [0, 1].
+ * losses: out, HOST array of n_alphas floats.  best_index: out, HOST, index of the first least loss
+ * (a loss that is not finite is never chosen unless all are).  scratch: device memory of at least
+ * awq_search_scratch_bytes(M, N, K, group) bytes, 256-byte aligned, owned by the caller.
+ * The call enqueues on `stream` and then SYNCHRONIZES it (the result is returned on the host); it
+ * must not run inside a stream capture.  A registered workspace is used as awq_linear uses it.
+ * Errors: those of awq_quantize_pack and awq_linear; AWQ_ERR_BAD_ARGUMENT for a bad list or a
+ * scratch that is too small; AWQ_ERR_CUDA if cuBLAS fails.
+ */
+size_t awq_search_scratch_bytes(int M, int N, int K, int group);
+int awq_search_alpha(const void* W, const float* act_mean_abs, const void* X, int M, int N, int K, int group,
+                     const float* alphas, int n_alphas, float* losses, int* best_index,
+                     void* scratch, size_t scratch_bytes, void* stream);
+
 /* Workspace (scratch for partial sums and arrival counters).
  * awq_workspace_bytes: bytes awq_linear can use for this problem (0 if none).  For M <= 16 the
  * split-K matrix-vector kernel REQUIRES them.  For M > 128 with N a multiple of 256 they are

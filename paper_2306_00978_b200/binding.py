@@ -23,7 +23,7 @@ EXPORTS = (
     "awq_channel_scale", "awq_linear", "awq_linear_path", "awq_workspace_bytes",
     "awq_set_workspace", "awq_unpack_canonical", "awq_poll_status", "awq_status_string",
     "awq_last_cuda_error", "awq_layout_version", "awq_launch_count", "awq_linear_gemv_static",
-    "awq_linear_multi",
+    "awq_linear_multi", "awq_search_scratch_bytes", "awq_search_alpha",
 )
 
 
@@ -57,6 +57,8 @@ def lib() -> ctypes.CDLL:
     L.awq_linear_path.restype, L.awq_linear_path.argtypes = i, [vp, vp, vp, vp, vp, i, i, i, i, i, vp]
     L.awq_linear_gemv_static.restype, L.awq_linear_gemv_static.argtypes = i, [vp, vp, vp, vp, vp, i, i, i, i, vp]
     L.awq_linear_multi.restype, L.awq_linear_multi.argtypes = i, [vp, vp, i, i, i, i, vp]
+    L.awq_search_scratch_bytes.restype, L.awq_search_scratch_bytes.argtypes = sz, [i, i, i, i]
+    L.awq_search_alpha.restype, L.awq_search_alpha.argtypes = i, [vp, vp, vp, i, i, i, i, vp, i, vp, vp, vp, sz, vp]
     L.awq_workspace_bytes.restype, L.awq_workspace_bytes.argtypes = sz, [i, i, i, i]
     L.awq_set_workspace.restype, L.awq_set_workspace.argtypes = i, [vp, sz]
     L.awq_unpack_canonical.restype, L.awq_unpack_canonical.argtypes = i, [vp, vp, vp, i, i, i, vp, vp, vp, vp]
@@ -197,6 +199,29 @@ def linear_gemv_static(x: torch.Tensor, qweight: torch.Tensor, scales: torch.Ten
         _dev(out, torch.float16, "out"), M, N, K, int(group), _stream())
     _check(rc, "awq_linear_gemv_static")
     return out
+
+
+def search_alpha(W: torch.Tensor, act_mean_abs: torch.Tensor, X: torch.Tensor, group: int, alphas):
+    """awq_search_alpha (Sec. 3.2): returns (losses as a list of floats, index of the first least loss)."""
+    N, K = W.shape
+    M = X.shape[0]
+    n = len(alphas)
+    need = int(lib().awq_search_scratch_bytes(M, N, K, int(group)))
+    if need == 0:
+        raise AwqError(f"shape N={N}, K={K}, group={group} is not accepted")
+    scratch = torch.empty(need, dtype=torch.uint8, device=W.device)
+    if M <= 16:
+        ensure_workspace(workspace_bytes(M, N, K, group))
+    elif M > 128:
+        ensure_workspace(workspace_bytes(M, N, K, group))
+    a = (ctypes.c_float * n)(*[float(v) for v in alphas])
+    losses = (ctypes.c_float * n)()
+    best = ctypes.c_int(0)
+    rc = lib().awq_search_alpha(_dev(W, torch.float16, "W"), _dev(act_mean_abs, torch.float32, "act_mean_abs"),
+                                _dev(X, torch.float16, "X"), M, N, K, int(group), a, n, losses,
+                                ctypes.byref(best), scratch.data_ptr(), need, _stream())
+    _check(rc, "awq_search_alpha")
+    return [float(v) for v in losses], int(best.value)
 
 
 def unpack_canonical(qweight, scales, zeros, N: int, K: int, group: int):

@@ -250,6 +250,50 @@ int awq_linear(const void* x, const void* qweight, const void* scales, const voi
     return awq_linear_path(x, qweight, scales, zeros, y, M, N, K, group, AWQ_PATH_AUTO, stream);
 }
 
+size_t awq_search_scratch_bytes(int M, int N, int K, int group) {
+    if (check_shape(N, K, group) != AWQ_OK || M < 1) return 0;
+    return search_scratch_bytes(M, N, K, group);
+}
+
+int awq_search_alpha(const void* W, const float* act_mean_abs, const void* X, int M, int N, int K, int group,
+                     const float* alphas, int n_alphas, float* losses, int* best_index,
+                     void* scratch, size_t scratch_bytes, void* stream) {
+    if (int rc = check_shape(N, K, group)) return rc;
+    if (M < 1) return AWQ_ERR_BAD_SHAPE;
+    if (!W || !act_mean_abs || !X || !alphas || !losses || !best_index || !scratch) return AWQ_ERR_NULL_POINTER;
+    if (n_alphas < 1 || n_alphas > kMaxSearchAlphas) return AWQ_ERR_BAD_ARGUMENT;
+    for (int i = 0; i < n_alphas; ++i)
+        if (!(alphas[i] >= 0.0f && alphas[i] <= 1.0f)) return AWQ_ERR_BAD_ARGUMENT;
+    if (scratch_bytes < search_scratch_bytes(M, N, K, group)) return AWQ_ERR_BAD_ARGUMENT;
+    if (!aligned16(W) || !aligned16(X) || (reinterpret_cast<uintptr_t>(scratch) & 255u) != 0) return AWQ_ERR_MISALIGNED;
+    const cudaStream_t st = (cudaStream_t)stream;
+    float *s, *yref, *dev_losses;
+    double* partials;
+    void *xs, *qw, *sc, *zp, *yq;
+    search_carve(scratch, M, N, K, group, &s, &xs, &qw, &sc, &zp, &yq, &yref, &partials, &dev_losses);
+    if (int rc = note_cuda(launch_reference_product(W, X, yref, M, N, K, st))) return rc;
+    for (int i = 0; i < n_alphas; ++i) {
+        if (int rc = awq_channel_scale(act_mean_abs, alphas[i], s, K, stream)) return rc;
+        if (int rc = awq_quantize_pack(W, act_mean_abs, alphas[i], group, qw, sc, zp, N, K, stream)) return rc;
+        if (int rc = note_cuda(launch_divide_by_scale(X, s, xs, M, K, st))) return rc;
+        if (int rc = awq_linear(xs, qw, sc, zp, yq, M, N, K, group, stream)) return rc;
+        if (int rc = note_cuda(launch_mean_squared_difference(yq, yref, (size_t)M * N, partials, dev_losses + i, st)))
+            return rc;
+    }
+    if (int rc = note_cuda(cudaMemcpyAsync(losses, dev_losses, (size_t)n_alphas * sizeof(float),
+                                           cudaMemcpyDeviceToHost, st)))
+        return rc;
+    if (int rc = note_cuda(cudaStreamSynchronize(st))) return rc;
+    int best = 0;
+    bool have = false;
+    for (int i = 0; i < n_alphas; ++i) {
+        if (!std::isfinite(losses[i])) continue;
+        if (!have || losses[i] < losses[best]) { best = i; have = true; }
+    }
+    *best_index = best;
+    return AWQ_OK;
+}
+
 int awq_unpack_canonical(const void* qweight, const void* scales, const void* zeros,
                          int N, int K, int group,
                          uint8_t* codes, uint16_t* scales_nk, uint8_t* zeros_nk, void* stream) {

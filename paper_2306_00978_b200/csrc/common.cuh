@@ -55,6 +55,17 @@ cudaError_t launch_gemv_splitk(const void* x, const void* qweight, const void* s
                                void* y, int M, int N, int K, int group, void* workspace,
                                unsigned int* status_word, int sms, cudaStream_t st);
 
+// scale search (search.cu)
+constexpr int kMaxSearchAlphas = 64;
+size_t search_scratch_bytes(int M, int N, int K, int group);
+void search_carve(void* base, int M, int N, int K, int group, float** s, void** xs, void** qweight,
+                  void** scales, void** zeros, void** yq, float** yref, double** partials, float** losses);
+cudaError_t launch_reference_product(const void* W, const void* X, float* yref, int M, int N, int K,
+                                     cudaStream_t st);
+cudaError_t launch_divide_by_scale(const void* X, const float* s, void* xs, int M, int K, cudaStream_t st);
+cudaError_t launch_mean_squared_difference(const void* yq, const float* yref, size_t n, double* partials,
+                                           float* out, cudaStream_t st);
+
 // the matrix-vector kernel's built-in scratch (no allocation): address on the current device
 cudaError_t gemv_static_scratch(void** out);
 int gemv_static_max_m();
