@@ -88,3 +88,24 @@ def test_decode_layer_7b_m1_sampled():
         rows, Wd = ref[name]
         x = x4 if K == 4096 else x11
         assert_parity(outs[name].cpu().numpy()[:, rows], orc.linear(x, Wd), f"7B {name} M=1")
+
+
+@pytest.mark.parametrize("name,K,N", list(synth.LLAMA2_70B_MLP))
+def test_70b_mlp_batch_sweep_sampled(name, K, N):
+    """configs[3]: the 70B MLP shapes over the small-batch sweep M in {1, 4, 8, 16} through
+    awq_linear's own dispatch (band kernel, split-K kernel, tensor-core kernel)."""
+    from paper_2306_00978_b200 import binding
+    seed = 4300 + (0 if name == "up_proj" else 1)
+    W, a, s = _layer(seed, N, K)
+    qw, sc, zp = binding.quantize_pack(to_cuda(W), to_cuda(a), ALPHA, GROUP)
+    rows = _sample_rows(np.random.default_rng(seed), N, count=48)
+    codes, zeros, scales = orc.quantize(W[rows], s, GROUP)
+    Wd = orc.dequantize(codes, zeros, scales, GROUP)
+    del W
+    x_all = synth.activations(seed, 16, K)
+    xs_all = (x_all.astype(np.float32) / s[None, :]).astype(np.float16)
+    for M in (1, 4, 8, 16):
+        xs = np.ascontiguousarray(xs_all[:M])
+        y = binding.linear(to_cuda(xs), qw, sc, zp, N, K, GROUP)
+        binding.poll_status()
+        assert_parity(y.cpu().numpy()[:, rows], orc.linear(xs, Wd), f"70B {name} M={M}")
