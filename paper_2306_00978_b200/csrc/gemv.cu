@@ -223,7 +223,7 @@ gemv_band_kernel(const BandProblems probs, const __half* __restrict__ x, int M, 
     const uint32_t bars = sbase + (uint32_t)lay.bar_off;
 
     const int ktiles = K / 64, ng = K / G;
-    const int upb = (ktiles + UT - 1) / UT;                           // units per band
+    const int upb = XREG ? 1 : (ktiles + UT - 1) / UT;                // units (stages) per band
     const int nbands = probs.first_band[probs.count];
     const int b0 = (int)(((unsigned)nbands * blockIdx.x) / gridDim.x);
     const int b1 = (int)(((unsigned)nbands * (blockIdx.x + 1)) / gridDim.x);
