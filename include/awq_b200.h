@@ -60,9 +60,11 @@ typedef enum AwqStatus {
 
 /* Which kernel awq_linear_path runs. */
 typedef enum AwqPath {
-    AWQ_PATH_AUTO = 0,          /* what awq_linear does: chosen from M */
+    AWQ_PATH_AUTO = 0,          /* what awq_linear does: the matrix-vector kernels for M <= 8 (and for
+                                   M <= 16 if a workspace of awq_workspace_bytes is registered), else
+                                   the tensor-core kernels */
     AWQ_PATH_GEMV = 1,          /* fused dequant matrix-vector kernel, M <= 16: band kernel when
-                                   M <= 4 and N/16 is not much below the SM count, else split-K */
+                                   M <= 8 and N/16 is not much below the SM count, else split-K */
     AWQ_PATH_GEMM = 2,          /* tcgen05 tensor-core kernel, any M >= 1: pairs of SMs
                                    (cta_group::2, 256 channels x 256 tokens per tile) when
                                    M > 128 and N is a multiple of 256, else one SM per tile */
@@ -102,13 +104,15 @@ int awq_channel_scale(const float* act_mean_abs, float alpha, float* s, int K, v
  * x: in, fp16 [M][K].  y: out, fp16 [M][N], fully overwritten; must not alias an input.
  * M <= 8 runs a matrix-vector kernel (HBM-bound; the 4-bit codes enter warp-level tensor-core
  * products exactly, accumulation, zero point and Delta in fp32, one rounding to fp16 at the
- * end), larger M the tcgen05 kernel ((q - z) * Delta rounded once to fp16, fp32 accumulation
- * in tensor memory).  Results are bit-reproducible.
- * The split-K matrix-vector kernel (used when N is small or M > 4) combines partial sums in a
+ * end), and so does 8 < M <= 16 when the registered workspace holds awq_workspace_bytes; larger
+ * M, or 8 < M <= 16 without that workspace, the tcgen05 kernel ((q - z) * Delta rounded once to
+ * fp16, fp32 accumulation in tensor memory).  Results are bit-reproducible.
+ * The split-K matrix-vector kernel (used when N is small or M > 8) combines partial sums in a
  * fixed order through the registered workspace; calls that use the workspace must not
  * overlap on the GPU (issue them on one stream).
- * Errors: AWQ_ERR_NO_WORKSPACE if that kernel is chosen and awq_workspace_bytes(M,N,K,group)
- * exceeds the registered size; shape / pointer errors as listed in AwqStatus.
+ * Errors: AWQ_ERR_NO_WORKSPACE if M <= 8, that kernel is chosen and
+ * awq_workspace_bytes(M,N,K,group) exceeds the registered size; shape / pointer errors as listed
+ * in AwqStatus.
  */
 int awq_linear(const void* x, const void* qweight, const void* scales, const void* zeros,
                void* y, int M, int N, int K, int group, void* stream);
@@ -118,7 +122,7 @@ int awq_linear(const void* x, const void* qweight, const void* scales, const voi
  * Q, K and V projections into a single kernel because at batch 1 a kernel's run time is
  * comparable to its launch overhead).  y_i = x . dequant(Wq_i)^T for i < count, count <= 4; all
  * matrices share K and `group`, each has its own N.  `problems` is a HOST array read during the
- * call.  For M <= 4 with enough output rows in total the matrices are served by ONE launch of
+ * call.  For M <= 8 with enough output rows in total the matrices are served by ONE launch of
  * the matrix-vector band kernel; otherwise this is the same as `count` awq_linear calls.  Each
  * output is what awq_linear would give with the band kernel (bit-identical when awq_linear picks
  * that kernel for the matrix on its own, within the usual tolerance otherwise).

@@ -19,7 +19,7 @@
 // first weight stages are in flight.  Nothing is rounded to fp16 before the output.
 //
 // Two work decompositions:
-//   gemv_band_kernel    M <= 4, N/16 not much smaller than the SM count.  A task is one 16-row
+//   gemv_band_kernel    M <= 8, N/16 not much smaller than the SM count.  A task is one 16-row
 //                       band over all of K (contiguous in the band-major weight layout); the 16
 //                       math warps split the columns of each stage and their sums meet in
 //                       shared memory - no traffic between blocks, no workspace.
@@ -152,6 +152,7 @@ template <int G, int TPW> struct BandStage {
 
 struct BandLayout {
     int stage_bytes, stages, xsum_off, red_off, bar_off, total;
+    int red_tokens;                  // tokens per reduction buffer row block: 4 (M <= 4) or 8
 };
 
 // Up to four weight matrices that share x, K and the group size (fused q/k/v or gate/up
@@ -191,7 +192,8 @@ inline BandLayout band_layout(int M, int K, bool x_in_registers) {
     BandLayout l;
     l.stage_bytes = ((St::kXOff + (x_in_registers ? 0 : M * St::kXRow) + 127) / 128) * 128;
     const int xsum = (K / 64 + St::kUT) * 8 * 4;        // + one stage of slack for ragged reads
-    const int red = 6 * kMathWarps * 4 * 16 * 4;        // one buffer per stage of [warp][token < 4][row] fp32
+    l.red_tokens = M <= 4 ? 4 : 8;
+    const int red = 6 * kMathWarps * l.red_tokens * 16 * 4;   // one buffer per stage of [warp][token][row] fp32
     int s = (kSmemBudget - xsum - red - 256) / l.stage_bytes;
     l.stages = s > 6 ? 6 : s;
     l.xsum_off = l.stages * l.stage_bytes;
@@ -331,13 +333,14 @@ gemv_band_kernel(const BandProblems probs, const __half* __restrict__ x, int M, 
                 if (j == upb - 1) {
                     if (!mbar_wait_relaxed(bars + 128u + 8u * stage, (req_phase >> stage) & 1u, ctl)) return;
                     req_phase ^= 1u << stage;
-                    const float* rb = red + stage * (kMathWarps * 4 * 16);
+                    const int rstride = lay.red_tokens * 16;            // floats per warp
+                    const float* rb = red + stage * (kMathWarps * rstride);
                     for (int idx = lane; idx < M * 16; idx += 32) {  // idx = token * 16 + row
                         float s0 = 0.0f, s1 = 0.0f, s2 = 0.0f, s3 = 0.0f;
 #pragma unroll
                         for (int w = 0; w < kMathWarps; w += 4) {
-                            s0 += rb[w * 64 + idx]; s1 += rb[(w + 1) * 64 + idx];
-                            s2 += rb[(w + 2) * 64 + idx]; s3 += rb[(w + 3) * 64 + idx];
+                            s0 += rb[w * rstride + idx]; s1 += rb[(w + 1) * rstride + idx];
+                            s2 += rb[(w + 2) * rstride + idx]; s3 += rb[(w + 3) * rstride + idx];
                         }
                         br.y[(size_t)(idx >> 4) * br.n + br.band * 16 + (idx & 15)] = __float2half_rn((s0 + s1) + (s2 + s3));
                     }
@@ -526,9 +529,10 @@ gemv_band_kernel(const BandProblems probs, const __half* __restrict__ x, int M, 
             }
             if (j == upb - 1) {
                 // the band's sums go to the reduction buffer of its last stage: red[stage][warp][token][row]
-                // (tokens 4..7 of the fragment do not exist in this kernel: M <= 4)
-                float* rb = red + stage * (kMathWarps * 4 * 16) + warp * 64;
-                if (t < 2) {
+                // (only the tokens the buffer has room for: 4 when M <= 4, else all 8 of the fragment)
+                const int rstride = lay.red_tokens * 16;
+                float* rb = red + stage * (kMathWarps * rstride) + warp * rstride;
+                if (2 * t < lay.red_tokens) {
 #pragma unroll
                     for (int i = 0; i < 4; ++i) {
                         if (ONE && (i & 1)) continue;
@@ -868,7 +872,7 @@ cudaError_t allow_big_smem(Kernel kernel, bool (&done)[64]) {
 bool gemv_uses_band_kernel(int M, int N, int sms) {
     // one 16-row band per task: needs enough bands to occupy the SMs, and few tokens (every
     // band re-reads its slice of x from L2)
-    return M <= 4 && (N / 16) * 4 >= sms * 3;
+    return M <= 8 && (N / 16) * 4 >= sms * 3;
 }
 
 size_t gemv_workspace_bytes(int M) {
@@ -921,7 +925,9 @@ cudaError_t launch_gemv_band(const void* x, const GemvMatrix* mats, int count, i
     pr.first_band[kMaxMulti] = bands;
     for (int i = count; i <= kMaxMulti; ++i) pr.first_band[i] = bands;
     const int blocks = bands < sms ? bands : sms;
-    const int tpw = M <= 2 ? 4 : 2;                            // 64 or 32 k-tiles per stage
+    // 64 k-tiles per stage while the stage's x slices stay small (M <= 2) or x lives in registers
+    // (K = 4096: a band is one such stage); else 32
+    const int tpw = (M <= 2 || K == 64 * 16 * 4) ? 4 : 2;
     cudaError_t e = cudaSuccess;
     // programmatic stream serialization: this launch may begin while the kernel in front of it in
     // the stream is still finishing (see the kernel: it waits before it touches x or y)

@@ -19,12 +19,15 @@ def _run(case, path, packed=None):
 
 GEMV_CASES = [
     # N, K, M, G, alpha  - several tiles, ragged k-tile counts, both groups, all token counts.
-    # PATH_GEMV picks the band kernel for the large-N, M <= 4 cases and the split-K kernel for
+    # PATH_GEMV picks the band kernel for the large-N, M <= 8 cases and the split-K kernel for
     # the others; PATH_GEMV_SPLITK forces the split-K kernel on all of them.
     (128, 128, 1, 128, 0.5), (128, 384, 1, 64, 0.5), (256, 640, 3, 128, 0.0), (384, 1152, 8, 64, 1.0),
     (1024, 1408, 5, 128, 0.5), (512, 2048, 16, 128, 0.5), (256, 896, 9, 64, 0.5),
     (4096, 4096, 1, 128, 0.5), (4096, 4096, 2, 64, 0.5), (4096, 4096, 4, 128, 0.0),
     (2048, 1152, 3, 64, 0.5), (2432, 8320, 1, 128, 0.5), (11008, 4096, 1, 128, 0.5),
+    # band kernel with 5..8 tokens: x in registers (K = 4096) and x through the stages
+    (4096, 4096, 8, 128, 0.5), (4096, 4096, 5, 64, 0.5), (11008, 4096, 6, 128, 0.5),
+    (2432, 8320, 7, 128, 0.5), (2432, 1152, 8, 64, 0.5),
 ]
 
 
@@ -119,7 +122,38 @@ def test_auto_dispatch_and_special_values():
         assert np.allclose(y[:, 200], ref[:, 200], rtol=2e-3, atol=1e-5)
 
 
-@pytest.mark.parametrize("M,G", [(1, 128), (3, 64)])
+def test_auto_dispatch_between_9_and_16_tokens():
+    """awq_linear with 9..16 tokens runs the split-K matrix-vector kernel when a workspace is
+    registered and the tensor-core kernel when none is: each bit-equal to its forced path."""
+    import torch
+    from paper_2306_00978_b200 import binding
+    L = binding.lib()
+    case = Case(77, 1024, 1408, 12, 128, 0.5)
+    qw, sc, zp = oracle_packed_to_cuda(case)
+    x = to_cuda(case.x)
+    forced_gemv = binding.linear(x, qw, sc, zp, case.N, case.K, case.group, path=binding.PATH_GEMV)
+    forced_gemm = binding.linear(x, qw, sc, zp, case.N, case.K, case.group, path=binding.PATH_GEMM)
+    with_ws = binding.linear(x, qw, sc, zp, case.N, case.K, case.group)      # binding registers a workspace
+    assert torch.equal(with_ws, forced_gemv)
+    y = torch.empty_like(forced_gemm)
+    torch.cuda.synchronize()
+    saved = binding._workspace.pop(torch.cuda.current_device(), None)
+    assert L.awq_set_workspace(None, 0) == 0
+    try:
+        rc = L.awq_linear(x.data_ptr(), qw.data_ptr(), sc.data_ptr(), zp.data_ptr(), y.data_ptr(),
+                          case.M, case.N, case.K, case.group, None)
+        assert rc == 0
+        binding.poll_status()
+    finally:
+        if saved is not None:
+            assert L.awq_set_workspace(saved.data_ptr(), saved.numel()) == 0
+            binding._workspace[torch.cuda.current_device()] = saved
+    assert torch.equal(y, forced_gemm)
+    assert_parity(y.cpu().numpy(), case.y_ref(), "auto M=12 without workspace")
+    assert_parity(with_ws.cpu().numpy(), case.y_ref(), "auto M=12 with workspace")
+
+
+@pytest.mark.parametrize("M,G", [(1, 128), (3, 64), (7, 128)])
 def test_multi_matrix_call(M, G):
     """awq_linear_multi: three matrices reading the same x in one launch; each output against
     the oracle, and bit-equal to the single call where that also runs the band kernel."""
