@@ -164,6 +164,7 @@ int awq_linear_path(const void* x, const void* qweight, const void* scales, cons
         return AWQ_ERR_BAD_ARGUMENT;
     const bool automatic = path == AWQ_PATH_AUTO;
     path = resolve_path(M, K, path);
+    if (path != AWQ_PATH_GEMM && path != AWQ_PATH_GEMM_1SM && (M > 16 || K > 65536)) return AWQ_ERR_BAD_SHAPE;
     DeviceState* d;
     if (int rc = device_state(&d)) return rc;
     if (automatic && M > 8 && M <= 16 && K <= 65536) {
@@ -173,7 +174,6 @@ int awq_linear_path(const void* x, const void* qweight, const void* scales, cons
         if (d->workspace_bytes >= gemv_workspace_bytes(M)) path = AWQ_PATH_GEMV;
     }
     const bool tensor_path = path == AWQ_PATH_GEMM || path == AWQ_PATH_GEMM_1SM;
-    if (!tensor_path && (M > 16 || K > 65536)) return AWQ_ERR_BAD_SHAPE;
     const cudaStream_t st = (cudaStream_t)stream;
     if (path == AWQ_PATH_GEMV && gemv_uses_band_kernel(M, N, d->sms)) {
         const GemvMatrix one = {qweight, scales, zeros, y, N};
