@@ -203,6 +203,62 @@ inline BandLayout band_layout(int M, int K, bool x_in_registers) {
     return l;
 }
 
+// One full stage of one math warp: the warp's TPW k-tiles (GPW whole groups) of the band's 16
+// rows times x, added to acc.  Straight-line code, one accumulation chain per group, the groups'
+// products interleaved word by word so that no MMA waits for the one before it.  Kx / Ky are
+// 2^-24 times the sums of x over each group for the lane's two accumulator columns (tokens 2t
+// and 2t+1).
+template <int G, int TPW, bool ONE>
+__device__ __forceinline__ void band_full_stage(const unsigned char* st, int o_w, int o_sc, int o_z,
+                                                const uint2 (&xr)[TPW][4],
+                                                const float (&Kx)[(TPW + G / 64 - 1) / (G / 64)],
+                                                const float (&Ky)[(TPW + G / 64 - 1) / (G / 64)],
+                                                float (&acc)[4]) {
+    constexpr int TPG = G / 64;
+    constexpr int GPW = (TPW + TPG - 1) / TPG;
+    float c[GPW][4];
+    uint4 pk[TPW];
+#pragma unroll
+    for (int v = 0; v < TPW; ++v) pk[v] = *reinterpret_cast<const uint4*>(st + o_w + v * 512);
+#pragma unroll
+    for (int v = 0; v < TPG; ++v)
+#pragma unroll
+        for (int jw = 0; jw < 4; ++jw)
+#pragma unroll
+            for (int q = 0; q < GPW; ++q) {
+                const int tile = q * TPG + v;
+                const uint32_t w = (jw == 0) ? pk[tile].x : (jw == 1) ? pk[tile].y : (jw == 2) ? pk[tile].z : pk[tile].w;
+                const uint32_t w8 = w >> 8;
+                const uint32_t bb0 = xr[tile][jw].x, bb1 = xr[tile][jw].y;
+                if (v == 0 && jw == 0)
+                    mma_16816_first(c[q], w & 0x000F000Fu, w & 0x00F000F0u, w8 & 0x000F000Fu,
+                                    w8 & 0x00F000F0u, bb0, bb1);
+                else
+                    mma_16816(c[q], w & 0x000F000Fu, w & 0x00F000F0u, w8 & 0x000F000Fu,
+                              w8 & 0x00F000F0u, bb0, bb1);
+            }
+    // per group: Delta * (2^24 D - z X); integers below 2^23 become floats without a conversion
+    // instruction; the lower rows' codes entered the product 16 times too large (mask 0xF0) and
+    // their zero point is read 16 times too large as well, so one factor serves both
+#pragma unroll
+    for (int q = 0; q < GPW; ++q) {
+        const float d_up = __half2float(*reinterpret_cast<const __half*>(st + o_sc + q * 32));
+        const float d_lo = __half2float(*reinterpret_cast<const __half*>(st + o_sc + q * 32 + 16));
+        const uint32_t zb = st[o_z + q * 16];
+        const float z_up = __uint_as_float(0x4B000000u | (zb & 0xFu)) - 8388608.0f;
+        const float z_lo16 = __uint_as_float(0x4B000000u | (zb & 0xF0u)) - 8388608.0f;   // 16 * z
+        const float su = d_up * 16777216.0f, sl = d_lo * 1048576.0f;
+        const float kx = Kx[q];
+        acc[0] = fmaf(su, fmaf(-z_up, kx, c[q][0]), acc[0]);
+        acc[2] = fmaf(sl, fmaf(-z_lo16, kx, c[q][2]), acc[2]);
+        if (!ONE) {
+            const float ky = Ky[q];
+            acc[1] = fmaf(su, fmaf(-z_up, ky, c[q][1]), acc[1]);
+            acc[3] = fmaf(sl, fmaf(-z_lo16, ky, c[q][3]), acc[3]);
+        }
+    }
+}
+
 // TPW = k-tiles per math warp and stage (stage = 16 * TPW k-tiles).  M <= 8 tokens (one token tile).
 // ONE: M == 1, the sums of the second token column of each accumulator fragment are not formed.
 // XREG: K == 64 * 16 * TPW, i.e. a band is exactly one stage and a math warp meets the same
@@ -233,7 +289,9 @@ gemv_band_kernel(const BandProblems probs, const __half* __restrict__ x, int M, 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x < (unsigned)S) {
         mbar_init(bars + 8u * threadIdx.x, 1);                      // full: the copy warp's byte count
-        mbar_init(bars + 64u + 8u * threadIdx.x, kMathWarps + 1);   // empty: math warps and the flush warp
+        // empty: math warps and the flush warp; with one-stage bands the flush warp alone (it has
+        // seen every math warp's flush_req arrival on the same stage)
+        mbar_init(bars + 64u + 8u * threadIdx.x, XREG ? 1 : kMathWarps + 1);
         mbar_init(bars + 128u + 8u * threadIdx.x, kMathWarps);      // flush_req: a band's sums are in red[stage]
         mbar_fence_init();
     } else if (threadIdx.x == 32) {
@@ -329,7 +387,7 @@ gemv_band_kernel(const BandProblems probs, const __half* __restrict__ x, int M, 
         for (int task = b0; task < b1; ++task) {
             const BandRef br = band_ref(probs, task);
             for (int j = 0; j < upb; ++j) {
-                if (!mbar_wait_relaxed(bars + 8u * stage, phase, ctl)) return;
+                if (!XREG && !mbar_wait_relaxed(bars + 8u * stage, phase, ctl)) return;
                 if (j == upb - 1) {
                     if (!mbar_wait_relaxed(bars + 128u + 8u * stage, (req_phase >> stage) & 1u, ctl)) return;
                     req_phase ^= 1u << stage;
@@ -379,7 +437,7 @@ gemv_band_kernel(const BandProblems probs, const __half* __restrict__ x, int M, 
             for (int jw = 0; jw < 4; ++jw)
                 xr[v][jw] = __ldg(reinterpret_cast<const uint2*>(xg + v * 64 + jw * 16));
     }
-    float XxR[GPW], XyR[GPW];                            // XREG: this warp's group sums of x
+    float XxR[GPW] = {}, XyR[GPW] = {};                  // XREG: 2^-24 times this warp's group sums of x
     if (XREG) {
         // the sums of x over this warp's groups (for the zero-point term) come straight from the
         // fragments: 16 values per lane and k-tile, the four lanes of a token, then each lane
@@ -397,6 +455,7 @@ gemv_band_kernel(const BandProblems probs, const __half* __restrict__ x, int M, 
                 }
             part += __shfl_xor_sync(0xFFFFFFFFu, part, 1);
             part += __shfl_xor_sync(0xFFFFFFFFu, part, 2);
+            part *= 1.0f / 16777216.0f;                  // the products carry 2^-24 (codes as subnormals)
             XxR[q] = __shfl_sync(0xFFFFFFFFu, part, 8 * t);
             XyR[q] = __shfl_sync(0xFFFFFFFFu, part, 8 * t + 4);
         }
@@ -406,93 +465,70 @@ gemv_band_kernel(const BandProblems probs, const __half* __restrict__ x, int M, 
         // measured slower.)
         tile_sums_of_x(x, xsum, M, K, 8, warp, kMathWarps, lane);
         named_barrier_sync(3, kMathThreads);
-#pragma unroll
-        for (int q = 0; q < GPW; ++q) { XxR[q] = 0.0f; XyR[q] = 0.0f; }
+    }
+
+    if constexpr (XREG) {
+        // ---- a band is one stage: one lean loop, every address advanced by increments
+        const uint32_t sb = (uint32_t)lay.stage_bytes;
+        const int rstride = lay.red_tokens * 16;
+        const bool store_ok = 2 * t < lay.red_tokens;
+        const unsigned char* st = smem;
+        const unsigned char* const st_end = smem + (uint32_t)S * sb;
+        float* rb = red + warp * rstride + 2 * t * 16 + g;             // red[stage][warp][token][row]
+        uint32_t bar = bars, phase = 0;                                 // full[stage]; flush_req[stage] at + 128
+        // odd bands of a matrix use the upper 8 bytes of the pair's zero-point block (every matrix
+        // has an even number of bands, so a band's parity inside its matrix is the task's parity)
+        int o_z = St::kZOff + warp * (GPW * 16) + (b0 & 1) * 8 + g;
+        for (int task = b0; task < b1; ++task) {
+            float acc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+            mbar_wait(bar, phase, ctl);
+            band_full_stage<G, TPW, ONE>(st, o_w, o_sc, o_z, xr, XxR, XyR, acc);
+            if (store_ok) {
+                rb[0] = acc[0];
+                rb[8] = acc[2];
+                if (!ONE) { rb[16] = acc[1]; rb[24] = acc[3]; }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar + 128u);                     // the flush warp frees the stage
+            o_z ^= 8;
+            st += sb; rb += kMathWarps * rstride; bar += 8u;
+            if (st == st_end) { st = smem; rb -= S * (kMathWarps * rstride); bar = bars; phase ^= 1u; }
+        }
+        return;
     }
 
     uint32_t stage = 0, phase = 0;
     for (int task = b0; task < b1; ++task) {
         float acc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-        // odd bands of a matrix use the upper 8 bytes of the pair's zero-point block
-        // (every matrix has an even number of bands - N is a multiple of 128 - so a band's parity
-        // inside its matrix is the task's parity)
         const int o_z = St::kZOff + warp * (GPW * 16) + (task & 1) * 8 + g;
         for (int j = 0; j < upb; ++j) {
             const int nt = min(UT, ktiles - j * UT) - warp * TPW;     // this warp's tiles: <= 0 .. TPW
             mbar_wait(bars + 8u * stage, phase, ctl);
             const unsigned char* st = smem + stage * (uint32_t)lay.stage_bytes;
             const float* xs = xs_lane + j * (UT * 8);
-            const bool full_stage = XREG || nt >= TPW;
-            float c[GPW][4];
-            float zu[GPW], zl[GPW];
-            uint4 pk[TPW];
-            if (full_stage) {
-                // ---- full stage: straight-line code, one accumulation chain per group, the
-                // groups' products interleaved word by word so that no MMA waits for the last
-#pragma unroll
-                for (int v = 0; v < TPW; ++v) pk[v] = *reinterpret_cast<const uint4*>(st + o_w + v * 512);
-                if (!XREG && tok_ok) {
+            if (nt >= TPW) {
+                if (tok_ok) {
 #pragma unroll
                     for (int v = 0; v < TPW; ++v)
 #pragma unroll
                         for (int jw = 0; jw < 4; ++jw)
                             xr[v][jw] = *reinterpret_cast<const uint2*>(st + o_x + v * 128 + jw * 32);
                 }
-#pragma unroll
-                for (int v = 0; v < TPG; ++v)
-#pragma unroll
-                    for (int jw = 0; jw < 4; ++jw)
-#pragma unroll
-                        for (int q = 0; q < GPW; ++q) {
-                            const int tile = q * TPG + v;
-                            const uint32_t w = (jw == 0) ? pk[tile].x : (jw == 1) ? pk[tile].y : (jw == 2) ? pk[tile].z : pk[tile].w;
-                            const uint32_t w8 = w >> 8;
-                            const uint32_t bb0 = xr[tile][jw].x, bb1 = xr[tile][jw].y;
-                            if (v == 0 && jw == 0)
-                                mma_16816_first(c[q], w & 0x000F000Fu, w & 0x00F000F0u, w8 & 0x000F000Fu,
-                                                w8 & 0x00F000F0u, bb0, bb1);
-                            else
-                                mma_16816(c[q], w & 0x000F000Fu, w & 0x00F000F0u, w8 & 0x000F000Fu,
-                                          w8 & 0x00F000F0u, bb0, bb1);
-                        }
-                // per group: scale term, then zero-point term (integers below 2^23 become floats
-                // without a conversion instruction)
+                float Kx[GPW], Ky[GPW];
 #pragma unroll
                 for (int q = 0; q < GPW; ++q) {
-                    const float d_up = __half2float(*reinterpret_cast<const __half*>(st + o_sc + q * 32));
-                    const float d_lo = __half2float(*reinterpret_cast<const __half*>(st + o_sc + q * 32 + 16));
-                    const uint32_t zb = st[o_z + q * 16];
-                    const float z_up = __uint_as_float(0x4B000000u | (zb & 0xFu)) - 8388608.0f;
-                    const float z_lo16 = __uint_as_float(0x4B000000u | (zb & 0xF0u)) - 8388608.0f;   // 16 * z
-                    zu[q] = d_up * z_up;
-                    zl[q] = (d_lo * 0.0625f) * z_lo16;
-                    const float su = d_up * 16777216.0f, sl = d_lo * 1048576.0f;
-                    acc[0] = fmaf(su, c[q][0], acc[0]);
-                    acc[2] = fmaf(sl, c[q][2], acc[2]);
-                    if (!ONE) {
-                        acc[1] = fmaf(su, c[q][1], acc[1]);
-                        acc[3] = fmaf(sl, c[q][3], acc[3]);
-                    }
-                }
+                    float Xx = 0.0f, Xy = 0.0f;
 #pragma unroll
-                for (int q = 0; q < GPW; ++q) {
-                    float Xx = XxR[q], Xy = XyR[q];
-                    if (!XREG) {
-#pragma unroll
-                        for (int v = 0; v < TPG; ++v) {
-                            const float2 X = *reinterpret_cast<const float2*>(xs + (q * TPG + v) * 8);
-                            Xx += X.x;
-                            Xy += X.y;
-                        }
+                    for (int v = 0; v < TPG; ++v) {
+                        const float2 X = *reinterpret_cast<const float2*>(xs + (q * TPG + v) * 8);
+                        Xx += X.x;
+                        Xy += X.y;
                     }
-                    acc[0] = fmaf(-zu[q], Xx, acc[0]);
-                    acc[2] = fmaf(-zl[q], Xx, acc[2]);
-                    if (!ONE) {
-                        acc[1] = fmaf(-zu[q], Xy, acc[1]);
-                        acc[3] = fmaf(-zl[q], Xy, acc[3]);
-                    }
+                    Kx[q] = Xx * (1.0f / 16777216.0f);
+                    Ky[q] = Xy * (1.0f / 16777216.0f);
                 }
-            } else if (!XREG && nt > 0) {
+                band_full_stage<G, TPW, ONE>(st, o_w, o_sc, o_z, xr, Kx, Ky, acc);
+            } else if (nt > 0) {
                 // ---- ragged last stage of a band: whole groups only (K % G == 0), one at a time
 #pragma unroll
                 for (int q = 0; q < GPW; ++q) {
