@@ -15,6 +15,8 @@ What is computed, and where it comes from
                      in the asymmetric min/max form with an integer zero point in
                      [0, 15] and Delta stored in fp16 (Sec. 3.2: "Delta and x are
                      represented in FP16").
+* search_clip        weight clipping (Sec. 3.2): per group, the range ratio of a given list that
+                     minimizes the squared quantization error of the group.
 * pack_* / unpack_*  eight 4-bit codes per 32-bit word in the order
                      w{0,2,4,6,1,3,5,7} (Sec. 4.2, SIMD-aware weight packing), inside
                      512-byte blocks (16 rows x 64 columns) whose 16-byte pieces are ordered
@@ -38,6 +40,13 @@ The search's norm is not named in the paper: the mean of the squared differences
 monotone function of the Frobenius norm has the same minimizer); diag(s)^-1 X is rounded to fp16
 once, because that is what the layer is given; the grid of alpha is an argument (the paper says
 "a grid size of 20" over [0, 1] without saying whether 1 is a grid point).
+Weight clipping is one sentence in the paper (the appendix it may have been detailed in is not
+part of the text): the reading here shrinks a group's [min, max] by a common ratio taken from a
+caller-given list, measures the error in the scaled weight space w' = w * s (the tensor that is
+actually quantized), unweighted, in fp32 in a fixed order so that the choice is reproducible bit
+for bit, and keeps the first best ratio.  INT3 (the paper's INT3-g128 tables) is the same
+quantizer on 8 levels (Delta = (max - min) / 7, z and q in [0, 7]); how the paper's kernels would
+store 3-bit codes is not described, here they occupy the 4-bit fields of the INT4 layout.
 Parity for these asymmetric details is unpinned by the paper (it prints no worked numeric
 example of Q); they are pinned by closed-form invariants, grid-aligned round trips and
 brute-force enumeration in tests/test_oracle_pins.py.
@@ -80,31 +89,41 @@ def channel_scale(act_mean_abs, alpha: float) -> np.ndarray:
 
 
 # --------------------------------------------------------------------- Eq. 2 - Eq. 4
-def quantize(W, s, group: int):
-    """Group-wise asymmetric INT4 round-to-nearest of W * diag(s).
+def quantize(W, s, group: int, clip=None, bits: int = 4):
+    """Group-wise asymmetric round-to-nearest of W * diag(s) on a grid of 2**bits levels.
 
     W fp16 [N][K]; s fp32 [K]; groups are `group` consecutive input channels of one
-    output row.  Returns (codes u8 [N][K], zeros u8 [N][K/group], scales fp16 [N][K/group]).
+    output row.  clip: None, or fp32 [N][K/group] of range ratios (Sec. 3.2, weight clipping):
+    a group's range becomes [r * min, r * max] (one fp32 multiply each) and values outside it
+    saturate at codes 0 and 2**bits - 1.  bits is 4 (INT4) or 3 (INT3).
+    Returns (codes u8 [N][K], zeros u8 [N][K/group], scales fp16 [N][K/group]).
     """
     W = np.asarray(W)
     assert W.dtype == np.float16 and W.ndim == 2
     N, K = W.shape
     assert K % group == 0
+    assert bits in (3, 4)
     ng = K // group
     s = np.asarray(s, dtype=np.float32)
     assert s.shape == (K,)
+    if clip is not None:
+        clip = np.asarray(clip)
+        assert clip.dtype == np.float32 and clip.shape == (N, ng)
 
     codes = np.empty((N, K), dtype=np.uint8)
     zeros = np.empty((N, ng), dtype=np.uint8)
     scales = np.empty((N, ng), dtype=np.float16)
     rows = max(1, (1 << 23) // K)                       # bound the fp32 temporaries
-    f15, f0 = np.float32(15.0), np.float32(0.0)
+    f15, f0 = np.float32((1 << bits) - 1), np.float32(0.0)    # top code: 15 (INT4) or 7 (INT3)
     for r0 in range(0, N, rows):
         r1 = min(N, r0 + rows)
         wp = W[r0:r1].astype(np.float32) * s[None, :]   # Eq. 3: w * s, one fp32 multiply
         wg = wp.reshape(r1 - r0, ng, group)
         mn = wg.min(axis=2)
         mx = wg.max(axis=2)
+        if clip is not None:
+            mn = mn * clip[r0:r1]
+            mx = mx * clip[r0:r1]
         with np.errstate(over="ignore", invalid="ignore", divide="ignore"):
             d16 = ((mx - mn) / f15).astype(np.float16)  # Delta, stored in fp16
             bad = ~np.isfinite(d16) | (d16 == 0)
@@ -211,11 +230,58 @@ def unpack_scales(packed, N: int, ng: int) -> np.ndarray:
     return np.ascontiguousarray(p.transpose(0, 2, 1).reshape(N, ng))
 
 
-def quantize_pack(W, act_mean_abs, alpha: float, group: int):
-    """The whole offline step: returns (qweight u32, scales fp16 [N/16][ng][16], zeros u8 [N/32][ng][16])."""
+def search_clip(W, s, group: int, ratios, bits: int = 4) -> np.ndarray:
+    """Weight clipping (Sec. 3.2: clipping that minimizes the squared error of quantization).
+
+    For every group and every ratio r of `ratios` the group of w' = W * diag(s) is quantized on
+    the range [r * min, r * max] and the squared error of the group is summed,
+        err(r) = sum over k ascending of (dequant(q_k) - w'_k) ** 2,
+    every step a single fp32 operation: dequant = (q - z) * Delta (one multiply), the difference,
+    its square, and the running sum.  The first ratio of least error is taken (a NaN error counts
+    as +inf).  Returns fp32 [N][K/group], each entry one of `ratios`.
+    """
+    W = np.asarray(W)
+    assert W.dtype == np.float16 and W.ndim == 2 and bits in (3, 4)
+    N, K = W.shape
+    ng = K // group
+    s = np.asarray(s, dtype=np.float32)
+    ratios = np.asarray(ratios, dtype=np.float32)
+    top, f0 = np.float32((1 << bits) - 1), np.float32(0.0)
+    wg = (W.astype(np.float32) * s[None, :]).reshape(N, ng, group)
+    mn0 = wg.min(axis=2)
+    mx0 = wg.max(axis=2)
+    best_err = np.full((N, ng), np.inf, dtype=np.float32)
+    best = np.zeros((N, ng), dtype=np.int64)
+    for i, r in enumerate(ratios):
+        mn = mn0 * r
+        mx = mx0 * r
+        with np.errstate(over="ignore", invalid="ignore", divide="ignore"):
+            d16 = ((mx - mn) / top).astype(np.float16)
+            bad = ~np.isfinite(d16) | (d16 == 0)
+            d = np.where(bad, np.float16(1.0), d16).astype(np.float16).astype(np.float32)
+            z = np.clip(np.rint((-mn) / d), f0, top)
+            err = np.zeros((N, ng), dtype=np.float32)
+            for k in range(group):                      # ascending k, fp32 running sum
+                w = wg[:, :, k]
+                q = np.clip(np.rint(w / d) + z, f0, top)
+                e = (q - z) * d - w
+                err = err + e * e
+        err = np.where(np.isnan(err), np.float32(np.inf), err)
+        if i == 0:
+            best_err = err
+        else:
+            better = err < best_err                     # strict: the first of equal errors stays
+            best = np.where(better, i, best)
+            best_err = np.where(better, err, best_err)
+    return ratios[best].astype(np.float32)
+
+
+def quantize_pack(W, act_mean_abs, alpha: float, group: int, clip=None, bits: int = 4):
+    """The whole offline step: returns (qweight u32, scales fp16 [N/16][ng][16], zeros u8 [N/32][ng][16]).
+    3-bit codes (bits = 3) are stored in the same 4-bit fields."""
     K = W.shape[1]
     a = np.ones(K, np.float32) if act_mean_abs is None else act_mean_abs
-    codes, zeros, scales = quantize(W, channel_scale(a, alpha), group)
+    codes, zeros, scales = quantize(W, channel_scale(a, alpha), group, clip=clip, bits=bits)
     return pack_qweight(codes), pack_scales(scales), pack_zeros(zeros)
 
 

@@ -492,3 +492,109 @@ def test_search_alpha_prefers_scaling_when_activations_have_outliers():
     flat = np.ones_like(a)
     lf, _ = orc.search_alpha(W, flat, X, 128, [0.0, 0.5, 1.0])
     assert lf[0] == lf[1] == lf[2]
+
+
+# ----------------------------------------------------------- weight clipping, 3-bit grid
+def _clip_example(sign):
+    """One group of 128 whose best clipping ratio and codes follow by hand: delta = 2^-6; the
+    values are 0, an outlier 20 delta and 126 values in {2, 6, 10, 14} delta.  On the full range
+    Delta = 20 delta / 15 = 4 delta / 3 and every v in {2, 6, 10, 14} sits half-way between two
+    levels (0.75 v = 1.5, 4.5, 7.5, 10.5): error (2 delta / 3)^2 each, 126 * 4/9 = 56 delta^2 in
+    all.  With ratio 0.75 the range is 15 delta, Delta = delta, every value but the outlier is a
+    level and the outlier saturates: error (5 delta)^2 = 25 delta^2 < 56 delta^2."""
+    delta = 2.0**-6
+    v = np.array([0] + [2, 6, 10, 14] * 31 + [2, 6, 20], dtype=np.float64)
+    assert v.size == 128
+    return (sign * v * delta).astype(np.float16)[None, :], v.astype(np.int64)
+
+
+@pytest.mark.parametrize("sign", [1, -1])
+def test_clip_worked_example(sign):
+    W, v = _clip_example(sign)
+    ones = np.ones(128, np.float32)
+    r = orc.search_clip(W, ones, 128, [1.0, 0.75])
+    assert r.shape == (1, 1) and r[0, 0] == np.float32(0.75)
+    codes, zeros, scales = orc.quantize(W, ones, 128, clip=r)
+    assert float(scales[0, 0]) == 2.0**-6
+    if sign > 0:
+        assert zeros[0, 0] == 0 and np.array_equal(codes[0], np.minimum(v, 15))
+    else:
+        assert zeros[0, 0] == 15 and np.array_equal(codes[0], 15 - np.minimum(v, 15))
+    # the other order of the list: same ratio
+    assert orc.search_clip(W, ones, 128, [0.75, 1.0])[0, 0] == np.float32(0.75)
+    # the clipped reconstruction misses only the outlier: 25 delta^2
+    back = orc.dequantize(codes, zeros, scales, 128)
+    assert np.isclose(((back - W.astype(np.float64)) ** 2).sum(), 25 * 2.0**-12, rtol=1e-12)
+
+
+def test_clip_ratio_one_is_the_plain_quantizer_and_ties_keep_the_first():
+    W, a = _gaussian_case(31, 64, 512)
+    s = orc.channel_scale(a, 0.5)
+    r = orc.search_clip(W, s, 128, [1.0])
+    assert (r == 1.0).all()
+    plain = orc.quantize(W, s, 128)
+    clipped = orc.quantize(W, s, 128, clip=r)
+    assert all(np.array_equal(p, c) for p, c in zip(plain, clipped))
+    # a list that repeats a ratio has equal errors for both copies: the choice must not change
+    r2 = orc.search_clip(W, s, 128, [0.9, 0.8, 0.9, 0.8])
+    r1 = orc.search_clip(W, s, 128, [0.9, 0.8])
+    assert np.array_equal(r1, r2)
+
+
+@pytest.mark.parametrize("bits,G", [(4, 128), (3, 64)])
+def test_clip_choice_is_the_least_error_through_an_independent_route(bits, G):
+    """The chosen ratio's error, recomputed in fp64 through quantize + dequantize (functions
+    pinned above), is the least over the list up to fp32 summation error, and never above the
+    unclipped error."""
+    N, K = 32, 512
+    W, a = _gaussian_case(33, N, K)
+    W = W.copy()
+    W[::3, ::37] *= np.float16(6.0)                         # a few outliers so that clipping pays
+    s = orc.channel_scale(a, 0.5)
+    ratios = np.linspace(1.0, 0.5, 11).astype(np.float32)
+    chosen = orc.search_clip(W, s, G, ratios, bits=bits)
+    assert np.isin(chosen, ratios).all()
+    wp = (W.astype(np.float32) * s[None, :]).astype(np.float64).reshape(N, K // G, G)
+    errs = []
+    for r in ratios:
+        clip = np.full((N, K // G), r, np.float32)
+        back = orc.dequantize(*orc.quantize(W, s, G, clip=clip, bits=bits), G).reshape(N, K // G, G)
+        errs.append(((back - wp) ** 2).sum(axis=2))
+    errs = np.stack(errs)                                    # [ratio][N][groups]
+    idx = np.argmax(ratios[:, None, None] == chosen[None], axis=0)
+    picked = np.take_along_axis(errs, idx[None], axis=0)[0]
+    assert (picked <= errs.min(axis=0) * (1 + 1e-4)).all()
+    assert (picked <= errs[0] * (1 + 1e-4)).all()
+    assert (idx > 0).mean() > 0.2                            # clipping is chosen for many groups
+
+
+def test_int3_grid_invariants_and_brute_force():
+    """bits = 3: codes and zero points stay in [0, 7], Delta is the fp16 rounding of range / 7,
+    the reconstruction error is at most half a step, and on tiny groups the codes minimise the
+    squared error over all 8^G code vectors for the oracle's own (Delta, z)."""
+    N, K, G = 64, 512, 128
+    W, a = _gaussian_case(35, N, K)
+    s = orc.channel_scale(a, 0.5)
+    codes, zeros, scales = orc.quantize(W, s, G, bits=3)
+    assert codes.max() == 7 and zeros.max() <= 7
+    wg = (W.astype(np.float64) * s.astype(np.float64)).reshape(N, K // G, G)
+    rng_ = (wg.max(axis=2) - wg.min(axis=2)) / 7.0
+    assert (np.abs(scales.astype(np.float64) - rng_) <= 2.0**-11 * rng_ * 1.0001).all()
+    back = orc.dequantize(codes, zeros, scales, G).reshape(N, K // G, G)
+    d = scales.astype(np.float64)[:, :, None]
+    assert (np.abs(wg - back) <= (0.5 + 7 * 2.0**-11) * d + 2.0**-22 * np.abs(wg) + 1e-12).all()
+    # a grid-aligned group round-trips exactly: levels {-3..4} * 2^-5
+    lv = (np.arange(-3, 5) * 2.0**-5).astype(np.float16)
+    Wg = np.tile(lv, 16)[None, :]
+    c, z, sc = orc.quantize(Wg, np.ones(128, np.float32), 128, bits=3)
+    assert z[0, 0] == 3 and float(sc[0, 0]) == 2.0**-5 and np.array_equal(c[0, :8], np.arange(8))
+    rng = np.random.default_rng(7)
+    vals = (rng.integers(-40, 41, size=(30, 3)) / 64.0).astype(np.float16)
+    vals = vals[(vals.max(axis=1) > 0) & (vals.min(axis=1) < 0)]
+    c, z, sc = orc.quantize(vals, np.ones(3, np.float32), 3, bits=3)
+    for r in range(vals.shape[0]):
+        dd, zz = Fraction(float(sc[r, 0])), int(z[r, 0])
+        w = [Fraction(float(v)) for v in vals[r]]
+        err = lambda qs: sum((wi - (qi - zz) * dd) ** 2 for wi, qi in zip(w, qs))
+        best = min(err(qs) for qs in itertools.product(range(8), repeat=3))
+        assert err([int(x) for x in c[r]]) <= best * (1 + Fraction(1, 2**20))
