@@ -317,6 +317,31 @@ def search_section():
             "best_alpha": alphas[best], "loss_best_over_loss_alpha0": losses[best] / losses[0]}
 
 
+def clip_section():
+    """Weight clipping (Sec. 3.2) on one 4096 -> 4096 layer: 20 range ratios per group, then the
+    clipped quantizer; CUDA events, best of 5."""
+    import torch
+    from paper_2306_00978_b200 import binding
+    N, K = 4096, 4096
+    W = torch.from_numpy(synth.weight(2000, N, K)).cuda()
+    a = torch.from_numpy(synth.act_mean_abs(2000, K)).cuda()
+    ratios = [1.0 - 0.5 * i / 19 for i in range(20)]
+    times = {"search": [], "quantize": []}
+    for _ in range(6):
+        e = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+        e[0].record()
+        r = binding.search_clip(W, a, ALPHA, GROUP, ratios)
+        e[1].record()
+        binding.quantize_pack(W, a, ALPHA, GROUP, clip_ratio=r)
+        e[2].record()
+        torch.cuda.synchronize()
+        times["search"].append(e[0].elapsed_time(e[1]))
+        times["quantize"].append(e[1].elapsed_time(e[2]))
+    return {"shape": f"{K}->{N}", "ratios": len(ratios), "search_ms": min(times["search"][1:]),
+            "clipped_quantize_ms": min(times["quantize"][1:]),
+            "groups_clipped_frac": float((r < 1.0).float().mean().item())}
+
+
 # ------------------------------------------------------------------- oracle (CPU) arm
 def _oracle_layer_inputs(max_rows=None):
     """Quantizes one decoder layer's matrices with the oracle; optionally only the first
@@ -536,6 +561,7 @@ def main():
         line["gemm_m2048"] = gemm_section(peaks)
         line["quantize_pack"] = quantize_section(peaks)
         line["alpha_search"] = search_section()
+        line["clip_search"] = clip_section()
         if world == 1:
             del graphs, e2e_graphs, layers
             torch.cuda.empty_cache()

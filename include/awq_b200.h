@@ -94,6 +94,37 @@ size_t awq_zeros_bytes(int N, int K, int group);
 int awq_quantize_pack(const void* W, const float* act_mean_abs, float alpha, int group,
                       void* qweight, void* scales, void* zeros, int N, int K, void* stream);
 
+/*
+ * The same offline step with the two variants the method also uses (Sec. 3.2 weight clipping;
+ * the INT3-g128 setting of the accuracy tables):
+ *   bits: 4 or 3.  bits = 3 quantizes to 8 levels (Delta = fp16_rne(range / 7), z and q in
+ *         [0,7]); the 3-bit codes occupy the same 4-bit fields, so the packed arrays, their
+ *         sizes and awq_linear are unchanged (the paper does not describe a 3-bit storage).
+ *   clip_ratio: NULL, or in, device, fp32 [N][K/group] (row-major): the group's range becomes
+ *         [r * min w', r * max w'] (one fp32 multiply each) before Delta and z are formed; values
+ *         outside saturate at codes 0 and 2^bits - 1.  awq_search_clip produces such an array.
+ * awq_quantize_pack(...) is awq_quantize_pack_ex(..., bits = 4, clip_ratio = NULL, ...).
+ * Errors: as awq_quantize_pack; AWQ_ERR_BAD_ARGUMENT for other `bits`.
+ */
+int awq_quantize_pack_ex(const void* W, const float* act_mean_abs, float alpha, int group, int bits,
+                         const float* clip_ratio, void* qweight, void* scales, void* zeros,
+                         int N, int K, void* stream);
+
+/*
+ * Weight clipping (Sec. 3.2: "weight clipping to minimize the MSE error of quantization"; the
+ * paper gives no algorithm, this is the reading used).  For every group of w' = fp32(W) * s and
+ * every ratio r_i of `ratios`, the group is quantized as awq_quantize_pack_ex would with
+ * clip_ratio = r_i, and
+ *   err_i = sum over k ascending of ((q_k - z) * Delta - w'_k)^2
+ * is formed in fp32, one IEEE operation per step (multiply, subtract, square, add), a NaN counting
+ * as +inf; clip_ratio[n][g] = the first r_i of least err_i.  The result is bit-reproducible.
+ * ratios: in, HOST, n_ratios values in (0, 1], 1 <= n_ratios <= 32, read during the call.
+ * clip_ratio: out, device, fp32 [N][K/group].  W, act_mean_abs, alpha, group, bits as above.
+ * Errors: AWQ_ERR_BAD_ARGUMENT for a bad list or `bits`; shape / pointer errors as listed in AwqStatus.
+ */
+int awq_search_clip(const void* W, const float* act_mean_abs, float alpha, int group, int bits,
+                    const float* ratios, int n_ratios, float* clip_ratio, int N, int K, void* stream);
+
 /* Eq. 5 alone: s[k] as used by awq_quantize_pack.  s: out, fp32 [K]. */
 int awq_channel_scale(const float* act_mean_abs, float alpha, float* s, int K, void* stream);
 

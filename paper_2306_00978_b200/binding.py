@@ -24,6 +24,7 @@ EXPORTS = (
     "awq_set_workspace", "awq_unpack_canonical", "awq_poll_status", "awq_status_string",
     "awq_last_cuda_error", "awq_layout_version", "awq_launch_count", "awq_linear_gemv_static",
     "awq_linear_multi", "awq_search_scratch_bytes", "awq_search_alpha",
+    "awq_quantize_pack_ex", "awq_search_clip",
 )
 
 
@@ -52,6 +53,8 @@ def lib() -> ctypes.CDLL:
     L.awq_scales_bytes.restype, L.awq_scales_bytes.argtypes = sz, [i, i, i]
     L.awq_zeros_bytes.restype, L.awq_zeros_bytes.argtypes = sz, [i, i, i]
     L.awq_quantize_pack.restype, L.awq_quantize_pack.argtypes = i, [vp, vp, f, i, vp, vp, vp, i, i, vp]
+    L.awq_quantize_pack_ex.restype, L.awq_quantize_pack_ex.argtypes = i, [vp, vp, f, i, i, vp, vp, vp, vp, i, i, vp]
+    L.awq_search_clip.restype, L.awq_search_clip.argtypes = i, [vp, vp, f, i, i, vp, i, vp, i, i, vp]
     L.awq_channel_scale.restype, L.awq_channel_scale.argtypes = i, [vp, f, vp, i, vp]
     L.awq_linear.restype, L.awq_linear.argtypes = i, [vp, vp, vp, vp, vp, i, i, i, i, vp]
     L.awq_linear_path.restype, L.awq_linear_path.argtypes = i, [vp, vp, vp, vp, vp, i, i, i, i, i, vp]
@@ -109,9 +112,10 @@ def channel_scale(act_mean_abs: Optional[torch.Tensor], alpha: float, K: int) ->
     return s
 
 
-def quantize_pack(W: torch.Tensor, act_mean_abs: Optional[torch.Tensor], alpha: float, group: int):
-    """awq_quantize_pack: returns (qweight u8 [N*K/2], scales fp16 [N/16][K/group][16],
-    zeros u8 [N/32][K/group][16])."""
+def quantize_pack(W: torch.Tensor, act_mean_abs: Optional[torch.Tensor], alpha: float, group: int,
+                  clip_ratio: Optional[torch.Tensor] = None, bits: int = 4):
+    """awq_quantize_pack / awq_quantize_pack_ex: returns (qweight u8 [N*K/2],
+    scales fp16 [N/16][K/group][16], zeros u8 [N/32][K/group][16])."""
     N, K = W.shape
     qb, sb, zb = packed_sizes(N, K, group)
     dev = W.device
@@ -119,10 +123,34 @@ def quantize_pack(W: torch.Tensor, act_mean_abs: Optional[torch.Tensor], alpha: 
     scales = torch.empty((N // 16, K // group, 16), dtype=torch.float16, device=dev)
     zeros = torch.empty((N // 32, K // group, 16), dtype=torch.uint8, device=dev)
     a = 0 if act_mean_abs is None else _dev(act_mean_abs, torch.float32, "act_mean_abs")
-    rc = lib().awq_quantize_pack(_dev(W, torch.float16, "W"), a, float(alpha), int(group),
-                                 qweight.data_ptr(), scales.data_ptr(), zeros.data_ptr(), N, K, _stream())
-    _check(rc, "awq_quantize_pack")
+    if clip_ratio is None and bits == 4:
+        rc = lib().awq_quantize_pack(_dev(W, torch.float16, "W"), a, float(alpha), int(group),
+                                     qweight.data_ptr(), scales.data_ptr(), zeros.data_ptr(), N, K, _stream())
+        _check(rc, "awq_quantize_pack")
+        return qweight, scales, zeros
+    c = 0
+    if clip_ratio is not None:
+        if tuple(clip_ratio.shape) != (N, K // group):
+            raise AwqError(f"clip_ratio: expected shape {(N, K // group)}")
+        c = _dev(clip_ratio, torch.float32, "clip_ratio")
+    rc = lib().awq_quantize_pack_ex(_dev(W, torch.float16, "W"), a, float(alpha), int(group), int(bits), c,
+                                    qweight.data_ptr(), scales.data_ptr(), zeros.data_ptr(), N, K, _stream())
+    _check(rc, "awq_quantize_pack_ex")
     return qweight, scales, zeros
+
+
+def search_clip(W: torch.Tensor, act_mean_abs: Optional[torch.Tensor], alpha: float, group: int,
+                ratios, bits: int = 4) -> torch.Tensor:
+    """awq_search_clip: per-group range ratios (fp32 [N][K/group], device) of least squared
+    quantization error, each one of `ratios` (a sequence of floats in (0, 1])."""
+    N, K = W.shape
+    out = torch.empty((N, K // group), dtype=torch.float32, device=W.device)
+    arr = (ctypes.c_float * len(ratios))(*[float(r) for r in ratios])
+    a = 0 if act_mean_abs is None else _dev(act_mean_abs, torch.float32, "act_mean_abs")
+    rc = lib().awq_search_clip(_dev(W, torch.float16, "W"), a, float(alpha), int(group), int(bits),
+                               ctypes.cast(arr, ctypes.c_void_p), len(ratios), out.data_ptr(), N, K, _stream())
+    _check(rc, "awq_search_clip")
+    return out
 
 
 def ensure_workspace(nbytes: int) -> None:

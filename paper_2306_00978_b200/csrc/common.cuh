@@ -27,9 +27,15 @@ void count_launch();
 
 // launchers (each returns the cudaError_t of the launch)
 cudaError_t launch_channel_scale(const float* a, float alpha, float* s, int K, cudaStream_t st);
-cudaError_t launch_quantize_pack(const __half* W, const float* a, float alpha, int group,
-                                 uint32_t* qweight, __half* scales, uint8_t* zeros,
+// bits: 4 or 3 (3-bit codes in the 4-bit fields); clip: optional per-group range ratios [N][K/group]
+cudaError_t launch_quantize_pack(const __half* W, const float* a, float alpha, int group, int bits,
+                                 const float* clip, uint32_t* qweight, __half* scales, uint8_t* zeros,
                                  int N, int K, cudaStream_t st);
+constexpr int kMaxClipRatios = 32;
+// ratios: HOST array of n_ratios <= kMaxClipRatios values; clip: device out, fp32 [N][K/group]
+cudaError_t launch_clip_search(const __half* W, const float* a, float alpha, int group, int bits,
+                               const float* ratios, int n_ratios, float* clip, int N, int K,
+                               cudaStream_t st);
 cudaError_t launch_unpack(const uint32_t* qweight, const __half* scales, const uint8_t* zeros,
                           int N, int K, int group, uint8_t* codes, uint16_t* scales_nk,
                           uint8_t* zeros_nk, cudaStream_t st);

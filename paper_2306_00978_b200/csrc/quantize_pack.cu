@@ -33,24 +33,25 @@ __device__ __forceinline__ uint2 ldg_stream(const uint2* p) {
     return v;
 }
 
-// Delta (fp16) and zero point of a group from its min and max.
-__device__ __forceinline__ void group_params(float mn, float mx, __half& d16, float& d, float& z) {
-    const float d32 = __fdiv_rn(__fsub_rn(mx, mn), 15.0f);
+// Delta (fp16) and zero point of a group from its min and max; `top` is the largest code
+// (15 for 4-bit, 7 for 3-bit grids).
+__device__ __forceinline__ void group_params(float mn, float mx, float top, __half& d16, float& d, float& z) {
+    const float d32 = __fdiv_rn(__fsub_rn(mx, mn), top);
     d16 = __float2half_rn(d32);
     const unsigned short bits = __half_as_ushort(d16);
     if ((bits & 0x7FFFu) == 0u || (bits & 0x7C00u) == 0x7C00u) d16 = __ushort_as_half(0x3C00u);
     d = __half2float(d16);
-    z = fminf(fmaxf(rintf(__fdiv_rn(-mn, d)), 0.0f), 15.0f);
+    z = fminf(fmaxf(rintf(__fdiv_rn(-mn, d)), 0.0f), top);
 }
 
 // q = clamp(rne(w / d) + z, 0, 15) with w / d the IEEE-rounded fp32 quotient.  `rd` = 1 / d
 // (rounded).  w * rd is within 2.5e-7 |w / d| of the quotient, so it rounds to the same integer
 // unless it lies within 1e-3 of a half-integer (or is large): only then is the division done.
-__device__ __forceinline__ uint32_t code_of(float w, float d, float rd, float z) {
+__device__ __forceinline__ uint32_t code_of(float w, float d, float rd, float z, float top) {
     const float t = __fmul_rn(w, rd);
     float r = rintf(t);
     if (!(fabsf(t - r) < 0.499f && fabsf(t) < 1024.0f)) r = rintf(__fdiv_rn(w, d));
-    return (uint32_t)fminf(fmaxf(__fadd_rn(r, z), 0.0f), 15.0f);
+    return (uint32_t)fminf(fmaxf(__fadd_rn(r, z), 0.0f), top);
 }
 
 // grid = (K/128, N/128), block = 256 (8 warps = 8 bands of the 128-row slab); three blocks per SM:
@@ -58,7 +59,8 @@ __device__ __forceinline__ uint32_t code_of(float w, float d, float rd, float z)
 template <int G>
 __global__ void __launch_bounds__(256, 3)
 quantize_pack_kernel(const __half* __restrict__ W, const float* __restrict__ a, float alpha,
-                     int mode, uint32_t* __restrict__ qweight, __half* __restrict__ scales,
+                     int mode, const float* __restrict__ clip, float top,
+                     uint32_t* __restrict__ qweight, __half* __restrict__ scales,
                      uint8_t* __restrict__ zeros, int N, int K) {
     __shared__ __align__(16) float s_sm[128];
     const int kblk = blockIdx.x, slab = blockIdx.y;
@@ -131,12 +133,26 @@ quantize_pack_kernel(const __half* __restrict__ W, const float* __restrict__ a, 
                 mx[ti][h] = fmaxf(mx[ti][h], __shfl_xor_sync(0xFFFFFFFFu, mx[ti][h], off));
             }
 
+    if (clip != nullptr) {
+        // weight clipping (Sec. 3.2): the group's range shrinks by its ratio, values outside saturate
+        const int ng = K / G;
+#pragma unroll
+        for (int ti = 0; ti < 2; ++ti)
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const int gi = (G == 64) ? kblk * 2 + ti : kblk;
+                const float r = __ldg(clip + (size_t)(n0 + 8 * h) * ng + gi);
+                mn[ti][h] = __fmul_rn(mn[ti][h], r);
+                mx[ti][h] = __fmul_rn(mx[ti][h], r);
+            }
+    }
+
 #pragma unroll
     for (int ti = 0; ti < 2; ++ti) {
         __half d16[2]; float d[2], z[2], rd[2];
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
-            group_params(mn[ti][h], mx[ti][h], d16[h], d[h], z[h]);
+            group_params(mn[ti][h], mx[ti][h], top, d16[h], d[h], z[h]);
             rd[h] = __frcp_rn(d[h]);
         }
 
@@ -150,10 +166,10 @@ quantize_pack_kernel(const __half* __restrict__ W, const float* __restrict__ a, 
             wprime(ti, 1, j, sv, wl);
             // slots (g,c) (g,c+1) (g+8,c) (g+8,c+1) (g,c+2) (g,c+3) (g+8,c+2) (g+8,c+3)
             // at nibbles 0, 4, 1, 5, 2, 6, 3, 7
-            words[j] = (code_of(wu[0], d[0], rd[0], z[0]) << 0) | (code_of(wu[1], d[0], rd[0], z[0]) << 16) |
-                       (code_of(wl[0], d[1], rd[1], z[1]) << 4) | (code_of(wl[1], d[1], rd[1], z[1]) << 20) |
-                       (code_of(wu[2], d[0], rd[0], z[0]) << 8) | (code_of(wu[3], d[0], rd[0], z[0]) << 24) |
-                       (code_of(wl[2], d[1], rd[1], z[1]) << 12) | (code_of(wl[3], d[1], rd[1], z[1]) << 28);
+            words[j] = (code_of(wu[0], d[0], rd[0], z[0], top) << 0) | (code_of(wu[1], d[0], rd[0], z[0], top) << 16) |
+                       (code_of(wl[0], d[1], rd[1], z[1], top) << 4) | (code_of(wl[1], d[1], rd[1], z[1], top) << 20) |
+                       (code_of(wu[2], d[0], rd[0], z[0], top) << 8) | (code_of(wu[3], d[0], rd[0], z[0], top) << 24) |
+                       (code_of(wl[2], d[1], rd[1], z[1], top) << 12) | (code_of(wl[3], d[1], rd[1], z[1], top) << 28);
         }
         // band-major: block (band, k-tile) is 512 bytes, a band's blocks are contiguous along K
         const size_t band = (size_t)slab * 8 + warp;
@@ -170,6 +186,81 @@ quantize_pack_kernel(const __half* __restrict__ W, const float* __restrict__ a, 
             zeros[((band >> 1) * ng + gi) * 16 + (band & 1) * 8 + g] =
                 (uint8_t)((uint32_t)z[0] | ((uint32_t)z[1] << 4));
         }
+    }
+}
+
+// Weight clipping (Sec. 3.2).  For every group of w' = w * s and every ratio r of the list, the
+// group is quantized on [r * min, r * max] and its squared error summed; the first ratio of least
+// error is written to clip[n][group].  The choice decides integer codes downstream, so the error
+// is defined operation by operation: dequant = (q - z) * Delta (one fp32 multiply), e = dequant -
+// w', err += e * e in fp32 over ascending k (no contraction), a NaN error counts as +inf.
+// grid = (ceil(K / 2048), N), block = 256: one row's chunk of w' in shared memory; a thread takes
+// one (group, ratio) pair at a time and walks the group's elements in order.
+constexpr int kClipChunk = 2048;
+struct ClipGrid {
+    float r[kMaxClipRatios];
+    int n;
+};
+
+template <int G>
+__global__ void __launch_bounds__(256)
+clip_search_kernel(const __half* __restrict__ W, const float* __restrict__ a, float alpha, int mode,
+                   const ClipGrid ratios, float top, float* __restrict__ clip, int N, int K) {
+    constexpr int kGroups = kClipChunk / G;
+    __shared__ float w_sm[kClipChunk];
+    __shared__ float mn_sm[kGroups], mx_sm[kGroups];
+    __shared__ float err_sm[kGroups * kMaxClipRatios];
+    const int n = blockIdx.y, k0 = blockIdx.x * kClipChunk;
+    const int cols = min(kClipChunk, K - k0);              // a multiple of 128: whole groups
+    const int ngr = cols / G;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    for (int i = threadIdx.x; i < cols; i += 256) {
+        const float sk = channel_scale_one(mode == kAlphaZero ? 1.0f : a[k0 + i], alpha, mode);
+        w_sm[i] = __fmul_rn(__half2float(W[(size_t)n * K + k0 + i]), sk);          // Eq. 3
+    }
+    __syncthreads();
+    for (int gi = warp; gi < ngr; gi += 8) {
+        float mn = INFINITY, mx = -INFINITY;
+#pragma unroll
+        for (int e = 0; e < G / 32; ++e) {
+            const float w = w_sm[gi * G + e * 32 + lane];
+            mn = fminf(mn, w);
+            mx = fmaxf(mx, w);
+        }
+#pragma unroll
+        for (int off = 16; off >= 1; off >>= 1) {
+            mn = fminf(mn, __shfl_xor_sync(0xFFFFFFFFu, mn, off));
+            mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, off));
+        }
+        if (lane == 0) { mn_sm[gi] = mn; mx_sm[gi] = mx; }
+    }
+    __syncthreads();
+    const int nr = ratios.n;
+    for (int item = threadIdx.x; item < ngr * nr; item += 256) {
+        const int gi = item / nr, i = item - gi * nr;
+        const float r = ratios.r[i];
+        __half d16;
+        float d, z;
+        group_params(__fmul_rn(mn_sm[gi], r), __fmul_rn(mx_sm[gi], r), top, d16, d, z);
+        const float* wg = w_sm + gi * G;
+        float err = 0.0f;
+#pragma unroll 4
+        for (int k = 0; k < G; ++k) {
+            const float w = wg[k];
+            const float q = fminf(fmaxf(__fadd_rn(rintf(__fdiv_rn(w, d)), z), 0.0f), top);
+            const float e = __fsub_rn(__fmul_rn(__fsub_rn(q, z), d), w);
+            err = __fadd_rn(err, __fmul_rn(e, e));
+        }
+        err_sm[gi * kMaxClipRatios + i] = (err != err) ? INFINITY : err;
+    }
+    __syncthreads();
+    if ((int)threadIdx.x < ngr) {
+        const float* e = err_sm + threadIdx.x * kMaxClipRatios;
+        int best = 0;
+        for (int i = 1; i < nr; ++i)
+            if (e[i] < e[best]) best = i;
+        clip[(size_t)n * (K / G) + k0 / G + threadIdx.x] = ratios.r[best];
     }
 }
 
@@ -204,15 +295,33 @@ cudaError_t launch_channel_scale(const float* a, float alpha, float* s, int K, c
     return cudaGetLastError();
 }
 
-cudaError_t launch_quantize_pack(const __half* W, const float* a, float alpha, int group,
-                                 uint32_t* qweight, __half* scales, uint8_t* zeros,
+cudaError_t launch_quantize_pack(const __half* W, const float* a, float alpha, int group, int bits,
+                                 const float* clip, uint32_t* qweight, __half* scales, uint8_t* zeros,
                                  int N, int K, cudaStream_t st) {
     const dim3 grid(K / 128, N / 128);
     const int mode = (int)alpha_mode(alpha);
+    const float top = (float)((1 << bits) - 1);
     if (group == 128)
-        quantize_pack_kernel<128><<<grid, 256, 0, st>>>(W, a, alpha, mode, qweight, scales, zeros, N, K);
+        quantize_pack_kernel<128><<<grid, 256, 0, st>>>(W, a, alpha, mode, clip, top, qweight, scales, zeros, N, K);
     else
-        quantize_pack_kernel<64><<<grid, 256, 0, st>>>(W, a, alpha, mode, qweight, scales, zeros, N, K);
+        quantize_pack_kernel<64><<<grid, 256, 0, st>>>(W, a, alpha, mode, clip, top, qweight, scales, zeros, N, K);
+    count_launch();
+    return cudaGetLastError();
+}
+
+cudaError_t launch_clip_search(const __half* W, const float* a, float alpha, int group, int bits,
+                               const float* ratios, int n_ratios, float* clip, int N, int K,
+                               cudaStream_t st) {
+    ClipGrid grid_r;
+    grid_r.n = n_ratios;
+    for (int i = 0; i < kMaxClipRatios; ++i) grid_r.r[i] = i < n_ratios ? ratios[i] : 1.0f;
+    const dim3 grid((K + kClipChunk - 1) / kClipChunk, N);
+    const int mode = (int)alpha_mode(alpha);
+    const float top = (float)((1 << bits) - 1);
+    if (group == 128)
+        clip_search_kernel<128><<<grid, 256, 0, st>>>(W, a, alpha, mode, grid_r, top, clip, N, K);
+    else
+        clip_search_kernel<64><<<grid, 256, 0, st>>>(W, a, alpha, mode, grid_r, top, clip, N, K);
     count_launch();
     return cudaGetLastError();
 }
