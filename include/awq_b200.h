@@ -228,6 +228,9 @@ int awq_search_alpha(const void* W, const float* act_mean_abs, const void* X, in
  * into equal ranges over all SM pairs (stream-K) and sums split tiles in a fixed order through the
  * workspace; without one, or with a smaller one, whole tiles go round-robin (same result up to
  * fp32 summation order, slower when the tile count is not a multiple of the pair count).
+ * For M <= 128 they are OPTIONAL as well: with them the tensor-core kernel splits each tile's K
+ * loop over several SMs (up to 16 splits, fp32 partial sums added in split order by whichever SM
+ * finishes a tile last), which is what keeps all SMs busy when N / 128 is below the SM count.
  * awq_set_workspace: registers caller-owned device memory for the current device; the first
  * 4096 bytes are cleared with a synchronous cudaMemset.  Pass (NULL, 0) to unregister.
  * The memory must stay valid until it is unregistered or replaced. */

@@ -179,8 +179,7 @@ def linear(x: torch.Tensor, qweight: torch.Tensor, scales: torch.Tensor, zeros: 
     if x.shape[1] != K:
         raise AwqError("x must be [M][K]")
     y = out if out is not None else torch.empty((M, N), dtype=torch.float16, device=x.device)
-    if (M <= 16 and path not in (PATH_GEMM, PATH_GEMM_1SM)) or (M > 128 and path in (PATH_AUTO, PATH_GEMM)):
-        ensure_workspace(workspace_bytes(M, N, K, group))
+    ensure_workspace(workspace_bytes(M, N, K, group))         # required (split-K GEMV) or optional (GEMM)
     args = (_dev(x, torch.float16, "x"), _dev(qweight, torch.uint8, "qweight"),
             _dev(scales, torch.float16, "scales"), _dev(zeros, torch.uint8, "zeros"),
             _dev(y, torch.float16, "y"), M, N, K, int(group))

@@ -148,17 +148,17 @@ static int resolve_path(int M, int K, int path) {
 
 size_t awq_workspace_bytes(int M, int N, int K, int group) {
     if (check_shape(N, K, group) != AWQ_OK || M < 1) return 0;
-    if (M > 16) {
-        // optional: with it the tensor-core kernel spreads its tiles evenly over the SM pairs
-        int dev = 0, sms = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess ||
-            cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
-            (void)cudaGetLastError();
-            sms = 160;                       // no device to ask: an upper bound for this GPU family
-        }
-        return gemm_workspace_bytes(M, N, sms);
+    // optional for the tensor-core kernels: with it they spread their work evenly over the SMs
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
+        (void)cudaGetLastError();
+        sms = 160;                           // no device to ask: an upper bound for this GPU family
     }
-    return gemv_workspace_bytes(M);
+    const size_t gemm = gemm_workspace_bytes(M, N, sms);
+    if (M > 16) return gemm;
+    const size_t gemv = gemv_workspace_bytes(M);   // required by the split-K matrix-vector kernel
+    return gemv > gemm ? gemv : gemm;
 }
 
 int awq_set_workspace(void* dev_ptr, size_t bytes) {

@@ -42,6 +42,11 @@ namespace awq {
 namespace {
 
 constexpr int kGemmThreads = 512;
+constexpr int kMaxSplits = 16;                  // split-K factor of a tile (M <= 128)
+#ifndef AWQ_DEQUANT_UNROLL
+#define AWQ_DEQUANT_UNROLL 2
+#endif
+constexpr int kDequantUnroll = AWQ_DEQUANT_UNROLL;   // k-blocks a dequantizer warp handles per iteration
 
 template <int BN> struct GemmCfg {
     static constexpr int kXTileBytes = BN * kBK * 2;
@@ -64,7 +69,8 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ CUtensorMap w_map,
             const __grid_constant__ CUtensorMap y_map,
             const __half* __restrict__ scales, const unsigned char* __restrict__ zeros,
-            int M, int N, int K, unsigned int* status_word) {
+            int M, int N, int K, int splits, float* __restrict__ partials,
+            unsigned int* __restrict__ counters, unsigned int* status_word) {
     using Cfg = GemmCfg<BN>;
     constexpr int S = Cfg::kStages;
     constexpr int NACC = Cfg::kNumAcc;
@@ -89,7 +95,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ C
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int m_tiles = (M + BN - 1) / BN;
     const int total_tiles = (N / 128) * m_tiles;
-    const int nkb = K / kBK;
+    // split-K: a work item is (tile, split); split sp of a tile covers the groups
+    // [sp * ng / splits, (sp + 1) * ng / splits), i.e. whole groups and at least one
+    constexpr int KPG = G / kBK;                    // k-blocks per group
+    const int ng = K / G;
+    const int total_items = total_tiles * splits;
+    auto kb_begin = [&](int sp) { return (int)(((long long)sp * ng) / splits) * KPG; };
 
     if (threadIdx.x == 0) {
         s_abort = 0u;
@@ -114,9 +125,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ C
             uint32_t stage = 0, phase = 0;
             unsigned int issued = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+            for (int item = blockIdx.x; item < total_items && ok; item += gridDim.x) {
+                const int tile = item / splits, sp = item - tile * splits;
                 const int slab = tile / m_tiles, mt = tile % m_tiles;
-                for (int kb = 0; kb < nkb; ++kb) {
+                const int kb1 = kb_begin(sp + 1);
+                for (int kb = kb_begin(sp); kb < kb1; ++kb) {
                     if (!mbar_wait(empty(stage), phase ^ 1u, ctl)) { ok = false; break; }
                     const uint32_t bar = raw_full(stage);
                     mbar_arrive_expect_tx(bar, Cfg::kTxBytes);
@@ -145,13 +158,15 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ C
             uint32_t stage = 0, phase = 0;
             int local = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++local) {
+            for (int item = blockIdx.x; item < total_items && ok; item += gridDim.x, ++local) {
+                const int sp = item % splits;
+                const int kb0 = kb_begin(sp), kb1 = kb_begin(sp + 1);
                 const int b = local % NACC;
                 const uint32_t use = (uint32_t)(local / NACC) & 1u;
                 if (!mbar_wait(acc_empty(b), use ^ 1u, ctl)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(b * BN);
-                for (int kb = 0; kb < nkb; ++kb) {
+                for (int kb = kb0; kb < kb1; ++kb) {
                     if (!mbar_wait(raw_full(stage), phase, ctl) || !mbar_wait(a_full(stage), phase, ctl)) {
                         ok = false; break;
                     }
@@ -161,7 +176,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ C
 #pragma unroll
                     for (int k = 0; k < kBK / 16; ++k)       // A: +8 columns, B: +32 bytes per K = 16 step
                         umma_f16_a_tmem(d_tmem, a_tmem + (uint32_t)(8 * k), bdesc + (uint64_t)(2 * k), idesc,
-                                        (kb | k) != 0 ? 1u : 0u);
+                                        (kb != kb0 || k != 0) ? 1u : 0u);
                     umma_commit(empty(stage));
                     if (++stage == S) { stage = 0; phase ^= 1u; }
                 }
@@ -176,56 +191,86 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ C
         const int wi = warp - 8, quad = wi & 3, hsel = wi >> 2;
         const int band = 2 * quad + hsel;               // bands 0..7 <-> TMEM lanes 16*band .. +15
         const int g = lane >> 2;
-        const int ng = K / G;
-        constexpr int KPG = G / kBK;                    // k-blocks per group
         const uint32_t taddr_band = tmem_base + ((uint32_t)(quad * 32 + hsel * 16) << 16) + (uint32_t)Cfg::kAColumn0;
         uint32_t stage = 0, phase = 0;
         bool ok = true;
-        for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+        for (int item = blockIdx.x; item < total_items && ok; item += gridDim.x) {
+            const int tile = item / splits, sp = item - tile * splits;
             const int slab = tile / m_tiles;
+            const int kb0 = kb_begin(sp), kb1 = kb_begin(sp + 1);
             // this lane's rows' parameters: scales [band][group][16], zero bytes [band pair][group][16]
             const unsigned short* sc_g = reinterpret_cast<const unsigned short*>(scales) +
                                          (size_t)(slab * 8 + band) * ng * 16 + g;
             const unsigned char* z_g = zeros + (size_t)(slab * 4 + (band >> 1)) * ng * 16 + (band & 1) * 8 + g;
-            // parameters of the current group and of the next two (fetched ahead of use)
-            uint32_t du = 0, dl = 0, zb = 0, du1, dl1, zb1, du2, dl2, zb2;
-            {
-                const int g1 = min(1, ng - 1);
-                du1 = __ldg(sc_g); dl1 = __ldg(sc_g + 8); zb1 = __ldg(z_g);
-                du2 = __ldg(sc_g + g1 * 16); dl2 = __ldg(sc_g + g1 * 16 + 8); zb2 = __ldg(z_g + g1 * 16);
+            // U k-blocks per iteration, so that their shared-memory reads, conversions and
+            // tensor-memory stores overlap (one k-block at a time is a chain of latencies: measured
+            // ~860 cycles per k-block).  The scales and zero points of an iteration's groups are
+            // fetched two iterations ahead.
+            constexpr int U = kDequantUnroll;
+            constexpr int GPI = U / KPG;                // groups per iteration
+            uint32_t du[GPI], dl[GPI], zb[GPI], du1[GPI], dl1[GPI], zb1[GPI], du2[GPI], dl2[GPI], zb2[GPI];
+            const int g0 = kb0 / KPG;
+#pragma unroll
+            for (int q = 0; q < GPI; ++q) {
+                const int ga = min(g0 + q, ng - 1), gb = min(g0 + GPI + q, ng - 1);
+                du[q] = dl[q] = zb[q] = 0u;
+                du1[q] = __ldg(sc_g + ga * 16); dl1[q] = __ldg(sc_g + ga * 16 + 8); zb1[q] = __ldg(z_g + ga * 16);
+                du2[q] = __ldg(sc_g + gb * 16); dl2[q] = __ldg(sc_g + gb * 16 + 8); zb2[q] = __ldg(z_g + gb * 16);
             }
-            for (int kb = 0; kb < nkb; ++kb) {
-                if (kb % KPG == 0) {
-                    du = du1; dl = dl1; zb = zb1;
-                    du1 = du2; dl1 = dl2; zb1 = zb2;
-                    const int g2 = min(kb / KPG + 2, ng - 1);
-                    du2 = __ldg(sc_g + g2 * 16); dl2 = __ldg(sc_g + g2 * 16 + 8); zb2 = __ldg(z_g + g2 * 16);
+            for (int kb = kb0; kb < kb1; kb += U) {
+                const int n = min(U, kb1 - kb);                    // k-blocks of this iteration
+#pragma unroll
+                for (int q = 0; q < GPI; ++q) {
+                    du[q] = du1[q]; dl[q] = dl1[q]; zb[q] = zb1[q];
+                    du1[q] = du2[q]; dl1[q] = dl2[q]; zb1[q] = zb2[q];
+                    const int gc = min(kb / KPG + 2 * GPI + q, ng - 1);
+                    du2[q] = __ldg(sc_g + gc * 16); dl2[q] = __ldg(sc_g + gc * 16 + 8); zb2[q] = __ldg(z_g + gc * 16);
                 }
-                ok = mbar_wait(raw_full(stage), phase, ctl);
+                uint32_t stg[U];
+                uint4 pk[U];
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    stg[u] = stage;
+                    if (u < n) {
+                        ok = ok && mbar_wait(raw_full(stage), phase, ctl);
+                        if (++stage == S) { stage = 0; phase ^= 1u; }
+                    }
+                }
                 ok = __all_sync(0xFFFFFFFFu, ok);
                 if (!ok) break;
-                const uint4 pk = *reinterpret_cast<const uint4*>(w_ptr(stage) + band * 512 + lane * 16);
-                const uint32_t d_up = du | (du << 16), d_lo = dl | (dl << 16);
-                const uint32_t zu = 0x6400u + (zb & 0xFu), zl = 0xD400u + ((zb >> 4) << 4);
-                const uint32_t zlo = zu | (zu << 16), zhi = zl | (zl << 16);
-                const uint32_t wds[4] = {pk.x, pk.y, pk.z, pk.w};
-                // per word j: (row g: c, c+1) (row g: c+2, c+3) (row g+8: c, c+1) (row g+8: c+2, c+3)
-                uint32_t v[16];
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    constexpr uint32_t kMagic = 0x64006400u, kSixteenth = 0x2C002C00u;
-                    const uint32_t w = wds[j], w8 = w >> 8;
-                    v[4 * j + 0] = hmul2_u32(hsub2_u32((w & 0x000F000Fu) | kMagic, zlo), d_up);
-                    v[4 * j + 1] = hmul2_u32(hsub2_u32((w8 & 0x000F000Fu) | kMagic, zlo), d_up);
-                    v[4 * j + 2] = hmul2_u32(hfma2_u32((w & 0x00F000F0u) | kMagic, kSixteenth, zhi), d_lo);
-                    v[4 * j + 3] = hmul2_u32(hfma2_u32((w8 & 0x00F000F0u) | kMagic, kSixteenth, zhi), d_lo);
+                for (int u = 0; u < U; ++u)
+                    if (u < n) pk[u] = *reinterpret_cast<const uint4*>(w_ptr(stg[u]) + band * 512 + lane * 16);
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    if (u < n) {
+                        const int q = u / KPG;
+                        const uint32_t d_up = du[q] | (du[q] << 16), d_lo = dl[q] | (dl[q] << 16);
+                        const uint32_t zu = 0x6400u + (zb[q] & 0xFu), zl = 0xD400u + ((zb[q] >> 4) << 4);
+                        const uint32_t zlo = zu | (zu << 16), zhi = zl | (zl << 16);
+                        const uint32_t wds[4] = {pk[u].x, pk[u].y, pk[u].z, pk[u].w};
+                        // per word j: (row g: c, c+1) (row g: c+2, c+3) (row g+8: c, c+1) (row g+8: c+2, c+3)
+                        uint32_t v[16];
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            constexpr uint32_t kMagic = 0x64006400u, kSixteenth = 0x2C002C00u;
+                            const uint32_t w = wds[j], w8 = w >> 8;
+                            v[4 * j + 0] = hmul2_u32(hsub2_u32((w & 0x000F000Fu) | kMagic, zlo), d_up);
+                            v[4 * j + 1] = hmul2_u32(hsub2_u32((w8 & 0x000F000Fu) | kMagic, zlo), d_up);
+                            v[4 * j + 2] = hmul2_u32(hfma2_u32((w & 0x00F000F0u) | kMagic, kSixteenth, zhi), d_lo);
+                            v[4 * j + 3] = hmul2_u32(hfma2_u32((w8 & 0x00F000F0u) | kMagic, kSixteenth, zhi), d_lo);
+                        }
+                        tmem_st_16x32cols(taddr_band + stg[u] * 32u, v);
+                    }
                 }
-                tmem_st_16x32cols(taddr_band + stage * 32u, v);
                 tmem_st_wait();
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(a_full(stage));
-                if (++stage == S) { stage = 0; phase ^= 1u; }
+                if (lane == 0) {
+#pragma unroll
+                    for (int u = 0; u < U; ++u)
+                        if (u < n) mbar_arrive(a_full(stg[u]));
+                }
             }
         }
     } else if (warp >= 4) {
@@ -234,7 +279,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ C
         int local = 0;
         int obuf = 0;
         bool ok = true;
-        for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++local) {
+        for (int item = blockIdx.x; item < total_items && ok; item += gridDim.x, ++local) {
+            const int tile = item / splits, sp = item - tile * splits;
             const int slab = tile / m_tiles, mt = tile % m_tiles;
             const int b = local % NACC;
             const uint32_t use = (uint32_t)(local / NACC) & 1u;
@@ -245,16 +291,59 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ C
             const int n0 = slab * 128 + quad * 32;
             const int m0 = mt * BN;
             const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(b * BN);
+            bool finish = true;                 // this warp writes its 32 channels of y
+            if (splits > 1) {
+                // split-K: the partial sums go to the workspace as fp32 [tile][split][token][channel];
+                // the warp whose arrival completes the (tile, quad) count adds all splits in split
+                // order - whichever arrives last, the sum is formed the same way - and nobody waits
+                float* mine = partials + ((size_t)(tile * splits + sp) * BN) * 128 + quad * 32 + lane;
+#pragma unroll 1
+                for (int c = 0; c < BN; c += 32) {
+                    uint32_t r[32];
+                    tmem_ld_32cols(taddr + (uint32_t)c, r);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) mine[(size_t)(c + i) * 128] = __uint_as_float(r[i]);
+                }
+                tc_fence_before();
+                __threadfence();
+                __syncwarp();
+                unsigned int old = 0;
+                if (lane == 0) {
+                    mbar_arrive(acc_empty(b));
+                    old = atomicAdd(counters + tile * 4 + quad, 1u);
+                }
+                old = __shfl_sync(0xFFFFFFFFu, old, 0);
+                finish = old == (unsigned int)(splits - 1);
+                if (finish) {
+                    __threadfence();
+                    if (lane == 0) counters[tile * 4 + quad] = 0u;      // ready for the next call
+                }
+            }
+            if (!finish) continue;
 #pragma unroll 1
             for (int c = 0; c < BN; c += 32) {
                 uint32_t r[32];
-                tmem_ld_32cols(taddr + (uint32_t)c, r);
-                tmem_ld_wait();
-                if (c + 32 >= BN) {
-                    // the accumulator is in registers: the MMA thread may start the next tile
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(acc_empty(b));
+                if (splits > 1) {
+                    const float* all = partials + ((size_t)tile * splits * BN + c) * 128 + quad * 32 + lane;
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__ldcg(all + (size_t)i * 128));
+#pragma unroll 1
+                    for (int q = 1; q < splits; ++q) {
+                        const float* p = all + (size_t)q * BN * 128;
+#pragma unroll
+                        for (int i = 0; i < 32; ++i)
+                            r[i] = __float_as_uint(__uint_as_float(r[i]) + __ldcg(p + (size_t)i * 128));
+                    }
+                } else {
+                    tmem_ld_32cols(taddr + (uint32_t)c, r);
+                    tmem_ld_wait();
+                    if (c + 32 >= BN) {
+                        // the accumulator is in registers: the MMA thread may start the next tile
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(acc_empty(b));
+                    }
                 }
                 // stage the 32 x 32 block as [token][channel] fp16 and hand it to the copy engine:
                 // one tensor store per block instead of 32 two-byte stores per thread (rows past
@@ -292,7 +381,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ C
 template <int G, int BN>
 cudaError_t launch_one(const CUtensorMap& map, const CUtensorMap& wmap, const CUtensorMap& ymap,
                        const void* scales, const void* zeros,
-                       int M, int N, int K, unsigned int* status_word, int sms, cudaStream_t st) {
+                       int M, int N, int K, int splits, void* workspace,
+                       unsigned int* status_word, int sms, cudaStream_t st) {
     using Cfg = GemmCfg<BN>;
     static bool attr_done[64] = {};
     int dev = 0;
@@ -303,13 +393,38 @@ cudaError_t launch_one(const CUtensorMap& map, const CUtensorMap& wmap, const CU
         if (e != cudaSuccess) return e;
         attr_done[dev & 63] = true;
     }
-    const int tiles = (N / 128) * ((M + BN - 1) / BN);
-    const int grid = tiles < sms ? tiles : sms;
+    const int items = (N / 128) * ((M + BN - 1) / BN) * splits;
+    const int grid = items < sms ? items : sms;
+    unsigned char* ws = static_cast<unsigned char*>(workspace);
     gemm_kernel<G, BN><<<grid, kGemmThreads, Cfg::kSmemBytes, st>>>(
         map, wmap, ymap, reinterpret_cast<const __half*>(scales),
-        reinterpret_cast<const unsigned char*>(zeros), M, N, K, status_word);
+        reinterpret_cast<const unsigned char*>(zeros), M, N, K, splits,
+        reinterpret_cast<float*>(ws + kCounterBytes), reinterpret_cast<unsigned int*>(ws), status_word);
     count_launch();
     return cudaGetLastError();
+}
+
+// Split-K factor of the one-SM kernel for M <= 128 (one token tile): with few 128-channel tiles
+// most SMs would idle and the busy ones would each dequantize a whole 128 x K slab.  The factor
+// minimizes rounds / splits, rounds = ceil(tiles * splits / SMs), with a small charge per split for
+// the fp32 partial sums (written and read once), within: at least four k-blocks per split, the
+// workspace at hand, one arrival counter per (tile, 32-channel quarter).
+int gemm_splits(int M, int N, int K, int group, int bn, int sms, size_t workspace_bytes) {
+    if (M > 128 || workspace_bytes <= kCounterBytes) return 1;
+    const int tiles = N / 128;
+    if (tiles * 4 > kMaxSlabs) return 1;
+    const int ng = K / group, nkb = K / kBK;
+    int best = 1;
+    double best_cost = 1e30;
+    for (int sp = 1; sp <= kMaxSplits; ++sp) {
+        if (sp > ng || nkb / sp < 4) break;
+        const size_t need = kCounterBytes + (size_t)tiles * sp * 128 * bn * sizeof(float);
+        if (sp > 1 && need > workspace_bytes) break;
+        const int rounds = (tiles * sp + sms - 1) / sms;
+        const double cost = (double)rounds / sp + (sp > 1 ? 0.02 * sp : 0.0);
+        if (cost < best_cost - 1e-9) { best_cost = cost; best = sp; }
+    }
+    return best;
 }
 
 }  // namespace
@@ -364,8 +479,9 @@ cudaError_t launch_gemm(const void* x, const void* qweight, const void* scales, 
         if (e != cudaSuccess || launched) return e;
     }
     if (!make_x_map(&map, bn) || !make_w_map(&wmap, 128)) return cudaErrorInvalidValue;
+    const int splits = gemm_splits(M, N, K, group, bn, sms, workspace ? workspace_bytes : 0);
 #define AWQ_GEMM_CASE(GG, BNN) \
-    return launch_one<GG, BNN>(map, wmap, ymap, scales, zeros, M, N, K, status_word, sms, st)
+    return launch_one<GG, BNN>(map, wmap, ymap, scales, zeros, M, N, K, splits, workspace, status_word, sms, st)
     if (group == 128) {
         switch (bn) { case 256: AWQ_GEMM_CASE(128, 256); case 128: AWQ_GEMM_CASE(128, 128);
                       case 64: AWQ_GEMM_CASE(128, 64); default: AWQ_GEMM_CASE(128, 32); }
@@ -377,7 +493,13 @@ cudaError_t launch_gemm(const void* x, const void* qweight, const void* scales, 
 }
 
 size_t gemm_workspace_bytes(int M, int N, int sms) {
-    return gemm_pair_applies(M, N) ? gemm_pair_workspace_bytes(sms) : 0;
+    if (gemm_pair_applies(M, N)) return gemm_pair_workspace_bytes(sms);
+    if (M > 128) return 0;
+    // split-K of the one-SM kernel: the most it can use for this M and N (any K)
+    const int bn = M > 64 ? 128 : M > 32 ? 64 : 32;
+    const int tiles = N / 128;
+    if (tiles * 4 > kMaxSlabs) return 0;
+    return kCounterBytes + (size_t)tiles * kMaxSplits * 128 * bn * sizeof(float);
 }
 
 }  // namespace awq

@@ -429,13 +429,39 @@ gemv_band_kernel(const BandProblems probs, const __half* __restrict__ x, int M, 
 #pragma unroll
         for (int jw = 0; jw < 4; ++jw) xr[v][jw] = make_uint2(0u, 0u);
 
-    if (XREG && tok_ok) {
-        const __half* xg = x + (size_t)g * K + (size_t)warp * (TPW * 64) + t * 4;
+    if constexpr (XREG) {
+        // Each token's slice of x for this warp (TPW k-tiles = 32 lanes x 16 bytes) is fetched with
+        // one coalesced 16-byte load per lane - every block asks L2 for the same few lines of x
+        // at the same moment, so the number of requests matters - and brought into fragment
+        // order through a private block of the reduction buffer, which is idle until the first
+        // band has been summed.
+        static_assert(TPW == 4, "the staging block holds 32 lanes x 16 bytes per token");
+        unsigned char* xst = reinterpret_cast<unsigned char*>(red) + warp * 512;
+        const uint4* xrow = reinterpret_cast<const uint4*>(x + (size_t)warp * (TPW * 64)) + lane;
 #pragma unroll
-        for (int v = 0; v < TPW; ++v)
+        for (int m0 = 0; m0 < 8; m0 += 4) {
+            if (m0 < M) {
+                uint4 row[4];
 #pragma unroll
-            for (int jw = 0; jw < 4; ++jw)
-                xr[v][jw] = __ldg(reinterpret_cast<const uint2*>(xg + v * 64 + jw * 16));
+                for (int i = 0; i < 4; ++i)
+                    if (m0 + i < M) row[i] = __ldg(xrow + (size_t)(m0 + i) * (K / 8));
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    if (m0 + i < M) {
+                        *reinterpret_cast<uint4*>(xst + lane * 16) = row[i];
+                        __syncwarp();
+                        if (g == m0 + i) {
+#pragma unroll
+                            for (int v = 0; v < TPW; ++v)
+#pragma unroll
+                                for (int jw = 0; jw < 4; ++jw)
+                                    xr[v][jw] = *reinterpret_cast<const uint2*>(xst + v * 128 + jw * 32 + t * 8);
+                        }
+                        __syncwarp();
+                    }
+                }
+            }
+        }
     }
     float XxR[GPW] = {}, XyR[GPW] = {};                  // XREG: 2^-24 times this warp's group sums of x
     if (XREG) {

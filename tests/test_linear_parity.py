@@ -51,6 +51,9 @@ GEMM_CASES = [
     (2560, 256, 2100, 128, 0.5), (2560, 384, 2100, 64, 0.5),
     # long K loops: with stream-K most pairs start or end inside a tile, some tiles are cut twice
     (512, 8192, 520, 128, 0.5), (1280, 6144, 1300, 64, 0.5),
+    # M <= 128 with a workspace: split-K of the one-SM kernel (several splits per tile, ragged
+    # group counts per split, more items than SMs)
+    (4096, 4096, 64, 128, 0.5), (1024, 2816, 33, 64, 0.5), (11008, 1408, 128, 128, 0.5), (2560, 1152, 20, 128, 0.5),
 ]
 
 
@@ -142,6 +145,10 @@ def test_auto_dispatch_between_9_and_16_tokens():
     try:
         rc = L.awq_linear(x.data_ptr(), qw.data_ptr(), sc.data_ptr(), zp.data_ptr(), y.data_ptr(),
                           case.M, case.N, case.K, case.group, None)
+        assert rc == 0
+        # the tensor-core kernel without a workspace (with one it splits K and sums in another order)
+        rc = L.awq_linear_path(x.data_ptr(), qw.data_ptr(), sc.data_ptr(), zp.data_ptr(), forced_gemm.data_ptr(),
+                               case.M, case.N, case.K, case.group, binding.PATH_GEMM, None)
         assert rc == 0
         binding.poll_status()
     finally:
