@@ -158,6 +158,7 @@ size_t awq_workspace_bytes(int M, int N, int K, int group) {
     const size_t gemm = gemm_workspace_bytes(M, N, sms);
     if (M > 16) return gemm;
     const size_t gemv = gemv_workspace_bytes(M);   // required by the split-K matrix-vector kernel
+    if (M <= 8) return gemv;                       // awq_linear never takes the tensor-core kernel here
     return gemv > gemm ? gemv : gemm;
 }
 

@@ -39,7 +39,9 @@ def test_sizes_and_layout_version(lib):
     assert lib.awq_qweight_bytes(100, 4096) == 0
     assert lib.awq_scales_bytes(4096, 4096, 32) == 0
     assert lib.awq_workspace_bytes(1, 4096, 4096, 128) > 4096
-    assert lib.awq_workspace_bytes(64, 4096, 4096, 128) == 0
+    # optional for M <= 128: split-K partial sums of the one-SM tensor-core kernel (16 splits at most)
+    assert lib.awq_workspace_bytes(64, 4096, 4096, 128) == 4096 + 32 * 16 * 128 * 64 * 4
+    assert lib.awq_workspace_bytes(12, 4096, 4096, 128) == 4096 + 32 * 16 * 128 * 32 * 4
     big = lib.awq_workspace_bytes(2048, 4096, 4096, 128)            # optional: stream-K partial tiles
     assert big > 4096 and (big - 4096) % (256 * 256 * 4) == 0
     assert lib.awq_workspace_bytes(2048, 4096 + 128, 4096, 128) == 0
