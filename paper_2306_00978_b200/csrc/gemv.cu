@@ -228,14 +228,17 @@ __device__ __forceinline__ void band_full_stage(const unsigned char* st, int o_w
             for (int q = 0; q < GPW; ++q) {
                 const int tile = q * TPG + v;
                 const uint32_t w = (jw == 0) ? pk[tile].x : (jw == 1) ? pk[tile].y : (jw == 2) ? pk[tile].z : pk[tile].w;
-                const uint32_t w8 = w >> 8;
+                // Integer and logic instructions issue at half the rate of fp32 ones and four masks
+                // plus a shift per word were the largest item of the stage, so the upper rows'
+                // operands keep their whole byte - the row-g code plus 16 times the row-(g+8) code of
+                // the same column, still an exact fp16 subnormal - and the lower rows' share is
+                // taken off once per group below; the byte permute replaces shift and mask.
+                const uint32_t w8 = __byte_perm(w, 0u, 0x4341u);            // bytes 1 and 3 of w
                 const uint32_t bb0 = xr[tile][jw].x, bb1 = xr[tile][jw].y;
                 if (v == 0 && jw == 0)
-                    mma_16816_first(c[q], w & 0x000F000Fu, w & 0x00F000F0u, w8 & 0x000F000Fu,
-                                    w8 & 0x00F000F0u, bb0, bb1);
+                    mma_16816_first(c[q], w & 0x00FF00FFu, w & 0x00F000F0u, w8, w8 & 0x00F000F0u, bb0, bb1);
                 else
-                    mma_16816(c[q], w & 0x000F000Fu, w & 0x00F000F0u, w8 & 0x000F000Fu,
-                              w8 & 0x00F000F0u, bb0, bb1);
+                    mma_16816(c[q], w & 0x00FF00FFu, w & 0x00F000F0u, w8, w8 & 0x00F000F0u, bb0, bb1);
             }
     // per group: Delta * (2^24 D - z X); integers below 2^23 become floats without a conversion
     // instruction; the lower rows' codes entered the product 16 times too large (mask 0xF0) and
@@ -249,11 +252,12 @@ __device__ __forceinline__ void band_full_stage(const unsigned char* st, int o_w
         const float z_lo16 = __uint_as_float(0x4B000000u | (zb & 0xF0u)) - 8388608.0f;   // 16 * z
         const float su = d_up * 16777216.0f, sl = d_lo * 1048576.0f;
         const float kx = Kx[q];
-        acc[0] = fmaf(su, fmaf(-z_up, kx, c[q][0]), acc[0]);
+        // c[q][0] holds sum (q_g + 16 q_{g+8}) x, c[q][2] holds sum 16 q_{g+8} x (both times 2^-24)
+        acc[0] = fmaf(su, fmaf(-z_up, kx, c[q][0] - c[q][2]), acc[0]);
         acc[2] = fmaf(sl, fmaf(-z_lo16, kx, c[q][2]), acc[2]);
         if (!ONE) {
             const float ky = Ky[q];
-            acc[1] = fmaf(su, fmaf(-z_up, ky, c[q][1]), acc[1]);
+            acc[1] = fmaf(su, fmaf(-z_up, ky, c[q][1] - c[q][3]), acc[1]);
             acc[3] = fmaf(sl, fmaf(-z_lo16, ky, c[q][3]), acc[3]);
         }
     }
