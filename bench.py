@@ -459,6 +459,53 @@ def one_shape(args):
     return 0
 
 
+def sweep(args):
+    """The full-shape sweep over the 7B layer's three distinct shapes: token counts 1 .. 8192 and
+    both group sizes through awq_linear (random packed weights, three rotating copies so that
+    small shapes do not sit in L2, eight calls per CUDA-graph replay, best of five replays).
+    One JSON object per line: microseconds, algorithmic GB/s, TFLOP/s."""
+    import torch
+    from paper_2306_00978_b200 import binding
+    shapes = [("q/k/v/o", 4096, 4096), ("gate/up", 4096, 11008), ("down", 11008, 4096)]
+    for group in (128, 64):
+        for name, K, N in shapes:
+            copies = []
+            for _ in range(3):
+                qw = torch.randint(0, 256, (N * K // 2,), dtype=torch.uint8, device="cuda")
+                sc = (torch.rand((N // 16, K // group, 16), device="cuda") * 0.01 + 0.001).half()
+                zp = torch.randint(0, 256, (N // 32, K // group, 16), dtype=torch.uint8, device="cuda")
+                copies.append((qw, sc, zp))
+            for M in (1, 2, 4, 8, 16, 32, 64, 128, 512, 2048, 8192):
+                x = torch.randn((M, K), device="cuda").half()
+                y = torch.empty((M, N), device="cuda", dtype=torch.float16)
+                calls = 8 if M <= 512 else 2
+                for i in range(3):
+                    binding.linear(x, *copies[i], N, K, group, out=y)
+                torch.cuda.synchronize()
+                graph, stream = torch.cuda.CUDAGraph(), torch.cuda.Stream()
+                with torch.cuda.stream(stream):
+                    with torch.cuda.graph(graph, stream=stream):
+                        for i in range(calls):
+                            binding.linear(x, *copies[i % 3], N, K, group, out=y)
+                torch.cuda.synchronize()
+                graph.replay()
+                torch.cuda.synchronize()
+                best = float("inf")
+                for _ in range(5):
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    e0.record()
+                    graph.replay()
+                    e1.record()
+                    torch.cuda.synchronize()
+                    best = min(best, e0.elapsed_time(e1) * 1e3 / calls)
+                binding.poll_status()
+                nbytes = N * K // 2 + (N * K // group) * 2 + (N * K // group) // 2 + M * K * 2 + M * N * 2
+                print(json.dumps({"shape": name, "K": K, "N": N, "group": group, "M": M, "us": round(best, 2),
+                                  "GBps": round(nbytes / best / 1e3, 1),
+                                  "TFLOPs": round(2 * M * N * K / best / 1e6, 1)}), flush=True)
+    return 0
+
+
 # --------------------------------------------------------------------------------- main
 def main():
     ap = argparse.ArgumentParser()
@@ -473,9 +520,13 @@ def main():
                          "weights (three rotating copies), then exit")
     ap.add_argument("--path", type=int, default=0, help="with --one: 0 auto, 1 GEMV, 2 GEMM, 3 split-K GEMV, 4 single-SM GEMM")
     ap.add_argument("--reps", type=int, default=3, help="with --one: passes over the three copies")
+    ap.add_argument("--sweep", action="store_true",
+                    help="per-shape table over the 7B layer shapes, M = 1 .. 8192, both group sizes; then exit")
     args = ap.parse_args()
     if args.one:
         return one_shape(args)
+    if args.sweep:
+        return sweep(args)
 
     if args.impl == "reference":
         return reference_arm(args)

@@ -66,16 +66,17 @@ __device__ __forceinline__ void mma_16816_first(float (&c)[4], uint32_t a0, uint
 // One 16-row x 64-column packed block (this lane's 16 bytes `pk`) times the matching 64
 // activations of MT*8 tokens (this lane's 4 x 8 bytes per token tile: word j of the piece
 // multiplies x[16j + 4t .. +3]):
-// c[mt][chain] receive D = sum q * 2^-24 x (rows g) and sum q * 2^-20 x (rows g+8).
+// c[mt][chain] receive D = sum (q_g + 16 q_{g+8}) * 2^-24 x (rows g: the whole byte is the
+// operand, see band_full_stage) and sum q_{g+8} * 2^-20 x (rows g+8); the caller subtracts.
 template <int MT, int NCH, bool FIRST = true>
 __device__ __forceinline__ void block_mma(const uint4& pk, const uint2 (&xq)[MT][4],
                                           float (&c)[MT][NCH][4]) {
     const uint32_t wds[4] = {pk.x, pk.y, pk.z, pk.w};
 #pragma unroll
     for (int jw = 0; jw < 4; ++jw) {
-        const uint32_t w = wds[jw], w8 = w >> 8;
-        const uint32_t a0 = w & 0x000F000Fu, a1 = w & 0x00F000F0u;
-        const uint32_t a2 = w8 & 0x000F000Fu, a3 = w8 & 0x00F000F0u;
+        const uint32_t w = wds[jw], w8 = __byte_perm(w, 0u, 0x4341u);     // bytes 1 and 3 of w
+        const uint32_t a0 = w & 0x00FF00FFu, a1 = w & 0x00F000F0u;
+        const uint32_t a2 = w8, a3 = w8 & 0x00F000F0u;
 #pragma unroll
         for (int mt = 0; mt < MT; ++mt) {
             const uint32_t b0 = xq[mt][jw].x, b1 = xq[mt][jw].y;
@@ -191,7 +192,9 @@ inline BandLayout band_layout(int M, int K, bool x_in_registers) {
     using St = BandStage<G, TPW>;
     BandLayout l;
     l.stage_bytes = ((St::kXOff + (x_in_registers ? 0 : M * St::kXRow) + 127) / 128) * 128;
-    const int xsum = (K / 64 + St::kUT) * 8 * 4;        // + one stage of slack for ragged reads
+    // per-k-tile sums of x (+ one stage of slack for ragged reads); with x in registers the region
+    // is the math warps' staging block for x instead (16 warps x 512 bytes)
+    const int xsum = x_in_registers ? kMathWarps * 512 : (K / 64 + St::kUT) * 8 * 4;
     l.red_tokens = M <= 4 ? 4 : 8;
     const int red = 6 * kMathWarps * l.red_tokens * 16 * 4;   // one buffer per stage of [warp][token][row] fp32
     int s = (kSmemBudget - xsum - red - 256) / l.stage_bytes;
@@ -437,10 +440,11 @@ gemv_band_kernel(const BandProblems probs, const __half* __restrict__ x, int M, 
         // Each token's slice of x for this warp (TPW k-tiles = 32 lanes x 16 bytes) is fetched with
         // one coalesced 16-byte load per lane - every block asks L2 for the same few lines of x
         // at the same moment, so the number of requests matters - and brought into fragment
-        // order through a private block of the reduction buffer, which is idle until the first
-        // band has been summed.
+        // order through the warp's private 512-byte block of shared memory (the region that holds
+        // the sums of x when x travels through the stages; not the reduction buffers: a warp that
+        // runs ahead may already be writing its sums there).
         static_assert(TPW == 4, "the staging block holds 32 lanes x 16 bytes per token");
-        unsigned char* xst = reinterpret_cast<unsigned char*>(red) + warp * 512;
+        unsigned char* xst = reinterpret_cast<unsigned char*>(xsum) + warp * 512;
         const uint4* xrow = reinterpret_cast<const uint4*>(x + (size_t)warp * (TPW * 64)) + lane;
 #pragma unroll
         for (int m0 = 0; m0 < 8; m0 += 4) {
@@ -586,10 +590,11 @@ gemv_band_kernel(const BandProblems probs, const __half* __restrict__ x, int M, 
                         const uint32_t zb = st[o_z + q * 16];
                         const float su = d_up * 16777216.0f, sl = d_lo * 1048576.0f;
                         const float zu = d_up * (float)(zb & 0xFu), zl = d_lo * (float)(zb >> 4);
-                        acc[0] = fmaf(su, c[0][0][0] + c[0][1][0], fmaf(-zu, Xx, acc[0]));
-                        acc[1] = fmaf(su, c[0][0][1] + c[0][1][1], fmaf(-zu, Xy, acc[1]));
-                        acc[2] = fmaf(sl, c[0][0][2] + c[0][1][2], fmaf(-zl, Xx, acc[2]));
-                        acc[3] = fmaf(sl, c[0][0][3] + c[0][1][3], fmaf(-zl, Xy, acc[3]));
+                        const float lo_x = c[0][0][2] + c[0][1][2], lo_y = c[0][0][3] + c[0][1][3];
+                        acc[0] = fmaf(su, (c[0][0][0] + c[0][1][0]) - lo_x, fmaf(-zu, Xx, acc[0]));
+                        acc[1] = fmaf(su, (c[0][0][1] + c[0][1][1]) - lo_y, fmaf(-zu, Xy, acc[1]));
+                        acc[2] = fmaf(sl, lo_x, fmaf(-zl, Xx, acc[2]));
+                        acc[3] = fmaf(sl, lo_y, fmaf(-zl, Xy, acc[3]));
                     }
                 }
             }
@@ -887,6 +892,8 @@ gemv_splitk_kernel(const unsigned char* __restrict__ qweight, const __half* __re
                         float d[4];
 #pragma unroll
                         for (int i = 0; i < 4; ++i) d[i] = (NCH == 2) ? c[mt][0][i] + c[mt][NCH - 1][i] : c[mt][0][i];
+                        d[0] -= d[2];                         // rows g carried the rows g+8 codes as well
+                        d[1] -= d[3];
                         acc[mt][0] = fmaf(su, d[0], fmaf(zu, X.x, acc[mt][0]));
                         acc[mt][1] = fmaf(su, d[1], fmaf(zu, X.y, acc[mt][1]));
                         acc[mt][2] = fmaf(sl, d[2], fmaf(zl, X.x, acc[mt][2]));

@@ -109,3 +109,36 @@ def test_70b_mlp_batch_sweep_sampled(name, K, N):
         y = binding.linear(to_cuda(xs), qw, sc, zp, N, K, GROUP)
         binding.poll_status()
         assert_parity(y.cpu().numpy()[:, rows], orc.linear(xs, Wd), f"70B {name} M={M}")
+
+
+SWEEP_SHAPES = [("q_proj", 4096, 4096), ("up_proj", 4096, 11008), ("down_proj", 11008, 4096)]
+
+
+@pytest.mark.parametrize("G,alpha", [(128, 0.5), (64, 1.0), (128, 0.0)])
+@pytest.mark.parametrize("name,K,N", SWEEP_SHAPES)
+def test_7b_shape_sweep_sampled(name, K, N, G, alpha):
+    """The full-shape sweep: the three distinct 7B layer shapes over the token counts
+    1 .. 8192 (every kernel and every dispatch branch), both group sizes and the three exact
+    alphas, through awq_linear; sampled channels, for large M sampled tokens as well."""
+    from paper_2306_00978_b200 import binding
+    seed = 7000 + K // 64 + N // 64 + G
+    W = synth.weight(seed, N, K)
+    a = synth.act_mean_abs(seed, K)
+    s = orc.channel_scale(a, alpha)
+    qw, sc, zp = binding.quantize_pack(to_cuda(W), to_cuda(a), alpha, G)
+    rng = np.random.default_rng(seed)
+    rows = _sample_rows(rng, N, count=40)
+    codes, zeros, scales = orc.quantize(W[rows], s, G)
+    Wdq = orc.dequantize(codes, zeros, scales, G)
+    Ms = (1, 2, 4, 8, 16, 32, 64, 128, 512, 2048, 8192)
+    x_all = synth.activations(seed, max(Ms), K)
+    xs_all = (x_all.astype(np.float32) / s[None, :]).astype(np.float16)
+    for M in Ms:
+        xs = xs_all[:M]
+        y = binding.linear(to_cuda(xs), qw, sc, zp, N, K, G)
+        binding.poll_status()
+        y = y.cpu().numpy()
+        toks = np.arange(M) if M <= 128 else np.unique(np.concatenate(
+            [rng.choice(M, size=64, replace=False), [0, 127, 128, 255, 256, M - 1]]))
+        y_ref = orc.linear(xs[toks], Wdq)
+        assert_parity(y[np.ix_(toks, rows)], y_ref, f"sweep {name} G={G} alpha={alpha} M={M}")
