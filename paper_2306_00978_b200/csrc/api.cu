@@ -192,9 +192,10 @@ int awq_linear_path(const void* x, const void* qweight, const void* scales, cons
     if (path != AWQ_PATH_GEMM && path != AWQ_PATH_GEMM_1SM && (M > 16 || K > 65536)) return AWQ_ERR_BAD_SHAPE;
     DeviceState* d;
     if (int rc = device_state(&d)) return rc;
-    if (automatic && M > 8 && M <= 16 && K <= 65536) {
-        // measured: up to 16 tokens the split-K matrix-vector kernel beats the tensor-core kernel
-        // (75 vs 115 us on 8192 -> 28672); it needs the workspace, the tensor-core kernel does not
+    if (automatic && M > 8 && M <= 16 && K <= 65536 && (size_t)N * (size_t)K >= ((size_t)1 << 27)) {
+        // measured at 16 tokens: on large matrices the split-K matrix-vector kernel beats the
+        // tensor-core kernel (74 vs 98 us on 8192 -> 28672), on small ones it loses (18.6 vs 13.6 us
+        // on 4096 -> 4096); it needs the workspace, the tensor-core kernel does not
         std::lock_guard<std::mutex> lock(g_mutex);
         if (d->workspace_bytes >= gemv_workspace_bytes(M)) path = AWQ_PATH_GEMV;
     }

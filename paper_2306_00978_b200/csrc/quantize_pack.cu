@@ -56,12 +56,13 @@ __device__ __forceinline__ uint32_t code_of(float w, float d, float rd, float z,
 
 // grid = (K/128, N/128), block = 256 (8 warps = 8 bands of the 128-row slab); three blocks per SM:
 // the kernel is latency-bound (loads, then arithmetic), measured 67.6 -> 53.2 us on 4096->11008
-template <int G>
+template <int G, int BITS, bool CLIP>
 __global__ void __launch_bounds__(256, 3)
 quantize_pack_kernel(const __half* __restrict__ W, const float* __restrict__ a, float alpha,
-                     int mode, const float* __restrict__ clip, float top,
+                     int mode, const float* __restrict__ clip,
                      uint32_t* __restrict__ qweight, __half* __restrict__ scales,
                      uint8_t* __restrict__ zeros, int N, int K) {
+    constexpr float top = (float)((1 << BITS) - 1);       // largest code
     __shared__ __align__(16) float s_sm[128];
     const int kblk = blockIdx.x, slab = blockIdx.y;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -133,7 +134,7 @@ quantize_pack_kernel(const __half* __restrict__ W, const float* __restrict__ a, 
                 mx[ti][h] = fmaxf(mx[ti][h], __shfl_xor_sync(0xFFFFFFFFu, mx[ti][h], off));
             }
 
-    if (clip != nullptr) {
+    if (CLIP) {
         // weight clipping (Sec. 3.2): the group's range shrinks by its ratio, values outside saturate
         const int ng = K / G;
 #pragma unroll
@@ -300,11 +301,18 @@ cudaError_t launch_quantize_pack(const __half* W, const float* a, float alpha, i
                                  int N, int K, cudaStream_t st) {
     const dim3 grid(K / 128, N / 128);
     const int mode = (int)alpha_mode(alpha);
-    const float top = (float)((1 << bits) - 1);
-    if (group == 128)
-        quantize_pack_kernel<128><<<grid, 256, 0, st>>>(W, a, alpha, mode, clip, top, qweight, scales, zeros, N, K);
-    else
-        quantize_pack_kernel<64><<<grid, 256, 0, st>>>(W, a, alpha, mode, clip, top, qweight, scales, zeros, N, K);
+#define AWQ_QP_LAUNCH(GG, BB, CC) \
+    quantize_pack_kernel<GG, BB, CC><<<grid, 256, 0, st>>>(W, a, alpha, mode, clip, qweight, scales, zeros, N, K)
+#define AWQ_QP_PICK(GG)                                                  \
+    do {                                                                 \
+        if (bits == 4 && !clip) AWQ_QP_LAUNCH(GG, 4, false);             \
+        else if (bits == 4) AWQ_QP_LAUNCH(GG, 4, true);                  \
+        else if (!clip) AWQ_QP_LAUNCH(GG, 3, false);                     \
+        else AWQ_QP_LAUNCH(GG, 3, true);                                 \
+    } while (0)
+    if (group == 128) AWQ_QP_PICK(128); else AWQ_QP_PICK(64);
+#undef AWQ_QP_PICK
+#undef AWQ_QP_LAUNCH
     count_launch();
     return cudaGetLastError();
 }

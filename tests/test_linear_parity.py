@@ -126,38 +126,44 @@ def test_auto_dispatch_and_special_values():
 
 
 def test_auto_dispatch_between_9_and_16_tokens():
-    """awq_linear with 9..16 tokens runs the split-K matrix-vector kernel when a workspace is
-    registered and the tensor-core kernel when none is: each bit-equal to its forced path."""
+    """awq_linear with 9..16 tokens: the tensor-core kernel on small matrices, and on large ones
+    (N * K >= 2^27) the split-K matrix-vector kernel if a workspace is registered.  Each result is
+    bit-equal to its forced path."""
     import torch
     from paper_2306_00978_b200 import binding
     L = binding.lib()
     case = Case(77, 1024, 1408, 12, 128, 0.5)
     qw, sc, zp = oracle_packed_to_cuda(case)
     x = to_cuda(case.x)
-    forced_gemv = binding.linear(x, qw, sc, zp, case.N, case.K, case.group, path=binding.PATH_GEMV)
+    auto = binding.linear(x, qw, sc, zp, case.N, case.K, case.group)
     forced_gemm = binding.linear(x, qw, sc, zp, case.N, case.K, case.group, path=binding.PATH_GEMM)
-    with_ws = binding.linear(x, qw, sc, zp, case.N, case.K, case.group)      # binding registers a workspace
-    assert torch.equal(with_ws, forced_gemv)
-    y = torch.empty_like(forced_gemm)
+    assert torch.equal(auto, forced_gemm)
+    assert_parity(auto.cpu().numpy(), case.y_ref(), "auto M=12, small matrix")
+    # a large matrix (random packed arrays: only the choice of kernel is checked here; parity at
+    # this size is covered by the 70B sweep)
+    N, K, G, M = 16384, 8192, 128, 12
+    qw = torch.randint(0, 256, (N * K // 2,), dtype=torch.uint8, device="cuda")
+    sc = (torch.rand((N // 16, K // G, 16), device="cuda") * 0.01 + 0.001).half()
+    zp = torch.randint(0, 256, (N // 32, K // G, 16), dtype=torch.uint8, device="cuda")
+    x = torch.randn((M, K), device="cuda").half()
+    with_ws = binding.linear(x, qw, sc, zp, N, K, G)                       # binding registers a workspace
+    assert torch.equal(with_ws, binding.linear(x, qw, sc, zp, N, K, G, path=binding.PATH_GEMV))
+    y = torch.empty_like(with_ws)
+    ref = torch.empty_like(with_ws)
     torch.cuda.synchronize()
     saved = binding._workspace.pop(torch.cuda.current_device(), None)
     assert L.awq_set_workspace(None, 0) == 0
     try:
-        rc = L.awq_linear(x.data_ptr(), qw.data_ptr(), sc.data_ptr(), zp.data_ptr(), y.data_ptr(),
-                          case.M, case.N, case.K, case.group, None)
-        assert rc == 0
-        # the tensor-core kernel without a workspace (with one it splits K and sums in another order)
-        rc = L.awq_linear_path(x.data_ptr(), qw.data_ptr(), sc.data_ptr(), zp.data_ptr(), forced_gemm.data_ptr(),
-                               case.M, case.N, case.K, case.group, binding.PATH_GEMM, None)
-        assert rc == 0
+        args = (x.data_ptr(), qw.data_ptr(), sc.data_ptr(), zp.data_ptr())
+        assert L.awq_linear(*args, y.data_ptr(), M, N, K, G, None) == 0
+        assert L.awq_linear_path(*args, ref.data_ptr(), M, N, K, G, binding.PATH_GEMM, None) == 0
         binding.poll_status()
     finally:
         if saved is not None:
             assert L.awq_set_workspace(saved.data_ptr(), saved.numel()) == 0
             binding._workspace[torch.cuda.current_device()] = saved
-    assert torch.equal(y, forced_gemm)
-    assert_parity(y.cpu().numpy(), case.y_ref(), "auto M=12 without workspace")
-    assert_parity(with_ws.cpu().numpy(), case.y_ref(), "auto M=12 with workspace")
+    assert torch.equal(y, ref)                                              # no workspace: tensor-core kernel
+    assert not torch.equal(y, with_ws)
 
 
 @pytest.mark.parametrize("M,G", [(1, 128), (3, 64), (7, 128)])
