@@ -8,13 +8,17 @@
 //
 // Math (both kernels).  Sixteen math warps.  The 16 bytes a lane reads from a stage are already
 // the A fragments of four warp-level m16n8k16 tensor-core products: thanks to the
-// w{0,2,4,6,1,3,5,7} nibble order, masking a packed word with 0x000F000F / 0x00F000F0 (before
-// and after one shift by 8) leaves two codes in the mantissa bits of an fp16x2 register, i.e.
-// the exact values q * 2^-24 (upper row) and q * 2^-20 (lower row) as fp16 subnormals.  Five
-// logic operations and one MMA per eight weights - the paper counts a shift, an AND and an FMA
-// per single weight.  x (up to 8 tokens per product) is the B operand, accumulation is fp32.
-// Zero point and scale are applied once per 64 columns in fp32:
-//   sum (q - z) x = 2^24 * D - z * X,   X = sum of x over those columns,
+// w{0,2,4,6,1,3,5,7} nibble order, every byte of a packed word holds the codes of rows g (low
+// nibble) and g+8 (high nibble) of one column, and bytes 0 / 2 and 1 / 3 line up with the two
+// halves of an fp16x2 register.  A byte in the mantissa bits of an fp16 is the exact subnormal
+// (q_g + 16 q_{g+8}) * 2^-24: the upper rows' operands are the bytes as they are (mask 0x00FF00FF,
+// or one byte permute for the odd bytes), the lower rows' operands the high nibbles alone (mask
+// 0x00F000F0 = 16 q_{g+8} * 2^-24), and the lower rows' sums are taken off the upper rows' once per
+// group.  Four integer-pipe operations and one MMA per eight weights - the paper counts a shift, an
+// AND and an FMA per single weight; the count matters because integer-pipe instructions dispatch at
+// half the fp32 rate and the stage time follows them.  x (up to 8 tokens per product) is the B
+// operand, accumulation is fp32.  Zero point and scale are applied once per group in fp32:
+//   sum (q - z) x = 2^24 * D - z * X,   X = sum of x over the group's columns,
 // where X is the same for every output row, so each block sums it once, in fp32, while its
 // first weight stages are in flight.  Nothing is rounded to fp16 before the output.
 //
