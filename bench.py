@@ -147,12 +147,25 @@ def build_layers(n_layers: int, seed0: int = 2000):
             s = binding.channel_scale(a, ALPHA, K)
             x = torch.from_numpy(synth.activations(xseed, 1, K)).cuda()
             xs = (x.float() / s[None, :]).half().contiguous()     # the caller's x / s
-            x_host = xs.cpu().pin_memory()
-            y = torch.empty((1, N), dtype=torch.float16, device="cuda")
-            y_host = torch.empty((1, N), dtype=torch.float16).pin_memory()
-            lin.append(dict(name=name, N=N, K=K, qw=qw, sc=sc, zp=zp, x=xs, x_host=x_host,
-                            y=y, y_host=y_host, x_dev_in=torch.empty_like(xs)))
+            lin.append(dict(name=name, N=N, K=K, qw=qw, sc=sc, zp=zp, x=xs))
             del W
+        # host-side view of a step (the e2e leg): the step's four activations in one pinned buffer,
+        # its seven outputs in another, one copy each way per step; the device tensors the calls
+        # read and write are views into the device-side images of the two buffers
+        firsts = [idxs[0] for idxs in STEP_CALLS]
+        x_host = torch.cat([lin[i]["x"].reshape(-1) for i in firsts]).cpu().pin_memory()
+        x_dev = torch.empty(x_host.numel(), dtype=torch.float16, device="cuda")
+        y_dev = torch.empty(sum(l["N"] for l in lin), dtype=torch.float16, device="cuda")
+        y_host = torch.empty(y_dev.numel(), dtype=torch.float16).pin_memory()
+        off = 0
+        for i in firsts:
+            lin[i]["x_dev_in"] = x_dev[off:off + lin[i]["K"]].view(1, -1)
+            off += lin[i]["K"]
+        off = 0
+        for l in lin:
+            l["y"] = y_dev[off:off + l["N"]].view(1, -1)
+            off += l["N"]
+        lin[0].update(x_host=x_host, x_dev=x_dev, y_dev=y_dev, y_host=y_host)
         layers.append(lin)
     torch.cuda.synchronize()
     return layers
@@ -165,25 +178,24 @@ STEP_CALLS = ((0, 1, 2), (3,), (4, 5), (6,))
 
 def run_step(layer, e2e=False):
     from paper_2306_00978_b200 import binding
+    if e2e:                                            # the step's inputs from pinned host memory
+        layer[0]["x_dev"].copy_(layer[0]["x_host"], non_blocking=True)
     for idxs in STEP_CALLS:
         first = layer[idxs[0]]
-        xin = first["x"]
-        if e2e:                                        # x from pinned host memory, every call
-            first["x_dev_in"].copy_(first["x_host"], non_blocking=True)
-            xin = first["x_dev_in"]
+        xin = first["x_dev_in"] if e2e else first["x"]
         if len(idxs) == 1:
             binding.linear(xin, first["qw"], first["sc"], first["zp"], first["N"], first["K"], GROUP,
                            out=first["y"])
         else:
             binding.linear_multi(xin, [(layer[i]["qw"], layer[i]["sc"], layer[i]["zp"], layer[i]["N"]) for i in idxs],
                                  first["K"], GROUP, outs=[layer[i]["y"] for i in idxs])
-        if e2e:
-            for i in idxs:
-                layer[i]["y_host"].copy_(layer[i]["y"], non_blocking=True)
+    if e2e:                                            # the step's outputs back to the host
+        layer[0]["y_host"].copy_(layer[0]["y_dev"], non_blocking=True)
 
 
 def run_step_e2e(layer):
-    """The same step through host buffers: x from pinned memory in, y back out, every call."""
+    """The same step through host buffers: the step's x from pinned memory in (one copy), its y
+    back out (one copy)."""
     run_step(layer, e2e=True)
 
 
