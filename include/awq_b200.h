@@ -245,7 +245,8 @@ int awq_unpack_canonical(const void* qweight, const void* scales, const void* ze
 
 /* Reads and clears the device status word of the current device (synchronizes the device).
  * Returns AWQ_OK, or AWQ_ERR_TIMEOUT if a kernel gave up a bounded wait since the last poll
- * (its output is then undefined), or AWQ_ERR_CUDA. */
+ * (its output is then undefined; the arrival counters at the head of the registered workspace
+ * are cleared again so that later calls start clean), or AWQ_ERR_CUDA. */
 int awq_poll_status(void);
 
 const char* awq_status_string(int status);

@@ -348,6 +348,16 @@ int awq_poll_status(void) {
     if (int rc = note_cuda(cudaMemcpy(&v, d->status_word, sizeof(v), cudaMemcpyDeviceToHost))) return rc;
     if (v != 0) {
         if (int rc = note_cuda(cudaMemset(d->status_word, 0, sizeof(v)))) return rc;
+        // a kernel that gave up may have left arrival counters half-way: start them afresh
+        void* ws = nullptr;
+        size_t ws_bytes = 0;
+        {
+            std::lock_guard<std::mutex> lock(g_mutex);
+            ws = d->workspace;
+            ws_bytes = d->workspace_bytes;
+        }
+        if (ws && ws_bytes >= kCounterBytes)
+            if (int rc = note_cuda(cudaMemset(ws, 0, kCounterBytes))) return rc;
         return AWQ_ERR_TIMEOUT;
     }
     return AWQ_OK;
