@@ -66,8 +66,9 @@ typedef enum AwqPath {
     AWQ_PATH_GEMV = 1,          /* fused dequant matrix-vector kernel, M <= 16: band kernel when
                                    M <= 8 and N/16 is not much below the SM count, else split-K */
     AWQ_PATH_GEMM = 2,          /* tcgen05 tensor-core kernel, any M >= 1: pairs of SMs
-                                   (cta_group::2, 256 channels x 256 tokens per tile) when
-                                   M > 128 and N is a multiple of 256, else one SM per tile */
+                                   (cta_group::2, 256 channels x 256 tokens per tile) when N is a
+                                   multiple of 256 and M > 128 (M > 64 from N = 8192, M >= 32 from
+                                   N = 16384), else one SM per tile */
     AWQ_PATH_GEMV_SPLITK = 3,   /* the split-K matrix-vector kernel, M <= 16 */
     AWQ_PATH_GEMM_1SM = 4       /* the tensor-core kernel with one SM per tile, any M >= 1 */
 } AwqPath;
@@ -223,7 +224,7 @@ int awq_search_alpha(const void* W, const float* act_mean_abs, const void* X, in
 
 /* Workspace (scratch for partial sums and arrival counters).
  * awq_workspace_bytes: bytes awq_linear can use for this problem (0 if none).  For M <= 16 the
- * split-K matrix-vector kernel REQUIRES them.  For M > 128 with N a multiple of 256 they are
+ * split-K matrix-vector kernel REQUIRES them.  Where the SM-pair tensor-core kernel runs (see AWQ_PATH_GEMM) they are
  * OPTIONAL: with a workspace of at least this size the tensor-core kernel cuts the tiles' K loops
  * into equal ranges over all SM pairs (stream-K) and sums split tiles in a fixed order through the
  * workspace; without one, or with a smaller one, whole tiles go round-robin (same result up to

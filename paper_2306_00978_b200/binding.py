@@ -237,10 +237,7 @@ def search_alpha(W: torch.Tensor, act_mean_abs: torch.Tensor, X: torch.Tensor, g
     if need == 0:
         raise AwqError(f"shape N={N}, K={K}, group={group} is not accepted")
     scratch = torch.empty(need, dtype=torch.uint8, device=W.device)
-    if M <= 16:
-        ensure_workspace(workspace_bytes(M, N, K, group))
-    elif M > 128:
-        ensure_workspace(workspace_bytes(M, N, K, group))
+    ensure_workspace(workspace_bytes(M, N, K, group))
     a = (ctypes.c_float * n)(*[float(v) for v in alphas])
     losses = (ctypes.c_float * n)()
     best = ctypes.c_int(0)

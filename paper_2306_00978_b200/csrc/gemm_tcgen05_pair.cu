@@ -553,7 +553,14 @@ cudaError_t launch_pair(const CUtensorMap& xmap, const CUtensorMap& wmap, const 
 
 }  // namespace
 
-bool gemm_pair_applies(int M, int N) { return M > 128 && N % 256 == 0; }
+// Above 128 tokens always; below, where the one-SM kernel's 128-channel tiles re-read x too often:
+// measured at M = 96 .. 128, 27.6 against 42 us on 4096 -> 11008; at M = 32 .. 128, 77 .. 84 against
+// 98 .. 117 us on 8192 -> 28672; but 26.5 against 13 .. 19 us on 4096 -> 4096 (few tiles: the
+// one-SM kernel with split-K wins).
+bool gemm_pair_applies(int M, int N) {
+    if (N % 256 != 0) return false;
+    return M > 128 || (M > 64 && N >= 8192) || (M >= 32 && N >= 16384);
+}
 
 // workspace with which the pair kernel balances its tiles over all SM pairs (stream-K)
 size_t gemm_pair_workspace_bytes(int sms) {

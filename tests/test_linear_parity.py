@@ -54,6 +54,8 @@ GEMM_CASES = [
     # M <= 128 with a workspace: split-K of the one-SM kernel (several splits per tile, ragged
     # group counts per split, more items than SMs)
     (4096, 4096, 64, 128, 0.5), (1024, 2816, 33, 64, 0.5), (11008, 1408, 128, 128, 0.5), (2560, 1152, 20, 128, 0.5),
+    # wide matrices at 33 .. 128 tokens: the SM-pair kernel with half-empty token tiles
+    (8192, 512, 100, 128, 0.5), (16384, 256, 40, 64, 0.5), (8192, 384, 64, 128, 0.5),
 ]
 
 
@@ -83,7 +85,7 @@ def _run_gemm_without_workspace(case):
 @pytest.mark.parametrize("mode", ["auto", "one-sm", "no-workspace"])
 @pytest.mark.parametrize("N,K,M,G,alpha", GEMM_CASES)
 def test_gemm_parity(N, K, M, G, alpha, mode):
-    """PATH_GEMM runs SM pairs when M > 128 and N % 256 == 0 (stream-K over the registered
+    """PATH_GEMM runs SM pairs when N % 256 == 0 and M > 128, or less on wide matrices (stream-K over the registered
     workspace, or whole tiles round-robin without one) and one SM per tile otherwise;
     PATH_GEMM_1SM forces the latter on every case."""
     from paper_2306_00978_b200 import binding
