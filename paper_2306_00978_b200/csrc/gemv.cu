@@ -866,42 +866,58 @@ gemv_splitk_kernel(const unsigned char* __restrict__ qweight, const __half* __re
             const unsigned char* xp[MT];
 #pragma unroll
             for (int mt = 0; mt < MT; ++mt) xp[mt] = st + x_off[mt];
+            // one accumulation per group (TPG k-tiles; K % 128 == 0 makes the warp's tile count a
+            // whole number of groups), then scale and zero point once per group
             constexpr int NCH = (MT == 1) ? 2 : 1;
 #pragma unroll
-            for (int v = 0; v < kWT; ++v) {
-                if (v < ntw) {
-                    const int tile = kWT * half + v;                   // k-tile inside the stage
-                    const uint4 pk = *reinterpret_cast<const uint4*>(st + w_off + v * 512);
-                    uint2 xq[MT][4];
+            for (int q2 = 0; q2 < kWT / TPG; ++q2) {
+                if (q2 * TPG < ntw) {
+                    float c[MT][NCH][4];
+                    float Xx[MT], Xy[MT];
 #pragma unroll
-                    for (int mt = 0; mt < MT; ++mt)
+                    for (int mt = 0; mt < MT; ++mt) { Xx[mt] = 0.0f; Xy[mt] = 0.0f; }
 #pragma unroll
-                        for (int jw = 0; jw < 4; ++jw) {
-                            // lanes without a token must not touch shared memory (see the band kernel)
-                            xq[mt][jw] = make_uint2(0u, 0u);
-                            if (tok_ok[mt]) xq[mt][jw] = *reinterpret_cast<const uint2*>(xp[mt] + v * 128 + jw * 32);
+                    for (int v2 = 0; v2 < TPG; ++v2) {
+                        const int v = q2 * TPG + v2;
+                        const int tile = kWT * half + v;               // k-tile inside the stage
+                        const uint4 pk = *reinterpret_cast<const uint4*>(st + w_off + v * 512);
+                        uint2 xq[MT][4];
+#pragma unroll
+                        for (int mt = 0; mt < MT; ++mt) {
+#pragma unroll
+                            for (int jw = 0; jw < 4; ++jw) {
+                                // lanes without a token must not touch shared memory (see the band kernel)
+                                xq[mt][jw] = make_uint2(0u, 0u);
+                                if (tok_ok[mt]) xq[mt][jw] = *reinterpret_cast<const uint2*>(xp[mt] + v * 128 + jw * 32);
+                            }
+                            const float2 X = *reinterpret_cast<const float2*>(
+                                xsum + (j * kUT + tile) * MTOK + mt * 8 + 2 * t);
+                            Xx[mt] += X.x;
+                            Xy[mt] += X.y;
                         }
-                    const int q = tile / TPG;
+                        if (v2 == 0) block_mma<MT, NCH, true>(pk, xq, c);
+                        else block_mma<MT, NCH, false>(pk, xq, c);
+                    }
+                    const int q = (kWT * half) / TPG + q2;             // group inside the stage
                     const float d_up = __half2float(*reinterpret_cast<const __half*>(st + sc_off + q * 32));
                     const float d_lo = __half2float(*reinterpret_cast<const __half*>(st + sc_off + q * 32 + 16));
                     const uint32_t zb = st[z_off + q * 16];
+                    // integers below 2^23 become floats without a conversion instruction
+                    const float z_up = __uint_as_float(0x4B000000u | (zb & 0xFu)) - 8388608.0f;
+                    const float z_lo16 = __uint_as_float(0x4B000000u | (zb & 0xF0u)) - 8388608.0f;   // 16 * z
                     const float su = d_up * 16777216.0f, sl = d_lo * 1048576.0f;
-                    const float zu = -d_up * (float)(zb & 0xFu), zl = -d_lo * (float)(zb >> 4);
-                    float c[MT][NCH][4];
-                    block_mma<MT, NCH>(pk, xq, c);
 #pragma unroll
                     for (int mt = 0; mt < MT; ++mt) {
-                        const float2 X = *reinterpret_cast<const float2*>(
-                            xsum + (j * kUT + tile) * MTOK + mt * 8 + 2 * t);
                         float d[4];
 #pragma unroll
                         for (int i = 0; i < 4; ++i) d[i] = (NCH == 2) ? c[mt][0][i] + c[mt][NCH - 1][i] : c[mt][0][i];
                         d[0] -= d[2];                         // rows g carried the rows g+8 codes as well
                         d[1] -= d[3];
-                        acc[mt][0] = fmaf(su, d[0], fmaf(zu, X.x, acc[mt][0]));
-                        acc[mt][1] = fmaf(su, d[1], fmaf(zu, X.y, acc[mt][1]));
-                        acc[mt][2] = fmaf(sl, d[2], fmaf(zl, X.x, acc[mt][2]));
-                        acc[mt][3] = fmaf(sl, d[3], fmaf(zl, X.y, acc[mt][3]));
+                        const float kx = Xx[mt] * (1.0f / 16777216.0f), ky = Xy[mt] * (1.0f / 16777216.0f);
+                        acc[mt][0] = fmaf(su, fmaf(-z_up, kx, d[0]), acc[mt][0]);
+                        acc[mt][1] = fmaf(su, fmaf(-z_up, ky, d[1]), acc[mt][1]);
+                        acc[mt][2] = fmaf(sl, fmaf(-z_lo16, kx, d[2]), acc[mt][2]);
+                        acc[mt][3] = fmaf(sl, fmaf(-z_lo16, ky, d[3]), acc[mt][3]);
                     }
                 }
             }

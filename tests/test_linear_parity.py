@@ -122,8 +122,10 @@ def test_auto_dispatch_and_special_values():
         ref = orc.linear(x, orc.dequantize(codes, zeros, scales, G))
         mask = np.ones(N, bool)
         mask[200] = False
-        # zero up to fp32 rounding of (sum q x) - z (sum x): far below one fp16 ulp of a typical output
-        assert np.abs(y[:, mask]).max() <= 1e-5
+        # zero up to fp32 rounding of (sum q x) - z (sum x), whose terms reach 255 |x| Delta per column
+        # (the upper rows' operands carry the lower rows' codes too): below one fp16 ulp of a
+        # typical output (|y| ~ 0.1: 6e-5)
+        assert np.abs(y[:, mask]).max() <= 4e-5
         assert np.allclose(y[:, 200], ref[:, 200], rtol=2e-3, atol=1e-5)
 
 
