@@ -620,7 +620,7 @@ def main():
                              "awq_linear_multi(gate,up), awq_linear(down); the rotating layers are replayed "
                              "back to back as one CUDA graph (layers_rotated steps per replay), a remainder of "
                              "steps as single-layer graphs"},
-        "roofline": {"bound": "hbm", "kernel": "gemv_band_kernel<128,4,true,true>", "achieved": achieved,
+        "roofline": {"bound": "hbm", "kernel": "gemv_band_kernel<128,4,true,true,5>", "achieved": achieved,
                      "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
                      "peak_source": peaks["source"], "frac_of_nominal_8000": achieved / NOMINAL_HBM_GBS,
                      "avg_launch_us": per_launch_s * 1e6,

@@ -275,7 +275,10 @@ __device__ __forceinline__ void band_full_stage(const unsigned char* st, int o_w
 // XREG: K == 64 * 16 * TPW, i.e. a band is exactly one stage and a math warp meets the same
 // k-tiles in every stage: its B fragments of x and its per-group sums of x are loaded once, from
 // global memory, and stay in registers; no x travels through the stages.
-template <int G, int TPW, bool ONE, bool XREG>
+// XS: 0, or (XREG only) the number of stages of the ring, known at compile time together with
+// 4-token reduction rows: the loop over the bands is then unrolled over one turn of the ring and
+// every stage, barrier and reduction address is a constant.
+template <int G, int TPW, bool ONE, bool XREG, int XS>
 __global__ void __launch_bounds__(kBandThreads, 1)
 gemv_band_kernel(const BandProblems probs, const __half* __restrict__ x, int M, int K,
                  const BandLayout lay, unsigned int* status_word) {
@@ -503,6 +506,37 @@ gemv_band_kernel(const BandProblems probs, const __half* __restrict__ x, int M, 
         // measured slower.)
         tile_sums_of_x(x, xsum, M, K, 8, warp, kMathWarps, lane);
         named_barrier_sync(3, kMathThreads);
+    }
+
+    if constexpr (XREG && XS > 0) {
+        // ---- a band is one stage and the ring has XS stages: one turn of the ring per outer
+        // iteration, all addresses constants of the slot
+        constexpr uint32_t SB = ((St::kXOff + 127) / 128) * 128;          // stage bytes (no x part)
+        constexpr int RS = 4 * 16;                                         // floats per warp in red[]
+        float* const rb0 = red + warp * RS + 2 * t * 16 + g;               // red[stage][warp][token][row]
+        const bool store_ok = t < 2;                                       // tokens 0 .. 3
+        int o_z = St::kZOff + warp * (GPW * 16) + (b0 & 1) * 8 + g;
+        uint32_t phase = 0;
+        for (int task = b0;;) {
+#pragma unroll
+            for (int sl = 0; sl < XS; ++sl) {
+                if (task >= b1) return;
+                float acc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+                mbar_wait(bars + 8u * sl, phase, ctl);
+                band_full_stage<G, TPW, ONE>(smem + sl * SB, o_w, o_sc, o_z, xr, XxR, XyR, acc);
+                if (store_ok) {
+                    float* rb = rb0 + sl * (kMathWarps * RS);
+                    rb[0] = acc[0];
+                    rb[8] = acc[2];
+                    if (!ONE) { rb[16] = acc[1]; rb[24] = acc[3]; }
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bars + 128u + 8u * sl);         // the flush warp frees the stage
+                o_z ^= 8;
+                ++task;
+            }
+            phase ^= 1u;
+        }
     }
 
     if constexpr (XREG) {
@@ -1038,11 +1072,19 @@ cudaError_t launch_gemv_band(const void* x, const GemvMatrix* mats, int count, i
         const BandLayout lay = band_layout<GG, TT>(M, K, XR);                                        \
         if (lay.stages < 2) return cudaErrorInvalidValue;      /* K too large for the x-sum table */ \
         static bool done[64] = {};                                                                   \
-        e = allow_big_smem(gemv_band_kernel<GG, TT, ONE1, XR>, done);                                \
-        if (e != cudaSuccess) return e;                                                              \
         cfg.dynamicSmemBytes = lay.total;                                                            \
-        e = cudaLaunchKernelEx(&cfg, gemv_band_kernel<GG, TT, ONE1, XR>, pr,                         \
-                               reinterpret_cast<const __half*>(x), M, K, lay, status_word);          \
+        if (XR && lay.stages == 5 && lay.red_tokens == 4) {                                          \
+            static bool done5[64] = {};                                                              \
+            e = allow_big_smem(gemv_band_kernel<GG, TT, ONE1, XR, (XR ? 5 : 0)>, done5);             \
+            if (e != cudaSuccess) return e;                                                          \
+            e = cudaLaunchKernelEx(&cfg, gemv_band_kernel<GG, TT, ONE1, XR, (XR ? 5 : 0)>, pr,       \
+                                   reinterpret_cast<const __half*>(x), M, K, lay, status_word);      \
+        } else {                                                                                     \
+            e = allow_big_smem(gemv_band_kernel<GG, TT, ONE1, XR, 0>, done);                         \
+            if (e != cudaSuccess) return e;                                                          \
+            e = cudaLaunchKernelEx(&cfg, gemv_band_kernel<GG, TT, ONE1, XR, 0>, pr,                  \
+                                   reinterpret_cast<const __half*>(x), M, K, lay, status_word);      \
+        }                                                                                            \
         if (e != cudaSuccess) return e;                                                              \
     } while (0)
     const bool xreg = tpw == 4 && K == 64 * 16 * 4;            // a band is exactly one stage
