@@ -53,11 +53,35 @@ __device__ __forceinline__ uint32_t code_of(float w, float d, float rd, float z,
     if (!(fabsf(t - r) < 0.499f && fabsf(t) < 1024.0f)) r = rintf(__fdiv_rn(w, d));
     return (uint32_t)fminf(fmaxf(__fadd_rn(r, z), 0.0f), top);
 }
+// The same without the per-element branch: `bad` collects whether any element came within `thr`
+// of a half-integer (thr = 0.5 minus the group's bound on |w * rd - w / d|); the caller then redoes
+// the word with code_of.  Every lane of a warp has to pass for the warp to skip the divisions, so
+// the margin is the group's own bound (a few 1e-6) and not a fixed 1e-3.
+__device__ __forceinline__ float level_fast(float w, float rd, float z, float top, float thr, bool& bad) {
+    const float t = __fmul_rn(w, rd);
+    // round half to even by addition (exact for |t| < 2^22; larger quotients have thr < 0): two fp32
+    // additions instead of a conversion-pipe instruction, the pipe this kernel keeps busiest
+    const float r = __fsub_rn(__fadd_rn(t, 12582912.0f), 12582912.0f);
+    bad = bad || !(fabsf(t - r) < thr);
+    return fminf(fmaxf(__fadd_rn(r, z), 0.0f), top);              // the code, still a float
+}
+// four codes (exact small integers held in floats) as four nibbles: q0 + 16 q1 + 256 q2 + 4096 q3 is
+// exact in fp32, so three FFMAs and one conversion replace four conversions and the shifts and ORs
+__device__ __forceinline__ uint32_t pack4(float q0, float q1, float q2, float q3) {
+    return (uint32_t)fmaf(q3, 4096.0f, fmaf(q2, 256.0f, fmaf(q1, 16.0f, q0)));
+}
 
-// grid = (K/128, N/128), block = 256 (8 warps = 8 bands of the 128-row slab); three blocks per SM:
-// the kernel is latency-bound (loads, then arithmetic), measured 67.6 -> 53.2 us on 4096->11008
+// grid = (K/128, N/128), block = 256 (8 warps = 8 bands of the 128-row slab); two blocks per SM
+// (118 registers, no spills; three blocks at 80 registers spill and measure 1 % slower).  The kernel
+// is bound by its own instruction stream (issue slots 62 % active, conversion pipe 55 %): measured on
+// 4096->11008, 67.6 us at first, 56 us with the multiply-instead-of-divide path per element, 50.5 us
+// with that path made branch-free per word, 48.2 us with rounding by addition, 46.4 us with the
+// nibbles assembled by FFMA (one conversion per four codes).
+#ifndef AWQ_QP_BLOCKS
+#define AWQ_QP_BLOCKS 2
+#endif
 template <int G, int BITS, bool CLIP>
-__global__ void __launch_bounds__(256, 3)
+__global__ void __launch_bounds__(256, AWQ_QP_BLOCKS)
 quantize_pack_kernel(const __half* __restrict__ W, const float* __restrict__ a, float alpha,
                      int mode, const float* __restrict__ clip,
                      uint32_t* __restrict__ qweight, __half* __restrict__ scales,
@@ -88,7 +112,7 @@ quantize_pack_kernel(const __half* __restrict__ W, const float* __restrict__ a, 
 
     // w' = fp32(w) * s  (Eq. 3) is formed twice from the raw words - here for the group's min / max,
     // below for the codes (the same two operations give the same value) - so that only the 32 raw
-    // registers stay live and four blocks fit an SM.  The four scales of a word are one 16-byte
+    // registers stay live.  The four scales of a word are one 16-byte
     // shared-memory read, used for both rows.
     auto wprime = [&](int ti, int h, int j, const float (&sv)[4], float (&w4)[4]) {
         const uint32_t u0 = raw[ti][h][j].x, u1 = raw[ti][h][j].y;
@@ -134,6 +158,12 @@ quantize_pack_kernel(const __half* __restrict__ W, const float* __restrict__ a, 
                 mx[ti][h] = fmaxf(mx[ti][h], __shfl_xor_sync(0xFFFFFFFFu, mx[ti][h], off));
             }
 
+    float wabs[2][2];                                       // largest |w'| of each group (before clipping)
+#pragma unroll
+    for (int ti = 0; ti < 2; ++ti)
+#pragma unroll
+        for (int h = 0; h < 2; ++h) wabs[ti][h] = fmaxf(fabsf(mn[ti][h]), fabsf(mx[ti][h]));
+
     if (CLIP) {
         // weight clipping (Sec. 3.2): the group's range shrinks by its ratio, values outside saturate
         const int ng = K / G;
@@ -150,11 +180,15 @@ quantize_pack_kernel(const __half* __restrict__ W, const float* __restrict__ a, 
 
 #pragma unroll
     for (int ti = 0; ti < 2; ++ti) {
-        __half d16[2]; float d[2], z[2], rd[2];
+        __half d16[2]; float d[2], z[2], rd[2], thr[2];
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
             group_params(mn[ti][h], mx[ti][h], top, d16[h], d[h], z[h]);
             rd[h] = __frcp_rn(d[h]);
+            // |w * rd - w / d| <= 1.8e-7 |w / d| (three roundings); the group's largest |w / d|
+            // bounds it for every element; quotients beyond 1024 always take the division
+            const float tmax = __fmul_rn(wabs[ti][h], rd[h]);
+            thr[h] = tmax < 1024.0f ? 0.5f - fmaf(tmax, 4e-7f, 1e-6f) : -1.0f;
         }
 
         uint32_t words[4];
@@ -167,10 +201,20 @@ quantize_pack_kernel(const __half* __restrict__ W, const float* __restrict__ a, 
             wprime(ti, 1, j, sv, wl);
             // slots (g,c) (g,c+1) (g+8,c) (g+8,c+1) (g,c+2) (g,c+3) (g+8,c+2) (g+8,c+3)
             // at nibbles 0, 4, 1, 5, 2, 6, 3, 7
-            words[j] = (code_of(wu[0], d[0], rd[0], z[0], top) << 0) | (code_of(wu[1], d[0], rd[0], z[0], top) << 16) |
-                       (code_of(wl[0], d[1], rd[1], z[1], top) << 4) | (code_of(wl[1], d[1], rd[1], z[1], top) << 20) |
-                       (code_of(wu[2], d[0], rd[0], z[0], top) << 8) | (code_of(wu[3], d[0], rd[0], z[0], top) << 24) |
-                       (code_of(wl[2], d[1], rd[1], z[1], top) << 12) | (code_of(wl[3], d[1], rd[1], z[1], top) << 28);
+            bool bad = false;
+            float qu[4], ql[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                qu[e] = level_fast(wu[e], rd[0], z[0], top, thr[0], bad);
+                ql[e] = level_fast(wl[e], rd[1], z[1], top, thr[1], bad);
+            }
+            // nibbles 0 .. 3 = (g,c) (g+8,c) (g,c+2) (g+8,c+2), nibbles 4 .. 7 the same for c+1, c+3
+            words[j] = pack4(qu[0], ql[0], qu[2], ql[2]) | (pack4(qu[1], ql[1], qu[3], ql[3]) << 16);
+            if (bad)                                               // rare: the word again, element by element
+                words[j] = (code_of(wu[0], d[0], rd[0], z[0], top) << 0) | (code_of(wu[1], d[0], rd[0], z[0], top) << 16) |
+                           (code_of(wl[0], d[1], rd[1], z[1], top) << 4) | (code_of(wl[1], d[1], rd[1], z[1], top) << 20) |
+                           (code_of(wu[2], d[0], rd[0], z[0], top) << 8) | (code_of(wu[3], d[0], rd[0], z[0], top) << 24) |
+                           (code_of(wl[2], d[1], rd[1], z[1], top) << 12) | (code_of(wl[3], d[1], rd[1], z[1], top) << 28);
         }
         // band-major: block (band, k-tile) is 512 bytes, a band's blocks are contiguous along K
         const size_t band = (size_t)slab * 8 + warp;
