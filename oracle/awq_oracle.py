@@ -47,6 +47,9 @@ actually quantized), unweighted, in fp32 in a fixed order so that the choice is 
 for bit, and keeps the first best ratio.  INT3 (the paper's INT3-g128 tables) is the same
 quantizer on 8 levels (Delta = (max - min) / 7, z and q in [0, 7]); how the paper's kernels would
 store 3-bit codes is not described, here they occupy the 4-bit fields of the INT4 layout.
+The symmetric grid is Eq. 2 as printed; since Round(w / Delta) then spans 2**bits + 1 values
+(-2**(bits-1) .. +2**(bits-1)), the single level +2**(bits-1) - reached only by a group's largest
+positive element - saturates at the top code.
 Parity for these asymmetric details is unpinned by the paper (it prints no worked numeric
 example of Q); they are pinned by closed-form invariants, grid-aligned round trips and
 brute-force enumeration in tests/test_oracle_pins.py.
@@ -89,8 +92,10 @@ def channel_scale(act_mean_abs, alpha: float) -> np.ndarray:
 
 
 # --------------------------------------------------------------------- Eq. 2 - Eq. 4
-def quantize(W, s, group: int, clip=None, bits: int = 4):
-    """Group-wise asymmetric round-to-nearest of W * diag(s) on a grid of 2**bits levels.
+def quantize(W, s, group: int, clip=None, bits: int = 4, symmetric: bool = False):
+    """Group-wise round-to-nearest of W * diag(s) on a grid of 2**bits levels: asymmetric (min / max
+    with a zero point), or symmetric (Eq. 2 as printed: Delta = max|w'| / 2**(bits-1), no offset;
+    stored with the fixed zero point 2**(bits-1), the level +2**(bits-1) saturating at the top code).
 
     W fp16 [N][K]; s fp32 [K]; groups are `group` consecutive input channels of one
     output row.  clip: None, or fp32 [N][K/group] of range ratios (Sec. 3.2, weight clipping):
@@ -124,6 +129,20 @@ def quantize(W, s, group: int, clip=None, bits: int = 4):
         if clip is not None:
             mn = mn * clip[r0:r1]
             mx = mx * clip[r0:r1]
+        if symmetric:
+            half = np.float32(1 << (bits - 1))
+            amax = np.maximum(np.abs(mn), np.abs(mx))
+            with np.errstate(over="ignore", invalid="ignore", divide="ignore"):
+                d16 = (amax / half).astype(np.float16)               # Eq. 2: Delta = max|w| / 2^(N-1)
+                bad = ~np.isfinite(d16) | (d16 == 0)
+                d16 = np.where(bad, np.float16(1.0), d16).astype(np.float16)
+                d = d16.astype(np.float32)
+                z = np.full_like(d, half)
+                q = np.clip(np.rint(wg / d[:, :, None]) + half, f0, f15)   # Eq. 2: Round(w / Delta)
+            codes[r0:r1] = q.reshape(r1 - r0, K).astype(np.uint8)
+            zeros[r0:r1] = z.astype(np.uint8)
+            scales[r0:r1] = d16
+            continue
         with np.errstate(over="ignore", invalid="ignore", divide="ignore"):
             d16 = ((mx - mn) / f15).astype(np.float16)  # Delta, stored in fp16
             bad = ~np.isfinite(d16) | (d16 == 0)
@@ -276,12 +295,12 @@ def search_clip(W, s, group: int, ratios, bits: int = 4) -> np.ndarray:
     return ratios[best].astype(np.float32)
 
 
-def quantize_pack(W, act_mean_abs, alpha: float, group: int, clip=None, bits: int = 4):
+def quantize_pack(W, act_mean_abs, alpha: float, group: int, clip=None, bits: int = 4, symmetric: bool = False):
     """The whole offline step: returns (qweight u32, scales fp16 [N/16][ng][16], zeros u8 [N/32][ng][16]).
     3-bit codes (bits = 3) are stored in the same 4-bit fields."""
     K = W.shape[1]
     a = np.ones(K, np.float32) if act_mean_abs is None else act_mean_abs
-    codes, zeros, scales = quantize(W, channel_scale(a, alpha), group, clip=clip, bits=bits)
+    codes, zeros, scales = quantize(W, channel_scale(a, alpha), group, clip=clip, bits=bits, symmetric=symmetric)
     return pack_qweight(codes), pack_scales(scales), pack_zeros(zeros)
 
 

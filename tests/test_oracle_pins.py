@@ -598,3 +598,41 @@ def test_int3_grid_invariants_and_brute_force():
         err = lambda qs: sum((wi - (qi - zz) * dd) ** 2 for wi, qi in zip(w, qs))
         best = min(err(qs) for qs in itertools.product(range(8), repeat=3))
         assert err([int(x) for x in c[r]]) <= best * (1 + Fraction(1, 2**20))
+
+
+# ------------------------------------------------------------------- symmetric grid (Eq. 2)
+def test_symmetric_grid_is_eq2():
+    """Eq. 2 as printed: Q(w) = Delta * Round(w / Delta), Delta = max|w| / 2^(N-1).  Pinned by a
+    grid-aligned group (codes known by hand), by exact zeros, by odd symmetry and by the half-step
+    error bound; the one level the 4-bit code cannot hold (+8) saturates."""
+    d = 2.0 ** -5
+    lv = np.arange(-8, 8)                                            # -8 .. 7: max|w| = 8 d, so Delta = d
+    Wg = (np.tile(lv, 8) * d).astype(np.float16)[None, :]
+    ones = np.ones(128, np.float32)
+    c, z, sc = orc.quantize(Wg, ones, 128, symmetric=True)
+    assert z[0, 0] == 8 and float(sc[0, 0]) == d
+    assert np.array_equal(c[0, :16], lv + 8)                         # code = Round(w / Delta) + 8
+    assert np.array_equal(orc.dequantize(c, z, sc, 128), Wg.astype(np.float64))      # round trip exact
+    # mirrored group: max at +8 d: that single element saturates at code 15 (value 7 d), the rest mirror
+    c2, z2, sc2 = orc.quantize((-Wg).astype(np.float16), ones, 128, symmetric=True)
+    assert float(sc2[0, 0]) == d and c2[0, 0] == 15
+    assert np.array_equal(c2[0, 1:16], 16 - c[0, 1:16])
+    # random groups: zero stays zero, |error| <= Delta / 2 (+ fp16 rounding of Delta) away from the top level
+    W, a = _gaussian_case(41, 64, 512)
+    W = W.copy()
+    W[:, ::17] = np.float16(0.0)
+    s = orc.channel_scale(a, 0.5)
+    c, z, sc = orc.quantize(W, s, 128, symmetric=True)
+    assert (z == 8).all()
+    back = orc.dequantize(c, z, sc, 128)
+    assert (back[:, ::17] == 0.0).all()
+    wp = W.astype(np.float64) * s.astype(np.float64)
+    dd = np.repeat(sc.astype(np.float64), 128, axis=1)
+    top_level = wp >= 7.5 * dd
+    assert (np.abs(wp - back)[~top_level] <= (0.5 + 8 * 2.0**-11) * dd[~top_level] + 1e-12).all()
+    assert (np.abs(wp - back)[top_level] <= (1.0 + 8 * 2.0**-11) * dd[top_level]).all()
+    amax = np.abs(wp).reshape(64, 4, 128).max(axis=2)
+    assert (np.abs(sc.astype(np.float64) - amax / 8.0) <= 2.0**-11 * amax / 8.0 * 1.0001).all()
+    # 3 bits: zero point 4, codes 0 .. 7
+    c3, z3, sc3 = orc.quantize(W, s, 128, bits=3, symmetric=True)
+    assert (z3 == 4).all() and c3.max() <= 7
