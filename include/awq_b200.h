@@ -101,14 +101,19 @@ int awq_quantize_pack(const void* W, const float* act_mean_abs, float alpha, int
  *   bits: 4 or 3.  bits = 3 quantizes to 8 levels (Delta = fp16_rne(range / 7), z and q in
  *         [0,7]); the 3-bit codes occupy the same 4-bit fields, so the packed arrays, their
  *         sizes and awq_linear are unchanged (the paper does not describe a 3-bit storage).
+ *   symmetric: 0, or 1 for the grid of Eq. 2 as printed: Delta = fp16_rne(max|w'| / 2^(bits-1)),
+ *         q = clamp(rne(w' / Delta) + 2^(bits-1), 0, 2^bits - 1) and the stored zero point is
+ *         2^(bits-1) for every group (Round(w'/Delta) spans 2^bits + 1 values; the largest,
+ *         reached only by a group's biggest positive element, saturates at the top code).
  *   clip_ratio: NULL, or in, device, fp32 [N][K/group] (row-major): the group's range becomes
  *         [r * min w', r * max w'] (one fp32 multiply each) before Delta and z are formed; values
  *         outside saturate at codes 0 and 2^bits - 1.  awq_search_clip produces such an array.
- * awq_quantize_pack(...) is awq_quantize_pack_ex(..., bits = 4, clip_ratio = NULL, ...).
- * Errors: as awq_quantize_pack; AWQ_ERR_BAD_ARGUMENT for other `bits`.
+ * awq_quantize_pack(...) is awq_quantize_pack_ex(..., bits = 4, symmetric = 0, clip_ratio = NULL, ...).
+ * awq_search_clip scores the asymmetric grid only; with symmetric = 1 a clip_ratio shrinks max|w'|.
+ * Errors: as awq_quantize_pack; AWQ_ERR_BAD_ARGUMENT for other `bits` or `symmetric`.
  */
 int awq_quantize_pack_ex(const void* W, const float* act_mean_abs, float alpha, int group, int bits,
-                         const float* clip_ratio, void* qweight, void* scales, void* zeros,
+                         int symmetric, const float* clip_ratio, void* qweight, void* scales, void* zeros,
                          int N, int K, void* stream);
 
 /*

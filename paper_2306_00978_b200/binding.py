@@ -53,7 +53,7 @@ def lib() -> ctypes.CDLL:
     L.awq_scales_bytes.restype, L.awq_scales_bytes.argtypes = sz, [i, i, i]
     L.awq_zeros_bytes.restype, L.awq_zeros_bytes.argtypes = sz, [i, i, i]
     L.awq_quantize_pack.restype, L.awq_quantize_pack.argtypes = i, [vp, vp, f, i, vp, vp, vp, i, i, vp]
-    L.awq_quantize_pack_ex.restype, L.awq_quantize_pack_ex.argtypes = i, [vp, vp, f, i, i, vp, vp, vp, vp, i, i, vp]
+    L.awq_quantize_pack_ex.restype, L.awq_quantize_pack_ex.argtypes = i, [vp, vp, f, i, i, i, vp, vp, vp, vp, i, i, vp]
     L.awq_search_clip.restype, L.awq_search_clip.argtypes = i, [vp, vp, f, i, i, vp, i, vp, i, i, vp]
     L.awq_channel_scale.restype, L.awq_channel_scale.argtypes = i, [vp, f, vp, i, vp]
     L.awq_linear.restype, L.awq_linear.argtypes = i, [vp, vp, vp, vp, vp, i, i, i, i, vp]
@@ -113,7 +113,7 @@ def channel_scale(act_mean_abs: Optional[torch.Tensor], alpha: float, K: int) ->
 
 
 def quantize_pack(W: torch.Tensor, act_mean_abs: Optional[torch.Tensor], alpha: float, group: int,
-                  clip_ratio: Optional[torch.Tensor] = None, bits: int = 4):
+                  clip_ratio: Optional[torch.Tensor] = None, bits: int = 4, symmetric: bool = False):
     """awq_quantize_pack / awq_quantize_pack_ex: returns (qweight u8 [N*K/2],
     scales fp16 [N/16][K/group][16], zeros u8 [N/32][K/group][16])."""
     N, K = W.shape
@@ -123,7 +123,7 @@ def quantize_pack(W: torch.Tensor, act_mean_abs: Optional[torch.Tensor], alpha: 
     scales = torch.empty((N // 16, K // group, 16), dtype=torch.float16, device=dev)
     zeros = torch.empty((N // 32, K // group, 16), dtype=torch.uint8, device=dev)
     a = 0 if act_mean_abs is None else _dev(act_mean_abs, torch.float32, "act_mean_abs")
-    if clip_ratio is None and bits == 4:
+    if clip_ratio is None and bits == 4 and not symmetric:
         rc = lib().awq_quantize_pack(_dev(W, torch.float16, "W"), a, float(alpha), int(group),
                                      qweight.data_ptr(), scales.data_ptr(), zeros.data_ptr(), N, K, _stream())
         _check(rc, "awq_quantize_pack")
@@ -133,7 +133,8 @@ def quantize_pack(W: torch.Tensor, act_mean_abs: Optional[torch.Tensor], alpha: 
         if tuple(clip_ratio.shape) != (N, K // group):
             raise AwqError(f"clip_ratio: expected shape {(N, K // group)}")
         c = _dev(clip_ratio, torch.float32, "clip_ratio")
-    rc = lib().awq_quantize_pack_ex(_dev(W, torch.float16, "W"), a, float(alpha), int(group), int(bits), c,
+    rc = lib().awq_quantize_pack_ex(_dev(W, torch.float16, "W"), a, float(alpha), int(group), int(bits),
+                                    int(bool(symmetric)), c,
                                     qweight.data_ptr(), scales.data_ptr(), zeros.data_ptr(), N, K, _stream())
     _check(rc, "awq_quantize_pack_ex")
     return qweight, scales, zeros

@@ -102,11 +102,11 @@ int awq_channel_scale(const float* act_mean_abs, float alpha, float* s, int K, v
 }
 
 int awq_quantize_pack_ex(const void* W, const float* act_mean_abs, float alpha, int group, int bits,
-                         const float* clip_ratio, void* qweight, void* scales, void* zeros,
+                         int symmetric, const float* clip_ratio, void* qweight, void* scales, void* zeros,
                          int N, int K, void* stream) {
     if (!(alpha >= 0.0f && alpha <= 1.0f)) return AWQ_ERR_BAD_ALPHA;
     if (int rc = check_shape(N, K, group)) return rc;
-    if (bits != 3 && bits != 4) return AWQ_ERR_BAD_ARGUMENT;
+    if ((bits != 3 && bits != 4) || (symmetric != 0 && symmetric != 1)) return AWQ_ERR_BAD_ARGUMENT;
     if (!W || !qweight || !scales || !zeros || (!act_mean_abs && alpha != 0.0f)) return AWQ_ERR_NULL_POINTER;
     if (!aligned16(W) || !aligned16(qweight) || !aligned16(scales) || !aligned16(zeros) ||
         (reinterpret_cast<uintptr_t>(act_mean_abs) & 3u) || (reinterpret_cast<uintptr_t>(clip_ratio) & 3u))
@@ -114,14 +114,14 @@ int awq_quantize_pack_ex(const void* W, const float* act_mean_abs, float alpha, 
     DeviceState* d;
     if (int rc = device_state(&d)) return rc;
     return note_cuda(launch_quantize_pack(reinterpret_cast<const __half*>(W), act_mean_abs, alpha, group, bits,
-                                          clip_ratio, reinterpret_cast<uint32_t*>(qweight),
+                                          symmetric != 0, clip_ratio, reinterpret_cast<uint32_t*>(qweight),
                                           reinterpret_cast<__half*>(scales),
                                           reinterpret_cast<uint8_t*>(zeros), N, K, (cudaStream_t)stream));
 }
 
 int awq_quantize_pack(const void* W, const float* act_mean_abs, float alpha, int group,
                       void* qweight, void* scales, void* zeros, int N, int K, void* stream) {
-    return awq_quantize_pack_ex(W, act_mean_abs, alpha, group, 4, nullptr, qweight, scales, zeros, N, K, stream);
+    return awq_quantize_pack_ex(W, act_mean_abs, alpha, group, 4, 0, nullptr, qweight, scales, zeros, N, K, stream);
 }
 
 int awq_search_clip(const void* W, const float* act_mean_abs, float alpha, int group, int bits,

@@ -29,7 +29,7 @@ void count_launch();
 cudaError_t launch_channel_scale(const float* a, float alpha, float* s, int K, cudaStream_t st);
 // bits: 4 or 3 (3-bit codes in the 4-bit fields); clip: optional per-group range ratios [N][K/group]
 cudaError_t launch_quantize_pack(const __half* W, const float* a, float alpha, int group, int bits,
-                                 const float* clip, uint32_t* qweight, __half* scales, uint8_t* zeros,
+                                 bool symmetric, const float* clip, uint32_t* qweight, __half* scales, uint8_t* zeros,
                                  int N, int K, cudaStream_t st);
 constexpr int kMaxClipRatios = 32;
 // ratios: HOST array of n_ratios <= kMaxClipRatios values; clip: device out, fp32 [N][K/group]

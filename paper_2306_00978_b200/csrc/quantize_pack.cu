@@ -80,7 +80,8 @@ __device__ __forceinline__ uint32_t pack4(float q0, float q1, float q2, float q3
 #ifndef AWQ_QP_BLOCKS
 #define AWQ_QP_BLOCKS 2
 #endif
-template <int G, int BITS, bool CLIP>
+// SYM: the symmetric grid of Eq. 2 (Delta = max|w'| / 2^(BITS-1), fixed zero point 2^(BITS-1))
+template <int G, int BITS, bool CLIP, bool SYM>
 __global__ void __launch_bounds__(256, AWQ_QP_BLOCKS)
 quantize_pack_kernel(const __half* __restrict__ W, const float* __restrict__ a, float alpha,
                      int mode, const float* __restrict__ clip,
@@ -183,7 +184,17 @@ quantize_pack_kernel(const __half* __restrict__ W, const float* __restrict__ a, 
         __half d16[2]; float d[2], z[2], rd[2], thr[2];
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
-            group_params(mn[ti][h], mx[ti][h], top, d16[h], d[h], z[h]);
+            if (SYM) {
+                constexpr float half_levels = (float)(1 << (BITS - 1));
+                const float d32 = __fdiv_rn(fmaxf(fabsf(mn[ti][h]), fabsf(mx[ti][h])), half_levels);
+                d16[h] = __float2half_rn(d32);
+                const unsigned short bits = __half_as_ushort(d16[h]);
+                if ((bits & 0x7FFFu) == 0u || (bits & 0x7C00u) == 0x7C00u) d16[h] = __ushort_as_half(0x3C00u);
+                d[h] = __half2float(d16[h]);
+                z[h] = half_levels;
+            } else {
+                group_params(mn[ti][h], mx[ti][h], top, d16[h], d[h], z[h]);
+            }
             rd[h] = __frcp_rn(d[h]);
             // |w * rd - w / d| <= 1.8e-7 |w / d| (three roundings); the group's largest |w / d|
             // bounds it for every element; quotients beyond 1024 always take the division
@@ -341,21 +352,26 @@ cudaError_t launch_channel_scale(const float* a, float alpha, float* s, int K, c
 }
 
 cudaError_t launch_quantize_pack(const __half* W, const float* a, float alpha, int group, int bits,
-                                 const float* clip, uint32_t* qweight, __half* scales, uint8_t* zeros,
+                                 bool symmetric, const float* clip, uint32_t* qweight, __half* scales, uint8_t* zeros,
                                  int N, int K, cudaStream_t st) {
     const dim3 grid(K / 128, N / 128);
     const int mode = (int)alpha_mode(alpha);
-#define AWQ_QP_LAUNCH(GG, BB, CC) \
-    quantize_pack_kernel<GG, BB, CC><<<grid, 256, 0, st>>>(W, a, alpha, mode, clip, qweight, scales, zeros, N, K)
+#define AWQ_QP_LAUNCH(GG, BB, CC, SS) \
+    quantize_pack_kernel<GG, BB, CC, SS><<<grid, 256, 0, st>>>(W, a, alpha, mode, clip, qweight, scales, zeros, N, K)
+#define AWQ_QP_PICK2(GG, SS)                                             \
+    do {                                                                 \
+        if (bits == 4 && !clip) AWQ_QP_LAUNCH(GG, 4, false, SS);         \
+        else if (bits == 4) AWQ_QP_LAUNCH(GG, 4, true, SS);              \
+        else if (!clip) AWQ_QP_LAUNCH(GG, 3, false, SS);                 \
+        else AWQ_QP_LAUNCH(GG, 3, true, SS);                             \
+    } while (0)
 #define AWQ_QP_PICK(GG)                                                  \
     do {                                                                 \
-        if (bits == 4 && !clip) AWQ_QP_LAUNCH(GG, 4, false);             \
-        else if (bits == 4) AWQ_QP_LAUNCH(GG, 4, true);                  \
-        else if (!clip) AWQ_QP_LAUNCH(GG, 3, false);                     \
-        else AWQ_QP_LAUNCH(GG, 3, true);                                 \
+        if (symmetric) AWQ_QP_PICK2(GG, true); else AWQ_QP_PICK2(GG, false); \
     } while (0)
     if (group == 128) AWQ_QP_PICK(128); else AWQ_QP_PICK(64);
 #undef AWQ_QP_PICK
+#undef AWQ_QP_PICK2
 #undef AWQ_QP_LAUNCH
     count_launch();
     return cudaGetLastError();

@@ -66,7 +66,8 @@ def test_argument_errors_need_no_gpu(lib):
     assert lib.awq_search_clip(one, one, 0.5, 128, 4, ctypes.cast(bad, ctypes.c_void_p), 2, one, 128, 128, None) == 10
     assert lib.awq_search_clip(one, one, 0.5, 128, 5, ctypes.cast(ok, ctypes.c_void_p), 2, one, 128, 128, None) == 10
     assert lib.awq_search_clip(one, one, 0.5, 128, 4, ctypes.cast(ok, ctypes.c_void_p), 33, one, 128, 128, None) == 10
-    assert lib.awq_quantize_pack_ex(one, one, 0.5, 128, 2, None, one, one, one, 128, 128, None) == 10
+    assert lib.awq_quantize_pack_ex(one, one, 0.5, 128, 2, 0, None, one, one, one, 128, 128, None) == 10
+    assert lib.awq_quantize_pack_ex(one, one, 0.5, 128, 4, 2, None, one, one, one, 128, 128, None) == 10
     assert lib.awq_linear_path(one, one, one, one, one, 1, 128, 128, 128, 7, None) == 10
     assert lib.awq_linear_path(one, one, one, one, one, 17, 128, 128, 128, 3, None) == 2
     assert b"group" in lib.awq_status_string(3)

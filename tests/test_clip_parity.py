@@ -90,3 +90,31 @@ def test_clipping_lowers_the_layer_error_on_weights_with_outliers():
         y = binding.linear(xd, *packed, N, K, G).cpu().numpy().astype(np.float64)
         errs.append(float(((y - y_ref) ** 2).mean()))
     assert errs[1] < 0.9 * errs[0]
+
+
+@pytest.mark.parametrize("N,K,G,bits,clipped", [(256, 512, 128, 4, False), (384, 640, 64, 4, True),
+                                               (1024, 4096, 128, 3, False), (4096, 4096, 128, 4, False)])
+def test_symmetric_quantizer_bit_exact_and_layer_parity(N, K, G, bits, clipped):
+    """The symmetric grid of Eq. 2 (zero point fixed at 2^(bits-1)): packed arrays bit-identical to
+    the oracle, with and without clipping ratios; the layer kernels on them within tolerance."""
+    from paper_2306_00978_b200 import binding
+    seed = 1300 + N + K + bits
+    W, a = _inputs(seed, N, K)
+    clip = None
+    if clipped:
+        rng = np.random.default_rng(seed)
+        clip = rng.choice(np.asarray(RATIOS, dtype=np.float32), size=(N, K // G)).astype(np.float32)
+    got = binding.quantize_pack(to_cuda(W), to_cuda(a), 0.5, G, bits=bits, symmetric=True,
+                                clip_ratio=None if clip is None else to_cuda(clip))
+    want = orc.quantize_pack(W, a, 0.5, G, clip=clip, bits=bits, symmetric=True)
+    _packed_equal(got, want)
+    if N <= 1024:
+        s = orc.channel_scale(a, 0.5)
+        codes, zeros, scales = orc.quantize(W, s, G, clip=clip, bits=bits, symmetric=True)
+        assert (zeros == (1 << (bits - 1))).all()
+        Wdq = orc.dequantize(codes, zeros, scales, G)
+        for M in (2, 33):
+            x = (synth.activations(seed, M, K).astype(np.float32) / s[None, :]).astype(np.float16)
+            y = binding.linear(to_cuda(x), *got, N, K, G)
+            binding.poll_status()
+            assert_parity(y.cpu().numpy(), orc.linear(x, Wdq), f"symmetric N={N} K={K} M={M}")
