@@ -374,21 +374,23 @@ def clip_section():
 
 
 # ------------------------------------------------------------------- oracle (CPU) arm
-def _oracle_layer_inputs(max_rows=None):
+def _oracle_layer_inputs(max_rows=None, col_div=1):
     """Quantizes one decoder layer's matrices with the oracle; optionally only the first
-    `max_rows` output rows of each (whole 128-row slabs), to bound the work."""
+    `max_rows` output rows (whole 128-row slabs) and the first K / col_div input channels (whole
+    128-column blocks) of each, to bound the work."""
     from oracle import awq_oracle as orc
     items = []
     for idx, (name, K, N) in enumerate(synth.LLAMA2_7B_LAYER):
         seed = 2000 + idx
         n = N if max_rows is None else min(N, max_rows)
-        W = synth.weight(seed, N, K)[:n]
-        a = synth.act_mean_abs(seed, K)
+        kc = max(128, (K // col_div) // 128 * 128)
+        W = np.ascontiguousarray(synth.weight(seed, N, K)[:n, :kc])
+        a = synth.act_mean_abs(seed, K)[:kc]
         s = orc.channel_scale(a, ALPHA)
-        x = synth.activations(seed, 1, K)
+        x = synth.activations(seed, 1, K)[:, :kc]
         xs = (x.astype(np.float32) / s[None, :]).astype(np.float16)
         qw, sc, zp = orc.quantize_pack(W, a, ALPHA, GROUP)
-        items.append((n, K, xs, qw, sc, zp))
+        items.append((n, kc, xs, qw, sc, zp))
     return items
 
 
@@ -426,13 +428,17 @@ def reference_arm(args):
     if rank != 0:
         return 0
     steps, warmup = max(1, args.steps), max(0, args.warmup)
-    # size the per-step sample so that the whole run stays within a few minutes
+    # size the per-step sample so that the whole run stays within a few minutes: rows first (down
+    # to one 128-row slab of each matrix), then input channels; about 50 ns per weight on 8 cores
     budget = 150.0 / (steps + warmup)
-    rows = 1024
-    per_row_s = 12 * 1.7 / 4096           # about 1.7 s per 4096x4096 matrix on 8 cores
-    while rows > 128 and rows * per_row_s > budget:
+    rows, col_div = 1024, 1
+    weights_per_row = sum(K for (_name, K, _N) in synth.LLAMA2_7B_LAYER)
+    cost = lambda r, c: r * weights_per_row / c * 50e-9
+    while rows > 128 and cost(rows, col_div) > budget:
         rows //= 2
-    items = _oracle_layer_inputs(max_rows=rows)
+    while col_div < 32 and cost(rows, col_div) > budget:
+        col_div *= 2
+    items = _oracle_layer_inputs(max_rows=rows, col_div=col_div)
     nbytes = sum(algorithmic_bytes(n, K, 1) for (n, K, *_rest) in items)
     for _ in range(warmup):
         _oracle_step(items)
@@ -446,13 +452,13 @@ def reference_arm(args):
     except Exception:
         cores = os.cpu_count() or 1
     value = nbytes / sec / 1e9
-    sample = (f"each step = first {rows} output rows of each of the 7 linears of one layer at M=1 "
-              f"through the CPU oracle")
+    sample = (f"each step = first {rows} output rows" + (f" x first 1/{col_div} of the input channels" if col_div > 1 else "") +
+              " of each of the 7 linears of one layer at M=1 through the CPU oracle")
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
             "steps": steps, "warmup": warmup, "ms_per_step": sec * 1e3, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
             "config": {"workload": "llama2-7b decoder-layer linears, M=1, g128, alpha=0.5 (bounded sample)",
-                       "rows_per_linear": rows},
+                       "rows_per_linear": rows, "input_channel_fraction": 1.0 / col_div},
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": int(cores), "kind": "oracle",
                              "sample": sample},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
