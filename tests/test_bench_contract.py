@@ -1,0 +1,47 @@
+"""The output contract of bench.py: one JSON line with the agreed keys.  The reference arm (the CPU
+oracle on a bounded sample) runs anywhere; the GPU arm is checked on a short run."""
+import json
+import os
+import subprocess
+import sys
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+BASE_KEYS = {"metric", "value", "unit", "n_gpus", "steps", "warmup", "ms_per_step", "higher_is_better",
+             "scaling", "vs_baseline", "dtype", "data", "config", "e2e", "gpu_launches", "cpu_baseline"}
+
+
+def _run(args, timeout):
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), *args], capture_output=True,
+                         text=True, timeout=timeout, cwd=ROOT)
+    assert out.returncode == 0, out.stderr[-2000:]
+    lines = [l for l in out.stdout.splitlines() if l.strip()]
+    assert len(lines) == 1, lines
+    return json.loads(lines[0])
+
+
+def test_reference_arm_line():
+    d = _run(["--impl", "reference", "--steps", "3", "--warmup", "1"], 600)
+    assert BASE_KEYS <= set(d) and d["impl"] == "reference"
+    assert d["steps"] == 3 and d["warmup"] == 1 and d["n_gpus"] == 1
+    assert d["value"] > 0 and d["unit"] == "GB/s" and d["higher_is_better"] is True
+    assert d["cpu_baseline"]["kind"] == "oracle" and d["cpu_baseline"]["value"] == d["value"]
+    assert d["e2e"] == {"value": d["value"], "unit": d["unit"], "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}
+    assert d["config"]["workload"].startswith("llama2-7b")
+
+
+@pytest.mark.gpu
+def test_gpu_arm_line():
+    d = _run(["--steps", "40", "--warmup", "5", "--layers", "2"], 900)
+    assert BASE_KEYS | {"roofline", "clocks"} <= set(d)
+    assert d["steps"] == 40 and d["warmup"] == 5 and d["n_gpus"] == 1 and d["scaling"] == "weak"
+    assert d["gpu_launches"] == 4 * 40
+    r = d["roofline"]
+    assert r["bound"] == "hbm" and r["unit"] == "GB/s" and abs(r["frac"] - r["achieved"] / r["peak"]) < 1e-9
+    assert 0.9 < r["traffic"] / r["algorithmic_bytes_per_launch"] < 1.1
+    assert d["e2e"]["h2d_bytes_per_step"] == 46592 and d["e2e"]["d2h_bytes_per_step"] == 84992
+    assert 0 < d["e2e"]["value"] < d["value"]
+    assert d["cpu_baseline"]["kind"] == "oracle" and d["cpu_baseline"]["cores"] >= 1
+    assert d["config"]["workload"].startswith("llama2-7b") and "model" not in d["config"]
+    assert set(d["clocks"]) >= {"sm_mhz", "sm_max_mhz", "reasons"}
