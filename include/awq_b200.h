@@ -22,12 +22,17 @@
  * band - is contiguous along K)
  *  qweight: N*K/2 bytes.  Block (band, kt) = rows 16*band..+15, columns 64*kt..+63 is 512
  *    bytes at ((n/16)*(K/64) + k/64) * 512.  A block is 32 pieces of 16 bytes, piece index
- *    4*g + t (g = 0..7, t = 0..3) holding rows g and g+8 of the band and columns 16t..16t+15 of
- *    the block.  32-bit word j of a piece holds columns c = 16t+4j .. +3 of both rows as eight
- *    4-bit slots
+ *    4*g + t (g = 0..7, t = 0..3) holding rows g and g+8 of the band.  32-bit word j (j = 0..3,
+ *    little-endian, at byte 4j of the piece) holds columns c = 16j+4t .. +3 of the block for
+ *    both rows - so the four pieces of a row pair interleave along K in runs of four columns,
+ *    and word j of all four pieces together covers columns 16j..16j+15 - as eight 4-bit slots
  *      (g,c) (g,c+1) (g+8,c) (g+8,c+1) (g,c+2) (g,c+3) (g+8,c+2) (g+8,c+3),
  *    slot e stored at bits 4p..4p+3 with p = {0,4,1,5,2,6,3,7}[e]  (read from the low
  *    nibble up, the slots appear in the order 0,2,4,6,1,3,5,7 - the GPU order of Sec. 4.2).
+ *    As one formula: code (n,k) sits in the byte at
+ *      ((n/16)*(K/64) + k/64)*512 + 16*(4*(n%8) + (k%16)/4) + 4*((k%64)/16) + {0,2,1,3}[k%4],
+ *    in its low nibble if n%16 < 8, else in its high nibble: every byte holds the codes of rows
+ *    g and g+8 of one column.
  *  scales: fp16 [N/16][K/group][16] (band, group, row in band).
  *  zeros:  bytes [N/32][K/group][16]: per pair of bands and group, bytes 0-7 belong to the even
  *    band, 8-15 to the odd one; byte n%8 of a band holds the zero point of row n (n%16 < 8)
@@ -117,8 +122,8 @@ int awq_quantize_pack_ex(const void* W, const float* act_mean_abs, float alpha, 
                          int N, int K, void* stream);
 
 /*
- * Weight clipping (Sec. 3.2: "weight clipping to minimize the MSE error of quantization"; the
- * paper gives no algorithm, this is the reading used).  For every group of w' = fp32(W) * s and
+ * Weight clipping (Sec. 3.2 names it in one sentence - clipping chosen to minimise the squared
+ * quantization error - and gives no algorithm; this is the reading used).  For every group of w' = fp32(W) * s and
  * every ratio r_i of `ratios`, the group is quantized as awq_quantize_pack_ex would with
  * clip_ratio = r_i, and
  *   err_i = sum over k ascending of ((q_k - z) * Delta - w'_k)^2

@@ -13,8 +13,8 @@ What is computed, and where it comes from
 * quantize           w' = w * s folded into the weight (Eq. 3, Eq. 4), then the
                      group-wise round-to-nearest grid Delta * Round(w'/Delta)   (Eq. 2),
                      in the asymmetric min/max form with an integer zero point in
-                     [0, 15] and Delta stored in fp16 (Sec. 3.2: "Delta and x are
-                     represented in FP16").
+                     [0, 15] and Delta stored in fp16 (Sec. 3.2 keeps Delta and the
+                     activations in half precision).
 * search_clip        weight clipping (Sec. 3.2): per group, the range ratio of a given list that
                      minimizes the squared quantization error of the group.
 * pack_* / unpack_*  eight 4-bit codes per 32-bit word in the order
@@ -38,8 +38,8 @@ group's raw min and max are used (the range is not widened to contain 0); a dege
 group (Delta rounds to 0 or is not finite) takes Delta = 1.  w * s stays in fp32.
 The search's norm is not named in the paper: the mean of the squared differences is used (any
 monotone function of the Frobenius norm has the same minimizer); diag(s)^-1 X is rounded to fp16
-once, because that is what the layer is given; the grid of alpha is an argument (the paper says
-"a grid size of 20" over [0, 1] without saying whether 1 is a grid point).
+once, because that is what the layer is given; the grid of alpha is an argument (Sec. 3.2 searches
+20 grid points over [0, 1] and does not say whether 1 is one of them).
 Weight clipping is one sentence in the paper (the appendix it may have been detailed in is not
 part of the text): the reading here shrinks a group's [min, max] by a common ratio taken from a
 caller-given list, measures the error in the scaled weight space w' = w * s (the tensor that is

@@ -196,6 +196,62 @@ def test_pack_matches_location_formula_and_round_trips():
     assert orc.qweight_location(16, 0, 192)[0] == 3 * 128
 
 
+def _layout_table(golden_dir):
+    rows = {"qweight": [], "zeros": [], "scales": []}
+    with open(os.path.join(golden_dir, "packed_layout.txt")) as f:
+        for line in f:
+            line = line.strip()
+            if not line or line.startswith("#"):
+                continue
+            kind, *vals = line.split()
+            rows[kind].append(tuple(int(v) for v in vals))
+    return rows
+
+
+def test_packed_layout_against_hand_derived_table(golden_dir):
+    """The layout is a free choice, so what pins it is its written definition: the table was worked
+    out by hand from the prose of the public header, entry by entry, and covers every index of the
+    formula (row in band, upper / lower row, column inside a word, word in piece, piece in block,
+    block along K, band): a swapped pair of indices or a wrong nibble table fails here."""
+    t = _layout_table(golden_dir)
+    assert len(t["qweight"]) >= 12
+    nib_seen = set()
+    for (n, k, K, byte, half) in t["qweight"]:
+        wi, p = orc.qweight_location(n, k, K)
+        assert (4 * wi + p // 2, p % 2) == (byte, half), (n, k)
+        nib_seen.add(p)
+        # the same through the array routine: a single non-zero code lands in that nibble only
+        N = 16 * (n // 16 + 1)
+        N += (-N) % 16
+        codes = np.zeros((N, K), np.uint8)
+        codes[n, k] = 0xF
+        raw = orc.pack_qweight(codes).astype("<u4").view(np.uint8)
+        want = np.zeros_like(raw)
+        want[byte] = 0xF0 if half else 0x0F
+        assert np.array_equal(raw, want), (n, k)
+        # and the closed form printed in the header
+        closed = ((n // 16) * (K // 64) + k // 64) * 512 + 16 * (4 * (n % 8) + (k % 16) // 4) \
+            + 4 * ((k % 64) // 16) + (0, 2, 1, 3)[k % 4]
+        assert closed == byte and (n % 16 >= 8) == bool(half)
+    assert nib_seen == set(range(8))                     # every entry of the nibble table is exercised
+    for (n, gi, ng, byte, half) in t["zeros"]:
+        assert orc.zeros_location(n, gi, ng) == (byte, half), (n, gi)
+        N = 32 * (n // 32 + 1)
+        z = np.zeros((N, ng), np.uint8)
+        z[n, gi] = 0xF
+        raw = orc.pack_zeros(z).reshape(-1)
+        want = np.zeros_like(raw)
+        want[byte] = 0xF0 if half else 0x0F
+        assert np.array_equal(raw, want), (n, gi)
+    for (n, gi, ng, idx) in t["scales"]:
+        assert orc.scales_location(n, gi, ng) == idx, (n, gi)
+        N = 16 * (n // 16 + 1)
+        sc = np.zeros((N, ng), np.float16)
+        sc[n, gi] = 1.0
+        raw = orc.pack_scales(sc).reshape(-1)
+        assert raw[idx] == 1.0 and np.count_nonzero(raw) == 1, (n, gi)
+
+
 def test_zero_and_scale_packing():
     rng = np.random.default_rng(5)
     N, ng = 256, 3
