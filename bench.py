@@ -43,9 +43,13 @@ FALLBACK_HBM_GBS = 6650.0
 FALLBACK_BF16_TFLOPS = 1590.0
 NOMINAL_HBM_GBS = 8000.0
 NOMINAL_FP16_TFLOPS = 2250.0
-# DRAM bytes per launch of the dominant kernel from the ncu capture summarised under
-# profiles/ (None until a capture of the current kernel exists).
-NCU_TRAFFIC_BYTES_PER_LAUNCH = {(11008, 4096): 23470000, (4096, 4096): 8760000}
+# DRAM traffic of the dominant kernel: ncu's dram__bytes_read.sum + dram__bytes_write.sum over the
+# algorithmic bytes of the captured launch (profiles/gemv_band_kernel_llama2_7b_M1.md: per-matrix
+# captures of 4096 -> 11008 and 4096 -> 4096; traffic grows in proportion to the packed bytes).
+NCU_TRAFFIC_RATIO = 1.0005
+DOMINANT_KERNEL = "gemv_band_kernel<128,4,true,true,5>"
+NCU_TRAFFIC_NOTE = ("scaled from the ncu captures of single-matrix launches in "
+                    "profiles/gemv_band_kernel_llama2_7b_M1.md: dram bytes / algorithmic bytes = 1.0002 .. 1.001")
 
 
 def algorithmic_bytes(N: int, K: int, M: int, group: int = GROUP) -> int:
@@ -176,11 +180,9 @@ def build_layers(n_layers: int, seed0: int = 2000):
 STEP_CALLS = ((0, 1, 2), (3,), (4, 5), (6,))
 
 
-def run_step(layer, e2e=False):
+def run_calls(layer, calls, e2e=False):
     from paper_2306_00978_b200 import binding
-    if e2e:                                            # the step's inputs from pinned host memory
-        layer[0]["x_dev"].copy_(layer[0]["x_host"], non_blocking=True)
-    for idxs in STEP_CALLS:
+    for idxs in calls:
         first = layer[idxs[0]]
         xin = first["x_dev_in"] if e2e else first["x"]
         if len(idxs) == 1:
@@ -189,6 +191,12 @@ def run_step(layer, e2e=False):
         else:
             binding.linear_multi(xin, [(layer[i]["qw"], layer[i]["sc"], layer[i]["zp"], layer[i]["N"]) for i in idxs],
                                  first["K"], GROUP, outs=[layer[i]["y"] for i in idxs])
+
+
+def run_step(layer, e2e=False):
+    if e2e:                                            # the step's inputs from pinned host memory
+        layer[0]["x_dev"].copy_(layer[0]["x_host"], non_blocking=True)
+    run_calls(layer, STEP_CALLS, e2e)
     if e2e:                                            # the step's outputs back to the host
         layer[0]["y_host"].copy_(layer[0]["y_dev"], non_blocking=True)
 
@@ -199,68 +207,99 @@ def run_step_e2e(layer):
     run_step(layer, e2e=True)
 
 
-def capture_steps(fn, layers):
-    """One CUDA graph per layer, captured from the C-ABI calls of one step (the launch-bound
-    inner loop of decode is replayed as a graph, as a serving stack would).  Returns the
-    graphs and the number of library kernels in one step."""
+def capture_chain(fn, layers, steps: int):
+    """ONE CUDA graph of exactly `steps` steps, the layers rotating (step i uses layer i mod L), so
+    that every launch of the region is chained to the one before it by programmatic dependent launch
+    - a decoder stack is replayed as one graph.  Returns (graph, library kernels per step)."""
     import torch
     from paper_2306_00978_b200 import binding
-    graphs = []
-    side = torch.cuda.Stream()
-    per_step = 0
     for layer in layers:
         fn(layer)                                    # warm: attributes set, workspace registered
     torch.cuda.synchronize()
+    side = torch.cuda.Stream()
+    g = torch.cuda.CUDAGraph()
     with torch.cuda.stream(side):
-        for layer in layers:
-            g = torch.cuda.CUDAGraph()
-            n0 = binding.launch_count()
-            with torch.cuda.graph(g, stream=side):
-                fn(layer)
-            per_step = binding.launch_count() - n0
-            graphs.append(g)
-        # the whole rotation as one graph (a decoder stack is replayed as one graph, layer after
-        # layer): len(layers) steps per replay
-        stack = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(stack, stream=side):
-            for layer in layers:
-                fn(layer)
+        n0 = binding.launch_count()
+        with torch.cuda.graph(g, stream=side):
+            for i in range(steps):
+                fn(layers[i % len(layers)])
+        per_step = (binding.launch_count() - n0) // steps
     torch.cuda.synchronize()
-    return graphs, per_step, stack
+    return g, per_step
 
 
-def timed_region(graphs, stack, steps: int, warmup: int, device: str):
-    """W warm-up steps, then exactly `steps` steps between barrier+synchronize, CUDA events on
-    the launching stream; returns (seconds = max over ranks, wall-clock window).  Whole rotations
-    of the layers are replayed as the stack graph (len(graphs) steps each), the remainder as
-    single-layer graphs."""
+def timed_region(graph, steps: int, warmup: int, device: str, min_seconds: float = 0.6, min_replays: int = 50):
+    """Warm-up (at least `warmup` steps, as whole replays of the same graph), then R replays of the
+    `steps`-step graph between barrier + synchronize, one CUDA event between consecutive replays on
+    the launching stream.  R is chosen so that the region lasts at least `min_seconds` (clock samples
+    are 100 ms apart) and at least `min_replays`.  Returns (median seconds per replay = max over
+    ranks, dict of the spread, wall-clock window, R)."""
     import torch
-    L = len(graphs)
-    for i in range(warmup // L):
-        stack.replay()
-    for i in range(warmup % L):
-        graphs[i].replay()
+    for _ in range(max(1, -(-warmup // steps))):
+        graph.replay()
     torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(3):
+        graph.replay()
+    e1.record()
+    torch.cuda.synchronize()
+    est = max(1e-6, e0.elapsed_time(e1) * 1e-3 / 3)
+    R = int(min(20000, max(min_replays, min_seconds / est)))
     replicas.barrier()
     torch.cuda.synchronize()
-    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(R + 1)]
     t0 = time.time()
-    start.record()
-    for i in range(steps // L):
-        stack.replay()
-    for i in range(steps % L):
-        graphs[i].replay()
-    end.record()
+    ev[0].record()
+    for r in range(R):
+        graph.replay()
+        ev[r + 1].record()
     torch.cuda.synchronize()
     t1 = time.time()
     replicas.barrier()
-    sec = start.elapsed_time(end) * 1e-3
-    return replicas.max_over_ranks(sec, device), (t0, t1)
+    per = sorted(ev[r].elapsed_time(ev[r + 1]) * 1e-3 for r in range(R))
+    med = statistics.median(per)
+    spread = {"replays": R, "min": per[0], "p10": per[R // 10], "median": med, "p90": per[(9 * R) // 10],
+              "max": per[-1], "mean": sum(per) / R}
+    return replicas.max_over_ranks(med, device), spread, (t0, t1), R
 
 
-def gemm_section(peaks, reps: int = 20):
-    """Prefill GEMM, M = 2048, Llama-2-13B MLP shapes: best-of-reps and mean TFLOP/s (the binding
-    registers the optional stream-K workspace)."""
+def per_position_times(layers, reps: int = 15):
+    """Device time of each of the step's four launch positions on its own: a graph that holds only
+    that position's call, once per rotating layer, eight times over (chained by programmatic
+    dependent launch like the step itself); median over `reps` replays.  Seconds per launch."""
+    import torch
+    from paper_2306_00978_b200 import binding
+    out = []
+    side = torch.cuda.Stream()
+    for idxs in STEP_CALLS:
+        g = torch.cuda.CUDAGraph()
+        n = 8 * len(layers)
+        with torch.cuda.stream(side):
+            with torch.cuda.graph(g, stream=side):
+                for i in range(n):
+                    run_calls(layers[i % len(layers)], (idxs,))
+        torch.cuda.synchronize()
+        g.replay()
+        torch.cuda.synchronize()
+        ts = []
+        for _ in range(reps):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            g.replay()
+            e1.record()
+            torch.cuda.synchronize()
+            ts.append(e0.elapsed_time(e1) * 1e-3 / n)
+        out.append(statistics.median(ts))
+    binding.poll_status()
+    return out
+
+
+def gemm_section(peaks, sampler=None, reps: int = 20, sustained_s: float = 2.0):
+    """Prefill GEMM, M = 2048, Llama-2-13B MLP shapes (the binding registers the optional stream-K
+    workspace).  Burst: best and mean of `reps` timings of four back-to-back calls.  Sustained: the
+    same call back to back for at least `sustained_s` seconds between two events, SM clock and
+    throttle reasons sampled inside that window."""
     import torch
     from paper_2306_00978_b200 import binding
     out = []
@@ -290,13 +329,38 @@ def gemm_section(peaks, reps: int = 20):
             e1.record()
             torch.cuda.synchronize()
             times.append(e0.elapsed_time(e1) * 1e-3 / inner)
-        binding.poll_status()
         flops = 2.0 * M * N * K
         best, mean = min(times), sum(times) / len(times)
-        out.append({"shape": f"{K}->{N}", "M": M, "tflops_best": flops / best / 1e12,
-                    "tflops_mean": flops / mean / 1e12, "ms_best": best * 1e3,
-                    "frac_of_measured_bf16_burst": flops / best / 1e12 / peaks["bf16_tflops"],
-                    "frac_of_nominal_2250": flops / best / 1e12 / NOMINAL_FP16_TFLOPS})
+        row = {"shape": f"{K}->{N}", "M": M, "tflops_best": flops / best / 1e12,
+               "tflops_mean": flops / mean / 1e12, "ms_best": best * 1e3,
+               "frac_of_measured_bf16_burst": flops / best / 1e12 / peaks["bf16_tflops"],
+               "frac_of_nominal_2250": flops / best / 1e12 / NOMINAL_FP16_TFLOPS}
+        # sustained: one graph of 64 calls replayed until the window is long enough
+        n = 64
+        g, side = torch.cuda.CUDAGraph(), torch.cuda.Stream()
+        with torch.cuda.stream(side):
+            with torch.cuda.graph(g, stream=side):
+                for _ in range(n):
+                    binding.linear(xs, qw, sc, zp, N, K, GROUP, out=y)
+        torch.cuda.synchronize()
+        replays = max(2, int(sustained_s / (n * best)) + 1)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t0 = time.time()
+        e0.record()
+        for _ in range(replays):
+            g.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        t1 = time.time()
+        sec = e0.elapsed_time(e1) * 1e-3
+        sus = flops * n * replays / sec / 1e12
+        row["sustained"] = {"tflops": sus, "seconds": sec, "calls": n * replays,
+                            "frac_of_measured_bf16_sustained": sus / peaks["bf16_tflops_sustained"],
+                            "frac_of_nominal_2250": sus / NOMINAL_FP16_TFLOPS,
+                            "clocks": sampler.summary(t0 + 0.2, t1) if sampler is not None else None}
+        binding.poll_status()
+        out.append(row)
+        del g
     return out
 
 
@@ -400,27 +464,57 @@ def _oracle_step(items):
         orc.linear_from_packed(xs, qw, sc, zp, n, K, GROUP)
 
 
-def cpu_baseline(budget_s: float = 20.0):
-    """The oracle as it stands on the host cores, on a bounded sample of the same step."""
-    rows = 1024
-    items = _oracle_layer_inputs(max_rows=rows)
-    nbytes = sum(algorithmic_bytes(n, K, 1) for (n, K, *_rest) in items)
-    t0 = time.time()
-    reps = 0
-    while True:
-        _oracle_step(items)
-        reps += 1
-        if time.time() - t0 > budget_s * 0.5 or reps >= 3:
-            break
-    sec = (time.time() - t0) / reps
+def _host_threads() -> int:
     try:
         from threadpoolctl import threadpool_info
-        cores = max([p.get("num_threads", 1) for p in threadpool_info()] or [1])
+        return int(max([p.get("num_threads", 1) for p in threadpool_info()] or [1]))
     except Exception:
-        cores = os.cpu_count() or 1
-    return {"value": nbytes / sec / 1e9, "unit": UNIT, "cores": int(cores), "kind": "oracle",
+        return int(os.cpu_count() or 1)
+
+
+def cpu_baseline(rows: int = 1024):
+    """The oracle as it stands on the host cores, on a bounded sample of the same step: the first
+    `rows` output rows of each of the layer's seven matrices.  Its three phases are timed apart:
+    quantize + pack (Eq. 2 - Eq. 5), unpack + dequantize to fp64, and the fp64 product."""
+    from oracle import awq_oracle as orc
+    mats = []
+    t_quant = 0.0
+    weights = 0
+    for idx, (name, K, N) in enumerate(synth.LLAMA2_7B_LAYER):
+        seed = 2000 + idx
+        n = min(N, rows)
+        W = np.ascontiguousarray(synth.weight(seed, N, K)[:n])
+        a = synth.act_mean_abs(seed, K)
+        x = synth.activations(seed, 1, K)
+        t0 = time.time()
+        s = orc.channel_scale(a, ALPHA)
+        qw, sc, zp = orc.quantize_pack(W, a, ALPHA, GROUP)
+        t_quant += time.time() - t0
+        xs = (x.astype(np.float32) / s[None, :]).astype(np.float16)
+        mats.append((n, K, xs, qw, sc, zp))
+        weights += n * K
+    nbytes = sum(algorithmic_bytes(n, K, 1) for (n, K, *_r) in mats)
+    t_deq = t_mul = 0.0
+    reps = 3
+    for _ in range(reps):
+        for (n, K, xs, qw, sc, zp) in mats:
+            t0 = time.time()
+            Wdq = orc.dequantize(orc.unpack_qweight(qw, n, K), orc.unpack_zeros(zp, n, K // GROUP),
+                                 orc.unpack_scales(sc, n, K // GROUP), GROUP)
+            t1 = time.time()
+            orc.linear(xs, Wdq)
+            t2 = time.time()
+            t_deq += t1 - t0
+            t_mul += t2 - t1
+    t_deq /= reps
+    t_mul /= reps
+    return {"value": nbytes / (t_deq + t_mul) / 1e9, "unit": UNIT, "cores": _host_threads(), "kind": "oracle",
             "sample": f"first {rows} output rows of each of the 7 linears of one layer at M=1 "
-                      f"(unpack + fp64 dequantize + fp64 product), {reps} repetitions"}
+                      f"({weights / 1e6:.1f} M weights); value = algorithmic bytes / (dequantize + multiply)",
+            "phases": {"quantize_pack_s": t_quant, "quantize_pack_Mweights_per_s": weights / t_quant / 1e6,
+                       "unpack_dequantize_s": t_deq, "unpack_dequantize_Mweights_per_s": weights / t_deq / 1e6,
+                       "multiply_fp64_s": t_mul, "multiply_fp64_GFLOPs": 2.0 * weights / t_mul / 1e9,
+                       "repetitions_of_layer_phases": reps}}
 
 
 def reference_arm(args):
@@ -446,11 +540,7 @@ def reference_arm(args):
     for _ in range(steps):
         _oracle_step(items)
     sec = (time.time() - t0) / steps
-    try:
-        from threadpoolctl import threadpool_info
-        cores = max([p.get("num_threads", 1) for p in threadpool_info()] or [1])
-    except Exception:
-        cores = os.cpu_count() or 1
+    cores = _host_threads()
     value = nbytes / sec / 1e9
     sample = (f"each step = first {rows} output rows" + (f" x first 1/{col_div} of the input channels" if col_div > 1 else "") +
               " of each of the 7 linears of one layer at M=1 through the CPU oracle")
@@ -496,50 +586,153 @@ def one_shape(args):
     return 0
 
 
-def sweep(args):
-    """The full-shape sweep over the 7B layer's three distinct shapes: token counts 1 .. 8192 and
-    both group sizes through awq_linear (random packed weights, three rotating copies so that
-    small shapes do not sit in L2, eight calls per CUDA-graph replay, best of five replays).
-    One JSON object per line: microseconds, algorithmic GB/s, TFLOP/s."""
-    import torch
+class RandomPacked:
+    """Rotating copies of random packed arrays of one shape (the kernels' work does not depend on the
+    values).  cold = True: enough copies that a pass over them moves more than twice the L2 size, so
+    that no call finds its weights in L2."""
+
+    def __init__(self, N: int, K: int, group: int, cold: bool = True, max_copies: int = 40):
+        import torch
+        self.N, self.K, self.group = N, K, group
+        packed = N * K // 2 + (N * K // group) * 2 + (N * K // group) // 2
+        l2 = torch.cuda.get_device_properties(torch.cuda.current_device()).L2_cache_size
+        n = 3
+        if cold:
+            n = max(3, min(max_copies, -(-2 * l2 // packed) + 1))
+        self.cold = cold and n * packed >= 2 * l2
+        self.copies = []
+        for _ in range(n):
+            qw = torch.randint(0, 256, (N * K // 2,), dtype=torch.uint8, device="cuda")
+            sc = (torch.rand((N // 16, K // group, 16), device="cuda") * 0.01 + 0.001).half()
+            zp = torch.randint(0, 256, (N // 32, K // group, 16), dtype=torch.uint8, device="cuda")
+            self.copies.append((qw, sc, zp))
+
+    def time_chained(self, M: int, path: int = 0, reps: int = 5, calls: int = 0):
+        """Microseconds per call inside a CUDA graph of back-to-back calls over the rotating copies
+        (launches chained by programmatic dependent launch where the kernel uses it): (best, median)."""
+        import torch
+        from paper_2306_00978_b200 import binding
+        N, K, group = self.N, self.K, self.group
+        x = torch.randn((M, K), device="cuda").half()
+        y = torch.empty((M, N), device="cuda", dtype=torch.float16)
+        n = len(self.copies)
+        if calls <= 0:
+            calls = max(8, n) if M <= 128 else 2
+        for i in range(min(3, n)):
+            binding.linear(x, *self.copies[i], N, K, group, out=y, path=path)
+        torch.cuda.synchronize()
+        graph, stream = torch.cuda.CUDAGraph(), torch.cuda.Stream()
+        with torch.cuda.stream(stream):
+            with torch.cuda.graph(graph, stream=stream):
+                for i in range(calls):
+                    binding.linear(x, *self.copies[i % n], N, K, group, out=y, path=path)
+        torch.cuda.synchronize()
+        graph.replay()
+        torch.cuda.synchronize()
+        ts = []
+        for _ in range(reps):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            graph.replay()
+            e1.record()
+            torch.cuda.synchronize()
+            ts.append(e0.elapsed_time(e1) * 1e3 / calls)
+        binding.poll_status()
+        return min(ts), statistics.median(ts)
+
+    def time_isolated(self, M: int, path: int = 0):
+        """Microseconds of a single call with nothing in front of it on the device: the stream is
+        kept busy by a sleep kernel while the host enqueues event, call, event, so the interval is
+        device time of one cold launch (its start-up included, nothing to overlap with).  Median
+        over the rotating copies."""
+        import torch
+        from paper_2306_00978_b200 import binding
+        N, K, group = self.N, self.K, self.group
+        x = torch.randn((M, K), device="cuda").half()
+        y = torch.empty((M, N), device="cuda", dtype=torch.float16)
+        binding.linear(x, *self.copies[0], N, K, group, out=y, path=path)
+        torch.cuda.synchronize()
+        ts = []
+        for i in range(len(self.copies)):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda._sleep(400000)
+            e0.record()
+            binding.linear(x, *self.copies[i], N, K, group, out=y, path=path)
+            e1.record()
+            torch.cuda.synchronize()
+            ts.append(e0.elapsed_time(e1) * 1e3)
+        binding.poll_status()
+        return statistics.median(ts)
+
+
+def _point(N, K, M, group, us, peaks):
+    """One measured call as absolute numbers and fractions of both rooflines."""
+    nbytes = algorithmic_bytes(N, K, M, group)
+    gbs, tf = nbytes / us / 1e3, 2.0 * M * N * K / us / 1e6
+    d = {"us": round(us, 2), "GBps": round(gbs, 1), "TFLOPs": round(tf, 2)}
+    if M <= 64:          # HBM-bound side of the ridge (about 70 tokens)
+        d["frac_hbm_measured"] = round(gbs / peaks["hbm_gbs"], 4)
+        d["frac_hbm_8000"] = round(gbs / NOMINAL_HBM_GBS, 4)
+    if M >= 64:
+        d["frac_tensor_measured_burst"] = round(tf / peaks["bf16_tflops"], 4)
+        d["frac_tensor_2250"] = round(tf / NOMINAL_FP16_TFLOPS, 4)
+    return d
+
+
+def config1_section(peaks):
+    """configs[0]: a single 4096 -> 4096 linear at M = 1, as an isolated launch and chained."""
+    rp = RandomPacked(4096, 4096, GROUP)
+    iso = rp.time_isolated(1)
+    best, med = rp.time_chained(1)
+    return {"shape": "4096->4096", "M": 1, "group": GROUP, "cold_l2": rp.cold, "copies": len(rp.copies),
+            "isolated": _point(4096, 4096, 1, GROUP, iso, peaks),
+            "chained": _point(4096, 4096, 1, GROUP, med, peaks), "chained_best_us": round(best, 2)}
+
+
+def config4_section(peaks):
+    """configs[3]: the Llama-2-70B MLP shapes over M = 1, 4, 8, 16 on both forced paths and as
+    awq_linear dispatches them (graph of chained calls over rotating copies, median of 5)."""
     from paper_2306_00978_b200 import binding
-    shapes = [("q/k/v/o", 4096, 4096), ("gate/up", 4096, 11008), ("down", 11008, 4096)]
-    for group in (128, 64):
-        for name, K, N in shapes:
-            copies = []
-            for _ in range(3):
-                qw = torch.randint(0, 256, (N * K // 2,), dtype=torch.uint8, device="cuda")
-                sc = (torch.rand((N // 16, K // group, 16), device="cuda") * 0.01 + 0.001).half()
-                zp = torch.randint(0, 256, (N // 32, K // group, 16), dtype=torch.uint8, device="cuda")
-                copies.append((qw, sc, zp))
-            for M in (1, 2, 4, 8, 16, 32, 64, 128, 512, 2048, 8192):
-                x = torch.randn((M, K), device="cuda").half()
-                y = torch.empty((M, N), device="cuda", dtype=torch.float16)
-                calls = 8 if M <= 512 else 2
-                for i in range(3):
-                    binding.linear(x, *copies[i], N, K, group, out=y)
-                torch.cuda.synchronize()
-                graph, stream = torch.cuda.CUDAGraph(), torch.cuda.Stream()
-                with torch.cuda.stream(stream):
-                    with torch.cuda.graph(graph, stream=stream):
-                        for i in range(calls):
-                            binding.linear(x, *copies[i % 3], N, K, group, out=y)
-                torch.cuda.synchronize()
-                graph.replay()
-                torch.cuda.synchronize()
-                best = float("inf")
-                for _ in range(5):
-                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                    e0.record()
-                    graph.replay()
-                    e1.record()
-                    torch.cuda.synchronize()
-                    best = min(best, e0.elapsed_time(e1) * 1e3 / calls)
-                binding.poll_status()
-                nbytes = N * K // 2 + (N * K // group) * 2 + (N * K // group) // 2 + M * K * 2 + M * N * 2
-                print(json.dumps({"shape": name, "K": K, "N": N, "group": group, "M": M, "us": round(best, 2),
-                                  "GBps": round(nbytes / best / 1e3, 1),
-                                  "TFLOPs": round(2 * M * N * K / best / 1e6, 1)}), flush=True)
+    rows = []
+    for name, K, N in synth.LLAMA2_70B_MLP:
+        rp = RandomPacked(N, K, GROUP)
+        for M in (1, 4, 8, 16):
+            r = {"shape": f"{K}->{N}", "M": M}
+            for label, path in (("gemv", binding.PATH_GEMV), ("gemm", binding.PATH_GEMM), ("auto", binding.PATH_AUTO)):
+                _, med = rp.time_chained(M, path=path, calls=8)
+                r[label] = _point(N, K, M, GROUP, med, peaks)
+            rows.append(r)
+        del rp
+    return rows
+
+
+SWEEP_SHAPES = (("q/k/v/o", 4096, 4096), ("gate/up", 4096, 11008), ("down", 11008, 4096))
+SWEEP_M = (1, 2, 4, 8, 16, 32, 64, 128, 512, 2048, 8192)
+
+
+def sweep_rows(peaks, groups=(128, 64), reps: int = 5):
+    """configs[4]: the 7B layer's three distinct shapes x token counts 1 .. 8192 x both group sizes
+    through awq_linear (alpha only changes the values of the packed arrays, not the run time: the
+    sweep's parity over alpha in {0, 0.5, 1} is a test).  Cold-L2 rotation for M <= 128."""
+    import torch
+    for group in groups:
+        for name, K, N in SWEEP_SHAPES:
+            rp = RandomPacked(N, K, group)
+            for M in SWEEP_M:
+                best, med = rp.time_chained(M, reps=reps)
+                row = {"shape": name, "K": K, "N": N, "group": group, "M": M}
+                row.update(_point(N, K, M, group, best, peaks))
+                row["us_median"] = round(med, 2)
+                yield row
+            del rp
+            torch.cuda.empty_cache()
+
+
+def sweep(args):
+    """The full-shape sweep, one JSON object per line."""
+    peaks = load_peaks()
+    for row in sweep_rows(peaks):
+        print(json.dumps(row), flush=True)
     return 0
 
 
@@ -584,40 +777,31 @@ def main():
     layers = build_layers(args.layers)
     step_bytes = sum(algorithmic_bytes(l["N"], l["K"], 1) for l in layers[0])
     packed_bytes = sum(l["qw"].numel() + l["sc"].numel() * 2 + l["zp"].numel() for l in layers[0])
+    l2_bytes = torch.cuda.get_device_properties(local_rank).L2_cache_size
 
     sampler = ClockSampler(local_rank)
     if rank == 0:
         sampler.start()
         time.sleep(0.3)
-    graphs, launches_per_step, stack = capture_steps(run_step, layers)
-    e2e_graphs, _, e2e_stack = capture_steps(run_step_e2e, layers)
-    sec, (w0, w1) = timed_region(graphs, stack, steps, warmup, device)
-    e2e_sec, _ = timed_region(e2e_graphs, e2e_stack, steps, warmup, device)
-    launches = launches_per_step * steps
+    graph, launches_per_step = capture_chain(run_step, layers, steps)
+    sec, spread, (w0, w1), R = timed_region(graph, steps, warmup, device)
+    del graph
+    e2e_graph, _ = capture_chain(run_step_e2e, layers, steps)
+    e2e_sec, e2e_spread, _, _ = timed_region(e2e_graph, steps, warmup, device, min_seconds=0.3, min_replays=20)
+    del e2e_graph
+    launches = launches_per_step * steps * R
     clocks = None
     if rank == 0:
-        if w1 - w0 < 1.0:
-            # the timed region is too short for 100 ms clock samples: keep the same load
-            # running (untimed) for about a second and sample that instead
-            w0 = time.time()
-            while time.time() - w0 < 1.2:
-                for i in range(50):
-                    stack.replay()
-                torch.cuda.synchronize()
-            w1 = time.time()
-            clocks_note = "sampled over ~1.2 s of the same steps run right after the timed region"
-        else:
-            clocks_note = "sampled during the timed region"
         time.sleep(0.15)
-        sampler.stop()
         clocks = sampler.summary(w0, w1)
-        clocks["note"] = clocks_note
+        clocks["note"] = f"sampled during the timed region ({w1 - w0:.2f} s)"
     binding.poll_status()
+    pos_sec = per_position_times(layers) if rank == 0 else None
 
-    value = replicas.aggregate_throughput(step_bytes * steps, sec) / 1e9
-    e2e_value = replicas.aggregate_throughput(step_bytes * steps, e2e_sec) / 1e9
-    per_launch_s = sec / max(1, launches)
-    achieved = step_bytes * steps / sec / 1e9         # one GPU's algorithmic GB/s over the region
+    value = replicas.aggregate_throughput(step_bytes, sec / steps) / 1e9
+    e2e_value = replicas.aggregate_throughput(step_bytes, e2e_sec / steps) / 1e9
+    achieved_step = step_bytes * steps / sec / 1e9      # one GPU's algorithmic GB/s over the region
+    rotation = args.layers * packed_bytes
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warmup,
         "ms_per_step": sec / steps * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -625,38 +809,73 @@ def main():
         "config": {"workload": "llama2-7b decoder-layer linears (q,k,v,o 4096->4096; gate,up 4096->11008; "
                                "down 11008->4096), M=1, g128, alpha=0.5",
                    "layers_rotated": args.layers, "packed_bytes_per_layer": packed_bytes,
-                   "l2_policy": f"weights rotate over {args.layers} layers "
-                                f"({args.layers * packed_bytes / 1e6:.0f} MB > 2 x 126 MB L2)",
+                   "l2_policy": f"weights rotate over {args.layers} layers = {rotation / 1e6:.0f} MB, "
+                                + ("more" if rotation > 2 * l2_bytes else "NOT more")
+                                + f" than 2 x the {l2_bytes / 1e6:.0f} MB L2"
+                                + ("" if rotation > 2 * l2_bytes else " (weights partly L2-resident: not a valid HBM figure)"),
                    "algorithmic_bytes_per_step": step_bytes, "parallelism": f"replicas x{world}",
                    "launch": "each step is 4 C-ABI calls: awq_linear_multi(q,k,v), awq_linear(o), "
-                             "awq_linear_multi(gate,up), awq_linear(down); the rotating layers are replayed "
-                             "back to back as one CUDA graph (layers_rotated steps per replay), a remainder of "
-                             "steps as single-layer graphs"},
-        "roofline": {"bound": "hbm", "kernel": "gemv_band_kernel<128,4,true,true,5>", "achieved": achieved,
-                     "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
-                     "peak_source": peaks["source"], "frac_of_nominal_8000": achieved / NOMINAL_HBM_GBS,
-                     "avg_launch_us": per_launch_s * 1e6,
-                     # per launch, averaged over the step's launches, from the per-matrix captures
-                     # in profiles/gemv_band_kernel_llama2_7b_M1.md (4x 4096^2, 3x 4096x11008)
-                     "traffic": (4 * NCU_TRAFFIC_BYTES_PER_LAUNCH[(4096, 4096)] +
-                                 3 * NCU_TRAFFIC_BYTES_PER_LAUNCH[(11008, 4096)]) / max(1, launches_per_step),
-                     "algorithmic_bytes_per_launch": step_bytes / max(1, launches_per_step)},
+                             "awq_linear_multi(gate,up), awq_linear(down); the `steps` steps (layers rotating) are "
+                             "ONE CUDA graph, all launches chained by programmatic dependent launch",
+                   "timing": f"the {steps}-step graph replayed {R} times, one CUDA event between replays; "
+                             "ms_per_step = median replay time / steps"},
+        "replay_seconds": spread,
         "e2e": {"value": e2e_value, "unit": UNIT,
                 "h2d_bytes_per_step": sum(2 * layers[0][idxs[0]]["K"] for idxs in STEP_CALLS),
-                "d2h_bytes_per_step": sum(2 * l["N"] for l in layers[0])},
+                "d2h_bytes_per_step": sum(2 * l["N"] for l in layers[0]),
+                "replays": e2e_spread["replays"]},
         "gpu_launches": launches,
         "clocks": clocks,
     }
+    if rank == 0:
+        # the dominant kernel: the K = 4096 instantiation of the band kernel serves three of the four
+        # launch positions (q+k+v, o, gate+up) and most of the step's bytes and time
+        pos_bytes = [sum(algorithmic_bytes(layers[0][i]["N"], layers[0][i]["K"], 1) for i in idxs)
+                     - 2 * layers[0][idxs[0]]["K"] * (len(idxs) - 1) for idxs in STEP_CALLS]
+        dom = [0, 1, 2]
+        dom_bytes = sum(pos_bytes[i] for i in dom) / len(dom)
+        dom_sec = sum(pos_sec[i] for i in dom) / len(dom)
+        achieved = dom_bytes / dom_sec / 1e9
+        line["roofline"] = {
+            "bound": "hbm", "kernel": DOMINANT_KERNEL, "achieved": achieved,
+            "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
+            "peak_source": peaks["source"], "frac_of_nominal_8000": achieved / NOMINAL_HBM_GBS,
+            "avg_launch_us": dom_sec * 1e6, "algorithmic_bytes_per_launch": dom_bytes,
+            "how": "average over this kernel's three launch positions of the step (q+k+v, o, gate+up), each "
+                   "timed with CUDA events on a graph that holds only that position, chained over the "
+                   "rotating layers",
+            "traffic": dom_bytes * NCU_TRAFFIC_RATIO,
+            "traffic_note": NCU_TRAFFIC_NOTE,
+            "per_position": [{"calls": "+".join(layers[0][i]["name"] for i in idxs), "us": pos_sec[k] * 1e6,
+                              "algorithmic_bytes": pos_bytes[k], "GBps": pos_bytes[k] / pos_sec[k] / 1e9,
+                              "frac": pos_bytes[k] / pos_sec[k] / 1e9 / peaks["hbm_gbs"]}
+                             for k, idxs in enumerate(STEP_CALLS)],
+            "step": {"achieved": achieved_step, "frac": achieved_step / peaks["hbm_gbs"],
+                     "frac_of_nominal_8000": achieved_step / NOMINAL_HBM_GBS,
+                     "sum_of_positions_us": sum(pos_sec) * 1e6}}
     if rank == 0 and not args.skip_extras:
-        line["gemm_m2048"] = gemm_section(peaks)
+        del layers
+        torch.cuda.empty_cache()
+        line["config1_single_linear"] = config1_section(peaks)
+        line["config4_70b_mlp"] = config4_section(peaks)
+        torch.cuda.empty_cache()
+        rows = list(sweep_rows(peaks, reps=3))
+        cols = ["shape", "group", "M", "us", "GBps", "TFLOPs"]
+        line["config5_sweep"] = {"columns": cols, "rows": [[r[c] for c in cols] for r in rows],
+                                 "note": "awq_linear, automatic dispatch, best of 3 graph replays; cold-L2 rotation "
+                                         "for M <= 128; alpha does not enter the run time"}
+        torch.cuda.empty_cache()
         line["quantize_pack"] = quantize_section(peaks)
         line["alpha_search"] = search_section()
         line["clip_search"] = clip_section()
+        # last of the GPU sections: its sustained leg runs the GPU into the power cap, and the SM
+        # clock stays low for a while afterwards
+        line["gemm_m2048"] = gemm_section(peaks, sampler)
         if world == 1:
-            del graphs, e2e_graphs, layers
             torch.cuda.empty_cache()
             line["cpu_baseline"] = cpu_baseline()
     if rank == 0:
+        sampler.stop()
         print(json.dumps(line), flush=True)
     replicas.barrier()
     replicas.shutdown()

@@ -152,6 +152,16 @@ int awq_channel_scale(const float* act_mean_abs, float alpha, float* s, int K, v
  * The split-K matrix-vector kernel (used when N is small or M > 8) combines partial sums in a
  * fixed order through the registered workspace; calls that use the workspace must not
  * overlap on the GPU (issue them on one stream).
+ * Stream order.  x and y follow plain stream order.  The packed arrays are treated as constants
+ * of the layer: the band matrix-vector kernel (M <= 8, N / 16 not far below the SM count) is
+ * launched with programmatic stream serialization and starts copying qweight, scales and zeros
+ * into shared memory BEFORE the work in front of it in the stream has completed; only its reads
+ * of x and its writes of y wait for that work.  The library covers its own writers: the first
+ * layer call after an awq_quantize_pack / awq_quantize_pack_ex on the same device is launched
+ * fully serialized.  A caller who produces packed arrays by other means (its own kernel, a
+ * copy) must make sure they are complete before the operation that directly precedes
+ * awq_linear in the stream begins - a stream or event synchronization, or any other kernel in
+ * between that does not itself signal programmatic launch completion early, is enough.
  * Errors: AWQ_ERR_NO_WORKSPACE if M <= 8, that kernel is chosen and
  * awq_workspace_bytes(M,N,K,group) exceeds the registered size; shape / pointer errors as listed
  * in AwqStatus.
@@ -208,6 +218,11 @@ int awq_linear_path(const void* x, const void* qweight, const void* scales, cons
  */
 int awq_linear_gemv_static(const void* x, const void* qweight, const void* scales, const void* zeros,
                             void* y, int M, int N, int K, int group, void* stream);
+/* Test aid for the entry point above (the paper has no counterpart): overwrites the arrival
+ * counters at the head of the built-in scratch with the byte `value` on `stream`, as a call that
+ * was cut short might leave them; awq_linear_gemv_static must still give the right result.
+ * Allocates nothing. */
+int awq_static_scratch_fill(int value, void* stream);
 
 /*
  * Scale search (Sec. 3.2).  For each alpha_i of `alphas`: s = s_X^alpha_i (Eq. 5, s_X = act_mean_abs),

@@ -24,7 +24,7 @@ EXPORTS = (
     "awq_set_workspace", "awq_unpack_canonical", "awq_poll_status", "awq_status_string",
     "awq_last_cuda_error", "awq_layout_version", "awq_launch_count", "awq_linear_gemv_static",
     "awq_linear_multi", "awq_search_scratch_bytes", "awq_search_alpha",
-    "awq_quantize_pack_ex", "awq_search_clip",
+    "awq_quantize_pack_ex", "awq_search_clip", "awq_static_scratch_fill",
 )
 
 
@@ -59,6 +59,7 @@ def lib() -> ctypes.CDLL:
     L.awq_linear.restype, L.awq_linear.argtypes = i, [vp, vp, vp, vp, vp, i, i, i, i, vp]
     L.awq_linear_path.restype, L.awq_linear_path.argtypes = i, [vp, vp, vp, vp, vp, i, i, i, i, i, vp]
     L.awq_linear_gemv_static.restype, L.awq_linear_gemv_static.argtypes = i, [vp, vp, vp, vp, vp, i, i, i, i, vp]
+    L.awq_static_scratch_fill.restype, L.awq_static_scratch_fill.argtypes = i, [i, vp]
     L.awq_linear_multi.restype, L.awq_linear_multi.argtypes = i, [vp, vp, i, i, i, i, vp]
     L.awq_search_scratch_bytes.restype, L.awq_search_scratch_bytes.argtypes = sz, [i, i, i, i]
     L.awq_search_alpha.restype, L.awq_search_alpha.argtypes = i, [vp, vp, vp, i, i, i, i, vp, i, vp, vp, vp, sz, vp]
@@ -227,6 +228,11 @@ def linear_gemv_static(x: torch.Tensor, qweight: torch.Tensor, scales: torch.Ten
         _dev(out, torch.float16, "out"), M, N, K, int(group), _stream())
     _check(rc, "awq_linear_gemv_static")
     return out
+
+
+def static_scratch_fill(value: int) -> None:
+    """awq_static_scratch_fill: test aid, dirties the built-in scratch's arrival counters."""
+    _check(lib().awq_static_scratch_fill(int(value), _stream()), "awq_static_scratch_fill")
 
 
 def search_alpha(W: torch.Tensor, act_mean_abs: torch.Tensor, X: torch.Tensor, group: int, alphas):

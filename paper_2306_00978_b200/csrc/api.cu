@@ -21,6 +21,10 @@ struct DeviceState {
     unsigned int* status_word = nullptr;   // device address of g_status on this device
     int cc_major = -1;
     int sms = 0;
+    // Set when one of this library's kernels that writes packed arrays (the quantizer) has been
+    // enqueued since the last matrix-vector launch: the band kernel prefetches weights before its
+    // stream dependency resolves, so the first launch after such a writer is fully serialized.
+    bool packed_written = false;
 };
 DeviceState g_dev[kMaxDevices];
 std::mutex g_mutex;
@@ -60,6 +64,14 @@ int device_state(DeviceState** out) {
     if (d.cc_major != 10) return AWQ_ERR_WRONG_DEVICE;
     *out = &d;
     return AWQ_OK;
+}
+
+// True once after a packed-array writer of this library was enqueued on the device.
+bool take_packed_written(DeviceState* d) {
+    std::lock_guard<std::mutex> lock(g_mutex);
+    const bool w = d->packed_written;
+    d->packed_written = false;
+    return w;
 }
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -113,6 +125,10 @@ int awq_quantize_pack_ex(const void* W, const float* act_mean_abs, float alpha, 
         return AWQ_ERR_MISALIGNED;
     DeviceState* d;
     if (int rc = device_state(&d)) return rc;
+    {
+        std::lock_guard<std::mutex> lock(g_mutex);
+        d->packed_written = true;
+    }
     return note_cuda(launch_quantize_pack(reinterpret_cast<const __half*>(W), act_mean_abs, alpha, group, bits,
                                           symmetric != 0, clip_ratio, reinterpret_cast<uint32_t*>(qweight),
                                           reinterpret_cast<__half*>(scales),
@@ -203,8 +219,10 @@ int awq_linear_path(const void* x, const void* qweight, const void* scales, cons
     const cudaStream_t st = (cudaStream_t)stream;
     if (path == AWQ_PATH_GEMV && gemv_uses_band_kernel(M, N, d->sms)) {
         const GemvMatrix one = {qweight, scales, zeros, y, N};
-        return note_cuda(launch_gemv_band(x, &one, 1, M, K, group, d->status_word, d->sms, st));
+        return note_cuda(launch_gemv_band(x, &one, 1, M, K, group, d->status_word, d->sms,
+                                          take_packed_written(d), st));
     }
+    (void)take_packed_written(d);               // every other kernel is plainly stream-ordered
     if (path == AWQ_PATH_GEMV || path == AWQ_PATH_GEMV_SPLITK) {
         void* ws = nullptr;
         {
@@ -245,6 +263,14 @@ int awq_linear_gemv_static(const void* x, const void* qweight, const void* scale
                                         d->status_word, d->sms, st));
 }
 
+int awq_static_scratch_fill(int value, void* stream) {
+    DeviceState* d;
+    if (int rc = device_state(&d)) return rc;
+    void* scratch = nullptr;
+    if (int rc = note_cuda(gemv_static_scratch(&scratch))) return rc;
+    return note_cuda(cudaMemsetAsync(scratch, value & 0xFF, kCounterBytes, (cudaStream_t)stream));
+}
+
 int awq_linear_multi(const void* x, const AwqLinearProblem* problems, int count,
                      int M, int K, int group, void* stream) {
     if (!problems || !x) return AWQ_ERR_NULL_POINTER;
@@ -268,7 +294,7 @@ int awq_linear_multi(const void* x, const AwqLinearProblem* problems, int count,
             mats[i] = GemvMatrix{problems[i].qweight, problems[i].scales, problems[i].zeros, problems[i].y,
                                  problems[i].N};
         return note_cuda(launch_gemv_band(x, mats, count, M, K, group, d->status_word, d->sms,
-                                          (cudaStream_t)stream));
+                                          take_packed_written(d), (cudaStream_t)stream));
     }
     // otherwise one call per matrix, as awq_linear would run it
     for (int i = 0; i < count; ++i) {

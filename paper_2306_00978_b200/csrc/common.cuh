@@ -54,9 +54,11 @@ struct GemvMatrix {                      // one packed weight matrix and its out
 };
 bool gemv_uses_band_kernel(int M, int N, int sms);
 size_t gemv_workspace_bytes(int M);
-// `count` matrices (1..kMaxMulti) sharing x, K and the group size, in one launch
+// `count` matrices (1..kMaxMulti) sharing x, K and the group size, in one launch.
+// serialize: launch without programmatic stream serialization (the kernel then starts only after
+// everything in front of it in the stream has completed, its weight prefetch included).
 cudaError_t launch_gemv_band(const void* x, const GemvMatrix* mats, int count, int M, int K, int group,
-                             unsigned int* status_word, int sms, cudaStream_t st);
+                             unsigned int* status_word, int sms, bool serialize, cudaStream_t st);
 cudaError_t launch_gemv_splitk(const void* x, const void* qweight, const void* scales, const void* zeros,
                                void* y, int M, int N, int K, int group, void* workspace,
                                unsigned int* status_word, int sms, cudaStream_t st);

@@ -1035,7 +1035,7 @@ cudaError_t gemv_static_scratch(void** out) {
 }
 
 cudaError_t launch_gemv_band(const void* x, const GemvMatrix* mats, int count, int M, int K, int group,
-                             unsigned int* status_word, int sms, cudaStream_t st) {
+                             unsigned int* status_word, int sms, bool serialize, cudaStream_t st) {
     BandProblems pr;
     pr.count = count;
     int bands = 0;
@@ -1066,7 +1066,7 @@ cudaError_t launch_gemv_band(const void* x, const GemvMatrix* mats, int count, i
     cfg.blockDim = dim3(kBandThreads);
     cfg.stream = st;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = serialize ? 0 : 1;
 #define AWQ_BAND_LAUNCH(GG, TT, ONE1, XR)                                                            \
     do {                                                                                             \
         const BandLayout lay = band_layout<GG, TT>(M, K, XR);                                        \
