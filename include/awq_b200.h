@@ -230,8 +230,10 @@ int awq_static_scratch_fill(int value, void* stream);
  *   loss_i = mean over (m, n) of ( awq_linear(fp16(X / s), Wq)[m][n] - sum_k X[m][k] W[n][k] )^2   (Eq. 4;
  * the paper does not name its norm: the mean squared difference has the same minimizer as any other
  * monotone function of the Frobenius norm).  The quantizer and the layer are the library's own
- * kernels, so the search scores exactly what deployment runs; the fp16 reference product is a cuBLAS
- * GEMM with fp32 accumulation.  The paper uses 20 grid points over [0, 1]; the grid is the caller's.
+ * kernels, so the search scores exactly what deployment runs; the fp16 reference product W X is a
+ * dense GEMM kernel of this library with fp32 accumulation and output.  Nothing is allocated: all
+ * intermediate arrays live in `scratch`.  The paper uses 20 grid points over [0, 1]; the grid is the
+ * caller's.
  * W: in, fp16 [N][K] (device).  act_mean_abs: in, fp32 [K] (device).  X: in, fp16 [M][K] calibration
  * activations (device), M >= 1.  alphas: in, HOST array of n_alphas <= 64 values in [0, 1].
  * losses: out, HOST array of n_alphas floats.  best_index: out, HOST, index of the first least loss
@@ -240,7 +242,7 @@ int awq_static_scratch_fill(int value, void* stream);
  * The call enqueues on `stream` and then SYNCHRONIZES it (the result is returned on the host); it
  * must not run inside a stream capture.  A registered workspace is used as awq_linear uses it.
  * Errors: those of awq_quantize_pack and awq_linear; AWQ_ERR_BAD_ARGUMENT for a bad list or a
- * scratch that is too small; AWQ_ERR_CUDA if cuBLAS fails.
+ * scratch that is too small.
  */
 size_t awq_search_scratch_bytes(int M, int N, int K, int group);
 int awq_search_alpha(const void* W, const float* act_mean_abs, const void* X, int M, int N, int K, int group,
@@ -274,6 +276,17 @@ int awq_unpack_canonical(const void* qweight, const void* scales, const void* ze
  * (its output is then undefined; the arrival counters at the head of the registered workspace
  * are cleared again so that later calls start clean), or AWQ_ERR_CUDA. */
 int awq_poll_status(void);
+
+/* How long a device-side wait (on a copy, on another block's partial sums) may last before the
+ * kernel gives it up, records AWQ_ERR_TIMEOUT for awq_poll_status and runs to its end: default
+ * about two seconds; 0 restores the default.  Applies to the current device; synchronizes it. */
+int awq_set_wait_limit_us(unsigned int microseconds);
+/* Test aid for the time-out path (no fault, trap or endless loop is involved): the next split-K
+ * matrix-vector launch on the current device (awq_linear_path with AWQ_PATH_GEMV_SPLITK, or
+ * awq_linear where it picks that kernel) announces 16 bytes more on each stage's copy barrier than
+ * its copies deliver, so its first wait runs into the limit set with awq_set_wait_limit_us; the
+ * kernel then returns by itself with undefined output.  One launch only; later calls are normal. */
+int awq_test_stall_next_gemv(void);
 
 const char* awq_status_string(int status);
 /* Text of the last CUDA error seen by the calling thread's library calls ("" if none). */

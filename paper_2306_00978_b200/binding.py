@@ -25,6 +25,7 @@ EXPORTS = (
     "awq_last_cuda_error", "awq_layout_version", "awq_launch_count", "awq_linear_gemv_static",
     "awq_linear_multi", "awq_search_scratch_bytes", "awq_search_alpha",
     "awq_quantize_pack_ex", "awq_search_clip", "awq_static_scratch_fill",
+    "awq_set_wait_limit_us", "awq_test_stall_next_gemv",
 )
 
 
@@ -60,6 +61,8 @@ def lib() -> ctypes.CDLL:
     L.awq_linear_path.restype, L.awq_linear_path.argtypes = i, [vp, vp, vp, vp, vp, i, i, i, i, i, vp]
     L.awq_linear_gemv_static.restype, L.awq_linear_gemv_static.argtypes = i, [vp, vp, vp, vp, vp, i, i, i, i, vp]
     L.awq_static_scratch_fill.restype, L.awq_static_scratch_fill.argtypes = i, [i, vp]
+    L.awq_set_wait_limit_us.restype, L.awq_set_wait_limit_us.argtypes = i, [ctypes.c_uint]
+    L.awq_test_stall_next_gemv.restype, L.awq_test_stall_next_gemv.argtypes = i, []
     L.awq_linear_multi.restype, L.awq_linear_multi.argtypes = i, [vp, vp, i, i, i, i, vp]
     L.awq_search_scratch_bytes.restype, L.awq_search_scratch_bytes.argtypes = sz, [i, i, i, i]
     L.awq_search_alpha.restype, L.awq_search_alpha.argtypes = i, [vp, vp, vp, i, i, i, i, vp, i, vp, vp, vp, sz, vp]
@@ -228,6 +231,11 @@ def linear_gemv_static(x: torch.Tensor, qweight: torch.Tensor, scales: torch.Ten
         _dev(out, torch.float16, "out"), M, N, K, int(group), _stream())
     _check(rc, "awq_linear_gemv_static")
     return out
+
+
+def set_wait_limit_us(us: int) -> None:
+    """awq_set_wait_limit_us: limit of a device-side wait (0 = default)."""
+    _check(lib().awq_set_wait_limit_us(int(us)), "awq_set_wait_limit_us")
 
 
 def static_scratch_fill(value: int) -> None:

@@ -57,7 +57,7 @@ def build(force: bool = False, verbose: bool = False, out: str = LIB_PATH, extra
         failed |= p.returncode != 0
     if failed:
         raise RuntimeError("nvcc failed")
-    link = [_nvcc(), "-shared", "-o", out, *objs, "-lcudart", "-lcublas", "-Xcompiler", "-fPIC"]
+    link = [_nvcc(), "-shared", "-o", out, *objs, "-lcudart", "-Xcompiler", "-fPIC"]
     subprocess.run(link, check=True)
     return out
 

@@ -21,6 +21,7 @@ struct DeviceState {
     unsigned int* status_word = nullptr;   // device address of g_status on this device
     int cc_major = -1;
     int sms = 0;
+    int tx_surplus_once = 0;               // time-out test: see awq_test_stall_next_gemv
     // Set when one of this library's kernels that writes packed arrays (the quantizer) has been
     // enqueued since the last matrix-vector launch: the band kernel prefetches weights before its
     // stream dependency resolves, so the first launch after such a writer is fully serialized.
@@ -29,7 +30,9 @@ struct DeviceState {
 DeviceState g_dev[kMaxDevices];
 std::mutex g_mutex;
 
-__device__ unsigned int g_status;          // 0, or a code written by a kernel that gave up a wait
+// [0]: 0, or a code written by a kernel that gave up a wait; [1]: limit of a device-side wait in
+// microseconds (0 = the built-in default)
+__device__ unsigned int g_status[2];
 
 int note_cuda(cudaError_t e) {
     if (e == cudaSuccess) return AWQ_OK;
@@ -53,7 +56,7 @@ int device_state(DeviceState** out) {
             void* p = nullptr;
             e = cudaGetSymbolAddress(&p, g_status);
             if (e != cudaSuccess) return note_cuda(e);
-            e = cudaMemset(p, 0, sizeof(unsigned int));
+            e = cudaMemset(p, 0, 2 * sizeof(unsigned int));
             if (e != cudaSuccess) return note_cuda(e);
             d.status_word = reinterpret_cast<unsigned int*>(p);
         }
@@ -230,8 +233,14 @@ int awq_linear_path(const void* x, const void* qweight, const void* scales, cons
             if (d->workspace_bytes < gemv_workspace_bytes(M)) return AWQ_ERR_NO_WORKSPACE;
             ws = d->workspace;
         }
+        int surplus = 0;
+        {
+            std::lock_guard<std::mutex> lock(g_mutex);
+            surplus = d->tx_surplus_once;
+            d->tx_surplus_once = 0;
+        }
         return note_cuda(launch_gemv_splitk(x, qweight, scales, zeros, y, M, N, K, group, ws, d->status_word,
-                                            d->sms, st));
+                                            d->sms, st, surplus));
     }
     void* ws = nullptr;
     size_t ws_bytes = 0;
@@ -261,6 +270,21 @@ int awq_linear_gemv_static(const void* x, const void* qweight, const void* scale
     if (int rc = note_cuda(cudaMemsetAsync(scratch, 0, kCounterBytes, st))) return rc;
     return note_cuda(launch_gemv_splitk(x, qweight, scales, zeros, y, M, N, K, group, scratch,
                                         d->status_word, d->sms, st));
+}
+
+int awq_set_wait_limit_us(unsigned int microseconds) {
+    DeviceState* d;
+    if (int rc = device_state(&d)) return rc;
+    if (int rc = note_cuda(cudaDeviceSynchronize())) return rc;
+    return note_cuda(cudaMemcpy(d->status_word + 1, &microseconds, sizeof(microseconds), cudaMemcpyHostToDevice));
+}
+
+int awq_test_stall_next_gemv(void) {
+    DeviceState* d;
+    if (int rc = device_state(&d)) return rc;
+    std::lock_guard<std::mutex> lock(g_mutex);
+    d->tx_surplus_once = 16;
+    return AWQ_OK;
 }
 
 int awq_static_scratch_fill(int value, void* stream) {

@@ -6,7 +6,7 @@
 
 namespace awq {
 
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // a wait gives up after ~2 s
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // a wait gives up after ~2 s by default
 constexpr unsigned int kTimeoutCode = 0x57A17u;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -50,20 +50,31 @@ __device__ __forceinline__ unsigned long long global_ns() {
 }
 
 struct WaitCtl {
-    unsigned int* status;            // device status word (global memory)
+    unsigned int* status;            // device status words (global memory): [0] code, [1] wait limit in us (0: default)
     volatile unsigned int* abort;    // block-wide "giving up" flag (shared memory)
 };
+// How long a wait may last: the default, or what awq_set_wait_limit_us stored (read on the slow
+// path only, i.e. by a wait that is already waiting).
+__device__ __forceinline__ unsigned long long wait_limit_ns(const WaitCtl& ctl) {
+    const unsigned int us = *reinterpret_cast<volatile unsigned int*>(ctl.status + 1);
+    return us ? (unsigned long long)us * 1000ull : kWaitLimitNs;
+}
+// Limit of the end-of-block drain (copies already issued must land before the block exits).
+__device__ __forceinline__ unsigned long long drain_limit_ns(const WaitCtl& ctl) {
+    const unsigned long long lim = wait_limit_ns(ctl);
+    return lim < 200000000ull ? lim : 200000000ull;
+}
 
 // Bounded wait on an mbarrier phase.  Returns false once the block is giving up: either this
 // wait ran out of time (it then records the time-out) or another thread's did.
 static __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, const WaitCtl& ctl) {
     if (*ctl.abort) return false;
-    const unsigned long long t0 = global_ns();
+    const unsigned long long t0 = global_ns(), limit = wait_limit_ns(ctl);
     for (unsigned int i = 1;; ++i) {
         if (mbar_try_wait(bar, parity)) return true;
         if ((i & 63u) == 0u) {
             if (*ctl.abort) return false;
-            if (global_ns() - t0 > kWaitLimitNs) {
+            if (global_ns() - t0 > limit) {
                 *ctl.abort = 1u;
                 atomicExch(ctl.status, kTimeoutCode);
                 return false;
@@ -80,12 +91,12 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const W
 // warps): sleep between polls so that the spinning does not take issue slots from the math warps.
 __device__ __forceinline__ bool mbar_wait_relaxed(uint32_t bar, uint32_t parity, const WaitCtl& ctl) {
     if (mbar_try_wait(bar, parity)) return true;
-    const unsigned long long t0 = global_ns();
+    const unsigned long long t0 = global_ns(), limit = wait_limit_ns(ctl);
     for (;;) {
         __nanosleep(128);
         if (mbar_try_wait(bar, parity)) return true;
         if (*ctl.abort) return false;
-        if (global_ns() - t0 > kWaitLimitNs) {
+        if (global_ns() - t0 > limit) {
             *ctl.abort = 1u;
             atomicExch(ctl.status, kTimeoutCode);
             return false;

@@ -59,9 +59,10 @@ size_t gemv_workspace_bytes(int M);
 // everything in front of it in the stream has completed, its weight prefetch included).
 cudaError_t launch_gemv_band(const void* x, const GemvMatrix* mats, int count, int M, int K, int group,
                              unsigned int* status_word, int sms, bool serialize, cudaStream_t st);
+// tx_surplus: 0, or (time-out test only) bytes announced on every stage's barrier beyond what the copies bring
 cudaError_t launch_gemv_splitk(const void* x, const void* qweight, const void* scales, const void* zeros,
                                void* y, int M, int N, int K, int group, void* workspace,
-                               unsigned int* status_word, int sms, cudaStream_t st);
+                               unsigned int* status_word, int sms, cudaStream_t st, int tx_surplus = 0);
 
 // scale search (search.cu)
 constexpr int kMaxSearchAlphas = 64;

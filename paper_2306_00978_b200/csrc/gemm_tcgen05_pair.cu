@@ -375,7 +375,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constan
                 const unsigned long long t0 = global_ns();
                 while (ld_acquire_u32(f) < 16u) {                   // 16 epilogue warps of that pair
                     if (*ctl.abort) { ok = false; break; }
-                    if (global_ns() - t0 > kWaitLimitNs) {
+                    if (global_ns() - t0 > wait_limit_ns(ctl)) {
                         *ctl.abort = 1u;
                         atomicExch(ctl.status, kTimeoutCode);
                         ok = false;

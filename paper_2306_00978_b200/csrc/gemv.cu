@@ -382,7 +382,7 @@ gemv_band_kernel(const BandProblems probs, const __half* __restrict__ x, int M, 
         for (int i = 0; i < pending; ++i) {
             if (stage == 0) { stage = S - 1; phase ^= 1u; } else { --stage; }
             const unsigned long long t0 = global_ns();
-            while (!mbar_try_wait(bars + 8u * stage, phase) && global_ns() - t0 < 200000000ull) {}
+            while (!mbar_try_wait(bars + 8u * stage, phase) && global_ns() - t0 < drain_limit_ns(ctl)) {}
         }
         return;
     }
@@ -708,7 +708,7 @@ __global__ void __launch_bounds__(kSplitkThreads, 1)
 gemv_splitk_kernel(const unsigned char* __restrict__ qweight, const __half* __restrict__ scales,
                    const unsigned char* __restrict__ zeros, const __half* __restrict__ x,
                    __half* __restrict__ y, float* __restrict__ partial, unsigned int* __restrict__ counters,
-                   int M, int N, int K, const SplitkLayout lay, unsigned int* status_word) {
+                   int M, int N, int K, const SplitkLayout lay, unsigned int* status_word, int tx_surplus) {
     extern __shared__ __align__(128) unsigned char smem[];
     __shared__ unsigned int s_abort;
     __shared__ unsigned int s_last;
@@ -765,7 +765,9 @@ gemv_splitk_kernel(const unsigned char* __restrict__ qweight, const __half* __re
             const uint32_t bar = bars + 8u * stage;
             if (lane == 0) {
                 mbar_wait_relaxed(bars + 64u + 8u * stage, phase ^ 1u, ctl);
-                mbar_arrive_expect_tx(bar, (uint32_t)(nt * kTileBytes + ngr * (256 + 64) + M * nt * 128));
+                // tx_surplus is 0 except in the time-out test, which announces more bytes than the
+                // copies below bring so that the stage never completes
+                mbar_arrive_expect_tx(bar, (uint32_t)(nt * kTileBytes + ngr * (256 + 64) + M * nt * 128 + tx_surplus));
             }
             __syncwarp();
             const int gi0 = kt * 64 / G;
@@ -793,7 +795,7 @@ gemv_splitk_kernel(const unsigned char* __restrict__ qweight, const __half* __re
         for (int i = 0; i < pending; ++i) {
             if (stage == 0) { stage = S - 1; phase ^= 1u; } else { --stage; }
             const unsigned long long t0 = global_ns();
-            while (!mbar_try_wait(bars + 8u * stage, phase) && global_ns() - t0 < 200000000ull) {}
+            while (!mbar_try_wait(bars + 8u * stage, phase) && global_ns() - t0 < drain_limit_ns(ctl)) {}
         }
         return;
     }
@@ -1105,7 +1107,7 @@ cudaError_t launch_gemv_band(const void* x, const GemvMatrix* mats, int count, i
 
 cudaError_t launch_gemv_splitk(const void* x, const void* qweight, const void* scales, const void* zeros,
                                void* y, int M, int N, int K, int group, void* workspace,
-                               unsigned int* status_word, int sms, cudaStream_t st) {
+                               unsigned int* status_word, int sms, cudaStream_t st, int tx_surplus) {
     const int ktiles = K / 64;
     const int ups = (ktiles + kUT - 1) / kUT;
     const int units = (N / 128) * ups;
@@ -1131,7 +1133,7 @@ cudaError_t launch_gemv_splitk(const void* x, const void* qweight, const void* s
         gemv_splitk_kernel<GG, MTT><<<blocks, kSplitkThreads, lay.total, st>>>(                      \
             reinterpret_cast<const unsigned char*>(qweight), reinterpret_cast<const __half*>(scales), \
             reinterpret_cast<const unsigned char*>(zeros), reinterpret_cast<const __half*>(x),       \
-            reinterpret_cast<__half*>(y), partial, counters, M, N, K, lay, status_word);             \
+            reinterpret_cast<__half*>(y), partial, counters, M, N, K, lay, status_word, tx_surplus); \
     } while (0)
     if (group == 128) { if (M <= 8) AWQ_SPLITK_LAUNCH(128, 1); else AWQ_SPLITK_LAUNCH(128, 2); }
     else              { if (M <= 8) AWQ_SPLITK_LAUNCH(64, 1);  else AWQ_SPLITK_LAUNCH(64, 2); }

@@ -2,11 +2,9 @@
 // (Eq. 5), quantize W diag(s) with the library's own quantizer, run the library's own layer on
 // diag(s)^-1 X, and measure the output error against the fp16 layer W X (Eq. 4).  Everything
 // that the search evaluates is therefore exactly what deployment will run.  The reference product
-// W X is a plain dense GEMM and comes from cuBLAS (fp16 inputs, fp32 accumulate and output).
-#include <cublas_v2.h>
-
-#include <mutex>
-
+// W X is a plain dense fp16 GEMM with fp32 accumulation and output; it runs once per search, on
+// a small warp-level tensor-core kernel of this file (no library call, no allocation).
+#include "async_copy.cuh"
 #include "common.cuh"
 
 namespace awq {
@@ -94,15 +92,97 @@ SearchScratch carve(void* base, int M, int N, int K, int group) {
     return r;
 }
 
-cublasHandle_t cublas_for_current_device(cublasStatus_t* status) {
-    static std::mutex mu;
-    static cublasHandle_t handles[64] = {};
-    int dev = 0;
-    cudaGetDevice(&dev);
-    std::lock_guard<std::mutex> lock(mu);
-    *status = CUBLAS_STATUS_SUCCESS;
-    if (!handles[dev & 63]) *status = cublasCreate(&handles[dev & 63]);
-    return handles[dev & 63];
+// ---------------------------------------------------------------- dense reference product
+// C[m][n] = sum_k X[m][k] * W[n][k]: both operands have K contiguous, which is the row / column
+// operand form of the warp-level m16n8k16 product.  128 tokens x 128 channels per block, 32
+// input channels per step, two shared-memory buffers filled by 16-byte asynchronous copies, eight
+// warps of 64 x 32 outputs each.  Rows of 80 bytes keep the 8 x 16-byte row reads of a matrix
+// load on distinct banks.
+constexpr int kRefBM = 128, kRefBN = 128, kRefBK = 32, kRefRow = 80;   // bytes per staged row
+constexpr int kRefTile = 128 * kRefRow;                                // one operand tile of one buffer
+
+__device__ __forceinline__ void cp_async_16(uint32_t dst, const void* src, bool valid) {
+    const int n = valid ? 16 : 0;                                     // 0: the 16 bytes are zero-filled
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(n) : "memory");
+}
+__device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+
+__global__ void __launch_bounds__(256)
+reference_product_kernel(const __half* __restrict__ W, const __half* __restrict__ X, float* __restrict__ C,
+                         int M, int N, int K) {
+    __shared__ __align__(16) unsigned char sm[2 * 2 * kRefTile];      // [buffer][X tile | W tile]
+    const uint32_t sbase = smem_u32(sm);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int m0 = blockIdx.y * kRefBM, n0 = blockIdx.x * kRefBN;
+    const int wm = (warp >> 2) * 64, wn = (warp & 3) * 32;            // this warp's corner inside the tile
+
+    auto fill = [&](int buf, int k0) {
+        // 128 rows x 4 pieces of 16 bytes per operand: two pieces of each operand per thread
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+            const int piece = tid + i * 256, row = piece >> 2, c = piece & 3;
+            const uint32_t dst = sbase + buf * (2 * kRefTile) + row * kRefRow + c * 16;
+            const bool ok = m0 + row < M;
+            cp_async_16(dst, X + (size_t)(ok ? m0 + row : 0) * K + k0 + c * 8, ok);
+            cp_async_16(dst + kRefTile, W + (size_t)(n0 + row) * K + k0 + c * 8, true);
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+    };
+
+    float acc[4][4][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) acc[i][j][e] = 0.0f;
+
+    const int steps = K / kRefBK;
+    fill(0, 0);
+    for (int s = 0; s < steps; ++s) {
+        if (s + 1 < steps) {
+            fill((s + 1) & 1, (s + 1) * kRefBK);
+            asm volatile("cp.async.wait_group 1;" ::: "memory");
+        } else {
+            asm volatile("cp.async.wait_group 0;" ::: "memory");
+        }
+        __syncthreads();
+        const uint32_t xa = sbase + (s & 1) * (2 * kRefTile), wa = xa + kRefTile;
+#pragma unroll
+        for (int kk = 0; kk < kRefBK; kk += 16) {
+            uint32_t a[4][4], b[2][4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i)   // rows wm + 16 i + (lane % 16), columns kk + 8 (lane / 16)
+                ldmatrix_x4(a[i], xa + (wm + 16 * i + (lane & 15)) * kRefRow + (kk + 8 * (lane >> 4)) * 2);
+#pragma unroll
+            for (int j = 0; j < 2; ++j)   // channels wn + 16 j + (lane % 8) + 8 (lane / 16), columns kk + 8 ((lane / 8) % 2)
+                ldmatrix_x4(b[j], wa + (wn + 16 * j + (lane & 7) + 8 * (lane >> 4)) * kRefRow + (kk + 8 * ((lane >> 3) & 1)) * 2);
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const uint32_t b0 = b[j >> 1][2 * (j & 1)], b1 = b[j >> 1][2 * (j & 1) + 1];
+                    asm volatile(
+                        "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                        : "+f"(acc[i][j][0]), "+f"(acc[i][j][1]), "+f"(acc[i][j][2]), "+f"(acc[i][j][3])
+                        : "r"(a[i][0]), "r"(a[i][1]), "r"(a[i][2]), "r"(a[i][3]), "r"(b0), "r"(b1));
+                }
+        }
+        __syncthreads();                                              // the buffer is refilled two steps on
+    }
+    const int g = lane >> 2, t = lane & 3;
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int col = n0 + wn + 8 * j + 2 * t;
+            const int r0 = m0 + wm + 16 * i + g, r1 = r0 + 8;
+            if (r0 < M) *reinterpret_cast<float2*>(C + (size_t)r0 * N + col) = make_float2(acc[i][j][0], acc[i][j][1]);
+            if (r1 < M) *reinterpret_cast<float2*>(C + (size_t)r1 * N + col) = make_float2(acc[i][j][2], acc[i][j][3]);
+        }
 }
 
 }  // namespace
@@ -114,15 +194,11 @@ size_t search_scratch_bytes(int M, int N, int K, int group) {
 // y_ref[m][n] = sum_k X[m][k] W[n][k], fp32 [M][N] row-major.
 cudaError_t launch_reference_product(const void* W, const void* X, float* yref, int M, int N, int K,
                                      cudaStream_t st) {
-    cublasStatus_t cs;
-    cublasHandle_t h = cublas_for_current_device(&cs);
-    if (cs != CUBLAS_STATUS_SUCCESS) return cudaErrorInitializationError;
-    if (cublasSetStream(h, st) != CUBLAS_STATUS_SUCCESS) return cudaErrorUnknown;
-    const float one = 1.0f, zero = 0.0f;
-    // column-major view: C^T (N x M) = W^T-view (N x K) * X-view (K x M)
-    cs = cublasGemmEx(h, CUBLAS_OP_T, CUBLAS_OP_N, N, M, K, &one, W, CUDA_R_16F, K, X, CUDA_R_16F, K, &zero,
-                      yref, CUDA_R_32F, N, CUBLAS_COMPUTE_32F, CUBLAS_GEMM_DEFAULT);
-    return cs == CUBLAS_STATUS_SUCCESS ? cudaSuccess : cudaErrorUnknown;
+    const dim3 grid((unsigned)(N / kRefBN), (unsigned)((M + kRefBM - 1) / kRefBM));
+    reference_product_kernel<<<grid, 256, 0, st>>>(reinterpret_cast<const __half*>(W),
+                                                   reinterpret_cast<const __half*>(X), yref, M, N, K);
+    count_launch();
+    return cudaGetLastError();
 }
 
 cudaError_t launch_divide_by_scale(const void* X, const float* s, void* xs, int M, int K, cudaStream_t st) {
