@@ -149,9 +149,10 @@ def build_layers(n_layers: int, seed0: int = 2000):
             a = torch.from_numpy(synth.act_mean_abs(xseed, K)).cuda()
             qw, sc, zp = binding.quantize_pack(W, a, ALPHA, GROUP)
             s = binding.channel_scale(a, ALPHA, K)
+            # the raw activation: the step's calls scale it by 1 / s themselves (awq_linear*_scaled,
+            # step S6 folded into the matrix-vector kernel)
             x = torch.from_numpy(synth.activations(xseed, 1, K)).cuda()
-            xs = (x.float() / s[None, :]).half().contiguous()     # the caller's x / s
-            lin.append(dict(name=name, N=N, K=K, qw=qw, sc=sc, zp=zp, x=xs))
+            lin.append(dict(name=name, N=N, K=K, qw=qw, sc=sc, zp=zp, x=x, s=binding.inverse_channel_scale(a, ALPHA, K)))
             del W
         # host-side view of a step (the e2e leg): the step's four activations in one pinned buffer,
         # its seven outputs in another, one copy each way per step; the device tensors the calls
@@ -185,12 +186,9 @@ def run_calls(layer, calls, e2e=False):
     for idxs in calls:
         first = layer[idxs[0]]
         xin = first["x_dev_in"] if e2e else first["x"]
-        if len(idxs) == 1:
-            binding.linear(xin, first["qw"], first["sc"], first["zp"], first["N"], first["K"], GROUP,
-                           out=first["y"])
-        else:
-            binding.linear_multi(xin, [(layer[i]["qw"], layer[i]["sc"], layer[i]["zp"], layer[i]["N"]) for i in idxs],
-                                 first["K"], GROUP, outs=[layer[i]["y"] for i in idxs])
+        binding.linear_multi_scaled(xin, first["s"],
+                                    [(layer[i]["qw"], layer[i]["sc"], layer[i]["zp"], layer[i]["N"]) for i in idxs],
+                                    first["K"], GROUP, outs=[layer[i]["y"] for i in idxs])
 
 
 def run_step(layer, e2e=False):
@@ -775,7 +773,10 @@ def main():
     steps = max(1, args.steps)
 
     layers = build_layers(args.layers)
-    step_bytes = sum(algorithmic_bytes(l["N"], l["K"], 1) for l in layers[0])
+    # each operand once per matrix as in the roofline table, plus the inverse channel scales (fp32 [K])
+    # that each of the four calls reads
+    step_bytes = sum(algorithmic_bytes(l["N"], l["K"], 1) for l in layers[0]) + \
+        sum(4 * layers[0][idxs[0]]["K"] for idxs in STEP_CALLS)
     packed_bytes = sum(l["qw"].numel() + l["sc"].numel() * 2 + l["zp"].numel() for l in layers[0])
     l2_bytes = torch.cuda.get_device_properties(local_rank).L2_cache_size
 
@@ -814,9 +815,10 @@ def main():
                                 + f" than 2 x the {l2_bytes / 1e6:.0f} MB L2"
                                 + ("" if rotation > 2 * l2_bytes else " (weights partly L2-resident: not a valid HBM figure)"),
                    "algorithmic_bytes_per_step": step_bytes, "parallelism": f"replicas x{world}",
-                   "launch": "each step is 4 C-ABI calls: awq_linear_multi(q,k,v), awq_linear(o), "
-                             "awq_linear_multi(gate,up), awq_linear(down); the `steps` steps (layers rotating) are "
-                             "ONE CUDA graph, all launches chained by programmatic dependent launch",
+                   "launch": "each step is 4 C-ABI calls: awq_linear_multi_scaled(q,k,v), awq_linear_scaled(o), "
+                             "awq_linear_multi_scaled(gate,up), awq_linear_scaled(down) on the UNDIVIDED activations "
+                             "(x / s is folded into the kernels: 4 launches per step); the `steps` steps (layers "
+                             "rotating) are ONE CUDA graph, all launches chained by programmatic dependent launch",
                    "timing": f"the {steps}-step graph replayed {R} times, one CUDA event between replays; "
                              "ms_per_step = median replay time / steps"},
         "replay_seconds": spread,
@@ -831,7 +833,8 @@ def main():
         # the dominant kernel: the K = 4096 instantiation of the band kernel serves three of the four
         # launch positions (q+k+v, o, gate+up) and most of the step's bytes and time
         pos_bytes = [sum(algorithmic_bytes(layers[0][i]["N"], layers[0][i]["K"], 1) for i in idxs)
-                     - 2 * layers[0][idxs[0]]["K"] * (len(idxs) - 1) for idxs in STEP_CALLS]
+                     - 2 * layers[0][idxs[0]]["K"] * (len(idxs) - 1) + 4 * layers[0][idxs[0]]["K"]
+                     for idxs in STEP_CALLS]
         dom = [0, 1, 2]
         dom_bytes = sum(pos_bytes[i] for i in dom) / len(dom)
         dom_sec = sum(pos_sec[i] for i in dom) / len(dom)

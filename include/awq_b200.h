@@ -189,6 +189,35 @@ typedef struct AwqLinearProblem {
 int awq_linear_multi(const void* x, const AwqLinearProblem* problems, int count,
                      int M, int K, int group, void* stream);
 
+/*
+ * The layer with diag(s)^-1 folded in (Sec. 3.2: the inverse scale goes into a neighbouring operator,
+ * so that no separate pass over the activations and no extra kernel launch is needed; Sec. 4.2: at
+ * batch 1 a launch costs as much as the kernel).
+ *   y = awq_linear(x', ...),   x'[m][k] = fp16_rne(fp32(x[m][k]) * inv_s[k])   (one fp32 multiply, one rounding)
+ * - bit for bit what the caller would get by forming x' itself and calling awq_linear /
+ * awq_linear_multi.  x: in, fp16 [M][K], NOT scaled.  inv_s: in, device, fp32 [K], 16-byte aligned:
+ * 1 / s for the alpha the weights were quantized with (awq_inverse_channel_scale gives the correctly
+ * rounded reciprocal of what awq_channel_scale gives); like the packed arrays it is a constant of
+ * the layer and may be read before the stream dependency resolves.  (A multiplication, not the
+ * division x / s: eight IEEE divisions per thread in the start-up of a launch that lasts a few
+ * microseconds cost 0.3 - 1.5 us per launch; x * (1 / s) and x / s differ in the last bit of the fp16
+ * result for a few elements in a thousand, which the method does not care about as long as the
+ * quantizer's s and this inv_s belong together.)
+ * Where the band matrix-vector kernel serves the call (M <= 8, enough output rows) and can keep x
+ * on chip (K = 4096, or M <= 2 and M * K small enough for shared memory) the scaling happens while
+ * the kernel fetches x: no extra launch, no extra memory.  Otherwise x' is first written to
+ * x_scratch (device, fp16 [M][K], caller-owned) by a small kernel and the plain call follows;
+ * x_scratch may be NULL if awq_linear_scaled_needs_scratch(M, N, K, group) returns 0 (for the
+ * multi call: N = the sum of the matrices' N), else AWQ_ERR_NULL_POINTER.
+ */
+int awq_linear_scaled(const void* x, const float* inv_s, void* x_scratch, const void* qweight, const void* scales,
+                      const void* zeros, void* y, int M, int N, int K, int group, void* stream);
+int awq_linear_multi_scaled(const void* x, const float* inv_s, void* x_scratch, const AwqLinearProblem* problems,
+                            int count, int M, int K, int group, void* stream);
+/* inv_s[k] = fp32(1 / s[k]) (correctly rounded), s as awq_channel_scale gives it.  inv_s: out, fp32 [K]. */
+int awq_inverse_channel_scale(const float* act_mean_abs, float alpha, float* inv_s, int K, void* stream);
+int awq_linear_scaled_needs_scratch(int M, int N, int K, int group);
+
 /* Same as awq_linear with the kernel forced (for the small-batch crossover measurement).
  * A matrix-vector path with M > 16 or K > 65536 returns AWQ_ERR_BAD_SHAPE. */
 int awq_linear_path(const void* x, const void* qweight, const void* scales, const void* zeros,

@@ -26,6 +26,8 @@ EXPORTS = (
     "awq_linear_multi", "awq_search_scratch_bytes", "awq_search_alpha",
     "awq_quantize_pack_ex", "awq_search_clip", "awq_static_scratch_fill",
     "awq_set_wait_limit_us", "awq_test_stall_next_gemv",
+    "awq_linear_scaled", "awq_linear_multi_scaled", "awq_linear_scaled_needs_scratch",
+    "awq_inverse_channel_scale",
 )
 
 
@@ -63,6 +65,10 @@ def lib() -> ctypes.CDLL:
     L.awq_static_scratch_fill.restype, L.awq_static_scratch_fill.argtypes = i, [i, vp]
     L.awq_set_wait_limit_us.restype, L.awq_set_wait_limit_us.argtypes = i, [ctypes.c_uint]
     L.awq_test_stall_next_gemv.restype, L.awq_test_stall_next_gemv.argtypes = i, []
+    L.awq_linear_scaled.restype, L.awq_linear_scaled.argtypes = i, [vp, vp, vp, vp, vp, vp, vp, i, i, i, i, vp]
+    L.awq_linear_multi_scaled.restype, L.awq_linear_multi_scaled.argtypes = i, [vp, vp, vp, vp, i, i, i, i, vp]
+    L.awq_inverse_channel_scale.restype, L.awq_inverse_channel_scale.argtypes = i, [vp, f, vp, i, vp]
+    L.awq_linear_scaled_needs_scratch.restype, L.awq_linear_scaled_needs_scratch.argtypes = i, [i, i, i, i]
     L.awq_linear_multi.restype, L.awq_linear_multi.argtypes = i, [vp, vp, i, i, i, i, vp]
     L.awq_search_scratch_bytes.restype, L.awq_search_scratch_bytes.argtypes = sz, [i, i, i, i]
     L.awq_search_alpha.restype, L.awq_search_alpha.argtypes = i, [vp, vp, vp, i, i, i, i, vp, i, vp, vp, vp, sz, vp]
@@ -114,6 +120,14 @@ def channel_scale(act_mean_abs: Optional[torch.Tensor], alpha: float, K: int) ->
     a = 0 if act_mean_abs is None else _dev(act_mean_abs, torch.float32, "act_mean_abs")
     _check(lib().awq_channel_scale(a, float(alpha), s.data_ptr(), K, _stream()), "awq_channel_scale")
     return s
+
+
+def inverse_channel_scale(act_mean_abs: Optional[torch.Tensor], alpha: float, K: int) -> torch.Tensor:
+    """1 / s as awq_linear_scaled wants it (the correctly rounded reciprocal of channel_scale)."""
+    inv = torch.empty(K, dtype=torch.float32, device="cuda")
+    a = 0 if act_mean_abs is None else _dev(act_mean_abs, torch.float32, "act_mean_abs")
+    _check(lib().awq_inverse_channel_scale(a, float(alpha), inv.data_ptr(), K, _stream()), "awq_inverse_channel_scale")
+    return inv
 
 
 def quantize_pack(W: torch.Tensor, act_mean_abs: Optional[torch.Tensor], alpha: float, group: int,
@@ -213,6 +227,31 @@ def linear_multi(x: torch.Tensor, mats, K: int, group: int, outs=None):
     rc = lib().awq_linear_multi(_dev(x, torch.float16, "x"), ctypes.byref(arr), len(mats), M, K, int(group),
                                 _stream())
     _check(rc, "awq_linear_multi")
+    return outs
+
+
+def linear_multi_scaled(x: torch.Tensor, inv_s: torch.Tensor, mats, K: int, group: int, outs=None,
+                        x_scratch: Optional[torch.Tensor] = None):
+    """awq_linear_multi_scaled (awq_linear_scaled for one matrix): x is NOT scaled; the product
+    fp16(fp32(x) * inv_s) is folded into the matrix-vector kernel where it can be, else formed
+    by a small kernel into `x_scratch` (allocated here if it is needed and not given)."""
+    M = x.shape[0]
+    s = inv_s
+    if x.shape[1] != K or s.numel() != K:
+        raise AwqError("x must be [M][K] and inv_s [K]")
+    if outs is None:
+        outs = [torch.empty((M, m[3]), dtype=torch.float16, device=x.device) for m in mats]
+    if x_scratch is None and lib().awq_linear_scaled_needs_scratch(M, sum(m[3] for m in mats), K, int(group)):
+        x_scratch = torch.empty_like(x)
+    ensure_workspace(max(workspace_bytes(M, m[3], K, group) for m in mats))
+    arr = (_Problem * len(mats))()
+    for k, ((qw, sc, zp, N), y) in enumerate(zip(mats, outs)):
+        arr[k] = _Problem(_dev(qw, torch.uint8, "qweight"), _dev(sc, torch.float16, "scales"),
+                          _dev(zp, torch.uint8, "zeros"), _dev(y, torch.float16, "y"), int(N))
+    rc = lib().awq_linear_multi_scaled(_dev(x, torch.float16, "x"), _dev(s, torch.float32, "s"),
+                                       0 if x_scratch is None else _dev(x_scratch, torch.float16, "x_scratch"),
+                                       ctypes.byref(arr), len(mats), M, K, int(group), _stream())
+    _check(rc, "awq_linear_multi_scaled")
     return outs
 
 

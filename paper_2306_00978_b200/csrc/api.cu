@@ -333,6 +333,64 @@ int awq_linear(const void* x, const void* qweight, const void* scales, const voi
     return awq_linear_path(x, qweight, scales, zeros, y, M, N, K, group, AWQ_PATH_AUTO, stream);
 }
 
+// ---- the layer with diag(s)^-1 folded in (Sec. 3.2: the inverse scale goes into the operator in front)
+static bool scaled_call_folds(int M, int total_n, int K, int group, int sms) {
+    return M <= 8 && K <= 65536 && gemv_uses_band_kernel(M, total_n, sms) && gemv_band_folds_scale(M, K, group);
+}
+
+int awq_linear_scaled_needs_scratch(int M, int N, int K, int group) {
+    if (check_shape(N, K, group) != AWQ_OK || M < 1) return 1;
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return 1;
+    }
+    return scaled_call_folds(M, N, K, group, sms) ? 0 : 1;
+}
+
+int awq_linear_multi_scaled(const void* x, const float* inv_s, void* x_scratch, const AwqLinearProblem* problems,
+                            int count, int M, int K, int group, void* stream) {
+    if (!problems || !x || !inv_s) return AWQ_ERR_NULL_POINTER;
+    if (count < 1 || count > kMaxMulti) return AWQ_ERR_BAD_ARGUMENT;
+    int total_n = 0;
+    for (int i = 0; i < count; ++i) {
+        const AwqLinearProblem& p = problems[i];
+        if (int rc = check_shape(p.N, K, group)) return rc;
+        if (!p.qweight || !p.scales || !p.zeros || !p.y) return AWQ_ERR_NULL_POINTER;
+        if (!aligned16(p.qweight) || !aligned16(p.scales) || !aligned16(p.zeros) || !aligned16(p.y))
+            return AWQ_ERR_MISALIGNED;
+        total_n += p.N;
+    }
+    if (M < 1 || (long long)M * K > (1LL << 40)) return AWQ_ERR_BAD_SHAPE;
+    if (!aligned16(x) || !aligned16(inv_s) || !aligned16(x_scratch)) return AWQ_ERR_MISALIGNED;
+    DeviceState* d;
+    if (int rc = device_state(&d)) return rc;
+    if (scaled_call_folds(M, total_n, K, group, d->sms)) {
+        GemvMatrix mats[kMaxMulti];
+        for (int i = 0; i < count; ++i)
+            mats[i] = GemvMatrix{problems[i].qweight, problems[i].scales, problems[i].zeros, problems[i].y,
+                                 problems[i].N};
+        return note_cuda(launch_gemv_band(x, mats, count, M, K, group, d->status_word, d->sms,
+                                          take_packed_written(d), (cudaStream_t)stream, inv_s));
+    }
+    // no kernel to fold it into: scale first (one more launch), then the plain calls
+    if (!x_scratch) return AWQ_ERR_NULL_POINTER;
+    if (int rc = note_cuda(launch_multiply_by_inverse(x, inv_s, x_scratch, M, K, (cudaStream_t)stream))) return rc;
+    return awq_linear_multi(x_scratch, problems, count, M, K, group, stream);
+}
+
+int awq_linear_scaled(const void* x, const float* inv_s, void* x_scratch, const void* qweight, const void* scales,
+                      const void* zeros, void* y, int M, int N, int K, int group, void* stream) {
+    const AwqLinearProblem one = {qweight, scales, zeros, y, N};
+    return awq_linear_multi_scaled(x, inv_s, x_scratch, &one, 1, M, K, group, stream);
+}
+
+int awq_inverse_channel_scale(const float* act_mean_abs, float alpha, float* inv_s, int K, void* stream) {
+    if (int rc = awq_channel_scale(act_mean_abs, alpha, inv_s, K, stream)) return rc;
+    return note_cuda(launch_inverse_scale(inv_s, inv_s, K, (cudaStream_t)stream));
+}
+
 size_t awq_search_scratch_bytes(int M, int N, int K, int group) {
     if (check_shape(N, K, group) != AWQ_OK || M < 1) return 0;
     return search_scratch_bytes(M, N, K, group);

@@ -57,8 +57,12 @@ size_t gemv_workspace_bytes(int M);
 // `count` matrices (1..kMaxMulti) sharing x, K and the group size, in one launch.
 // serialize: launch without programmatic stream serialization (the kernel then starts only after
 // everything in front of it in the stream has completed, its weight prefetch included).
+// sdiv: nullptr, or the inverse channel scales (fp32 [K], device): the kernel multiplies x by them
+// while it fetches it; only where gemv_band_folds_scale(M, K, group) holds.
 cudaError_t launch_gemv_band(const void* x, const GemvMatrix* mats, int count, int M, int K, int group,
-                             unsigned int* status_word, int sms, bool serialize, cudaStream_t st);
+                             unsigned int* status_word, int sms, bool serialize, cudaStream_t st,
+                             const float* sdiv = nullptr);
+bool gemv_band_folds_scale(int M, int K, int group);
 // tx_surplus: 0, or (time-out test only) bytes announced on every stage's barrier beyond what the copies bring
 cudaError_t launch_gemv_splitk(const void* x, const void* qweight, const void* scales, const void* zeros,
                                void* y, int M, int N, int K, int group, void* workspace,
@@ -72,6 +76,9 @@ void search_carve(void* base, int M, int N, int K, int group, float** s, void** 
 cudaError_t launch_reference_product(const void* W, const void* X, float* yref, int M, int N, int K,
                                      cudaStream_t st);
 cudaError_t launch_divide_by_scale(const void* X, const float* s, void* xs, int M, int K, cudaStream_t st);
+// xs = fp16_rne(fp32(X) * inv_s); inverse_scale: inv_s = fp32(1 / s), correctly rounded
+cudaError_t launch_multiply_by_inverse(const void* X, const float* inv_s, void* xs, int M, int K, cudaStream_t st);
+cudaError_t launch_inverse_scale(const float* s, float* inv_s, int K, cudaStream_t st);
 cudaError_t launch_mean_squared_difference(const void* yq, const float* yref, size_t n, double* partials,
                                            float* out, cudaStream_t st);
 

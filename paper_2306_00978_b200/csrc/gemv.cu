@@ -158,6 +158,8 @@ template <int G, int TPW> struct BandStage {
 struct BandLayout {
     int stage_bytes, stages, xsum_off, red_off, bar_off, total;
     int red_tokens;                  // tokens per reduction buffer row block: 4 (M <= 4) or 8
+    int x_row, xg_off;               // x resident in shared memory: bytes per token row; offset of the
+                                     // per-group sums of x, fp32 [K / G][4 tokens], behind the rows
 };
 
 // Up to four weight matrices that share x, K and the group size (fused q/k/v or gate/up
@@ -192,22 +194,50 @@ __device__ __forceinline__ BandRef band_ref(const BandProblems& pr, int task) {
     return r;
 }
 template <int G, int TPW>
-inline BandLayout band_layout(int M, int K, bool x_in_registers) {
+inline BandLayout band_layout(int M, int K, bool x_in_registers, bool x_resident = false) {
     using St = BandStage<G, TPW>;
     BandLayout l;
-    l.stage_bytes = ((St::kXOff + (x_in_registers ? 0 : M * St::kXRow) + 127) / 128) * 128;
+    l.stage_bytes = ((St::kXOff + ((x_in_registers || x_resident) ? 0 : M * St::kXRow) + 127) / 128) * 128;
     // per-k-tile sums of x (+ one stage of slack for ragged reads); with x in registers the region
-    // is the math warps' staging block for x instead (16 warps x 512 bytes)
-    const int xsum = x_in_registers ? kMathWarps * 512 : (K / 64 + St::kUT) * 8 * 4;
+    // is the math warps' staging block for x instead (16 warps x 512 bytes); with x resident in
+    // shared memory it holds the M rows of x (padded against bank conflicts) and the group sums
+    l.x_row = K * 2 + 32;
+    l.xg_off = ((M * l.x_row + 127) / 128) * 128;
+    const int xsum = x_resident ? l.xg_off + (K / G) * 16
+                                : (x_in_registers ? kMathWarps * 512 : (K / 64 + St::kUT) * 8 * 4);
     l.red_tokens = M <= 4 ? 4 : 8;
     const int red = 6 * kMathWarps * l.red_tokens * 16 * 4;   // one buffer per stage of [warp][token][row] fp32
-    int s = (kSmemBudget - xsum - red - 256) / l.stage_bytes;
+    int s = (kSmemBudget - xsum - red - 256 - 128) / l.stage_bytes;
     l.stages = s > 6 ? 6 : s;
     l.xsum_off = l.stages * l.stage_bytes;
-    l.red_off = l.xsum_off + xsum;
+    l.red_off = ((l.xsum_off + xsum + 127) / 128) * 128;
     l.bar_off = l.red_off + red;
     l.total = l.bar_off + 256;
+    l.xg_off += l.xsum_off;
     return l;
+}
+
+// A read-only 16-byte load that stays where it is written (the compiler may otherwise sink a plain
+// load below the dependency wait, towards its first use).
+__device__ __forceinline__ float4 ld_const_f4(const float* p) {
+    float4 v;
+    asm volatile("ld.global.nc.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(p));
+    return v;
+}
+
+// Eight activations times their inverse channel scales: fp16_rne(fp32(x) * inv_s), one fp32
+// multiply and one rounding per element (the caller's side of Eq. 4, folded into the fetch of x).
+__device__ __forceinline__ uint4 scale8(const uint4& h, const float4& s0, const float4& s1) {
+    const float sv[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
+    const uint32_t w[4] = {h.x, h.y, h.z, h.w};
+    uint32_t o[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&w[e]));
+        const __half2 r = __floats2half2_rn(__fmul_rn(f.x, sv[2 * e]), __fmul_rn(f.y, sv[2 * e + 1]));
+        o[e] = *reinterpret_cast<const uint32_t*>(&r);
+    }
+    return make_uint4(o[0], o[1], o[2], o[3]);
 }
 
 // One full stage of one math warp: the warp's TPW k-tiles (GPW whole groups) of the band's 16
@@ -278,10 +308,17 @@ __device__ __forceinline__ void band_full_stage(const unsigned char* st, int o_w
 // XS: 0, or (XREG only) the number of stages of the ring, known at compile time together with
 // 4-token reduction rows: the loop over the bands is then unrolled over one turn of the ring and
 // every stage, barrier and reduction address is a constant.
-template <int G, int TPW, bool ONE, bool XREG, int XS>
+// XSM (not with XREG; M <= 4): x stays resident in shared memory for the whole launch instead of
+// travelling through the stages slice by slice: each math warp fetches, once, exactly the
+// columns it multiplies (the same k-tiles of every stage of every band) and forms their group
+// sums, so no x copy, no per-stage x bytes on the barriers and no block-wide barrier is needed.
+// sdiv: nullptr, or the inverse channel scales 1 / s (fp32 [K]): x is then multiplied by them while it
+// is fetched (XREG and XSM only), fp16_rne(fp32(x) * inv_s), which folds the caller's diag(s)^-1 into
+// this kernel.
+template <int G, int TPW, bool ONE, bool XREG, int XS, bool XSM = false>
 __global__ void __launch_bounds__(kBandThreads, 1)
 gemv_band_kernel(const BandProblems probs, const __half* __restrict__ x, int M, int K,
-                 const BandLayout lay, unsigned int* status_word) {
+                 const BandLayout lay, unsigned int* status_word, const float* __restrict__ sdiv) {
     extern __shared__ __align__(128) unsigned char smem[];
     __shared__ unsigned int s_abort;
     using St = BandStage<G, TPW>;
@@ -289,6 +326,7 @@ gemv_band_kernel(const BandProblems probs, const __half* __restrict__ x, int M, 
     constexpr int TPG = G / 64;                         // k-tiles per group
     constexpr int GPW = (TPW + TPG - 1) / TPG;          // groups touched by one warp in a stage
     static_assert(TPW % TPG == 0, "a warp's tiles must cover whole groups");
+    static_assert(!(XREG && XSM), "x lives either in registers or in shared memory");
     const int S = lay.stages;
     const uint32_t sbase = smem_u32(smem);
     // barriers: full[s] at 8s, empty[s] at 64 + 8s, flush_req[s] at 128 + 8s
@@ -329,7 +367,7 @@ gemv_band_kernel(const BandProblems probs, const __half* __restrict__ x, int M, 
     if (warp == kMathWarps + 2) {
         // ---------------------------------------------------------------- x-copy warp
         // lane m < M copies token m's slice of x for each stage (counted on the stage's barrier)
-        if (XREG) return;
+        if (XREG || XSM) return;
         asm volatile("griddepcontrol.wait;" ::: "memory");
         uint32_t stage = 0, phase = 0;
         for (int task = b0; task < b1; ++task) {
@@ -362,7 +400,7 @@ gemv_band_kernel(const BandProblems probs, const __half* __restrict__ x, int M, 
                 const uint32_t bar = bars + 8u * stage;
                 if (lane == 0) {
                     mbar_wait_relaxed(bars + 64u + 8u * stage, phase ^ 1u, ctl);
-                    mbar_arrive_expect_tx(bar, (uint32_t)(nt * 512 + ngr * 48 + (XREG ? 0 : M * nt * 128)));
+                    mbar_arrive_expect_tx(bar, (uint32_t)(nt * 512 + ngr * 48 + ((XREG || XSM) ? 0 : M * nt * 128)));
                 }
                 __syncwarp();
                 const int gi0 = kt * 64 / G;
@@ -387,6 +425,28 @@ gemv_band_kernel(const BandProblems probs, const __half* __restrict__ x, int M, 
         return;
     }
 
+    // the channel scales are constants of the layer like the weights: with x in registers a lane
+    // fetches the eight it needs before the dependency wait
+    // (x resident in shared memory: the scales of the first batch of stage positions)
+    constexpr int JB = ONE ? 4 : 2;                              // stage positions fetched per batch
+    float4 sd0 = make_float4(1.0f, 1.0f, 1.0f, 1.0f), sd1 = sd0;
+    float4 sa[XSM ? JB : 1], sb[XSM ? JB : 1];
+    if (XREG && sdiv != nullptr && warp < kMathWarps) {
+        sd0 = ld_const_f4(sdiv + warp * (TPW * 64) + lane * 8);
+        sd1 = ld_const_f4(sdiv + warp * (TPW * 64) + lane * 8 + 4);
+    }
+    if (XSM && warp < kMathWarps) {
+#pragma unroll
+        for (int jj = 0; jj < JB; ++jj) {
+            const int col = (jj * UT + warp * TPW) * 64 + lane * 8;
+            sa[jj] = make_float4(1.0f, 1.0f, 1.0f, 1.0f);
+            sb[jj] = sa[jj];
+            if (sdiv != nullptr && jj < upb && lane * 8 < TPW * 64 && col < K) {
+                sa[jj] = ld_const_f4(sdiv + col);
+                sb[jj] = ld_const_f4(sdiv + col + 4);
+            }
+        }
+    }
     asm volatile("griddepcontrol.wait;" ::: "memory");
     float* xsum = reinterpret_cast<float*>(smem + lay.xsum_off);
 
@@ -460,6 +520,11 @@ gemv_band_kernel(const BandProblems probs, const __half* __restrict__ x, int M, 
 #pragma unroll
                 for (int i = 0; i < 4; ++i)
                     if (m0 + i < M) row[i] = __ldg(xrow + (size_t)(m0 + i) * (K / 8));
+                if (sdiv != nullptr) {
+#pragma unroll
+                    for (int i = 0; i < 4; ++i)
+                        if (m0 + i < M) row[i] = scale8(row[i], sd0, sd1);
+                }
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
                     if (m0 + i < M) {
@@ -500,6 +565,64 @@ gemv_band_kernel(const BandProblems probs, const __half* __restrict__ x, int M, 
             XxR[q] = __shfl_sync(0xFFFFFFFFu, part, 8 * t);
             XyR[q] = __shfl_sync(0xFFFFFFFFu, part, 8 * t + 4);
         }
+    } else if (XSM) {
+        // This warp's columns of x - TPW k-tiles at the same place of every stage of a band - from
+        // global memory into the resident rows, scaled by 1 / s on the way if asked, and the sums
+        // over each group (G / 8 lanes) into the table (times 2^-24: the products carry that
+        // factor).  Nobody else reads these columns, so a warp-level barrier is enough.
+        constexpr int LPG = G / 8;                              // lanes per group
+        constexpr int MT = ONE ? 1 : 4;
+        unsigned char* xb = smem + lay.xsum_off;
+        float* xg = reinterpret_cast<float*>(smem + lay.xg_off);
+        for (int j0 = 0; j0 < upb; j0 += JB) {
+            uint4 v[JB][MT];
+#pragma unroll
+            for (int jj = 0; jj < JB; ++jj) {
+                const int col = ((j0 + jj) * UT + warp * TPW) * 64 + lane * 8;
+                const bool valid = j0 + jj < upb && lane * 8 < TPW * 64 && col < K;
+                if (j0 > 0 && valid && sdiv != nullptr) {        // (the first batch's scales are there already)
+                    sa[jj] = ld_const_f4(sdiv + col);
+                    sb[jj] = ld_const_f4(sdiv + col + 4);
+                }
+#pragma unroll
+                for (int m = 0; m < MT; ++m) {
+                    v[jj][m] = make_uint4(0u, 0u, 0u, 0u);
+                    if (valid && m < M) v[jj][m] = __ldg(reinterpret_cast<const uint4*>(x + (size_t)m * K + col));
+                }
+            }
+#pragma unroll
+            for (int jj = 0; jj < JB; ++jj) {
+                const int col = ((j0 + jj) * UT + warp * TPW) * 64 + lane * 8;
+                const bool valid = j0 + jj < upb && lane * 8 < TPW * 64 && col < K;   // the same for all lanes of a group
+                float sum[MT];
+#pragma unroll
+                for (int m = 0; m < MT; ++m) {
+                    if (valid && m < M) {
+                        if (sdiv != nullptr) v[jj][m] = scale8(v[jj][m], sa[jj], sb[jj]);
+                        *reinterpret_cast<uint4*>(xb + m * lay.x_row + col * 2) = v[jj][m];
+                    }
+                    const uint32_t u[4] = {v[jj][m].x, v[jj][m].y, v[jj][m].z, v[jj][m].w};
+                    sum[m] = 0.0f;
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&u[e]));
+                        sum[m] += f.x + f.y;
+                    }
+#pragma unroll
+                    for (int off = LPG / 2; off >= 1; off >>= 1) sum[m] += __shfl_xor_sync(0xFFFFFFFFu, sum[m], off);
+                }
+                if (valid && (lane & (LPG - 1)) == 0) {
+                    float4 o = make_float4(sum[0] * (1.0f / 16777216.0f), 0.0f, 0.0f, 0.0f);
+                    if constexpr (!ONE) {
+                        o.y = sum[1] * (1.0f / 16777216.0f);
+                        o.z = sum[2] * (1.0f / 16777216.0f);
+                        o.w = sum[3] * (1.0f / 16777216.0f);
+                    }
+                    *reinterpret_cast<float4*>(xg + (col / G) * 4) = o;
+                }
+            }
+        }
+        __syncwarp();
     } else {
         // x sums per k-tile (the 16 math warps), while the first stages are in flight.  (Deferring
         // them behind the first stage's products, and polling barriers ahead of use, were both
@@ -578,17 +701,28 @@ gemv_band_kernel(const BandProblems probs, const __half* __restrict__ x, int M, 
             mbar_wait(bars + 8u * stage, phase, ctl);
             const unsigned char* st = smem + stage * (uint32_t)lay.stage_bytes;
             const float* xs = xs_lane + j * (UT * 8);
+            // x resident: this lane's fragments and its two tokens' group sums at stage position j
+            const unsigned char* xres = smem + lay.xsum_off + g * lay.x_row + ((j * UT + warp * TPW) * 64 + t * 4) * 2;
+            const float* xgs = reinterpret_cast<const float*>(smem + lay.xg_off) +
+                               ((j * UT + warp * TPW) * 64 / G) * 4 + 2 * (t & 1);
+            const unsigned char* xfrag = XSM ? xres : st + o_x;
             if (nt >= TPW) {
                 if (tok_ok) {
 #pragma unroll
                     for (int v = 0; v < TPW; ++v)
 #pragma unroll
                         for (int jw = 0; jw < 4; ++jw)
-                            xr[v][jw] = *reinterpret_cast<const uint2*>(st + o_x + v * 128 + jw * 32);
+                            xr[v][jw] = *reinterpret_cast<const uint2*>(xfrag + v * 128 + jw * 32);
                 }
                 float Kx[GPW], Ky[GPW];
 #pragma unroll
                 for (int q = 0; q < GPW; ++q) {
+                    if (XSM) {
+                        const float2 X = *reinterpret_cast<const float2*>(xgs + q * 4);
+                        Kx[q] = X.x;
+                        Ky[q] = X.y;
+                        continue;
+                    }
                     float Xx = 0.0f, Xy = 0.0f;
 #pragma unroll
                     for (int v = 0; v < TPG; ++v) {
@@ -615,11 +749,19 @@ gemv_band_kernel(const BandProblems probs, const __half* __restrict__ x, int M, 
                             if (tok_ok) {
 #pragma unroll
                                 for (int jw = 0; jw < 4; ++jw)
-                                    xq[0][jw] = *reinterpret_cast<const uint2*>(st + o_x + tile * 128 + jw * 32);
+                                    xq[0][jw] = *reinterpret_cast<const uint2*>(xfrag + tile * 128 + jw * 32);
                             }
-                            const float2 X = *reinterpret_cast<const float2*>(xs + tile * 8);
-                            Xx += X.x;
-                            Xy += X.y;
+                            if (XSM) {
+                                if (v == 0) {                      // the table holds 2^-24 times the group's sums
+                                    const float2 X = *reinterpret_cast<const float2*>(xgs + q * 4);
+                                    Xx = X.x * 16777216.0f;
+                                    Xy = X.y * 16777216.0f;
+                                }
+                            } else {
+                                const float2 X = *reinterpret_cast<const float2*>(xs + tile * 8);
+                                Xx += X.x;
+                                Xy += X.y;
+                            }
                             if (v == 0) block_mma<1, 2, true>(pk, xq, c);
                             else block_mma<1, 2, false>(pk, xq, c);
                         }
@@ -1036,8 +1178,21 @@ cudaError_t gemv_static_scratch(void** out) {
     return cudaSuccess;
 }
 
+// Whether the band kernel can take x unscaled and fold the multiplication by 1 / s into
+// its fetch of x (x in registers, or x resident in shared memory).
+bool gemv_band_folds_scale(int M, int K, int group) {
+    if (K == 64 * 16 * 4) return true;                          // x in registers, any M <= 8
+    // x resident in shared memory: measured faster than x through the stages for one and two
+    // tokens (7.7 against 7.9 us on 11008 -> 4096, 23.9 against 24.8 us on 8192 -> 28672 at M = 1),
+    // slower for three and four (two k-tiles per warp and stage), so it is built for M <= 2
+    if (M > 2) return false;
+    const BandLayout l = group == 128 ? band_layout<128, 4>(M, K, false, true) : band_layout<64, 4>(M, K, false, true);
+    return l.stages >= 4;
+}
+
 cudaError_t launch_gemv_band(const void* x, const GemvMatrix* mats, int count, int M, int K, int group,
-                             unsigned int* status_word, int sms, bool serialize, cudaStream_t st) {
+                             unsigned int* status_word, int sms, bool serialize, cudaStream_t st,
+                             const float* sdiv) {
     BandProblems pr;
     pr.count = count;
     int bands = 0;
@@ -1069,25 +1224,32 @@ cudaError_t launch_gemv_band(const void* x, const GemvMatrix* mats, int count, i
     cfg.stream = st;
     cfg.attrs = attr;
     cfg.numAttrs = serialize ? 0 : 1;
+    const __half* xh = reinterpret_cast<const __half*>(x);
+#define AWQ_BAND_GO(KERNEL, LAY)                                                                     \
+    do {                                                                                             \
+        static bool done[64] = {};                                                                   \
+        cfg.dynamicSmemBytes = (LAY).total;                                                          \
+        e = allow_big_smem(KERNEL, done);                                                            \
+        if (e != cudaSuccess) return e;                                                              \
+        e = cudaLaunchKernelEx(&cfg, KERNEL, pr, xh, M, K, LAY, status_word, sdiv);                  \
+        if (e != cudaSuccess) return e;                                                              \
+    } while (0)
 #define AWQ_BAND_LAUNCH(GG, TT, ONE1, XR)                                                            \
     do {                                                                                             \
         const BandLayout lay = band_layout<GG, TT>(M, K, XR);                                        \
-        if (lay.stages < 2) return cudaErrorInvalidValue;      /* K too large for the x-sum table */ \
-        static bool done[64] = {};                                                                   \
-        cfg.dynamicSmemBytes = lay.total;                                                            \
+        const BandLayout layr = band_layout<GG, TT>(M, K, false, true);                              \
         if (XR && lay.stages == 5 && lay.red_tokens == 4) {                                          \
-            static bool done5[64] = {};                                                              \
-            e = allow_big_smem(gemv_band_kernel<GG, TT, ONE1, XR, (XR ? 5 : 0)>, done5);             \
-            if (e != cudaSuccess) return e;                                                          \
-            e = cudaLaunchKernelEx(&cfg, gemv_band_kernel<GG, TT, ONE1, XR, (XR ? 5 : 0)>, pr,       \
-                                   reinterpret_cast<const __half*>(x), M, K, lay, status_word);      \
+            AWQ_BAND_GO((gemv_band_kernel<GG, TT, ONE1, XR, (XR ? 5 : 0), false>), lay);             \
+        } else if (XR) {                                                                             \
+            if (lay.stages < 2) return cudaErrorInvalidValue;                                        \
+            AWQ_BAND_GO((gemv_band_kernel<GG, TT, ONE1, XR, 0, false>), lay);                        \
+        } else if (M <= 2 && layr.stages >= 4) {                                                     \
+            AWQ_BAND_GO((gemv_band_kernel<GG, TT, ONE1, false, 0, !XR>), layr);                      \
         } else {                                                                                     \
-            e = allow_big_smem(gemv_band_kernel<GG, TT, ONE1, XR, 0>, done);                         \
-            if (e != cudaSuccess) return e;                                                          \
-            e = cudaLaunchKernelEx(&cfg, gemv_band_kernel<GG, TT, ONE1, XR, 0>, pr,                  \
-                                   reinterpret_cast<const __half*>(x), M, K, lay, status_word);      \
+            if (lay.stages < 2) return cudaErrorInvalidValue;  /* K too large for the x-sum table */ \
+            if (sdiv != nullptr) return cudaErrorInvalidValue; /* callers ask gemv_band_folds_scale */ \
+            AWQ_BAND_GO((gemv_band_kernel<GG, TT, ONE1, false, 0, false>), lay);                     \
         }                                                                                            \
-        if (e != cudaSuccess) return e;                                                              \
     } while (0)
     const bool xreg = tpw == 4 && K == 64 * 16 * 4;            // a band is exactly one stage
 #define AWQ_BAND_PICK(GG)                                                                            \
@@ -1101,6 +1263,7 @@ cudaError_t launch_gemv_band(const void* x, const GemvMatrix* mats, int count, i
     if (group == 128) AWQ_BAND_PICK(128); else AWQ_BAND_PICK(64);
 #undef AWQ_BAND_PICK
 #undef AWQ_BAND_LAUNCH
+#undef AWQ_BAND_GO
     count_launch();
     return cudaGetLastError();
 }

@@ -34,6 +34,29 @@ __global__ void divide_by_scale_kernel(const __half* __restrict__ X, const float
     reinterpret_cast<uint4*>(xs)[i] = make_uint4(o[0], o[1], o[2], o[3]);
 }
 
+// xs[m][k] = fp16_rne(fp32(X[m][k]) * inv_s[k]): what awq_linear_scaled computes inside the layer,
+// as a kernel of its own for the shapes whose kernel cannot fold it.
+__global__ void multiply_by_inverse_kernel(const __half* __restrict__ X, const float* __restrict__ inv_s,
+                                           __half* __restrict__ xs, size_t chunks, int K) {
+    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= chunks) return;
+    const int k0 = (int)((i * 8) % (size_t)K);
+    const uint4 h = reinterpret_cast<const uint4*>(X)[i];
+    const uint32_t w[4] = {h.x, h.y, h.z, h.w};
+    uint32_t o[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&w[e]));
+        const __half2 r = __floats2half2_rn(__fmul_rn(f.x, inv_s[k0 + 2 * e]), __fmul_rn(f.y, inv_s[k0 + 2 * e + 1]));
+        o[e] = *reinterpret_cast<const uint32_t*>(&r);
+    }
+    reinterpret_cast<uint4*>(xs)[i] = make_uint4(o[0], o[1], o[2], o[3]);
+}
+__global__ void inverse_scale_kernel(const float* __restrict__ s, float* __restrict__ inv_s, int K) {
+    const int k = blockIdx.x * blockDim.x + threadIdx.x;
+    if (k < K) inv_s[k] = __frcp_rn(s[k]);
+}
+
 // Sum of (y_q - y_ref)^2: every block adds a fixed, interleaved share of the elements in fp64
 // and the last kernel adds the blocks' sums in block order, so the loss is reproducible.
 __global__ void __launch_bounds__(256)
@@ -205,6 +228,20 @@ cudaError_t launch_divide_by_scale(const void* X, const float* s, void* xs, int 
     const size_t chunks = (size_t)M * K / 8;
     divide_by_scale_kernel<<<(unsigned)((chunks + 255) / 256), 256, 0, st>>>(
         reinterpret_cast<const __half*>(X), s, reinterpret_cast<__half*>(xs), chunks, K);
+    count_launch();
+    return cudaGetLastError();
+}
+
+cudaError_t launch_multiply_by_inverse(const void* X, const float* inv_s, void* xs, int M, int K, cudaStream_t st) {
+    const size_t chunks = (size_t)M * K / 8;
+    multiply_by_inverse_kernel<<<(unsigned)((chunks + 255) / 256), 256, 0, st>>>(
+        reinterpret_cast<const __half*>(X), inv_s, reinterpret_cast<__half*>(xs), chunks, K);
+    count_launch();
+    return cudaGetLastError();
+}
+
+cudaError_t launch_inverse_scale(const float* s, float* inv_s, int K, cudaStream_t st) {
+    inverse_scale_kernel<<<(K + 255) / 256, 256, 0, st>>>(s, inv_s, K);
     count_launch();
     return cudaGetLastError();
 }
