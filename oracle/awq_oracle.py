@@ -221,6 +221,55 @@ def unpack_qweight(words, N: int, K: int) -> np.ndarray:
     return a.transpose(0, 6, 2, 1, 4, 3, 5, 7).reshape(N, K)
 
 
+# ------------------------------------------------------------- 3-bit storage (INT3-g128 setting)
+def int3_location(n: int, k: int, K: int):
+    """Where the three bits of code (n, k) sit in the 3-bit array: [(word index, bit), ...] for
+    bit 0, 1, 2 of the code.
+
+    The paper's INT3 tables need codes of 3 bits; it does not describe a storage, this is the
+    layout used.  Blocks, bands and pieces are those of the 4-bit layout, but a piece is three
+    words instead of four: block (band, k // 64) is 96 words at (band * (K // 64) + k // 64) * 96,
+    piece (g, t) at word 3 * (4 g + t) of it.  With (j, p) the word and nibble that
+    `qweight_location` gives inside the piece: for j < 3 the code keeps its place, bits
+    4p .. 4p+2 of word j; for j = 3 (columns 48 .. 63 of the block) bit b of the code sits in the
+    spare top bit of nibble p of word b, i.e. bit 4p+3 of word b.
+    """
+    word4, p = qweight_location(n, k, K)
+    block, in_block = divmod(word4, WORDS_PER_BLOCK)
+    piece, j = divmod(in_block, 4)
+    base = block * 96 + piece * 3
+    if j < 3:
+        return [(base + j, 4 * p + b) for b in range(3)]
+    return [(base + b, 4 * p + 3) for b in range(3)]
+
+
+def pack_qweight_int3(codes) -> np.ndarray:
+    """codes u8 [N][K], all < 8 -> uint32 [N*K*3/32] in the layout of `int3_location`: of the four
+    nibble words w0 .. w3 of every 16-byte piece of the 4-bit layout, word b (b = 0, 1, 2) takes
+    bit b of w3's nibbles into the spare top bits of its own."""
+    codes = np.asarray(codes, dtype=np.uint8)
+    assert codes.max(initial=0) < 8
+    w = pack_qweight(codes).reshape(-1, 4)
+    out = np.empty((w.shape[0], 3), dtype=np.uint32)
+    ones = np.uint32(0x11111111)
+    for b in range(3):
+        out[:, b] = w[:, b] | (((w[:, 3] >> np.uint32(b)) & ones) << np.uint32(3))
+    return out.reshape(-1)
+
+
+def unpack_qweight_int3(words3, N: int, K: int) -> np.ndarray:
+    """Inverse of pack_qweight_int3."""
+    u = np.asarray(words3, dtype=np.uint32).reshape(-1, 3)
+    assert u.size == N * K * 3 // 32
+    w = np.empty((u.shape[0], 4), dtype=np.uint32)
+    ones, low = np.uint32(0x11111111), np.uint32(0x77777777)
+    w[:, 3] = 0
+    for b in range(3):
+        w[:, b] = u[:, b] & low
+        w[:, 3] |= ((u[:, b] >> np.uint32(3)) & ones) << np.uint32(b)
+    return unpack_qweight(w.reshape(-1), N, K)
+
+
 def pack_zeros(zeros) -> np.ndarray:
     """zeros u8 [N][ng] -> u8 [N/32][ng][16] in the layout of `zeros_location`."""
     zeros = np.asarray(zeros, dtype=np.uint8)

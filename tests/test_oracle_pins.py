@@ -197,7 +197,7 @@ def test_pack_matches_location_formula_and_round_trips():
 
 
 def _layout_table(golden_dir):
-    rows = {"qweight": [], "zeros": [], "scales": []}
+    rows = {"qweight": [], "zeros": [], "scales": [], "int3": []}
     with open(os.path.join(golden_dir, "packed_layout.txt")) as f:
         for line in f:
             line = line.strip()
@@ -250,6 +250,38 @@ def test_packed_layout_against_hand_derived_table(golden_dir):
         sc[n, gi] = 1.0
         raw = orc.pack_scales(sc).reshape(-1)
         assert raw[idx] == 1.0 and np.count_nonzero(raw) == 1, (n, gi)
+
+
+def test_int3_storage_against_hand_derived_table_and_round_trip(golden_dir):
+    t = _layout_table(golden_dir)
+    assert len(t["int3"]) >= 10
+    for (n, k, K, *pos) in t["int3"]:
+        want = [(pos[2 * b], pos[2 * b + 1]) for b in range(3)]              # (byte, bit in byte)
+        got = [(4 * w + bit // 8, bit % 8) for (w, bit) in orc.int3_location(n, k, K)]
+        assert got == want, (n, k)
+        N = 16 * (n // 16 + 1)
+        for b in range(3):                                                   # one code bit at a time
+            codes = np.zeros((N, K), np.uint8)
+            codes[n, k] = 1 << b
+            raw = orc.pack_qweight_int3(codes).astype("<u4").view(np.uint8)
+            expect = np.zeros_like(raw)
+            expect[want[b][0]] = 1 << want[b][1]
+            assert np.array_equal(raw, expect), (n, k, b)
+    rng = np.random.default_rng(11)
+    for N, K in [(128, 64), (256, 192)]:
+        codes = rng.integers(0, 8, size=(N, K), dtype=np.uint8)
+        words = orc.pack_qweight_int3(codes)
+        assert words.size == N * K * 3 // 32                                 # 3/8 byte per weight
+        assert np.array_equal(orc.unpack_qweight_int3(words, N, K), codes)
+        ref = [0] * words.size
+        seen = set()
+        for n in range(N):
+            for k in range(K):
+                for b, (w, bit) in enumerate(orc.int3_location(n, k, K)):
+                    assert (w, bit) not in seen
+                    seen.add((w, bit))
+                    ref[w] |= ((int(codes[n, k]) >> b) & 1) << bit
+        assert words.tolist() == ref
 
 
 def test_zero_and_scale_packing():
