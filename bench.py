@@ -704,6 +704,61 @@ def config4_section(peaks):
     return rows
 
 
+def int3_section(peaks):
+    """The layer on the 3-bit storage (band matrix-vector kernel, M = 1) next to the same shapes on
+    the 4-bit layout: microseconds, algorithmic GB/s of each and the bytes saved."""
+    import torch
+    from paper_2306_00978_b200 import binding
+    out = []
+    for (K, N) in ((4096, 11008), (8192, 28672)):
+        l2 = torch.cuda.get_device_properties(torch.cuda.current_device()).L2_cache_size
+        b3 = N * K * 3 // 8 + (N * K // GROUP) * 2 + (N * K // GROUP) // 2
+        n = max(3, -(-2 * l2 // b3) + 1)
+        copies = []
+        for _ in range(n):
+            q3 = torch.randint(0, 256, (N * K * 3 // 8,), dtype=torch.uint8, device="cuda")
+            sc = (torch.rand((N // 16, K // GROUP, 16), device="cuda") * 0.01 + 0.001).half()
+            zp = torch.randint(0, 120, (N // 32, K // GROUP, 16), dtype=torch.uint8, device="cuda")
+            copies.append((q3, sc, zp))
+        x = torch.randn((1, K), device="cuda").half()
+        y = torch.empty((1, N), device="cuda", dtype=torch.float16)
+        scratch = torch.empty(16, dtype=torch.uint8, device="cuda")
+        for i in range(3):
+            binding.linear_int3(x, *copies[i], N, K, GROUP, out=y, scratch=scratch)
+        torch.cuda.synchronize()
+        g, side = torch.cuda.CUDAGraph(), torch.cuda.Stream()
+        calls = max(8, n)
+        with torch.cuda.stream(side):
+            with torch.cuda.graph(g, stream=side):
+                for i in range(calls):
+                    binding.linear_int3(x, *copies[i % n], N, K, GROUP, out=y, scratch=scratch)
+        torch.cuda.synchronize()
+        g.replay()
+        ts = []
+        for _ in range(5):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            g.replay()
+            e1.record()
+            torch.cuda.synchronize()
+            ts.append(e0.elapsed_time(e1) * 1e3 / calls)
+        binding.poll_status()
+        us3 = statistics.median(ts)
+        del copies, g
+        torch.cuda.empty_cache()
+        rp = RandomPacked(N, K, GROUP)
+        _, us4 = rp.time_chained(1)
+        del rp
+        torch.cuda.empty_cache()
+        bytes3 = b3 + 2 * K + 2 * N
+        bytes4 = algorithmic_bytes(N, K, 1)
+        out.append({"shape": f"{K}->{N}", "M": 1, "int3_us": round(us3, 2), "int3_GBps": round(bytes3 / us3 / 1e3, 1),
+                    "int3_frac_hbm_measured": round(bytes3 / us3 / 1e3 / peaks["hbm_gbs"], 4),
+                    "int4_us": round(us4, 2), "int4_GBps": round(bytes4 / us4 / 1e3, 1),
+                    "bytes_int3": bytes3, "bytes_int4": bytes4, "bytes_saved_frac": round(1 - bytes3 / bytes4, 4)})
+    return out
+
+
 SWEEP_SHAPES = (("q/k/v/o", 4096, 4096), ("gate/up", 4096, 11008), ("down", 11008, 4096))
 SWEEP_M = (1, 2, 4, 8, 16, 32, 64, 128, 512, 2048, 8192)
 
@@ -868,6 +923,7 @@ def main():
                                  "note": "awq_linear, automatic dispatch, best of 3 graph replays; cold-L2 rotation "
                                          "for M <= 128; alpha does not enter the run time"}
         torch.cuda.empty_cache()
+        line["int3_storage"] = int3_section(peaks)
         line["quantize_pack"] = quantize_section(peaks)
         line["alpha_search"] = search_section()
         line["clip_search"] = clip_section()

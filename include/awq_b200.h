@@ -218,6 +218,32 @@ int awq_linear_multi_scaled(const void* x, const float* inv_s, void* x_scratch, 
 int awq_inverse_channel_scale(const float* act_mean_abs, float alpha, float* inv_s, int K, void* stream);
 int awq_linear_scaled_needs_scratch(int M, int N, int K, int group);
 
+/*
+ * 3-bit storage (the INT3-g128 setting of the paper's accuracy tables; the paper does not describe
+ * how its kernels would store 3-bit codes, this is the layout used).  awq_quantize_pack_ex with
+ * bits = 3 writes 3-bit codes into the 4-bit layout; awq_pack_int3 turns that array into the
+ * dense one of 3/8 byte per weight, awq_unpack_int3 back:
+ *  qweight3: N*K*3/8 bytes.  Bands, blocks and pieces are those of the 4-bit layout, but a block
+ *    (band, kt) is 384 bytes at ((n/16)*(K/64) + k/64) * 384 and piece 4*g + t is 12 bytes = three
+ *    little-endian words at byte 12*(4*g + t) of the block.  Let (j, p) be the word and the nibble
+ *    that the 4-bit layout gives code (n,k) inside its piece (j = (k%64)/16, p from the slot table
+ *    above).  For j < 3 the code keeps its place: bits 4p .. 4p+2 of word j.  For j = 3 (columns
+ *    48..63 of the block) bit b of the code (b = 0, 1, 2) sits in the spare top bit of nibble p of
+ *    word b: bit 4p+3 of word b.  In words: u_b = w_b | (((w_3 >> b) & 0x11111111) << 3).
+ *  scales and zeros are unchanged.
+ * awq_linear_int3: the layer on that storage.  Where the band matrix-vector kernel serves the call
+ * (M <= 8 and N / 16 not far below the SM count) it streams the 3-bit array itself, 25 % fewer
+ * weight bytes than the 4-bit layout; other shapes (split-K and tensor-core kernels read the
+ * 4-bit layout) are first expanded into qweight_scratch (device, awq_qweight_bytes(N, K) bytes,
+ * caller-owned; may be NULL when the band kernel applies, else AWQ_ERR_NULL_POINTER) and run as
+ * awq_linear.  Results equal awq_linear on the expanded array bit for bit where the same kernel runs.
+ */
+size_t awq_qweight_bytes_int3(int N, int K);
+int awq_pack_int3(const void* qweight, void* qweight3, int N, int K, void* stream);
+int awq_unpack_int3(const void* qweight3, void* qweight, int N, int K, void* stream);
+int awq_linear_int3(const void* x, const void* qweight3, const void* scales, const void* zeros, void* y,
+                    void* qweight_scratch, int M, int N, int K, int group, void* stream);
+
 /* Same as awq_linear with the kernel forced (for the small-batch crossover measurement).
  * A matrix-vector path with M > 16 or K > 65536 returns AWQ_ERR_BAD_SHAPE. */
 int awq_linear_path(const void* x, const void* qweight, const void* scales, const void* zeros,

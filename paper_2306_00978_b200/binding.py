@@ -27,7 +27,7 @@ EXPORTS = (
     "awq_quantize_pack_ex", "awq_search_clip", "awq_static_scratch_fill",
     "awq_set_wait_limit_us", "awq_test_stall_next_gemv",
     "awq_linear_scaled", "awq_linear_multi_scaled", "awq_linear_scaled_needs_scratch",
-    "awq_inverse_channel_scale",
+    "awq_inverse_channel_scale", "awq_qweight_bytes_int3", "awq_pack_int3", "awq_unpack_int3", "awq_linear_int3",
 )
 
 
@@ -68,6 +68,10 @@ def lib() -> ctypes.CDLL:
     L.awq_linear_scaled.restype, L.awq_linear_scaled.argtypes = i, [vp, vp, vp, vp, vp, vp, vp, i, i, i, i, vp]
     L.awq_linear_multi_scaled.restype, L.awq_linear_multi_scaled.argtypes = i, [vp, vp, vp, vp, i, i, i, i, vp]
     L.awq_inverse_channel_scale.restype, L.awq_inverse_channel_scale.argtypes = i, [vp, f, vp, i, vp]
+    L.awq_qweight_bytes_int3.restype, L.awq_qweight_bytes_int3.argtypes = sz, [i, i]
+    L.awq_pack_int3.restype, L.awq_pack_int3.argtypes = i, [vp, vp, i, i, vp]
+    L.awq_unpack_int3.restype, L.awq_unpack_int3.argtypes = i, [vp, vp, i, i, vp]
+    L.awq_linear_int3.restype, L.awq_linear_int3.argtypes = i, [vp, vp, vp, vp, vp, vp, i, i, i, i, vp]
     L.awq_linear_scaled_needs_scratch.restype, L.awq_linear_scaled_needs_scratch.argtypes = i, [i, i, i, i]
     L.awq_linear_multi.restype, L.awq_linear_multi.argtypes = i, [vp, vp, i, i, i, i, vp]
     L.awq_search_scratch_bytes.restype, L.awq_search_scratch_bytes.argtypes = sz, [i, i, i, i]
@@ -253,6 +257,37 @@ def linear_multi_scaled(x: torch.Tensor, inv_s: torch.Tensor, mats, K: int, grou
                                        ctypes.byref(arr), len(mats), M, K, int(group), _stream())
     _check(rc, "awq_linear_multi_scaled")
     return outs
+
+
+def pack_int3(qweight: torch.Tensor, N: int, K: int) -> torch.Tensor:
+    """awq_pack_int3: the 4-bit layout holding 3-bit codes -> the 3-bit storage (u8 [N*K*3/8])."""
+    out = torch.empty(int(lib().awq_qweight_bytes_int3(N, K)), dtype=torch.uint8, device=qweight.device)
+    _check(lib().awq_pack_int3(_dev(qweight, torch.uint8, "qweight"), out.data_ptr(), N, K, _stream()), "awq_pack_int3")
+    return out
+
+
+def unpack_int3(qweight3: torch.Tensor, N: int, K: int) -> torch.Tensor:
+    out = torch.empty(N * K // 2, dtype=torch.uint8, device=qweight3.device)
+    _check(lib().awq_unpack_int3(_dev(qweight3, torch.uint8, "qweight3"), out.data_ptr(), N, K, _stream()),
+           "awq_unpack_int3")
+    return out
+
+
+def linear_int3(x: torch.Tensor, qweight3: torch.Tensor, scales: torch.Tensor, zeros: torch.Tensor,
+                N: int, K: int, group: int, out: Optional[torch.Tensor] = None,
+                scratch: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """awq_linear_int3: the layer on the 3-bit storage (`scratch`, N*K/2 bytes, is allocated here
+    when the shape needs the expansion and none is given)."""
+    M = x.shape[0]
+    y = out if out is not None else torch.empty((M, N), dtype=torch.float16, device=x.device)
+    ensure_workspace(workspace_bytes(M, N, K, group))
+    if scratch is None:
+        scratch = torch.empty(N * K // 2, dtype=torch.uint8, device=x.device)
+    rc = lib().awq_linear_int3(_dev(x, torch.float16, "x"), _dev(qweight3, torch.uint8, "qweight3"),
+                               _dev(scales, torch.float16, "scales"), _dev(zeros, torch.uint8, "zeros"),
+                               _dev(y, torch.float16, "y"), scratch.data_ptr(), M, N, K, int(group), _stream())
+    _check(rc, "awq_linear_int3")
+    return y
 
 
 def linear_gemv_static(x: torch.Tensor, qweight: torch.Tensor, scales: torch.Tensor, zeros: torch.Tensor,

@@ -386,6 +386,58 @@ int awq_linear_scaled(const void* x, const float* inv_s, void* x_scratch, const 
     return awq_linear_multi_scaled(x, inv_s, x_scratch, &one, 1, M, K, group, stream);
 }
 
+// ---- 3-bit storage
+size_t awq_qweight_bytes_int3(int N, int K) {
+    return check_shape(N, K, 128) == AWQ_OK ? (size_t)N * K / 8 * 3 : 0;
+}
+
+int awq_pack_int3(const void* qweight, void* qweight3, int N, int K, void* stream) {
+    if (int rc = check_shape(N, K, 128)) return rc;
+    if (!qweight || !qweight3) return AWQ_ERR_NULL_POINTER;
+    if (!aligned16(qweight) || !aligned16(qweight3)) return AWQ_ERR_MISALIGNED;
+    DeviceState* d;
+    if (int rc = device_state(&d)) return rc;
+    {
+        std::lock_guard<std::mutex> lock(g_mutex);
+        d->packed_written = true;
+    }
+    return note_cuda(launch_pack_int3(qweight, qweight3, N, K, (cudaStream_t)stream));
+}
+
+int awq_unpack_int3(const void* qweight3, void* qweight, int N, int K, void* stream) {
+    if (int rc = check_shape(N, K, 128)) return rc;
+    if (!qweight || !qweight3) return AWQ_ERR_NULL_POINTER;
+    if (!aligned16(qweight) || !aligned16(qweight3)) return AWQ_ERR_MISALIGNED;
+    DeviceState* d;
+    if (int rc = device_state(&d)) return rc;
+    {
+        std::lock_guard<std::mutex> lock(g_mutex);
+        d->packed_written = true;
+    }
+    return note_cuda(launch_unpack_int3(qweight3, qweight, N, K, (cudaStream_t)stream));
+}
+
+int awq_linear_int3(const void* x, const void* qweight3, const void* scales, const void* zeros, void* y,
+                    void* qweight_scratch, int M, int N, int K, int group, void* stream) {
+    if (int rc = check_shape(N, K, group)) return rc;
+    if (M < 1 || (long long)M * K > (1LL << 40) || (long long)M * N > (1LL << 40)) return AWQ_ERR_BAD_SHAPE;
+    if (!x || !qweight3 || !scales || !zeros || !y) return AWQ_ERR_NULL_POINTER;
+    if (!aligned16(x) || !aligned16(qweight3) || !aligned16(scales) || !aligned16(zeros) || !aligned16(y) ||
+        !aligned16(qweight_scratch))
+        return AWQ_ERR_MISALIGNED;
+    DeviceState* d;
+    if (int rc = device_state(&d)) return rc;
+    if (M <= 8 && K <= 65536 && gemv_uses_band_kernel(M, N, d->sms)) {
+        const GemvMatrix one = {qweight3, scales, zeros, y, N};
+        return note_cuda(launch_gemv_band(x, &one, 1, M, K, group, d->status_word, d->sms,
+                                          take_packed_written(d), (cudaStream_t)stream, nullptr, 3));
+    }
+    // every other kernel reads the 4-bit layout: expand first (one more launch), then the plain call
+    if (!qweight_scratch) return AWQ_ERR_NULL_POINTER;
+    if (int rc = awq_unpack_int3(qweight3, qweight_scratch, N, K, stream)) return rc;
+    return awq_linear(x, qweight_scratch, scales, zeros, y, M, N, K, group, stream);
+}
+
 int awq_inverse_channel_scale(const float* act_mean_abs, float alpha, float* inv_s, int K, void* stream) {
     if (int rc = awq_channel_scale(act_mean_abs, alpha, inv_s, K, stream)) return rc;
     return note_cuda(launch_inverse_scale(inv_s, inv_s, K, (cudaStream_t)stream));

@@ -40,6 +40,10 @@ cudaError_t launch_unpack(const uint32_t* qweight, const __half* scales, const u
                           int N, int K, int group, uint8_t* codes, uint16_t* scales_nk,
                           uint8_t* zeros_nk, cudaStream_t st);
 
+// 3-bit storage <-> the 4-bit layout holding 3-bit codes (N * K / 32 pieces of 16 / 12 bytes)
+cudaError_t launch_pack_int3(const void* q4, void* q3, int N, int K, cudaStream_t st);
+cudaError_t launch_unpack_int3(const void* q3, void* q4, int N, int K, cudaStream_t st);
+
 constexpr int kGemvMaxBlocks = 256;      // upper bound on the split-K matrix-vector kernel's grid
 
 // Matrix-vector kernels.  The band kernel needs no workspace; the split-K kernel needs
@@ -55,13 +59,14 @@ struct GemvMatrix {                      // one packed weight matrix and its out
 bool gemv_uses_band_kernel(int M, int N, int sms);
 size_t gemv_workspace_bytes(int M);
 // `count` matrices (1..kMaxMulti) sharing x, K and the group size, in one launch.
+// bits: 4, or 3 for qweight in the 3-bit storage (384 bytes per block).
 // serialize: launch without programmatic stream serialization (the kernel then starts only after
 // everything in front of it in the stream has completed, its weight prefetch included).
 // sdiv: nullptr, or the inverse channel scales (fp32 [K], device): the kernel multiplies x by them
 // while it fetches it; only where gemv_band_folds_scale(M, K, group) holds.
 cudaError_t launch_gemv_band(const void* x, const GemvMatrix* mats, int count, int M, int K, int group,
                              unsigned int* status_word, int sms, bool serialize, cudaStream_t st,
-                             const float* sdiv = nullptr);
+                             const float* sdiv = nullptr, int bits = 4);
 bool gemv_band_folds_scale(int M, int K, int group);
 // tx_surplus: 0, or (time-out test only) bytes announced on every stage's barrier beyond what the copies bring
 cudaError_t launch_gemv_splitk(const void* x, const void* qweight, const void* scales, const void* zeros,

@@ -146,10 +146,11 @@ constexpr int kBandThreads = kMathThreads + 96;        // + weight-copy warp + f
 
 // Stage layout of the band kernel, fixed at compile time by TPW (k-tiles per math warp and
 // stage) and the group size, so that every shared-memory read is base + immediate.
-template <int G, int TPW> struct BandStage {
+// TB: bytes of a packed block (16 rows x 64 columns): 512 for 4-bit codes, 384 for the 3-bit storage.
+template <int G, int TPW, int TB = 512> struct BandStage {
     static constexpr int kUT = 16 * TPW;                // k-tiles per stage
     static constexpr int kGroups = kUT * 64 / G;
-    static constexpr int kScOff = kUT * 512;            // [group][16] fp16
+    static constexpr int kScOff = kUT * TB;             // [group][16] fp16
     static constexpr int kZOff = kScOff + kGroups * 32; // [group][16] bytes (a pair of bands)
     static constexpr int kXOff = kZOff + kGroups * 16;  // [token][kXRow]
     static constexpr int kXRow = kUT * 128 + 16;        // padded against bank conflicts
@@ -193,9 +194,9 @@ __device__ __forceinline__ BandRef band_ref(const BandProblems& pr, int task) {
     r.band = task - pr.first_band[p];
     return r;
 }
-template <int G, int TPW>
+template <int G, int TPW, int TB = 512>
 inline BandLayout band_layout(int M, int K, bool x_in_registers, bool x_resident = false) {
-    using St = BandStage<G, TPW>;
+    using St = BandStage<G, TPW, TB>;
     BandLayout l;
     l.stage_bytes = ((St::kXOff + ((x_in_registers || x_resident) ? 0 : M * St::kXRow) + 127) / 128) * 128;
     // per-k-tile sums of x (+ one stage of slack for ragged reads); with x in registers the region
@@ -240,12 +241,31 @@ __device__ __forceinline__ uint4 scale8(const uint4& h, const float4& s0, const 
     return make_uint4(o[0], o[1], o[2], o[3]);
 }
 
+// A lane's packed piece of one block as the four nibble words of the 4-bit layout.  3-bit storage
+// (TB = 384): three words per piece, the fourth word's bits ride in the spare top bits of the
+// nibbles of the other three.
+template <int TB>
+__device__ __forceinline__ uint4 load_piece(const unsigned char* p) {
+    if constexpr (TB == 512) {
+        return *reinterpret_cast<const uint4*>(p);
+    } else {
+        const uint32_t u0 = *reinterpret_cast<const uint32_t*>(p), u1 = *reinterpret_cast<const uint32_t*>(p + 4),
+                       u2 = *reinterpret_cast<const uint32_t*>(p + 8);
+        uint4 w;
+        w.x = u0 & 0x77777777u;
+        w.y = u1 & 0x77777777u;
+        w.z = u2 & 0x77777777u;
+        w.w = ((u0 >> 3) & 0x11111111u) | ((u1 >> 2) & 0x22222222u) | ((u2 >> 1) & 0x44444444u);
+        return w;
+    }
+}
+
 // One full stage of one math warp: the warp's TPW k-tiles (GPW whole groups) of the band's 16
 // rows times x, added to acc.  Straight-line code, one accumulation chain per group, the groups'
 // products interleaved word by word so that no MMA waits for the one before it.  Kx / Ky are
 // 2^-24 times the sums of x over each group for the lane's two accumulator columns (tokens 2t
 // and 2t+1).
-template <int G, int TPW, bool ONE>
+template <int G, int TPW, bool ONE, int TB = 512>
 __device__ __forceinline__ void band_full_stage(const unsigned char* st, int o_w, int o_sc, int o_z,
                                                 const uint2 (&xr)[TPW][4],
                                                 const float (&Kx)[(TPW + G / 64 - 1) / (G / 64)],
@@ -256,7 +276,7 @@ __device__ __forceinline__ void band_full_stage(const unsigned char* st, int o_w
     float c[GPW][4];
     uint4 pk[TPW];
 #pragma unroll
-    for (int v = 0; v < TPW; ++v) pk[v] = *reinterpret_cast<const uint4*>(st + o_w + v * 512);
+    for (int v = 0; v < TPW; ++v) pk[v] = load_piece<TB>(st + o_w + v * TB);
 #pragma unroll
     for (int v = 0; v < TPG; ++v)
 #pragma unroll
@@ -315,13 +335,14 @@ __device__ __forceinline__ void band_full_stage(const unsigned char* st, int o_w
 // sdiv: nullptr, or the inverse channel scales 1 / s (fp32 [K]): x is then multiplied by them while it
 // is fetched (XREG and XSM only), fp16_rne(fp32(x) * inv_s), which folds the caller's diag(s)^-1 into
 // this kernel.
-template <int G, int TPW, bool ONE, bool XREG, int XS, bool XSM = false>
+// TB: 512 (4-bit codes) or 384 (the 3-bit storage, see load_piece).
+template <int G, int TPW, bool ONE, bool XREG, int XS, bool XSM = false, int TB = 512>
 __global__ void __launch_bounds__(kBandThreads, 1)
 gemv_band_kernel(const BandProblems probs, const __half* __restrict__ x, int M, int K,
                  const BandLayout lay, unsigned int* status_word, const float* __restrict__ sdiv) {
     extern __shared__ __align__(128) unsigned char smem[];
     __shared__ unsigned int s_abort;
-    using St = BandStage<G, TPW>;
+    using St = BandStage<G, TPW, TB>;
     constexpr int UT = St::kUT;
     constexpr int TPG = G / 64;                         // k-tiles per group
     constexpr int GPW = (TPW + TPG - 1) / TPG;          // groups touched by one warp in a stage
@@ -400,12 +421,12 @@ gemv_band_kernel(const BandProblems probs, const __half* __restrict__ x, int M, 
                 const uint32_t bar = bars + 8u * stage;
                 if (lane == 0) {
                     mbar_wait_relaxed(bars + 64u + 8u * stage, phase ^ 1u, ctl);
-                    mbar_arrive_expect_tx(bar, (uint32_t)(nt * 512 + ngr * 48 + ((XREG || XSM) ? 0 : M * nt * 128)));
+                    mbar_arrive_expect_tx(bar, (uint32_t)(nt * TB + ngr * 48 + ((XREG || XSM) ? 0 : M * nt * 128)));
                 }
                 __syncwarp();
                 const int gi0 = kt * 64 / G;
                 if (lane == 0)
-                    bulk_load_hint(dst, br.qweight + ((size_t)band * ktiles + kt) * 512, (uint32_t)(nt * 512), bar, once);
+                    bulk_load_hint(dst, br.qweight + ((size_t)band * ktiles + kt) * TB, (uint32_t)(nt * TB), bar, once);
                 else if (lane == 1)
                     bulk_load_hint(dst + St::kScOff, br.scales + ((size_t)band * ng + gi0) * 16, (uint32_t)(ngr * 32), bar, once);
                 else if (lane == 2)
@@ -490,7 +511,7 @@ gemv_band_kernel(const BandProblems probs, const __half* __restrict__ x, int M, 
     const int g = lane >> 2, t = lane & 3;
     const bool tok_ok = g < M;
     // this lane's fixed byte offsets inside a stage
-    const int o_w = warp * (TPW * 512) + lane * 16;
+    const int o_w = warp * (TPW * TB) + lane * (TB / 32);
     const int o_sc = St::kScOff + warp * (GPW * 32) + g * 2;
     const int o_x = St::kXOff + g * St::kXRow + warp * (TPW * 128) + t * 8;
     const float* xs_lane = xsum + warp * (TPW * 8) + 2 * t;
@@ -646,7 +667,7 @@ gemv_band_kernel(const BandProblems probs, const __half* __restrict__ x, int M, 
                 if (task >= b1) return;
                 float acc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
                 mbar_wait(bars + 8u * sl, phase, ctl);
-                band_full_stage<G, TPW, ONE>(smem + sl * SB, o_w, o_sc, o_z, xr, XxR, XyR, acc);
+                band_full_stage<G, TPW, ONE, TB>(smem + sl * SB, o_w, o_sc, o_z, xr, XxR, XyR, acc);
                 if (store_ok) {
                     float* rb = rb0 + sl * (kMathWarps * RS);
                     rb[0] = acc[0];
@@ -677,7 +698,7 @@ gemv_band_kernel(const BandProblems probs, const __half* __restrict__ x, int M, 
         for (int task = b0; task < b1; ++task) {
             float acc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
             mbar_wait(bar, phase, ctl);
-            band_full_stage<G, TPW, ONE>(st, o_w, o_sc, o_z, xr, XxR, XyR, acc);
+            band_full_stage<G, TPW, ONE, TB>(st, o_w, o_sc, o_z, xr, XxR, XyR, acc);
             if (store_ok) {
                 rb[0] = acc[0];
                 rb[8] = acc[2];
@@ -733,7 +754,7 @@ gemv_band_kernel(const BandProblems probs, const __half* __restrict__ x, int M, 
                     Kx[q] = Xx * (1.0f / 16777216.0f);
                     Ky[q] = Xy * (1.0f / 16777216.0f);
                 }
-                band_full_stage<G, TPW, ONE>(st, o_w, o_sc, o_z, xr, Kx, Ky, acc);
+                band_full_stage<G, TPW, ONE, TB>(st, o_w, o_sc, o_z, xr, Kx, Ky, acc);
             } else if (nt > 0) {
                 // ---- ragged last stage of a band: whole groups only (K % G == 0), one at a time
 #pragma unroll
@@ -744,7 +765,7 @@ gemv_band_kernel(const BandProblems probs, const __half* __restrict__ x, int M, 
 #pragma unroll
                         for (int v = 0; v < TPG; ++v) {
                             const int tile = q * TPG + v;
-                            const uint4 pk = *reinterpret_cast<const uint4*>(st + o_w + tile * 512);
+                            const uint4 pk = load_piece<TB>(st + o_w + tile * TB);
                             uint2 xq[1][4] = {{make_uint2(0u, 0u), make_uint2(0u, 0u), make_uint2(0u, 0u), make_uint2(0u, 0u)}};
                             if (tok_ok) {
 #pragma unroll
@@ -1192,7 +1213,7 @@ bool gemv_band_folds_scale(int M, int K, int group) {
 
 cudaError_t launch_gemv_band(const void* x, const GemvMatrix* mats, int count, int M, int K, int group,
                              unsigned int* status_word, int sms, bool serialize, cudaStream_t st,
-                             const float* sdiv) {
+                             const float* sdiv, int bits) {
     BandProblems pr;
     pr.count = count;
     int bands = 0;
@@ -1234,33 +1255,34 @@ cudaError_t launch_gemv_band(const void* x, const GemvMatrix* mats, int count, i
         e = cudaLaunchKernelEx(&cfg, KERNEL, pr, xh, M, K, LAY, status_word, sdiv);                  \
         if (e != cudaSuccess) return e;                                                              \
     } while (0)
-#define AWQ_BAND_LAUNCH(GG, TT, ONE1, XR)                                                            \
+#define AWQ_BAND_LAUNCH(GG, TT, ONE1, XR, TBB)                                                       \
     do {                                                                                             \
-        const BandLayout lay = band_layout<GG, TT>(M, K, XR);                                        \
-        const BandLayout layr = band_layout<GG, TT>(M, K, false, true);                              \
-        if (XR && lay.stages == 5 && lay.red_tokens == 4) {                                          \
-            AWQ_BAND_GO((gemv_band_kernel<GG, TT, ONE1, XR, (XR ? 5 : 0), false>), lay);             \
+        const BandLayout lay = band_layout<GG, TT, TBB>(M, K, XR);                                   \
+        const BandLayout layr = band_layout<GG, TT, TBB>(M, K, false, true);                         \
+        if (XR && lay.stages == (TBB == 512 ? 5 : 6) && lay.red_tokens == 4) {                       \
+            AWQ_BAND_GO((gemv_band_kernel<GG, TT, ONE1, XR, (XR ? (TBB == 512 ? 5 : 6) : 0), false, TBB>), lay); \
         } else if (XR) {                                                                             \
             if (lay.stages < 2) return cudaErrorInvalidValue;                                        \
-            AWQ_BAND_GO((gemv_band_kernel<GG, TT, ONE1, XR, 0, false>), lay);                        \
+            AWQ_BAND_GO((gemv_band_kernel<GG, TT, ONE1, XR, 0, false, TBB>), lay);                   \
         } else if (M <= 2 && layr.stages >= 4) {                                                     \
-            AWQ_BAND_GO((gemv_band_kernel<GG, TT, ONE1, false, 0, !XR>), layr);                      \
+            AWQ_BAND_GO((gemv_band_kernel<GG, TT, ONE1, false, 0, !XR, TBB>), layr);                 \
         } else {                                                                                     \
             if (lay.stages < 2) return cudaErrorInvalidValue;  /* K too large for the x-sum table */ \
             if (sdiv != nullptr) return cudaErrorInvalidValue; /* callers ask gemv_band_folds_scale */ \
-            AWQ_BAND_GO((gemv_band_kernel<GG, TT, ONE1, false, 0, false>), lay);                     \
+            AWQ_BAND_GO((gemv_band_kernel<GG, TT, ONE1, false, 0, false, TBB>), lay);                \
         }                                                                                            \
     } while (0)
     const bool xreg = tpw == 4 && K == 64 * 16 * 4;            // a band is exactly one stage
-#define AWQ_BAND_PICK(GG)                                                                            \
+#define AWQ_BAND_PICK(GG, TBB)                                                                       \
     do {                                                                                             \
-        if (tpw != 4) AWQ_BAND_LAUNCH(GG, 2, false, false);                                          \
-        else if (M == 1 && xreg) AWQ_BAND_LAUNCH(GG, 4, true, true);                                 \
-        else if (M == 1) AWQ_BAND_LAUNCH(GG, 4, true, false);                                        \
-        else if (xreg) AWQ_BAND_LAUNCH(GG, 4, false, true);                                          \
-        else AWQ_BAND_LAUNCH(GG, 4, false, false);                                                   \
+        if (tpw != 4) AWQ_BAND_LAUNCH(GG, 2, false, false, TBB);                                     \
+        else if (M == 1 && xreg) AWQ_BAND_LAUNCH(GG, 4, true, true, TBB);                            \
+        else if (M == 1) AWQ_BAND_LAUNCH(GG, 4, true, false, TBB);                                   \
+        else if (xreg) AWQ_BAND_LAUNCH(GG, 4, false, true, TBB);                                     \
+        else AWQ_BAND_LAUNCH(GG, 4, false, false, TBB);                                              \
     } while (0)
-    if (group == 128) AWQ_BAND_PICK(128); else AWQ_BAND_PICK(64);
+    if (bits == 3) { if (group == 128) AWQ_BAND_PICK(128, 384); else AWQ_BAND_PICK(64, 384); }
+    else           { if (group == 128) AWQ_BAND_PICK(128, 512); else AWQ_BAND_PICK(64, 512); }
 #undef AWQ_BAND_PICK
 #undef AWQ_BAND_LAUNCH
 #undef AWQ_BAND_GO

@@ -404,4 +404,40 @@ cudaError_t launch_unpack(const uint32_t* qweight, const __half* scales, const u
     return cudaGetLastError();
 }
 
+// ---- 3-bit storage: four nibble words of a piece (codes < 8) <-> three words.  One thread per piece.
+__global__ void pack_int3_kernel(const uint4* __restrict__ q4, uint32_t* __restrict__ q3, size_t pieces) {
+    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= pieces) return;
+    const uint4 w = q4[i];
+    q3[3 * i + 0] = (w.x & 0x77777777u) | ((w.w & 0x11111111u) << 3);
+    q3[3 * i + 1] = (w.y & 0x77777777u) | (((w.w >> 1) & 0x11111111u) << 3);
+    q3[3 * i + 2] = (w.z & 0x77777777u) | (((w.w >> 2) & 0x11111111u) << 3);
+}
+__global__ void unpack_int3_kernel(const uint32_t* __restrict__ q3, uint4* __restrict__ q4, size_t pieces) {
+    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= pieces) return;
+    const uint32_t u0 = q3[3 * i], u1 = q3[3 * i + 1], u2 = q3[3 * i + 2];
+    uint4 w;
+    w.x = u0 & 0x77777777u;
+    w.y = u1 & 0x77777777u;
+    w.z = u2 & 0x77777777u;
+    w.w = ((u0 >> 3) & 0x11111111u) | ((u1 >> 2) & 0x22222222u) | ((u2 >> 1) & 0x44444444u);
+    q4[i] = w;
+}
+
+cudaError_t launch_pack_int3(const void* q4, void* q3, int N, int K, cudaStream_t st) {
+    const size_t pieces = (size_t)N * K / 32;
+    pack_int3_kernel<<<(unsigned)((pieces + 255) / 256), 256, 0, st>>>(
+        reinterpret_cast<const uint4*>(q4), reinterpret_cast<uint32_t*>(q3), pieces);
+    count_launch();
+    return cudaGetLastError();
+}
+cudaError_t launch_unpack_int3(const void* q3, void* q4, int N, int K, cudaStream_t st) {
+    const size_t pieces = (size_t)N * K / 32;
+    unpack_int3_kernel<<<(unsigned)((pieces + 255) / 256), 256, 0, st>>>(
+        reinterpret_cast<const uint32_t*>(q3), reinterpret_cast<uint4*>(q4), pieces);
+    count_launch();
+    return cudaGetLastError();
+}
+
 }  // namespace awq
