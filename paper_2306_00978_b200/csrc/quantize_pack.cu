@@ -53,195 +53,176 @@ __device__ __forceinline__ uint32_t code_of(float w, float d, float rd, float z,
     if (!(fabsf(t - r) < 0.499f && fabsf(t) < 1024.0f)) r = rintf(__fdiv_rn(w, d));
     return (uint32_t)fminf(fmaxf(__fadd_rn(r, z), 0.0f), top);
 }
-// The same without the per-element branch: `bad` collects whether any element came within `thr`
-// of a half-integer (thr = 0.5 minus the group's bound on |w * rd - w / d|); the caller then redoes
-// the word with code_of.  Every lane of a warp has to pass for the warp to skip the divisions, so
-// the margin is the group's own bound (a few 1e-6) and not a fixed 1e-3.
-__device__ __forceinline__ float level_fast(float w, float rd, float z, float top, float thr, bool& bad) {
-    const float t = __fmul_rn(w, rd);
-    // round half to even by addition (exact for |t| < 2^22; larger quotients have thr < 0): two fp32
-    // additions instead of a conversion-pipe instruction, the pipe this kernel keeps busiest
-    const float r = __fsub_rn(__fadd_rn(t, 12582912.0f), 12582912.0f);
-    bad = bad || !(fabsf(t - r) < thr);
-    return fminf(fmaxf(__fadd_rn(r, z), 0.0f), top);              // the code, still a float
-}
 // four codes (exact small integers held in floats) as four nibbles: q0 + 16 q1 + 256 q2 + 4096 q3 is
 // exact in fp32, so three FFMAs and one conversion replace four conversions and the shifts and ORs
 __device__ __forceinline__ uint32_t pack4(float q0, float q1, float q2, float q3) {
     return (uint32_t)fmaf(q3, 4096.0f, fmaf(q2, 256.0f, fmaf(q1, 16.0f, q0)));
 }
 
-// grid = (K/128, N/128), block = 256 (8 warps = 8 bands of the 128-row slab); two blocks per SM
-// (118 registers, no spills; three blocks at 80 registers spill and measure 1 % slower).  The kernel
-// is bound by its own instruction stream (issue slots 62 % active, conversion pipe 55 %): measured on
-// 4096->11008, 67.6 us at first, 56 us with the multiply-instead-of-divide path per element, 50.5 us
-// with that path made branch-free per word, 48.2 us with rounding by addition, 46.4 us with the
-// nibbles assembled by FFMA (one conversion per four codes).
-#ifndef AWQ_QP_BLOCKS
-#define AWQ_QP_BLOCKS 2
-#endif
-// SYM: the symmetric grid of Eq. 2 (Delta = max|w'| / 2^(BITS-1), fixed zero point 2^(BITS-1))
+// grid = (K/128, N/128), block = 512: warp w takes band w % 8 of the slab and block w / 8 of the
+// 128 columns, a lane 2 rows x 16 columns - exactly the data of the 16-byte packed piece it writes.
+// The products w' = w * s stay in registers (32), formed once; two blocks (32 warps) fit an SM.  For
+// G = 128 the two warps that share a group exchange their min / max through shared memory.  The
+// division w' / Delta is done only where it can matter: w' * (1 / Delta) rounds to the same integer
+// unless it lies within the group's own error bound of a half-integer; that test is collected per
+// packed word (`bad`), so there is no branch per element, and a word that fails is redone element
+// by element with the division (code_of).  Rounding is by adding 1.5 * 2^23 (the zero point rides
+// in the subtraction that follows), group min / max take three-input min / max instructions, the
+// nibbles of four codes are assembled by FFMA and converted once.
+// (An earlier form - one warp per 16 rows x 128 columns, 8 warps per block, w' formed twice - issued
+// about a third more instructions with half the resident warps and measured the same 45 us on
+// 4096 -> 11008: the kernel is bound by how many bytes its blocks keep in flight, not by its
+// instruction stream.)
+__device__ __forceinline__ float min3(float a, float b, float c) {
+    float d; asm("min.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c)); return d;
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float d; asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c)); return d;
+}
+// code (still a float) = clamp(rne(w * rd) + z): zc = 1.5 * 2^23 - z, so that (t + 1.5 * 2^23) - zc
+// is the rounded quotient plus the zero point, exactly
+__device__ __forceinline__ float level_fast2(float w, float rd, float zc, float top, float thr, bool& bad) {
+    const float t = __fmul_rn(w, rd);
+    const float u = __fadd_rn(t, 12582912.0f);
+    const float r = __fsub_rn(u, 12582912.0f);
+    bad = bad || !(fabsf(__fsub_rn(t, r)) < thr);
+    return fminf(fmaxf(__fsub_rn(u, zc), 0.0f), top);
+}
+
 template <int G, int BITS, bool CLIP, bool SYM>
-__global__ void __launch_bounds__(256, AWQ_QP_BLOCKS)
-quantize_pack_kernel(const __half* __restrict__ W, const float* __restrict__ a, float alpha,
-                     int mode, const float* __restrict__ clip,
-                     uint32_t* __restrict__ qweight, __half* __restrict__ scales,
-                     uint8_t* __restrict__ zeros, int N, int K) {
+__global__ void __launch_bounds__(512, 2)
+quantize_pack_tile_kernel(const __half* __restrict__ W, const float* __restrict__ a, float alpha,
+                          int mode, const float* __restrict__ clip,
+                          uint32_t* __restrict__ qweight, __half* __restrict__ scales,
+                          uint8_t* __restrict__ zeros, int N, int K) {
     constexpr float top = (float)((1 << BITS) - 1);       // largest code
     __shared__ __align__(16) float s_sm[128];
+    __shared__ float2 s_mm[2][128];                        // G = 128: [block of the pair][row of the slab] (min, max)
     const int kblk = blockIdx.x, slab = blockIdx.y;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int bw = warp & 7, ti = warp >> 3;
     const int g = lane >> 2, t = lane & 3;
-    const int n0 = slab * 128 + warp * 16 + g;            // this lane's upper row; lower = n0 + 8
+    const int n0 = slab * 128 + bw * 16 + g;               // this lane's upper row; lower = n0 + 8
     const int kbase = kblk * 128;
 
-    // issue the weight loads first: [tile][row h][word j] = columns 16j + 4t .. +3 of the tile
-    uint2 raw[2][2][4];
+    uint2 raw[2][4];                                       // [row h][word j] = columns 16j + 4t .. +3 of the block
 #pragma unroll
-    for (int ti = 0; ti < 2; ++ti)
+    for (int h = 0; h < 2; ++h)
 #pragma unroll
-        for (int h = 0; h < 2; ++h)
-#pragma unroll
-            for (int j = 0; j < 4; ++j)
-                raw[ti][h][j] = ldg_stream(reinterpret_cast<const uint2*>(
-                    W + (size_t)(n0 + 8 * h) * K + kbase + ti * 64 + 16 * j + 4 * t));
+        for (int j = 0; j < 4; ++j)
+            raw[h][j] = ldg_stream(reinterpret_cast<const uint2*>(
+                W + (size_t)(n0 + 8 * h) * K + kbase + ti * 64 + 16 * j + 4 * t));
     if (threadIdx.x < 128) {
         const int k = kbase + threadIdx.x;
         s_sm[threadIdx.x] = channel_scale_one(mode == kAlphaZero ? 1.0f : a[k], alpha, mode);
     }
     __syncthreads();
 
-    // w' = fp32(w) * s  (Eq. 3) is formed twice from the raw words - here for the group's min / max,
-    // below for the codes (the same two operations give the same value) - so that only the 32 raw
-    // registers stay live.  The four scales of a word are one 16-byte
-    // shared-memory read, used for both rows.
-    auto wprime = [&](int ti, int h, int j, const float (&sv)[4], float (&w4)[4]) {
-        const uint32_t u0 = raw[ti][h][j].x, u1 = raw[ti][h][j].y;
-        w4[0] = __fmul_rn(__half2float(__ushort_as_half((unsigned short)(u0 & 0xFFFFu))), sv[0]);
-        w4[1] = __fmul_rn(__half2float(__ushort_as_half((unsigned short)(u0 >> 16))), sv[1]);
-        w4[2] = __fmul_rn(__half2float(__ushort_as_half((unsigned short)(u1 & 0xFFFFu))), sv[2]);
-        w4[3] = __fmul_rn(__half2float(__ushort_as_half((unsigned short)(u1 >> 16))), sv[3]);
-    };
-    // group min / max: a row's group is spread over the 4 lanes t = 0..3 (and, for
-    // G = 128, over both tiles)
-    float mn[2][2], mx[2][2];
+    // w' = fp32(w) * s  (Eq. 3), once, and the min / max of this lane's 16 columns of each row
+    float wp[2][4][4];
+    float mn[2], mx[2];
 #pragma unroll
-    for (int ti = 0; ti < 2; ++ti) {
+    for (int h = 0; h < 2; ++h) { mn[h] = INFINITY; mx[h] = -INFINITY; }
 #pragma unroll
-        for (int h = 0; h < 2; ++h) { mn[ti][h] = INFINITY; mx[ti][h] = -INFINITY; }
+    for (int j = 0; j < 4; ++j) {
+        const float4 s4 = *reinterpret_cast<const float4*>(&s_sm[ti * 64 + 16 * j + 4 * t]);
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const float4 s4 = *reinterpret_cast<const float4*>(&s_sm[ti * 64 + 16 * j + 4 * t]);
-            const float sv[4] = {s4.x, s4.y, s4.z, s4.w};
-#pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                float w4[4];
-                wprime(ti, h, j, sv, w4);
-#pragma unroll
-                for (int e = 0; e < 4; ++e) { mn[ti][h] = fminf(mn[ti][h], w4[e]); mx[ti][h] = fmaxf(mx[ti][h], w4[e]); }
-            }
+        for (int h = 0; h < 2; ++h) {
+            const uint32_t u0 = raw[h][j].x, u1 = raw[h][j].y;
+            wp[h][j][0] = __fmul_rn(__half2float(__ushort_as_half((unsigned short)(u0 & 0xFFFFu))), s4.x);
+            wp[h][j][1] = __fmul_rn(__half2float(__ushort_as_half((unsigned short)(u0 >> 16))), s4.y);
+            wp[h][j][2] = __fmul_rn(__half2float(__ushort_as_half((unsigned short)(u1 & 0xFFFFu))), s4.z);
+            wp[h][j][3] = __fmul_rn(__half2float(__ushort_as_half((unsigned short)(u1 >> 16))), s4.w);
+            mn[h] = min3(mn[h], wp[h][j][0], wp[h][j][1]);
+            mn[h] = min3(mn[h], wp[h][j][2], wp[h][j][3]);
+            mx[h] = max3(mx[h], wp[h][j][0], wp[h][j][1]);
+            mx[h] = max3(mx[h], wp[h][j][2], wp[h][j][3]);
         }
     }
+#pragma unroll
+    for (int h = 0; h < 2; ++h)
+#pragma unroll
+        for (int off = 1; off <= 2; off <<= 1) {
+            mn[h] = fminf(mn[h], __shfl_xor_sync(0xFFFFFFFFu, mn[h], off));
+            mx[h] = fmaxf(mx[h], __shfl_xor_sync(0xFFFFFFFFu, mx[h], off));
+        }
     if (G == 128) {
+        // the group spans both blocks of the pair: the other half's min / max through shared memory
+        if (t == 0) {
+            s_mm[ti][bw * 16 + g] = make_float2(mn[0], mx[0]);
+            s_mm[ti][bw * 16 + g + 8] = make_float2(mn[1], mx[1]);
+        }
+        __syncthreads();
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
-            mn[0][h] = mn[1][h] = fminf(mn[0][h], mn[1][h]);
-            mx[0][h] = mx[1][h] = fmaxf(mx[0][h], mx[1][h]);
+            const float2 o = s_mm[ti ^ 1][bw * 16 + g + 8 * h];
+            mn[h] = fminf(mn[h], o.x);
+            mx[h] = fmaxf(mx[h], o.y);
         }
     }
+    float wabs[2];                                          // largest |w'| of each group (before clipping)
 #pragma unroll
-    for (int ti = 0; ti < 2; ++ti)
-#pragma unroll
-        for (int h = 0; h < 2; ++h)
-#pragma unroll
-            for (int off = 1; off <= 2; off <<= 1) {
-                mn[ti][h] = fminf(mn[ti][h], __shfl_xor_sync(0xFFFFFFFFu, mn[ti][h], off));
-                mx[ti][h] = fmaxf(mx[ti][h], __shfl_xor_sync(0xFFFFFFFFu, mx[ti][h], off));
-            }
-
-    float wabs[2][2];                                       // largest |w'| of each group (before clipping)
-#pragma unroll
-    for (int ti = 0; ti < 2; ++ti)
-#pragma unroll
-        for (int h = 0; h < 2; ++h) wabs[ti][h] = fmaxf(fabsf(mn[ti][h]), fabsf(mx[ti][h]));
-
+    for (int h = 0; h < 2; ++h) wabs[h] = fmaxf(fabsf(mn[h]), fabsf(mx[h]));
+    const int gi = (G == 64) ? kblk * 2 + ti : kblk;
+    const int ng = K / G;
     if (CLIP) {
-        // weight clipping (Sec. 3.2): the group's range shrinks by its ratio, values outside saturate
-        const int ng = K / G;
-#pragma unroll
-        for (int ti = 0; ti < 2; ++ti)
-#pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                const int gi = (G == 64) ? kblk * 2 + ti : kblk;
-                const float r = __ldg(clip + (size_t)(n0 + 8 * h) * ng + gi);
-                mn[ti][h] = __fmul_rn(mn[ti][h], r);
-                mx[ti][h] = __fmul_rn(mx[ti][h], r);
-            }
-    }
-
-#pragma unroll
-    for (int ti = 0; ti < 2; ++ti) {
-        __half d16[2]; float d[2], z[2], rd[2], thr[2];
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
-            if (SYM) {
-                constexpr float half_levels = (float)(1 << (BITS - 1));
-                const float d32 = __fdiv_rn(fmaxf(fabsf(mn[ti][h]), fabsf(mx[ti][h])), half_levels);
-                d16[h] = __float2half_rn(d32);
-                const unsigned short bits = __half_as_ushort(d16[h]);
-                if ((bits & 0x7FFFu) == 0u || (bits & 0x7C00u) == 0x7C00u) d16[h] = __ushort_as_half(0x3C00u);
-                d[h] = __half2float(d16[h]);
-                z[h] = half_levels;
-            } else {
-                group_params(mn[ti][h], mx[ti][h], top, d16[h], d[h], z[h]);
-            }
-            rd[h] = __frcp_rn(d[h]);
-            // |w * rd - w / d| <= 1.8e-7 |w / d| (three roundings); the group's largest |w / d|
-            // bounds it for every element; quotients beyond 1024 always take the division
-            const float tmax = __fmul_rn(wabs[ti][h], rd[h]);
-            thr[h] = tmax < 1024.0f ? 0.5f - fmaf(tmax, 4e-7f, 1e-6f) : -1.0f;
+            const float r = __ldg(clip + (size_t)(n0 + 8 * h) * ng + gi);
+            mn[h] = __fmul_rn(mn[h], r);
+            mx[h] = __fmul_rn(mx[h], r);
         }
-
-        uint32_t words[4];
+    }
+    __half d16[2]; float d[2], z[2], rd[2], thr[2], zc[2];
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const float4 s4 = *reinterpret_cast<const float4*>(&s_sm[ti * 64 + 16 * j + 4 * t]);
-            const float sv[4] = {s4.x, s4.y, s4.z, s4.w};
-            float wu[4], wl[4];                                  // rows g and g + 8, columns c .. c+3
-            wprime(ti, 0, j, sv, wu);
-            wprime(ti, 1, j, sv, wl);
-            // slots (g,c) (g,c+1) (g+8,c) (g+8,c+1) (g,c+2) (g,c+3) (g+8,c+2) (g+8,c+3)
-            // at nibbles 0, 4, 1, 5, 2, 6, 3, 7
-            bool bad = false;
-            float qu[4], ql[4];
+    for (int h = 0; h < 2; ++h) {
+        if (SYM) {
+            constexpr float half_levels = (float)(1 << (BITS - 1));
+            const float d32 = __fdiv_rn(fmaxf(fabsf(mn[h]), fabsf(mx[h])), half_levels);
+            d16[h] = __float2half_rn(d32);
+            const unsigned short bits = __half_as_ushort(d16[h]);
+            if ((bits & 0x7FFFu) == 0u || (bits & 0x7C00u) == 0x7C00u) d16[h] = __ushort_as_half(0x3C00u);
+            d[h] = __half2float(d16[h]);
+            z[h] = half_levels;
+        } else {
+            group_params(mn[h], mx[h], top, d16[h], d[h], z[h]);
+        }
+        rd[h] = __frcp_rn(d[h]);
+        zc[h] = 12582912.0f - z[h];                          // exact: z is a small integer
+        // |w * rd - w / d| <= 1.8e-7 |w / d| (three roundings); the group's largest |w / d|
+        // bounds it for every element; quotients beyond 1024 always take the division
+        const float tmax = __fmul_rn(wabs[h], rd[h]);
+        thr[h] = tmax < 1024.0f ? 0.5f - fmaf(tmax, 4e-7f, 1e-6f) : -1.0f;
+    }
+    uint32_t words[4];
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                qu[e] = level_fast(wu[e], rd[0], z[0], top, thr[0], bad);
-                ql[e] = level_fast(wl[e], rd[1], z[1], top, thr[1], bad);
-            }
-            // nibbles 0 .. 3 = (g,c) (g+8,c) (g,c+2) (g+8,c+2), nibbles 4 .. 7 the same for c+1, c+3
-            words[j] = pack4(qu[0], ql[0], qu[2], ql[2]) | (pack4(qu[1], ql[1], qu[3], ql[3]) << 16);
-            if (bad)                                               // rare: the word again, element by element
-                words[j] = (code_of(wu[0], d[0], rd[0], z[0], top) << 0) | (code_of(wu[1], d[0], rd[0], z[0], top) << 16) |
-                           (code_of(wl[0], d[1], rd[1], z[1], top) << 4) | (code_of(wl[1], d[1], rd[1], z[1], top) << 20) |
-                           (code_of(wu[2], d[0], rd[0], z[0], top) << 8) | (code_of(wu[3], d[0], rd[0], z[0], top) << 24) |
-                           (code_of(wl[2], d[1], rd[1], z[1], top) << 12) | (code_of(wl[3], d[1], rd[1], z[1], top) << 28);
+    for (int j = 0; j < 4; ++j) {
+        bool bad = false;
+        float qu[4], ql[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            qu[e] = level_fast2(wp[0][j][e], rd[0], zc[0], top, thr[0], bad);
+            ql[e] = level_fast2(wp[1][j][e], rd[1], zc[1], top, thr[1], bad);
         }
-        // band-major: block (band, k-tile) is 512 bytes, a band's blocks are contiguous along K
-        const size_t band = (size_t)slab * 8 + warp;
-        const size_t block = band * (K / 64) + (size_t)kblk * 2 + ti;
-        uint4* dst = reinterpret_cast<uint4*>(qweight) + block * 32 + lane;
-        *dst = make_uint4(words[0], words[1], words[2], words[3]);
-
-        if (t == 0 && (G == 64 || ti == 0)) {
-            // scales: [band][group][16]; zero bytes: [band pair][group][16], 8 per band
-            const int gi = (G == 64) ? kblk * 2 + ti : kblk;
-            const size_t ng = K / G;
-            scales[(band * ng + gi) * 16 + g] = d16[0];
-            scales[(band * ng + gi) * 16 + g + 8] = d16[1];
-            zeros[((band >> 1) * ng + gi) * 16 + (band & 1) * 8 + g] =
-                (uint8_t)((uint32_t)z[0] | ((uint32_t)z[1] << 4));
-        }
+        // nibbles 0 .. 3 = (g,c) (g+8,c) (g,c+2) (g+8,c+2), nibbles 4 .. 7 the same for c+1, c+3
+        words[j] = pack4(qu[0], ql[0], qu[2], ql[2]) | (pack4(qu[1], ql[1], qu[3], ql[3]) << 16);
+        if (bad)                                               // rare: the word again, element by element
+            words[j] = (code_of(wp[0][j][0], d[0], rd[0], z[0], top) << 0) | (code_of(wp[0][j][1], d[0], rd[0], z[0], top) << 16) |
+                       (code_of(wp[1][j][0], d[1], rd[1], z[1], top) << 4) | (code_of(wp[1][j][1], d[1], rd[1], z[1], top) << 20) |
+                       (code_of(wp[0][j][2], d[0], rd[0], z[0], top) << 8) | (code_of(wp[0][j][3], d[0], rd[0], z[0], top) << 24) |
+                       (code_of(wp[1][j][2], d[1], rd[1], z[1], top) << 12) | (code_of(wp[1][j][3], d[1], rd[1], z[1], top) << 28);
+    }
+    // band-major: block (band, k-tile) is 512 bytes, a band's blocks are contiguous along K
+    const size_t band = (size_t)slab * 8 + bw;
+    const size_t block = band * (K / 64) + (size_t)kblk * 2 + ti;
+    uint4* dst = reinterpret_cast<uint4*>(qweight) + block * 32 + lane;
+    *dst = make_uint4(words[0], words[1], words[2], words[3]);
+    if (t == 0 && (G == 64 || ti == 0)) {
+        // scales: [band][group][16]; zero bytes: [band pair][group][16], 8 per band
+        scales[(band * ng + gi) * 16 + g] = d16[0];
+        scales[(band * ng + gi) * 16 + g + 8] = d16[1];
+        zeros[((band >> 1) * ng + gi) * 16 + (band & 1) * 8 + g] =
+            (uint8_t)((uint32_t)z[0] | ((uint32_t)z[1] << 4));
     }
 }
 
@@ -357,7 +338,7 @@ cudaError_t launch_quantize_pack(const __half* W, const float* a, float alpha, i
     const dim3 grid(K / 128, N / 128);
     const int mode = (int)alpha_mode(alpha);
 #define AWQ_QP_LAUNCH(GG, BB, CC, SS) \
-    quantize_pack_kernel<GG, BB, CC, SS><<<grid, 256, 0, st>>>(W, a, alpha, mode, clip, qweight, scales, zeros, N, K)
+    quantize_pack_tile_kernel<GG, BB, CC, SS><<<grid, 512, 0, st>>>(W, a, alpha, mode, clip, qweight, scales, zeros, N, K)
 #define AWQ_QP_PICK2(GG, SS)                                             \
     do {                                                                 \
         if (bits == 4 && !clip) AWQ_QP_LAUNCH(GG, 4, false, SS);         \
