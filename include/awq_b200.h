@@ -65,9 +65,10 @@ typedef enum AwqStatus {
 
 /* Which kernel awq_linear_path runs. */
 typedef enum AwqPath {
-    AWQ_PATH_AUTO = 0,          /* what awq_linear does: the matrix-vector kernels for M <= 8 (and for
-                                   M <= 16 if N * K >= 2^27 and a workspace of awq_workspace_bytes is
-                                   registered), else the tensor-core kernels */
+    AWQ_PATH_AUTO = 0,          /* what awq_linear does: the matrix-vector kernels for M <= 8, the
+                                   chunked matrix-vector kernel for 9 <= M <= 16 if K is a multiple of
+                                   2048 and a workspace of awq_workspace_bytes is registered, else the
+                                   tensor-core kernels */
     AWQ_PATH_GEMV = 1,          /* fused dequant matrix-vector kernel, M <= 16: band kernel when
                                    M <= 8 and N/16 is not much below the SM count, else split-K */
     AWQ_PATH_GEMM = 2,          /* tcgen05 tensor-core kernel, any M >= 1: pairs of SMs
@@ -75,7 +76,10 @@ typedef enum AwqPath {
                                    multiple of 256 and M > 128 (M > 64 from N = 8192, M >= 32 from
                                    N = 16384), else one SM per tile */
     AWQ_PATH_GEMV_SPLITK = 3,   /* the split-K matrix-vector kernel, M <= 16 */
-    AWQ_PATH_GEMM_1SM = 4       /* the tensor-core kernel with one SM per tile, any M >= 1 */
+    AWQ_PATH_GEMM_1SM = 4,      /* the tensor-core kernel with one SM per tile, any M >= 1 */
+    AWQ_PATH_GEMV_MID = 5       /* the chunked matrix-vector kernel, M <= 32: a block owns a chunk of K,
+                                   keeps its slice of x in shared memory and streams band runs; needs
+                                   a workspace of awq_workspace_bytes (fp32 partial sums per chunk) */
 } AwqPath;
 
 /* Sizes of the packed arrays, in bytes (0 if the shape is not accepted). */
@@ -146,9 +150,11 @@ int awq_channel_scale(const float* act_mean_abs, float alpha, float* s, int K, v
  * x: in, fp16 [M][K].  y: out, fp16 [M][N], fully overwritten; must not alias an input.
  * M <= 8 runs a matrix-vector kernel (HBM-bound; the 4-bit codes enter warp-level tensor-core
  * products exactly, accumulation, zero point and Delta in fp32, one rounding to fp16 at the
- * end), and so does 8 < M <= 16 on a large matrix (N * K >= 2^27) when the registered workspace
- * holds awq_workspace_bytes; everything else the tcgen05 kernel ((q - z) * Delta rounded once to
- * fp16, fp32 accumulation in tensor memory).  Results are bit-reproducible.
+ * end), and so does 8 < M <= 16 with K a multiple of 2048 when the registered workspace holds
+ * awq_workspace_bytes (the chunked kernel, AWQ_PATH_GEMV_MID: same arithmetic, partial sums per
+ * chunk of K added in a fixed order by a second small kernel); everything else the tcgen05 kernel
+ * ((q - z) * Delta rounded once to fp16, fp32 accumulation in tensor memory).  Results are
+ * bit-reproducible.
  * The split-K matrix-vector kernel (used when N is small or M > 8) combines partial sums in a
  * fixed order through the registered workspace; calls that use the workspace must not
  * overlap on the GPU (issue them on one stream).

@@ -160,6 +160,16 @@ int awq_search_clip(const void* W, const float* act_mean_abs, float alpha, int g
                                         ratios, n_ratios, clip_ratio, N, K, (cudaStream_t)stream));
 }
 
+// Where the chunked matrix-vector kernel beats the other kernels (measured at 9 and 16 tokens:
+// 17.9 against 26 us on 4096 -> 11008, 12.3 against 13.6 us on 4096 -> 4096, 54 against 98 us
+// (tensor-core kernel) and 72 us (split-K matrix-vector kernel) on 8192 -> 28672, 60 against 102 us
+// on 28672 -> 8192; with a ragged last chunk it loses: 28 against 26 us on 11008 -> 4096; from 17
+// tokens on the tensor-core kernels are as fast or faster).
+static bool mid_kernel_preferred(int M, int N, int K) {
+    (void)N;
+    return M > 8 && M <= 16 && K % 2048 == 0;
+}
+
 static int resolve_path(int M, int K, int path) {
     if (path == AWQ_PATH_AUTO) return (M <= 8 && K <= 65536) ? AWQ_PATH_GEMV : AWQ_PATH_GEMM;
     return path;
@@ -174,7 +184,11 @@ size_t awq_workspace_bytes(int M, int N, int K, int group) {
         (void)cudaGetLastError();
         sms = 160;                           // no device to ask: an upper bound for this GPU family
     }
-    const size_t gemm = gemm_workspace_bytes(M, N, sms);
+    size_t gemm = gemm_workspace_bytes(M, N, sms);
+    if (M > 8 && M <= 32 && gemv_mid_applies(M, N, K, group, sms)) {
+        const size_t mid = gemv_mid_workspace_bytes(M, N, K);
+        if (mid > gemm) gemm = mid;
+    }
     if (M > 16) return gemm;
     const size_t gemv = gemv_workspace_bytes(M);   // required by the split-K matrix-vector kernel
     if (M <= 8) return gemv;                       // awq_linear never takes the tensor-core kernel here
@@ -204,19 +218,31 @@ int awq_linear_path(const void* x, const void* qweight, const void* scales, cons
     if (!aligned16(x) || !aligned16(qweight) || !aligned16(scales) || !aligned16(zeros) || !aligned16(y))
         return AWQ_ERR_MISALIGNED;
     if (path != AWQ_PATH_AUTO && path != AWQ_PATH_GEMV && path != AWQ_PATH_GEMM && path != AWQ_PATH_GEMV_SPLITK &&
-        path != AWQ_PATH_GEMM_1SM)
+        path != AWQ_PATH_GEMM_1SM && path != AWQ_PATH_GEMV_MID)
         return AWQ_ERR_BAD_ARGUMENT;
     const bool automatic = path == AWQ_PATH_AUTO;
     path = resolve_path(M, K, path);
-    if (path != AWQ_PATH_GEMM && path != AWQ_PATH_GEMM_1SM && (M > 16 || K > 65536)) return AWQ_ERR_BAD_SHAPE;
+    if (path == AWQ_PATH_GEMV_MID) {
+        if (M > 64 || K > 65536) return AWQ_ERR_BAD_SHAPE;
+    } else if (path != AWQ_PATH_GEMM && path != AWQ_PATH_GEMM_1SM && (M > 16 || K > 65536)) {
+        return AWQ_ERR_BAD_SHAPE;
+    }
     DeviceState* d;
     if (int rc = device_state(&d)) return rc;
-    if (automatic && M > 8 && M <= 16 && K <= 65536 && (size_t)N * (size_t)K >= ((size_t)1 << 27)) {
-        // measured at 16 tokens: on large matrices the split-K matrix-vector kernel beats the
-        // tensor-core kernel (74 vs 98 us on 8192 -> 28672), on small ones it loses (18.6 vs 13.6 us
-        // on 4096 -> 4096); it needs the workspace, the tensor-core kernel does not
+    if (automatic && mid_kernel_preferred(M, N, K) && gemv_mid_applies(M, N, K, group, d->sms)) {
         std::lock_guard<std::mutex> lock(g_mutex);
-        if (d->workspace_bytes >= gemv_workspace_bytes(M)) path = AWQ_PATH_GEMV;
+        if (d->workspace_bytes >= gemv_mid_workspace_bytes(M, N, K)) path = AWQ_PATH_GEMV_MID;
+    }
+    if (path == AWQ_PATH_GEMV_MID) {
+        if (!gemv_mid_applies(M, N, K, group, d->sms)) return AWQ_ERR_BAD_SHAPE;
+        void* ws = nullptr;
+        {
+            std::lock_guard<std::mutex> lock(g_mutex);
+            if (d->workspace_bytes < gemv_mid_workspace_bytes(M, N, K)) return AWQ_ERR_NO_WORKSPACE;
+            ws = d->workspace;
+        }
+        return note_cuda(launch_gemv_mid(x, qweight, scales, zeros, y, M, N, K, group, ws, d->status_word, d->sms,
+                                         take_packed_written(d), (cudaStream_t)stream));
     }
     const bool tensor_path = path == AWQ_PATH_GEMM || path == AWQ_PATH_GEMM_1SM;
     const cudaStream_t st = (cudaStream_t)stream;

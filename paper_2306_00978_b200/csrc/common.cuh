@@ -73,6 +73,14 @@ cudaError_t launch_gemv_splitk(const void* x, const void* qweight, const void* s
                                void* y, int M, int N, int K, int group, void* workspace,
                                unsigned int* status_word, int sms, cudaStream_t st, int tx_surplus = 0);
 
+// medium token counts (gemv_mid.cu): blocks own a chunk of K, partial sums per chunk in the
+// workspace (behind its counter head), a second kernel adds the chunks
+bool gemv_mid_applies(int M, int N, int K, int group, int sms);
+size_t gemv_mid_workspace_bytes(int M, int N, int K);
+cudaError_t launch_gemv_mid(const void* x, const void* qweight, const void* scales, const void* zeros, void* y,
+                            int M, int N, int K, int group, void* workspace, unsigned int* status_word, int sms,
+                            bool serialize, cudaStream_t st);
+
 // scale search (search.cu)
 constexpr int kMaxSearchAlphas = 64;
 size_t search_scratch_bytes(int M, int N, int K, int group);

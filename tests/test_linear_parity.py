@@ -197,9 +197,9 @@ def test_quantize_then_linear_back_to_back_on_one_stream():
 
 
 def test_auto_dispatch_between_9_and_16_tokens():
-    """awq_linear with 9..16 tokens: the tensor-core kernel on small matrices, and on large ones
-    (N * K >= 2^27) the split-K matrix-vector kernel if a workspace is registered.  Each result is
-    bit-equal to its forced path."""
+    """awq_linear with 9..16 tokens: the tensor-core kernel where K is not a multiple of 2048 (or no
+    workspace is registered), the chunked matrix-vector kernel otherwise.  Each result is bit-equal
+    to its forced path."""
     import torch
     from paper_2306_00978_b200 import binding
     L = binding.lib()
@@ -209,7 +209,13 @@ def test_auto_dispatch_between_9_and_16_tokens():
     auto = binding.linear(x, qw, sc, zp, case.N, case.K, case.group)
     forced_gemm = binding.linear(x, qw, sc, zp, case.N, case.K, case.group, path=binding.PATH_GEMM)
     assert torch.equal(auto, forced_gemm)
-    assert_parity(auto.cpu().numpy(), case.y_ref(), "auto M=12, small matrix")
+    assert_parity(auto.cpu().numpy(), case.y_ref(), "auto M=12, K not a multiple of 2048")
+    case = Case(78, 1024, 4096, 12, 128, 0.5)
+    qw, sc, zp = oracle_packed_to_cuda(case)
+    x = to_cuda(case.x)
+    auto = binding.linear(x, qw, sc, zp, case.N, case.K, case.group)
+    assert torch.equal(auto, binding.linear(x, qw, sc, zp, case.N, case.K, case.group, path=binding.PATH_GEMV_MID))
+    assert_parity(auto.cpu().numpy(), case.y_ref(), "auto M=12, chunked kernel")
     # a large matrix (random packed arrays: only the choice of kernel is checked here; parity at
     # this size is covered by the 70B sweep)
     N, K, G, M = 16384, 8192, 128, 12
@@ -218,7 +224,7 @@ def test_auto_dispatch_between_9_and_16_tokens():
     zp = torch.randint(0, 256, (N // 32, K // G, 16), dtype=torch.uint8, device="cuda")
     x = torch.randn((M, K), device="cuda").half()
     with_ws = binding.linear(x, qw, sc, zp, N, K, G)                       # binding registers a workspace
-    assert torch.equal(with_ws, binding.linear(x, qw, sc, zp, N, K, G, path=binding.PATH_GEMV))
+    assert torch.equal(with_ws, binding.linear(x, qw, sc, zp, N, K, G, path=binding.PATH_GEMV_MID))
     y = torch.empty_like(with_ws)
     ref = torch.empty_like(with_ws)
     torch.cuda.synchronize()
@@ -286,3 +292,23 @@ def test_missing_workspace_is_reported():
     if saved is not None:
         assert L.awq_set_workspace(saved.data_ptr(), saved.numel()) == 0
         binding._workspace[torch.cuda.current_device()] = saved
+
+
+@pytest.mark.parametrize("N,K,M,G", [
+    (512, 1024, 9, 128),      # half a chunk only
+    (1024, 1408, 16, 128),    # ragged second... first chunk: 22 k-tiles
+    (768, 4096, 17, 64),      # two token groups, four chunks of 1024
+    (512, 2304, 32, 128),     # ragged last chunk
+    (640, 2048, 24, 64),
+    (2432, 4096, 13, 128),    # more bands than blocks of a chunk
+    (128, 8192, 10, 128),     # fewer bands than blocks
+])
+def test_chunked_matrix_vector_kernel(N, K, M, G):
+    """AWQ_PATH_GEMV_MID: a block owns a chunk of K; partial sums per chunk, added by a second
+    kernel.  Parity with the oracle and bit-reproducibility."""
+    from paper_2306_00978_b200 import binding
+    case = Case(600 + N + K + M + G, N, K, M, G, 0.5)
+    y = _run(case, binding.PATH_GEMV_MID)
+    assert_parity(y, case.y_ref(), f"chunked N={N} K={K} M={M} G={G}")
+    y2 = _run(case, binding.PATH_GEMV_MID)
+    assert np.array_equal(y.view(np.uint16), y2.view(np.uint16))
