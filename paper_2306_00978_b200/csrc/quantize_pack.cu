@@ -8,6 +8,8 @@
 // no shared-memory transpose is needed.  Every
 // rounding point is an explicit IEEE operation (no contraction); the per-weight division is
 // replaced by a multiplication only where that provably rounds to the same integer.
+#include <type_traits>
+
 #include "common.cuh"
 
 namespace awq {
@@ -59,20 +61,26 @@ __device__ __forceinline__ uint32_t pack4(float q0, float q1, float q2, float q3
     return (uint32_t)fmaf(q3, 4096.0f, fmaf(q2, 256.0f, fmaf(q1, 16.0f, q0)));
 }
 
-// grid = (K/128, N/128), block = 512: warp w takes band w % 8 of the slab and block w / 8 of the
-// 128 columns, a lane 2 rows x 16 columns - exactly the data of the 16-byte packed piece it writes.
-// The products w' = w * s stay in registers (32), formed once; two blocks (32 warps) fit an SM.  For
+// grid = (K/128, N/32), block = 128: warp w takes band w % 2 of the block's 32 rows and block w / 2 of
+// the 128 columns, a lane 2 rows x 16 columns - exactly the data of the 16-byte packed piece it writes.
+// The products w' = w * s stay in registers (32), formed once (64 registers, 32 warps per SM).  For
 // G = 128 the two warps that share a group exchange their min / max through shared memory.  The
 // division w' / Delta is done only where it can matter: w' * (1 / Delta) rounds to the same integer
-// unless it lies within the group's own error bound of a half-integer; that test is collected per
-// packed word (`bad`), so there is no branch per element, and a word that fails is redone element
-// by element with the division (code_of).  Rounding is by adding 1.5 * 2^23 (the zero point rides
-// in the subtraction that follows), group min / max take three-input min / max instructions, the
-// nibbles of four codes are assembled by FFMA and converted once.
-// (An earlier form - one warp per 16 rows x 128 columns, 8 warps per block, w' formed twice - issued
-// about a third more instructions with half the resident warps and measured the same 45 us on
-// 4096 -> 11008: the kernel is bound by how many bytes its blocks keep in flight, not by its
-// instruction stream.)
+// unless it lies within the group's own error bound of a half-integer; that test is taken per
+// packed word and row (the largest distance of the word's products from their rounded values), so
+// there is no branch per element, and a word that fails is redone element by element with the
+// division (code_of).  Rounding is by adding 1.5 * 2^23 (the zero point rides in the subtraction
+// that follows), group min / max take three-input min / max instructions, clamping to [0, top] is
+// compiled in only for the warps one of whose groups can leave the range, the nibbles of four codes
+// are assembled by FFMA and converted once.
+// What bounds it (measured on 4096 -> 11008, 113.6 MB): a block loads, computes and stores in
+// phases, and the blocks of an SM run in step, so the loads overlap the arithmetic only as far as
+// the blocks drift apart.  With 512-thread blocks (two per SM) 45.4 us, whatever the instruction
+// count (a form with a third more instructions and half the warps: 45 us; a third fewer
+// integer-pipe instructions: 44.3 us); 256-thread blocks 41.6 us, 128-thread blocks 37.9 us, 64-thread
+// blocks 41.0 us (the 128 channel scales are then formed per 64 threads).  A persistent form whose
+// producer warp keeps six 32 KB tiles in flight by tensor-map copies for sixteen quantizing warps
+// measured 58 us: the arithmetic needs the 32 warps.
 __device__ __forceinline__ float min3(float a, float b, float c) {
     float d; asm("min.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c)); return d;
 }
@@ -81,28 +89,35 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
 }
 // code (still a float) = clamp(rne(w * rd) + z): zc = 1.5 * 2^23 - z, so that (t + 1.5 * 2^23) - zc
 // is the rounded quotient plus the zero point, exactly
-__device__ __forceinline__ float level_fast2(float w, float rd, float zc, float top, float thr, bool& bad) {
+// `dev` receives |t - rne(t)|, the distance that decides whether the product may stand for the
+// quotient; CLAMP = false where the group's smallest and largest element are known to stay in range.
+template <bool CLAMP>
+__device__ __forceinline__ float level_fast2(float w, float rd, float zc, float top, float& dev) {
     const float t = __fmul_rn(w, rd);
     const float u = __fadd_rn(t, 12582912.0f);
     const float r = __fsub_rn(u, 12582912.0f);
-    bad = bad || !(fabsf(__fsub_rn(t, r)) < thr);
-    return fminf(fmaxf(__fsub_rn(u, zc), 0.0f), top);
+    dev = fabsf(__fsub_rn(t, r));
+    const float q = __fsub_rn(u, zc);
+    return CLAMP ? fminf(fmaxf(q, 0.0f), top) : q;
 }
 
+constexpr int kQBands = 2;                                // bands (16 rows) per thread block
+constexpr int kQThreads = kQBands * 2 * 32;              // one warp per band and 64-column block
+
 template <int G, int BITS, bool CLIP, bool SYM>
-__global__ void __launch_bounds__(512, 2)
+__global__ void __launch_bounds__(kQThreads, 1024 / kQThreads)
 quantize_pack_tile_kernel(const __half* __restrict__ W, const float* __restrict__ a, float alpha,
                           int mode, const float* __restrict__ clip,
                           uint32_t* __restrict__ qweight, __half* __restrict__ scales,
                           uint8_t* __restrict__ zeros, int N, int K) {
     constexpr float top = (float)((1 << BITS) - 1);       // largest code
     __shared__ __align__(16) float s_sm[128];
-    __shared__ float2 s_mm[2][128];                        // G = 128: [block of the pair][row of the slab] (min, max)
-    const int kblk = blockIdx.x, slab = blockIdx.y;
+    __shared__ float2 s_mm[2][kQBands * 16];               // G = 128: [block of the pair][row] (min, max)
+    const int kblk = blockIdx.x;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int bw = warp & 7, ti = warp >> 3;
+    const int bw = warp % kQBands, ti = warp / kQBands;
     const int g = lane >> 2, t = lane & 3;
-    const int n0 = slab * 128 + bw * 16 + g;               // this lane's upper row; lower = n0 + 8
+    const int n0 = (blockIdx.y * kQBands + bw) * 16 + g;   // this lane's upper row; lower = n0 + 8
     const int kbase = kblk * 128;
 
     uint2 raw[2][4];                                       // [row h][word j] = columns 16j + 4t .. +3 of the block
@@ -112,9 +127,9 @@ quantize_pack_tile_kernel(const __half* __restrict__ W, const float* __restrict_
         for (int j = 0; j < 4; ++j)
             raw[h][j] = ldg_stream(reinterpret_cast<const uint2*>(
                 W + (size_t)(n0 + 8 * h) * K + kbase + ti * 64 + 16 * j + 4 * t));
-    if (threadIdx.x < 128) {
-        const int k = kbase + threadIdx.x;
-        s_sm[threadIdx.x] = channel_scale_one(mode == kAlphaZero ? 1.0f : a[k], alpha, mode);
+    for (int i = threadIdx.x; i < 128; i += kQThreads) {
+        const int k = kbase + i;
+        s_sm[i] = channel_scale_one(mode == kAlphaZero ? 1.0f : a[k], alpha, mode);
     }
     __syncthreads();
 
@@ -128,11 +143,12 @@ quantize_pack_tile_kernel(const __half* __restrict__ W, const float* __restrict_
         const float4 s4 = *reinterpret_cast<const float4*>(&s_sm[ti * 64 + 16 * j + 4 * t]);
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
-            const uint32_t u0 = raw[h][j].x, u1 = raw[h][j].y;
-            wp[h][j][0] = __fmul_rn(__half2float(__ushort_as_half((unsigned short)(u0 & 0xFFFFu))), s4.x);
-            wp[h][j][1] = __fmul_rn(__half2float(__ushort_as_half((unsigned short)(u0 >> 16))), s4.y);
-            wp[h][j][2] = __fmul_rn(__half2float(__ushort_as_half((unsigned short)(u1 & 0xFFFFu))), s4.z);
-            wp[h][j][3] = __fmul_rn(__half2float(__ushort_as_half((unsigned short)(u1 >> 16))), s4.w);
+            const float2 f01 = __half22float2(*reinterpret_cast<const __half2*>(&raw[h][j].x));
+            const float2 f23 = __half22float2(*reinterpret_cast<const __half2*>(&raw[h][j].y));
+            wp[h][j][0] = __fmul_rn(f01.x, s4.x);
+            wp[h][j][1] = __fmul_rn(f01.y, s4.y);
+            wp[h][j][2] = __fmul_rn(f23.x, s4.z);
+            wp[h][j][3] = __fmul_rn(f23.y, s4.w);
             mn[h] = min3(mn[h], wp[h][j][0], wp[h][j][1]);
             mn[h] = min3(mn[h], wp[h][j][2], wp[h][j][3]);
             mx[h] = max3(mx[h], wp[h][j][0], wp[h][j][1]);
@@ -194,26 +210,48 @@ quantize_pack_tile_kernel(const __half* __restrict__ W, const float* __restrict_
         const float tmax = __fmul_rn(wabs[h], rd[h]);
         thr[h] = tmax < 1024.0f ? 0.5f - fmaf(tmax, 4e-7f, 1e-6f) : -1.0f;
     }
-    uint32_t words[4];
+    // Clamping to [0, top] can only matter where the group's smallest or largest element leaves the
+    // range (the level is monotone in w'): rare without clipping - rne(max / Delta) + rne(-min / Delta)
+    // exceeds top only when both quotients sit on a tie - so the warp takes the clamped code only if one
+    // of its lanes needs it.
+    bool need_clamp = CLIP || SYM;
+    if (!need_clamp) {
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
-        bool bad = false;
-        float qu[4], ql[4];
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-            qu[e] = level_fast2(wp[0][j][e], rd[0], zc[0], top, thr[0], bad);
-            ql[e] = level_fast2(wp[1][j][e], rd[1], zc[1], top, thr[1], bad);
+        for (int h = 0; h < 2; ++h) {
+            float dummy;
+            const float qlo = level_fast2<false>(mn[h], rd[h], zc[h], top, dummy);
+            const float qhi = level_fast2<false>(mx[h], rd[h], zc[h], top, dummy);
+            need_clamp = need_clamp || !(qlo >= 0.0f && qhi <= top);
         }
-        // nibbles 0 .. 3 = (g,c) (g+8,c) (g,c+2) (g+8,c+2), nibbles 4 .. 7 the same for c+1, c+3
-        words[j] = pack4(qu[0], ql[0], qu[2], ql[2]) | (pack4(qu[1], ql[1], qu[3], ql[3]) << 16);
-        if (bad)                                               // rare: the word again, element by element
-            words[j] = (code_of(wp[0][j][0], d[0], rd[0], z[0], top) << 0) | (code_of(wp[0][j][1], d[0], rd[0], z[0], top) << 16) |
-                       (code_of(wp[1][j][0], d[1], rd[1], z[1], top) << 4) | (code_of(wp[1][j][1], d[1], rd[1], z[1], top) << 20) |
-                       (code_of(wp[0][j][2], d[0], rd[0], z[0], top) << 8) | (code_of(wp[0][j][3], d[0], rd[0], z[0], top) << 24) |
-                       (code_of(wp[1][j][2], d[1], rd[1], z[1], top) << 12) | (code_of(wp[1][j][3], d[1], rd[1], z[1], top) << 28);
+        need_clamp = __any_sync(0xFFFFFFFFu, need_clamp);
     }
+    uint32_t words[4];
+    auto quantize_words = [&](auto clamp_tag) {
+        constexpr bool CL = decltype(clamp_tag)::value;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            float qu[4], ql[4], du[4], dl[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                qu[e] = level_fast2<CL>(wp[0][j][e], rd[0], zc[0], top, du[e]);
+                ql[e] = level_fast2<CL>(wp[1][j][e], rd[1], zc[1], top, dl[e]);
+            }
+            // the word's largest distance from the rounded value, per row, decides
+            const float dmu = max3(max3(du[0], du[1], du[2]), du[3], 0.0f);
+            const float dml = max3(max3(dl[0], dl[1], dl[2]), dl[3], 0.0f);
+            const bool bad = !(dmu < thr[0]) || !(dml < thr[1]);
+            // nibbles 0 .. 3 = (g,c) (g+8,c) (g,c+2) (g+8,c+2), nibbles 4 .. 7 the same for c+1, c+3
+            words[j] = pack4(qu[0], ql[0], qu[2], ql[2]) | (pack4(qu[1], ql[1], qu[3], ql[3]) << 16);
+            if (bad)                                               // rare: the word again, element by element
+                words[j] = (code_of(wp[0][j][0], d[0], rd[0], z[0], top) << 0) | (code_of(wp[0][j][1], d[0], rd[0], z[0], top) << 16) |
+                           (code_of(wp[1][j][0], d[1], rd[1], z[1], top) << 4) | (code_of(wp[1][j][1], d[1], rd[1], z[1], top) << 20) |
+                           (code_of(wp[0][j][2], d[0], rd[0], z[0], top) << 8) | (code_of(wp[0][j][3], d[0], rd[0], z[0], top) << 24) |
+                           (code_of(wp[1][j][2], d[1], rd[1], z[1], top) << 12) | (code_of(wp[1][j][3], d[1], rd[1], z[1], top) << 28);
+        }
+    };
+    if (need_clamp) quantize_words(std::true_type{}); else quantize_words(std::false_type{});
     // band-major: block (band, k-tile) is 512 bytes, a band's blocks are contiguous along K
-    const size_t band = (size_t)slab * 8 + bw;
+    const size_t band = (size_t)blockIdx.y * kQBands + bw;
     const size_t block = band * (K / 64) + (size_t)kblk * 2 + ti;
     uint4* dst = reinterpret_cast<uint4*>(qweight) + block * 32 + lane;
     *dst = make_uint4(words[0], words[1], words[2], words[3]);
@@ -335,10 +373,10 @@ cudaError_t launch_channel_scale(const float* a, float alpha, float* s, int K, c
 cudaError_t launch_quantize_pack(const __half* W, const float* a, float alpha, int group, int bits,
                                  bool symmetric, const float* clip, uint32_t* qweight, __half* scales, uint8_t* zeros,
                                  int N, int K, cudaStream_t st) {
-    const dim3 grid(K / 128, N / 128);
+    const dim3 grid(K / 128, N / (16 * kQBands));
     const int mode = (int)alpha_mode(alpha);
 #define AWQ_QP_LAUNCH(GG, BB, CC, SS) \
-    quantize_pack_tile_kernel<GG, BB, CC, SS><<<grid, 512, 0, st>>>(W, a, alpha, mode, clip, qweight, scales, zeros, N, K)
+    quantize_pack_tile_kernel<GG, BB, CC, SS><<<grid, kQThreads, 0, st>>>(W, a, alpha, mode, clip, qweight, scales, zeros, N, K)
 #define AWQ_QP_PICK2(GG, SS)                                             \
     do {                                                                 \
         if (bits == 4 && !clip) AWQ_QP_LAUNCH(GG, 4, false, SS);         \
