@@ -66,9 +66,9 @@ typedef enum AwqStatus {
 /* Which kernel awq_linear_path runs. */
 typedef enum AwqPath {
     AWQ_PATH_AUTO = 0,          /* what awq_linear does: the matrix-vector kernels for M <= 8, the
-                                   chunked matrix-vector kernel for 9 <= M <= 16 if K is a multiple of
-                                   2048 and a workspace of awq_workspace_bytes is registered, else the
-                                   tensor-core kernels */
+                                   chunked matrix-vector kernel for 9 <= M <= 16 (up to 24 where
+                                   N * K >= 2^25) if a workspace of awq_workspace_bytes is registered,
+                                   else the tensor-core kernels */
     AWQ_PATH_GEMV = 1,          /* fused dequant matrix-vector kernel, M <= 16: band kernel when
                                    M <= 8 and N/16 is not much below the SM count, else split-K */
     AWQ_PATH_GEMM = 2,          /* tcgen05 tensor-core kernel, any M >= 1: pairs of SMs
@@ -77,9 +77,10 @@ typedef enum AwqPath {
                                    N = 16384), else one SM per tile */
     AWQ_PATH_GEMV_SPLITK = 3,   /* the split-K matrix-vector kernel, M <= 16 */
     AWQ_PATH_GEMM_1SM = 4,      /* the tensor-core kernel with one SM per tile, any M >= 1 */
-    AWQ_PATH_GEMV_MID = 5       /* the chunked matrix-vector kernel, M <= 32: a block owns a chunk of K,
-                                   keeps its slice of x in shared memory and streams band runs; needs
-                                   a workspace of awq_workspace_bytes (fp32 partial sums per chunk) */
+    AWQ_PATH_GEMV_MID = 5       /* the chunked matrix-vector kernel, 9 <= M <= 32: work units of 16 bands
+                                   x 1024 input channels, the unit's slice of x in shared memory, one
+                                   band per warp; needs a workspace of awq_workspace_bytes (fp32 partial
+                                   sums per chunk of K) */
 } AwqPath;
 
 /* Sizes of the packed arrays, in bytes (0 if the shape is not accepted). */
@@ -150,9 +151,9 @@ int awq_channel_scale(const float* act_mean_abs, float alpha, float* s, int K, v
  * x: in, fp16 [M][K].  y: out, fp16 [M][N], fully overwritten; must not alias an input.
  * M <= 8 runs a matrix-vector kernel (HBM-bound; the 4-bit codes enter warp-level tensor-core
  * products exactly, accumulation, zero point and Delta in fp32, one rounding to fp16 at the
- * end), and so does 8 < M <= 16 with K a multiple of 2048 when the registered workspace holds
+ * end), and so does 8 < M <= 16 (<= 24 where N * K >= 2^25) when the registered workspace holds
  * awq_workspace_bytes (the chunked kernel, AWQ_PATH_GEMV_MID: same arithmetic, partial sums per
- * chunk of K added in a fixed order by a second small kernel); everything else the tcgen05 kernel
+ * chunk of 1024 input channels added in a fixed order by a second small kernel); everything else the tcgen05 kernel
  * ((q - z) * Delta rounded once to fp16, fp32 accumulation in tensor memory).  Results are
  * bit-reproducible.
  * The split-K matrix-vector kernel (used when N is small or M > 8) combines partial sums in a

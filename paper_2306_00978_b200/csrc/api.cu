@@ -160,14 +160,14 @@ int awq_search_clip(const void* W, const float* act_mean_abs, float alpha, int g
                                         ratios, n_ratios, clip_ratio, N, K, (cudaStream_t)stream));
 }
 
-// Where the chunked matrix-vector kernel beats the other kernels (measured at 9 and 16 tokens:
-// 17.9 against 26 us on 4096 -> 11008, 12.3 against 13.6 us on 4096 -> 4096, 54 against 98 us
-// (tensor-core kernel) and 72 us (split-K matrix-vector kernel) on 8192 -> 28672, 60 against 102 us
-// on 28672 -> 8192; with a ragged last chunk it loses: 28 against 26 us on 11008 -> 4096; from 17
-// tokens on the tensor-core kernels are as fast or faster).
+// Where the chunked matrix-vector kernel beats the tensor-core kernels (measured, us, chunked against
+// tensor-core: at 16 tokens 10.9 / 13.5 on 4096 -> 4096, 17.4 / 25.9 on 4096 -> 11008, 20.9 / 26.2 on
+// 11008 -> 4096, 45 / 98 on 8192 -> 28672; at 24 tokens 14.0 / 13.9, 23.2 / 26.1, 27.4 / 26.2, 60.7 / 98;
+// at 32 tokens 17.6 / 13.8, 28.4 / 25.8, 33.4 / 26.4, 79 / 81).
 static bool mid_kernel_preferred(int M, int N, int K) {
-    (void)N;
-    return M > 8 && M <= 16 && K % 2048 == 0;
+    if (M <= 8) return false;
+    if (M <= 16) return true;
+    return M <= 24 && (long long)N * K >= (1LL << 25);
 }
 
 static int resolve_path(int M, int K, int path) {
@@ -223,7 +223,7 @@ int awq_linear_path(const void* x, const void* qweight, const void* scales, cons
     const bool automatic = path == AWQ_PATH_AUTO;
     path = resolve_path(M, K, path);
     if (path == AWQ_PATH_GEMV_MID) {
-        if (M > 64 || K > 65536) return AWQ_ERR_BAD_SHAPE;
+        if (M > 32 || K > 65536) return AWQ_ERR_BAD_SHAPE;
     } else if (path != AWQ_PATH_GEMM && path != AWQ_PATH_GEMM_1SM && (M > 16 || K > 65536)) {
         return AWQ_ERR_BAD_SHAPE;
     }

@@ -197,25 +197,19 @@ def test_quantize_then_linear_back_to_back_on_one_stream():
 
 
 def test_auto_dispatch_between_9_and_16_tokens():
-    """awq_linear with 9..16 tokens: the tensor-core kernel where K is not a multiple of 2048 (or no
-    workspace is registered), the chunked matrix-vector kernel otherwise.  Each result is bit-equal
-    to its forced path."""
+    """awq_linear with 9..16 tokens: the chunked matrix-vector kernel when a workspace is registered
+    (the binding registers one), the tensor-core kernel otherwise.  Each result is bit-equal to its
+    forced path."""
     import torch
     from paper_2306_00978_b200 import binding
     L = binding.lib()
-    case = Case(77, 1024, 1408, 12, 128, 0.5)
-    qw, sc, zp = oracle_packed_to_cuda(case)
-    x = to_cuda(case.x)
-    auto = binding.linear(x, qw, sc, zp, case.N, case.K, case.group)
-    forced_gemm = binding.linear(x, qw, sc, zp, case.N, case.K, case.group, path=binding.PATH_GEMM)
-    assert torch.equal(auto, forced_gemm)
-    assert_parity(auto.cpu().numpy(), case.y_ref(), "auto M=12, K not a multiple of 2048")
-    case = Case(78, 1024, 4096, 12, 128, 0.5)
-    qw, sc, zp = oracle_packed_to_cuda(case)
-    x = to_cuda(case.x)
-    auto = binding.linear(x, qw, sc, zp, case.N, case.K, case.group)
-    assert torch.equal(auto, binding.linear(x, qw, sc, zp, case.N, case.K, case.group, path=binding.PATH_GEMV_MID))
-    assert_parity(auto.cpu().numpy(), case.y_ref(), "auto M=12, chunked kernel")
+    for (N, K) in ((1024, 1408), (1024, 4096)):
+        case = Case(77 + K, N, K, 12, 128, 0.5)
+        qw, sc, zp = oracle_packed_to_cuda(case)
+        x = to_cuda(case.x)
+        auto = binding.linear(x, qw, sc, zp, case.N, case.K, case.group)
+        assert torch.equal(auto, binding.linear(x, qw, sc, zp, case.N, case.K, case.group, path=binding.PATH_GEMV_MID))
+        assert_parity(auto.cpu().numpy(), case.y_ref(), f"auto M=12, chunked kernel, K={K}")
     # a large matrix (random packed arrays: only the choice of kernel is checked here; parity at
     # this size is covered by the 70B sweep)
     N, K, G, M = 16384, 8192, 128, 12
@@ -295,17 +289,18 @@ def test_missing_workspace_is_reported():
 
 
 @pytest.mark.parametrize("N,K,M,G", [
-    (512, 1024, 9, 128),      # half a chunk only
-    (1024, 1408, 16, 128),    # ragged second... first chunk: 22 k-tiles
-    (768, 4096, 17, 64),      # two token groups, four chunks of 1024
-    (512, 2304, 32, 128),     # ragged last chunk
-    (640, 2048, 24, 64),
-    (2432, 4096, 13, 128),    # more bands than blocks of a chunk
-    (128, 8192, 10, 128),     # fewer bands than blocks
+    (512, 1024, 9, 128),      # one chunk
+    (1024, 1408, 16, 128),    # ragged second chunk (6 k-tiles)
+    (768, 4096, 17, 64),      # three token fragments, four chunks
+    (512, 2304, 32, 128),     # four token fragments, ragged last chunk
+    (640, 2048, 24, 64),      # 40 bands: a last unit of 8 bands
+    (2432, 4096, 13, 128),    # more units than blocks
+    (128, 8192, 10, 128),     # one unit of 8 bands per chunk
+    (4224, 1152, 9, 128),     # units crossing from one chunk to the next inside a block
 ])
 def test_chunked_matrix_vector_kernel(N, K, M, G):
-    """AWQ_PATH_GEMV_MID: a block owns a chunk of K; partial sums per chunk, added by a second
-    kernel.  Parity with the oracle and bit-reproducibility."""
+    """AWQ_PATH_GEMV_MID: units of 16 bands x 1024 input channels, one band per warp; partial sums
+    per chunk, added by a second kernel.  Parity with the oracle and bit-reproducibility."""
     from paper_2306_00978_b200 import binding
     case = Case(600 + N + K + M + G, N, K, M, G, 0.5)
     y = _run(case, binding.PATH_GEMV_MID)
