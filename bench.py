@@ -781,6 +781,25 @@ def sweep_rows(peaks, groups=(128, 64), reps: int = 5):
             torch.cuda.empty_cache()
 
 
+def quantize_only(args):
+    """A small, self-contained run of the quantize+pack kernel for ncu captures."""
+    import torch
+    from paper_2306_00978_b200 import binding
+    N, K = args.quantize_only
+    W = torch.from_numpy(synth.weight(2004, N, K)).cuda()
+    a = torch.from_numpy(synth.act_mean_abs(2004, K)).cuda()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for r in range(args.reps + 1):
+        if r == args.reps:
+            e0.record()
+        binding.quantize_pack(W, a, ALPHA, GROUP)
+    e1.record()
+    torch.cuda.synchronize()
+    nbytes = 2 * N * K + 4 * K + N * K // 2 + 2 * N * K // GROUP + N * K // (2 * GROUP)
+    print(json.dumps({"quantize_only": [N, K], "us_last_launch": e0.elapsed_time(e1) * 1e3, "algorithmic_bytes": nbytes}))
+    return 0
+
+
 def sweep(args):
     """The full-shape sweep, one JSON object per line."""
     peaks = load_peaks()
@@ -803,11 +822,15 @@ def main():
                          "weights (three rotating copies), then exit")
     ap.add_argument("--path", type=int, default=0, help="with --one: 0 auto, 1 GEMV, 2 GEMM, 3 split-K GEMV, 4 single-SM GEMM")
     ap.add_argument("--reps", type=int, default=3, help="with --one: passes over the three copies")
+    ap.add_argument("--quantize-only", nargs=2, type=int, metavar=("N", "K"),
+                    help="profiling aid: a few awq_quantize_pack launches on seeded weights of one shape, then exit")
     ap.add_argument("--sweep", action="store_true",
                     help="per-shape table over the 7B layer shapes, M = 1 .. 8192, both group sizes; then exit")
     args = ap.parse_args()
     if args.one:
         return one_shape(args)
+    if args.quantize_only:
+        return quantize_only(args)
     if args.sweep:
         return sweep(args)
 
