@@ -13,8 +13,7 @@ from typing import Optional, Tuple
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-# AWQ_B200_LIB selects another build of the same library (an experiment, a debug build)
-LIB_PATH = os.environ.get("AWQ_B200_LIB") or os.path.join(_HERE, "libawq_b200.so")
+LIB_PATH = os.path.join(_HERE, "libawq_b200.so")
 
 PATH_AUTO, PATH_GEMV, PATH_GEMM, PATH_GEMV_SPLITK, PATH_GEMM_1SM, PATH_GEMV_MID = 0, 1, 2, 3, 4, 5
 

@@ -34,17 +34,16 @@ def _stale() -> bool:
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def build(force: bool = False, verbose: bool = False, out: str = LIB_PATH, extra=()) -> str:
-    """Compile every kernel for sm_100a into one shared library; returns its path.
-    `extra` are additional nvcc flags (e.g. -D switches for an experiment), `out` the library
-    to write."""
-    if not force and not _stale() and out == LIB_PATH:
+def build(force: bool = False, verbose: bool = False) -> str:
+    """Compile every kernel for sm_100a into one shared library; returns its path."""
+    out = LIB_PATH
+    if not force and not _stale():
         return LIB_PATH
     objs = []
     procs = []
     for src in SOURCES:
         obj = os.path.join(CSRC, src.replace(".cu", ".o"))
-        cmd = [_nvcc(), *NVCC_FLAGS, *extra, "-c", os.path.join(CSRC, src), "-o", obj]
+        cmd = [_nvcc(), *NVCC_FLAGS, "-c", os.path.join(CSRC, src), "-o", obj]
         if verbose:
             cmd.insert(1, "-Xptxas=-v")
         procs.append((src, subprocess.Popen(cmd, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)))
@@ -63,7 +62,4 @@ def build(force: bool = False, verbose: bool = False, out: str = LIB_PATH, extra
 
 
 if __name__ == "__main__":
-    _extra = tuple(a for a in sys.argv[1:] if a.startswith("-D"))
-    _out = [a[6:] for a in sys.argv[1:] if a.startswith("--out=")]
-    print(build(force="--force" in sys.argv or bool(_extra), verbose="-v" in sys.argv,
-                out=_out[0] if _out else LIB_PATH, extra=_extra))
+    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))

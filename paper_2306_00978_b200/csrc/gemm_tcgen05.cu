@@ -43,10 +43,7 @@ namespace {
 
 constexpr int kGemmThreads = 512;
 constexpr int kMaxSplits = 16;                  // split-K factor of a tile (M <= 128)
-#ifndef AWQ_DEQUANT_UNROLL
-#define AWQ_DEQUANT_UNROLL 2
-#endif
-constexpr int kDequantUnroll = AWQ_DEQUANT_UNROLL;   // k-blocks a dequantizer warp handles per iteration
+constexpr int kDequantUnroll = 2;               // k-blocks a dequantizer warp handles per iteration
 
 template <int BN> struct GemmCfg {
     static constexpr int kXTileBytes = BN * kBK * 2;
