@@ -164,10 +164,18 @@ int awq_search_clip(const void* W, const float* act_mean_abs, float alpha, int g
 // tensor-core: at 16 tokens 10.9 / 13.5 on 4096 -> 4096, 17.4 / 25.9 on 4096 -> 11008, 20.9 / 26.2 on
 // 11008 -> 4096, 45 / 98 on 8192 -> 28672; at 24 tokens 14.0 / 13.9, 23.2 / 26.1, 27.4 / 26.2, 60.7 / 98;
 // at 32 tokens 17.6 / 13.8, 28.4 / 25.8, 33.4 / 26.4, 79 / 81).
+// With one token fragment its time does not depend on M (34 us on the 70B shapes for 1 .. 8 tokens),
+// while the band kernel's grows with the tokens that travel through its stages: on large matrices it
+// wins from 3 tokens (8192 -> 28672: 32.7 / 34.5 at 3, 33.9 / 39.0 at 5, 34.3 / 49.0 at 8), on middle-sized
+// ones from 5 (5120 -> 13824: 15.1 / 15.0 at 5, 15.5 / 19.1 at 8; 8192 -> 16384: 21.0 / 23.6 at 5); on
+// 4096 -> 11008 the band kernel wins up to 8 tokens (9.8 against 13.6).
 static bool mid_kernel_preferred(int M, int N, int K) {
-    if (M <= 8) return false;
+    const long long nk = (long long)N * K;
+    if (M <= 2) return false;
+    if (M <= 4) return nk > (1LL << 27);
+    if (M <= 8) return nk >= (1LL << 26);
     if (M <= 16) return true;
-    return M <= 24 && (long long)N * K >= (1LL << 25);
+    return M <= 24 && nk >= (1LL << 25);
 }
 
 static int resolve_path(int M, int K, int path) {
@@ -185,13 +193,11 @@ size_t awq_workspace_bytes(int M, int N, int K, int group) {
         sms = 160;                           // no device to ask: an upper bound for this GPU family
     }
     size_t gemm = gemm_workspace_bytes(M, N, sms);
-    if (M > 8 && M <= 32 && gemv_mid_applies(M, N, K, group, sms)) {
-        const size_t mid = gemv_mid_workspace_bytes(M, N, K);
-        if (mid > gemm) gemm = mid;
-    }
+    const size_t mid = (M <= 32 && gemv_mid_applies(M, N, K, group, sms)) ? gemv_mid_workspace_bytes(M, N, K) : 0;
+    if (M > 8 && mid > gemm) gemm = mid;
     if (M > 16) return gemm;
     const size_t gemv = gemv_workspace_bytes(M);   // required by the split-K matrix-vector kernel
-    if (M <= 8) return gemv;                       // awq_linear never takes the tensor-core kernel here
+    if (M <= 8) return gemv > mid ? gemv : mid;    // awq_linear never takes the tensor-core kernel here
     return gemv > gemm ? gemv : gemm;
 }
 

@@ -309,7 +309,7 @@ size_t gemv_mid_workspace_bytes(int M, int N, int K) {
 }
 bool gemv_mid_applies(int M, int N, int K, int group, int sms) {
     (void)N; (void)sms;
-    if (M < 9 || M > 32 || K > 65536) return false;
+    if (M < 1 || M > 32 || K > 65536) return false;
     return mid_layout(M, group).total <= kMidSmem && encode_fn() != nullptr;
 }
 
@@ -383,7 +383,8 @@ cudaError_t launch_gemv_mid(const void* x, const void* qweight, const void* scal
     } while (0)
 #define AWQ_MID_PICK(GG)                                                                            \
     do {                                                                                            \
-        if (lay.mtok <= 16) AWQ_MID_LAUNCH(GG, 2);                                                  \
+        if (lay.mtok <= 8) AWQ_MID_LAUNCH(GG, 1);                                                   \
+        else if (lay.mtok <= 16) AWQ_MID_LAUNCH(GG, 2);                                             \
         else if (lay.mtok <= 24) AWQ_MID_LAUNCH(GG, 3);                                             \
         else AWQ_MID_LAUNCH(GG, 4);                                                                 \
     } while (0)
