@@ -283,6 +283,10 @@ gemv_mid_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
 // y[m][n] = fp16(sum over the chunks, ascending, of partial[c][m][n]): four outputs per thread.
 __global__ void __launch_bounds__(256)
 gemv_mid_reduce_kernel(const float* __restrict__ partial, __half* __restrict__ y, int chunks, size_t mn) {
+    // launched with programmatic stream serialization behind the kernel above: it may be resident
+    // before that kernel has finished, and lets the launch behind it start its own weight copies
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const size_t i = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * 4;
     if (i >= mn) return;
     float4 s = *reinterpret_cast<const float4*>(partial + i);
@@ -393,8 +397,14 @@ cudaError_t launch_gemv_mid(const void* x, const void* qweight, const void* scal
 #undef AWQ_MID_LAUNCH
     count_launch();
     const size_t mn = (size_t)M * N;
-    gemv_mid_reduce_kernel<<<(unsigned)((mn / 4 + 255) / 256), 256, 0, st>>>(partial, reinterpret_cast<__half*>(y),
-                                                                             chunks, mn);
+    cudaLaunchConfig_t rcfg = {};
+    rcfg.gridDim = dim3((unsigned)((mn / 4 + 255) / 256));
+    rcfg.blockDim = dim3(256);
+    rcfg.stream = st;
+    rcfg.attrs = attr;
+    rcfg.numAttrs = 1;
+    e = cudaLaunchKernelEx(&rcfg, gemv_mid_reduce_kernel, (const float*)partial, reinterpret_cast<__half*>(y), chunks, mn);
+    if (e != cudaSuccess) return e;
     count_launch();
     return cudaGetLastError();
 }
