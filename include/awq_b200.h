@@ -67,8 +67,8 @@ typedef enum AwqStatus {
 typedef enum AwqPath {
     AWQ_PATH_AUTO = 0,          /* what awq_linear does: the matrix-vector kernels for M <= 8; the
                                    chunked matrix-vector kernel for 9 <= M <= 16 (up to 24 where
-                                   N * K >= 2^25), and on large matrices already from 3 tokens
-                                   (N * K > 2^27) or 5 tokens (N * K >= 2^26), if a workspace of
+                                   N * K >= 2^25), and where K > 4096 already from 3 tokens
+                                   (N * K >= 2^26) or 5 tokens (N * K >= 2^25), if a workspace of
                                    awq_workspace_bytes is registered; else the tensor-core kernels */
     AWQ_PATH_GEMV = 1,          /* fused dequant matrix-vector kernel, M <= 16: band kernel when
                                    M <= 8 and N/16 is not much below the SM count, else split-K */

@@ -164,16 +164,20 @@ int awq_search_clip(const void* W, const float* act_mean_abs, float alpha, int g
 // tensor-core: at 16 tokens 10.9 / 13.5 on 4096 -> 4096, 17.4 / 25.9 on 4096 -> 11008, 20.9 / 26.2 on
 // 11008 -> 4096, 45 / 98 on 8192 -> 28672; at 24 tokens 14.0 / 13.9, 23.2 / 26.1, 27.4 / 26.2, 60.7 / 98;
 // at 32 tokens 17.6 / 13.8, 28.4 / 25.8, 33.4 / 26.4, 79 / 81).
-// With one token fragment its time does not depend on M (34 us on the 70B shapes for 1 .. 8 tokens),
-// while the band kernel's grows with the tokens that travel through its stages: on large matrices it
-// wins from 3 tokens (8192 -> 28672: 32.7 / 34.5 at 3, 33.9 / 39.0 at 5, 34.3 / 49.0 at 8), on middle-sized
-// ones from 5 (5120 -> 13824: 15.1 / 15.0 at 5, 15.5 / 19.1 at 8; 8192 -> 16384: 21.0 / 23.6 at 5); on
-// 4096 -> 11008 the band kernel wins up to 8 tokens (9.8 against 13.6).
+// With one token fragment its time does not depend on M (32 us on the 70B shapes for 1 .. 8 tokens),
+// while the band kernel's grows with the tokens that travel through its stages.  Chunked / band, us:
+//   8192 -> 28672   3 tokens 31.3 / 34.5   5: 31.9 / 38.9   8: 32.5 / 49.1
+//   8192 -> 16384   3: 19.1 / 20.4   4: 19.2 / 20.7   8: 19.5 / 29.2
+//   8192 -> 8192    3: 13.0 / 13.0   4: 12.8 / 13.4   8: 13.2 / 18.7
+//   13824 -> 5120   3: 14.7 / 16.3   4: 14.8 / 17.5   8: 15.0 / 24.1
+//   5120 -> 13824   3: 13.6 / 13.4   4: 13.6 / 13.8   5: 13.7 / 15.1
+//   11008 -> 4096   4: 12.9 / 11.3   5: 13.1 / 12.9   6: 13.3 / 14.8   8: 13.1 / 16.1
+// With 4096 input channels the band kernel keeps x in registers and wins up to 8 tokens
+// (4096 -> 11008 at 8 tokens: 11.7 / 9.8; 4096 -> 4096: 6.5 / 6.9).
 static bool mid_kernel_preferred(int M, int N, int K) {
     const long long nk = (long long)N * K;
     if (M <= 2) return false;
-    if (M <= 4) return nk > (1LL << 27);
-    if (M <= 8) return nk >= (1LL << 26);
+    if (M <= 8) return K > 4096 && nk >= (M <= 4 ? (1LL << 26) : (1LL << 25));
     if (M <= 16) return true;
     return M <= 24 && nk >= (1LL << 25);
 }

@@ -29,7 +29,7 @@ namespace {
 constexpr int kMidMathWarps = 16;
 constexpr int kMidThreads = (kMidMathWarps + 1) * 32;   // + producer warp
 constexpr int kMidSmem = 220 * 1024;
-constexpr int kMidChunkTiles = 16;                       // k-tiles (64 columns) per chunk
+constexpr int kMidChunkTiles = 16;                       // k-tiles (64 columns) per chunk: 16, or 8 where that fills the SMs better
 constexpr int kMidStageTiles = 2;                        // k-tiles per stage and band
 constexpr int kMidStageBytes = kMidMathWarps * kMidStageTiles * 512;
 constexpr int kMidStages = 8;
@@ -58,12 +58,12 @@ struct MidLayout {
     int bar_off, total;
 };
 
-inline MidLayout mid_layout(int M, int group) {
+inline MidLayout mid_layout(int M, int group, int chunk_tiles = kMidChunkTiles) {
     MidLayout l;
     l.mtok = ((M + 7) / 8) * 8;
-    const int groups = kMidChunkTiles * 64 / group;       // 8 or 16
+    const int groups = chunk_tiles * 64 / group;
     l.x_off = kMidStages * kMidStageBytes;
-    l.x_row = kMidChunkTiles * 128 + 32;
+    l.x_row = chunk_tiles * 128 + 32;
     l.xg_off = l.x_off + ((l.mtok * l.x_row + 127) / 128) * 128;
     l.par_off = l.xg_off + ((groups * l.mtok * 4 + 127) / 128) * 128;
     l.z_in_par = kMidMathWarps * groups * 32;
@@ -73,8 +73,8 @@ inline MidLayout mid_layout(int M, int group) {
     return l;
 }
 
-// MT = 8-token B fragments per product (tokens rounded up to 8 MT).
-template <int G, int MT>
+// MT = 8-token B fragments per product (tokens rounded up to 8 MT); CT = k-tiles per chunk.
+template <int G, int MT, int CT>
 __global__ void __launch_bounds__(kMidThreads, 1)
 gemv_mid_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant__ CUtensorMap sc_map,
                 const __grid_constant__ CUtensorMap z_map, const __half* __restrict__ x,
@@ -83,14 +83,14 @@ gemv_mid_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
     extern __shared__ __align__(1024) unsigned char smem[];
     __shared__ unsigned int s_abort;
     constexpr int TPG = G / 64;                          // k-tiles per group
-    constexpr int GPC = kMidChunkTiles / TPG;            // groups per chunk
+    constexpr int GPC = CT / TPG;                        // groups per chunk
     constexpr int S = kMidStages;
     const uint32_t sbase = smem_u32(smem);
     // barriers: full[s] at 8s, empty[s] at 64 + 8s, par_full[b] at 128 + 8b, par_empty[b] at 160 + 8b
     const uint32_t bars = sbase + (uint32_t)lay.bar_off;
     const int ktiles = K / 64, nbands = N / 16;
     const int nbg = (nbands + kMidMathWarps - 1) / kMidMathWarps;
-    const int nchunks = (ktiles + kMidChunkTiles - 1) / kMidChunkTiles;
+    const int nchunks = (ktiles + CT - 1) / CT;
     const int units = nchunks * nbg;
     const int u0 = (int)(((long long)units * blockIdx.x) / gridDim.x);
     const int u1 = (int)(((long long)units * (blockIdx.x + 1)) / gridDim.x);
@@ -121,8 +121,8 @@ gemv_mid_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
         bool ok = true;
         for (int u = u0; u < u1 && ok; ++u) {
             const int c = u / nbg, bg = u - c * nbg;
-            const int kt0 = c * kMidChunkTiles;
-            const int nt = min(kMidChunkTiles, ktiles - kt0);
+            const int kt0 = c * CT;
+            const int nt = min(CT, ktiles - kt0);
             const uint32_t pb = (uint32_t)(u - u0) & 1u, puse = ((uint32_t)(u - u0) >> 1) & 1u;
             if (!mbar_wait_relaxed(bars + 160u + 8u * pb, puse ^ 1u, ctl)) break;
             const uint32_t pdst = sbase + (uint32_t)lay.par_off + pb * (uint32_t)lay.par_bytes;
@@ -163,8 +163,8 @@ gemv_mid_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
     int cur_chunk = -1;
     for (int u = u0; u < u1; ++u) {
         const int c = u / nbg, bg = u - c * nbg;
-        const int kt0 = c * kMidChunkTiles;
-        const int nt = min(kMidChunkTiles, ktiles - kt0);
+        const int kt0 = c * CT;
+        const int nt = min(CT, ktiles - kt0);
         if (c != cur_chunk) {
             // a new chunk: its slice of x (rows of nt * 64 halfs, absent tokens as zeros) and the sums
             // of x over each group and token, times 2^-24 (the products carry that factor)
@@ -303,13 +303,25 @@ gemv_mid_reduce_kernel(const float* __restrict__ partial, __half* __restrict__ y
 
 }  // namespace
 
-// Chunks of K (the workspace holds one fp32 [M][N] array per chunk).
-int gemv_mid_chunks(int M, int K) {
-    (void)M;
-    return (K / 64 + kMidChunkTiles - 1) / kMidChunkTiles;
+// k-tiles per chunk for a problem: 16, or 8 where the units (chunks x groups of 16 bands) then fill
+// the blocks' equal shares much better (the slowest block sets the time).  Halving the chunk doubles
+// the partial sums (M / 32 of the weight bytes at 8 k-tiles, written and read back) and the per-unit
+// work (x slice, scales, filling the ring), so the gain has to be large.  Measured at 16 tokens:
+// 4096 -> 4096 10.4 -> 7.9 us and 11008 -> 4096 18.7 -> 16.9 us (shares 0.43 -> 0.86 and
+// 0.59 -> 0.79 full), but 28672 -> 8192 43.7 -> 51.6 us (0.87 -> 0.93; 33.9 -> 39.5 us at 4 tokens).
+static int mid_chunk_tiles(int N, int K, int sms) {
+    const int nbg = (N / 16 + kMidMathWarps - 1) / kMidMathWarps;
+    auto efficiency = [&](int ct) {
+        const int units = ((K / 64 + ct - 1) / ct) * nbg;
+        const int blocks = units < sms ? units : sms;
+        const int worst = (units + blocks - 1) / blocks;
+        return (double)units / ((double)worst * sms);
+    };
+    return efficiency(8) > efficiency(16) + 0.15 ? 8 : 16;
 }
+// The workspace holds one fp32 [M][N] array per chunk; sized for the smaller chunk.
 size_t gemv_mid_workspace_bytes(int M, int N, int K) {
-    return kCounterBytes + (size_t)gemv_mid_chunks(M, K) * M * N * sizeof(float);
+    return kCounterBytes + (size_t)((K / 64 + 7) / 8) * M * N * sizeof(float);
 }
 bool gemv_mid_applies(int M, int N, int K, int group, int sms) {
     (void)N; (void)sms;
@@ -322,8 +334,9 @@ cudaError_t launch_gemv_mid(const void* x, const void* qweight, const void* scal
                             bool serialize, cudaStream_t st) {
     EncodeTiledFn enc = encode_fn();
     if (!enc) return cudaErrorNotSupported;
-    const MidLayout lay = mid_layout(M, group);
-    const int ng = K / group, gpc = kMidChunkTiles * 64 / group;
+    const int ct = mid_chunk_tiles(N, K, sms);
+    const MidLayout lay = mid_layout(M, group, ct);
+    const int ng = K / group, gpc = ct * 64 / group;
     const cuuint32_t estr[2] = {1, 1};
     CUtensorMap wmap, scmap, zmap;
     {
@@ -357,7 +370,7 @@ cudaError_t launch_gemv_mid(const void* x, const void* qweight, const void* scal
             return cudaErrorInvalidValue;
     }
     float* partial = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(workspace) + kCounterBytes);
-    const int chunks = gemv_mid_chunks(M, K);
+    const int chunks = (K / 64 + ct - 1) / ct;
     const int units = chunks * ((N / 16 + kMidMathWarps - 1) / kMidMathWarps);
     cudaLaunchConfig_t cfg = {};
     cudaLaunchAttribute attr[1];
@@ -370,30 +383,35 @@ cudaError_t launch_gemv_mid(const void* x, const void* qweight, const void* scal
     cfg.attrs = attr;
     cfg.numAttrs = serialize ? 0 : 1;
     cudaError_t e;
-#define AWQ_MID_LAUNCH(GG, MTT)                                                                     \
+#define AWQ_MID_LAUNCH2(GG, MTT)                                                                    \
+    do {                                                                                            \
+        if (ct == 16) AWQ_MID_LAUNCH(GG, MTT, 16); else AWQ_MID_LAUNCH(GG, MTT, 8);                 \
+    } while (0)
+#define AWQ_MID_LAUNCH(GG, MTT, CTT)                                                                \
     do {                                                                                            \
         static bool done[64] = {};                                                                  \
         int dev = 0;                                                                                \
         e = cudaGetDevice(&dev);                                                                    \
         if (e != cudaSuccess) return e;                                                             \
         if (!done[dev & 63]) {                                                                      \
-            e = cudaFuncSetAttribute(gemv_mid_kernel<GG, MTT>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMidSmem); \
+            e = cudaFuncSetAttribute(gemv_mid_kernel<GG, MTT, CTT>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMidSmem); \
             if (e != cudaSuccess) return e;                                                         \
             done[dev & 63] = true;                                                                  \
         }                                                                                           \
-        e = cudaLaunchKernelEx(&cfg, gemv_mid_kernel<GG, MTT>, wmap, scmap, zmap,                   \
+        e = cudaLaunchKernelEx(&cfg, gemv_mid_kernel<GG, MTT, CTT>, wmap, scmap, zmap,                   \
                                reinterpret_cast<const __half*>(x), partial, M, N, K, lay, status_word); \
         if (e != cudaSuccess) return e;                                                             \
     } while (0)
 #define AWQ_MID_PICK(GG)                                                                            \
     do {                                                                                            \
-        if (lay.mtok <= 8) AWQ_MID_LAUNCH(GG, 1);                                                   \
-        else if (lay.mtok <= 16) AWQ_MID_LAUNCH(GG, 2);                                             \
-        else if (lay.mtok <= 24) AWQ_MID_LAUNCH(GG, 3);                                             \
-        else AWQ_MID_LAUNCH(GG, 4);                                                                 \
+        if (lay.mtok <= 8) AWQ_MID_LAUNCH2(GG, 1);                                                  \
+        else if (lay.mtok <= 16) AWQ_MID_LAUNCH2(GG, 2);                                            \
+        else if (lay.mtok <= 24) AWQ_MID_LAUNCH2(GG, 3);                                            \
+        else AWQ_MID_LAUNCH2(GG, 4);                                                                \
     } while (0)
     if (group == 128) AWQ_MID_PICK(128); else AWQ_MID_PICK(64);
 #undef AWQ_MID_PICK
+#undef AWQ_MID_LAUNCH2
 #undef AWQ_MID_LAUNCH
     count_launch();
     const size_t mn = (size_t)M * N;
