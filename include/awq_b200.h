@@ -68,8 +68,10 @@ typedef enum AwqPath {
     AWQ_PATH_AUTO = 0,          /* what awq_linear does: the matrix-vector kernels for M <= 8; the
                                    chunked matrix-vector kernel for 9 <= M <= 16 (up to 24 where
                                    N * K >= 2^25), and where K > 4096 already from 3 tokens
-                                   (N * K >= 2^26) or 5 tokens (N * K >= 2^25), if a workspace of
-                                   awq_workspace_bytes is registered; else the tensor-core kernels */
+                                   (N * K >= 2^26) or 5 tokens (N * K >= 2^25), and the chunked
+                                   tensor-core kernel for the other M <= 64 (N a multiple of 128), if
+                                   a workspace of awq_workspace_bytes is registered; else the
+                                   tensor-core prefill kernels */
     AWQ_PATH_GEMV = 1,          /* fused dequant matrix-vector kernel, M <= 16: band kernel when
                                    M <= 8 and N/16 is not much below the SM count, else split-K */
     AWQ_PATH_GEMM = 2,          /* tcgen05 tensor-core kernel, any M >= 1: pairs of SMs
@@ -78,10 +80,13 @@ typedef enum AwqPath {
                                    N = 16384), else one SM per tile */
     AWQ_PATH_GEMV_SPLITK = 3,   /* the split-K matrix-vector kernel, M <= 16 */
     AWQ_PATH_GEMM_1SM = 4,      /* the tensor-core kernel with one SM per tile, any M >= 1 */
-    AWQ_PATH_GEMV_MID = 5       /* the chunked matrix-vector kernel, M <= 32: work units of 16 bands
+    AWQ_PATH_GEMV_MID = 5,      /* the chunked matrix-vector kernel, M <= 32: work units of 16 bands
                                    x 1024 input channels, the unit's slice of x in shared memory, one
                                    band per warp; needs a workspace of awq_workspace_bytes (fp32 partial
                                    sums per chunk of K) */
+    AWQ_PATH_GEMM_SKINNY = 6    /* the chunked tensor-core kernel, M <= 64, N a multiple of 128: work
+                                   units of 128 channels x a chunk of K, the chunk's slice of x resident
+                                   in shared memory; needs a workspace of awq_workspace_bytes */
 } AwqPath;
 
 /* Sizes of the packed arrays, in bytes (0 if the shape is not accepted). */

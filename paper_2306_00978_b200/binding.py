@@ -15,7 +15,7 @@ import torch
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libawq_b200.so")
 
-PATH_AUTO, PATH_GEMV, PATH_GEMM, PATH_GEMV_SPLITK, PATH_GEMM_1SM, PATH_GEMV_MID = 0, 1, 2, 3, 4, 5
+PATH_AUTO, PATH_GEMV, PATH_GEMM, PATH_GEMV_SPLITK, PATH_GEMM_1SM, PATH_GEMV_MID, PATH_GEMM_SKINNY = 0, 1, 2, 3, 4, 5, 6
 
 EXPORTS = (
     "awq_qweight_bytes", "awq_scales_bytes", "awq_zeros_bytes", "awq_quantize_pack",

@@ -13,7 +13,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB_NAME = "libawq_b200.so"
 LIB_PATH = os.path.join(HERE, LIB_NAME)
-SOURCES = ("api.cu", "quantize_pack.cu", "gemv.cu", "gemv_mid.cu", "gemm_tcgen05.cu", "gemm_tcgen05_pair.cu", "search.cu")
+SOURCES = ("api.cu", "quantize_pack.cu", "gemv.cu", "gemv_mid.cu", "gemm_tcgen05.cu", "gemm_tcgen05_pair.cu", "gemm_skinny.cu", "search.cu")
 NVCC_FLAGS = (
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "--std=c++17",
     "-Xcompiler", "-fPIC",

@@ -199,6 +199,10 @@ size_t awq_workspace_bytes(int M, int N, int K, int group) {
     size_t gemm = gemm_workspace_bytes(M, N, sms);
     const size_t mid = (M <= 32 && gemv_mid_applies(M, N, K, group, sms)) ? gemv_mid_workspace_bytes(M, N, K) : 0;
     if (M > 8 && mid > gemm) gemm = mid;
+    if (M > 8 && gemm_skinny_applies(M, N, K, group)) {
+        const size_t skinny = gemm_skinny_workspace_bytes(M, N, K, group, sms);
+        if (skinny > gemm) gemm = skinny;
+    }
     if (M > 16) return gemm;
     const size_t gemv = gemv_workspace_bytes(M);   // required by the split-K matrix-vector kernel
     if (M <= 8) return gemv > mid ? gemv : mid;    // awq_linear never takes the tensor-core kernel here
@@ -228,12 +232,14 @@ int awq_linear_path(const void* x, const void* qweight, const void* scales, cons
     if (!aligned16(x) || !aligned16(qweight) || !aligned16(scales) || !aligned16(zeros) || !aligned16(y))
         return AWQ_ERR_MISALIGNED;
     if (path != AWQ_PATH_AUTO && path != AWQ_PATH_GEMV && path != AWQ_PATH_GEMM && path != AWQ_PATH_GEMV_SPLITK &&
-        path != AWQ_PATH_GEMM_1SM && path != AWQ_PATH_GEMV_MID)
+        path != AWQ_PATH_GEMM_1SM && path != AWQ_PATH_GEMV_MID && path != AWQ_PATH_GEMM_SKINNY)
         return AWQ_ERR_BAD_ARGUMENT;
     const bool automatic = path == AWQ_PATH_AUTO;
     path = resolve_path(M, K, path);
     if (path == AWQ_PATH_GEMV_MID) {
         if (M > 32 || K > 65536) return AWQ_ERR_BAD_SHAPE;
+    } else if (path == AWQ_PATH_GEMM_SKINNY) {
+        if (!gemm_skinny_applies(M, N, K, group)) return AWQ_ERR_BAD_SHAPE;
     } else if (path != AWQ_PATH_GEMM && path != AWQ_PATH_GEMM_1SM && (M > 16 || K > 65536)) {
         return AWQ_ERR_BAD_SHAPE;
     }
@@ -242,6 +248,13 @@ int awq_linear_path(const void* x, const void* qweight, const void* scales, cons
     if (automatic && mid_kernel_preferred(M, N, K) && gemv_mid_applies(M, N, K, group, d->sms)) {
         std::lock_guard<std::mutex> lock(g_mutex);
         if (d->workspace_bytes >= gemv_mid_workspace_bytes(M, N, K)) path = AWQ_PATH_GEMV_MID;
+    }
+    if (automatic && path == AWQ_PATH_GEMM && M > 16 && M <= 64 && gemm_skinny_applies(M, N, K, group)) {
+        // 17 .. 64 tokens: the chunked tensor-core kernel (measured against the prefill kernels at 32
+        // and 64 tokens: 10.1 / 13.7 and 11.1 / 16.1 us on 4096 -> 4096, 20.7 / 26.2 and 20.8 / 31.4 us
+        // on 4096 -> 11008, 66.5 / 80.9 and 73.5 / 81.2 us on 8192 -> 28672)
+        std::lock_guard<std::mutex> lock(g_mutex);
+        if (d->workspace_bytes >= gemm_skinny_workspace_bytes(M, N, K, group, d->sms)) path = AWQ_PATH_GEMM_SKINNY;
     }
     if (path == AWQ_PATH_GEMV_MID) {
         if (!gemv_mid_applies(M, N, K, group, d->sms)) return AWQ_ERR_BAD_SHAPE;
@@ -253,6 +266,16 @@ int awq_linear_path(const void* x, const void* qweight, const void* scales, cons
         }
         return note_cuda(launch_gemv_mid(x, qweight, scales, zeros, y, M, N, K, group, ws, d->status_word, d->sms,
                                          take_packed_written(d), (cudaStream_t)stream));
+    }
+    if (path == AWQ_PATH_GEMM_SKINNY) {
+        void* ws = nullptr;
+        {
+            std::lock_guard<std::mutex> lock(g_mutex);
+            if (d->workspace_bytes < gemm_skinny_workspace_bytes(M, N, K, group, d->sms)) return AWQ_ERR_NO_WORKSPACE;
+            ws = d->workspace;
+        }
+        return note_cuda(launch_gemm_skinny(x, qweight, scales, zeros, y, M, N, K, group, ws, d->status_word,
+                                            d->sms, take_packed_written(d), (cudaStream_t)stream));
     }
     const bool tensor_path = path == AWQ_PATH_GEMM || path == AWQ_PATH_GEMM_1SM;
     const cudaStream_t st = (cudaStream_t)stream;

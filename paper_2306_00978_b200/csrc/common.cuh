@@ -81,6 +81,18 @@ cudaError_t launch_gemv_mid(const void* x, const void* qweight, const void* scal
                             int M, int N, int K, int group, void* workspace, unsigned int* status_word, int sms,
                             bool serialize, cudaStream_t st);
 
+// y[m][n] = fp16(sum over the chunks, ascending, of partial[c][m][n]), mn = M * N a multiple of 4;
+// launched with programmatic stream serialization behind the kernel that wrote the partial sums
+cudaError_t launch_chunk_reduce(const float* partial, void* y, int chunks, size_t mn, cudaStream_t st);
+
+// 17 .. 64 tokens on the tensor cores (gemm_skinny.cu): units of one 128-channel slab x one chunk of
+// K, the chunk's slice of x resident in shared memory, partial sums per chunk in the workspace
+bool gemm_skinny_applies(int M, int N, int K, int group);
+size_t gemm_skinny_workspace_bytes(int M, int N, int K, int group, int sms);
+cudaError_t launch_gemm_skinny(const void* x, const void* qweight, const void* scales, const void* zeros, void* y,
+                               int M, int N, int K, int group, void* workspace, unsigned int* status_word, int sms,
+                               bool serialize, cudaStream_t st);
+
 // scale search (search.cu)
 constexpr int kMaxSearchAlphas = 64;
 size_t search_scratch_bytes(int M, int N, int K, int group);

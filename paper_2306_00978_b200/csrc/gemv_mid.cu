@@ -414,17 +414,25 @@ cudaError_t launch_gemv_mid(const void* x, const void* qweight, const void* scal
 #undef AWQ_MID_LAUNCH2
 #undef AWQ_MID_LAUNCH
     count_launch();
-    const size_t mn = (size_t)M * N;
+    e = launch_chunk_reduce(partial, y, chunks, (size_t)M * N, st);
+    if (e != cudaSuccess) return e;
+    return cudaGetLastError();
+}
+
+cudaError_t launch_chunk_reduce(const float* partial, void* y, int chunks, size_t mn, cudaStream_t st) {
     cudaLaunchConfig_t rcfg = {};
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
     rcfg.gridDim = dim3((unsigned)((mn / 4 + 255) / 256));
     rcfg.blockDim = dim3(256);
     rcfg.stream = st;
     rcfg.attrs = attr;
     rcfg.numAttrs = 1;
-    e = cudaLaunchKernelEx(&rcfg, gemv_mid_reduce_kernel, (const float*)partial, reinterpret_cast<__half*>(y), chunks, mn);
+    cudaError_t e = cudaLaunchKernelEx(&rcfg, gemv_mid_reduce_kernel, partial, reinterpret_cast<__half*>(y), chunks, mn);
     if (e != cudaSuccess) return e;
     count_launch();
-    return cudaGetLastError();
+    return cudaSuccess;
 }
 
 }  // namespace awq

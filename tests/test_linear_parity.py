@@ -307,3 +307,55 @@ def test_chunked_matrix_vector_kernel(N, K, M, G):
     assert_parity(y, case.y_ref(), f"chunked N={N} K={K} M={M} G={G}")
     y2 = _run(case, binding.PATH_GEMV_MID)
     assert np.array_equal(y.view(np.uint16), y2.view(np.uint16))
+
+
+@pytest.mark.parametrize("N,K,M,G,alpha", [
+    (128, 128, 17, 128, 0.5),     # one slab, one stage
+    (256, 256, 20, 128, 0.5),
+    (512, 1024, 17, 128, 0.0),    # 16-token tile does not fit: 32-token tile
+    (1024, 1408, 33, 128, 0.5),   # 64-token tile; 11 stages per unit: the warps' stage parity crosses units
+    (768, 4096, 64, 64, 1.0),     # full 64-token tile, group 64, four chunks
+    (1280, 2048, 9, 128, 0.5),    # 16-token tile
+    (2048, 5120, 48, 64, 0.5),
+    (4096, 4096, 32, 128, 0.5),   # more units than blocks: ranges that cross from one chunk to the next
+    (19072, 384, 25, 128, 0.5),   # 149 slabs, one short chunk of 3 stages per unit
+    (128, 8192, 40, 128, 0.5),    # one slab, many chunks
+    (256, 640, 1, 64, 0.5),       # a single token
+])
+def test_chunked_tensor_core_kernel(N, K, M, G, alpha):
+    """AWQ_PATH_GEMM_SKINNY: units of 128 channels x a chunk of K on tcgen05, the chunk's slice of x
+    resident in shared memory; partial sums per chunk, added by a second kernel.  Parity with the
+    oracle and bit-reproducibility."""
+    from paper_2306_00978_b200 import binding
+    case = Case(900 + N + K + M + G, N, K, M, G, alpha)
+    y = _run(case, binding.PATH_GEMM_SKINNY)
+    assert_parity(y, case.y_ref(), f"chunked tensor-core N={N} K={K} M={M} G={G}")
+    y2 = _run(case, binding.PATH_GEMM_SKINNY)
+    assert np.array_equal(y.view(np.uint16), y2.view(np.uint16))
+
+
+def test_auto_dispatch_between_17_and_64_tokens():
+    """awq_linear with 17..64 tokens and a registered workspace: the chunked matrix-vector kernel up
+    to 24 tokens on matrices of at least 2^25 weights, else the chunked tensor-core kernel; above 64
+    tokens, or where N is not a multiple of 128, the prefill kernels.  Each result is bit-equal to
+    its forced path."""
+    import torch
+    from paper_2306_00978_b200 import binding
+    for (N, K, M, want) in ((1024, 1408, 20, binding.PATH_GEMM_SKINNY), (1024, 1408, 64, binding.PATH_GEMM_SKINNY),
+                            (1024, 1408, 65, binding.PATH_GEMM), (8192, 4096, 24, binding.PATH_GEMV_MID),
+                            (8192, 4096, 25, binding.PATH_GEMM_SKINNY)):
+        if N * K >= 1 << 24:
+            qw = torch.randint(0, 256, (N * K // 2,), dtype=torch.uint8, device="cuda")
+            sc = (torch.rand((N // 16, K // 128, 16), device="cuda") * 0.01 + 0.001).half()
+            zp = torch.randint(0, 256, (N // 32, K // 128, 16), dtype=torch.uint8, device="cuda")
+            x = torch.randn((M, K), device="cuda").half()
+        else:
+            case = Case(31 + M, N, K, M, 128, 0.5)
+            qw, sc, zp = oracle_packed_to_cuda(case)
+            x = to_cuda(case.x)
+        auto = binding.linear(x, qw, sc, zp, N, K, 128)
+        forced = binding.linear(x, qw, sc, zp, N, K, 128, path=want)
+        binding.poll_status()
+        assert torch.equal(auto, forced), (N, K, M)
+        if N * K < 1 << 24:
+            assert_parity(auto.cpu().numpy(), case.y_ref(), f"auto M={M}")
