@@ -869,7 +869,7 @@ def main():
     ap.add_argument("--one", nargs=3, type=int, metavar=("N", "K", "M"),
                     help="profiling aid: a few awq_linear launches of one shape on random packed "
                          "weights (three rotating copies), then exit")
-    ap.add_argument("--path", type=int, default=0, help="with --one: 0 auto, 1 GEMV, 2 GEMM, 3 split-K GEMV, 4 single-SM GEMM")
+    ap.add_argument("--path", type=int, default=0, help="with --one: 0 auto, 1 GEMV, 2 GEMM, 3 split-K GEMV, 4 single-SM GEMM, 5 chunked GEMV, 6 chunked tensor-core")
     ap.add_argument("--reps", type=int, default=3, help="with --one: passes over the three copies")
     ap.add_argument("--quantize-only", nargs=2, type=int, metavar=("N", "K"),
                     help="profiling aid: a few awq_quantize_pack launches on seeded weights of one shape, then exit")
