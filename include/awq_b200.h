@@ -15,8 +15,9 @@
  *  - Return value: AWQ_OK (0) or a positive AwqStatus code.  Nothing is printed, thrown
  *    or aborted.  awq_status_string() names a code.
  *  - Shapes: N (output channels) a multiple of 128, K (input channels) a multiple of 128,
- *    group 64 or 128, M >= 1.  W is fp16 [N][K] row-major, x fp16 [M][K] row-major,
- *    y fp16 [M][N] row-major.
+ *    group 64, 128, 256, 512 or 1024 (dividing K), M >= 1.  W is fp16 [N][K] row-major, x fp16
+ *    [M][K] row-major, y fp16 [M][N] row-major.  The paper's setting is 128; the searches
+ *    (awq_search_alpha, awq_search_clip) take 64 and 128 only.
  *
  * Packed layout (layout version 3, "band-major": all data of 16 consecutive output rows - a
  * band - is contiguous along K)
@@ -33,8 +34,10 @@
  *      ((n/16)*(K/64) + k/64)*512 + 16*(4*(n%8) + (k%16)/4) + 4*((k%64)/16) + {0,2,1,3}[k%4],
  *    in its low nibble if n%16 < 8, else in its high nibble: every byte holds the codes of rows
  *    g and g+8 of one column.
- *  scales: fp16 [N/16][K/group][16] (band, group, row in band).
- *  zeros:  bytes [N/32][K/group][16]: per pair of bands and group, bytes 0-7 belong to the even
+ *  Stored groups: scales and zero points are stored per group for group <= 128 and per 128
+ *    columns above (each group's entry group / 128 times in a row): G below is min(group, 128).
+ *  scales: fp16 [N/16][K/G][16] (band, stored group, row in band).
+ *  zeros:  bytes [N/32][K/G][16]: per pair of bands and stored group, bytes 0-7 belong to the even
  *    band, 8-15 to the odd one; byte n%8 of a band holds the zero point of row n (n%16 < 8)
  *    in its low nibble and of row n+8 in its high nibble.
  */
@@ -52,7 +55,7 @@ typedef enum AwqStatus {
     AWQ_OK = 0,
     AWQ_ERR_NULL_POINTER = 1,
     AWQ_ERR_BAD_SHAPE = 2,      /* N % 128, K % 128, K % group != 0, M < 1, or too large */
-    AWQ_ERR_BAD_GROUP = 3,      /* group not 64 or 128 */
+    AWQ_ERR_BAD_GROUP = 3,      /* group not 64, 128, 256, 512 or 1024 (the searches: not 64 or 128) */
     AWQ_ERR_BAD_ALPHA = 4,      /* alpha outside [0, 1] or NaN */
     AWQ_ERR_MISALIGNED = 5,     /* a pointer is not 16-byte aligned */
     AWQ_ERR_NO_WORKSPACE = 6,   /* the call needs more workspace than was registered */

@@ -270,6 +270,15 @@ def unpack_qweight_int3(words3, N: int, K: int) -> np.ndarray:
     return unpack_qweight(w.reshape(-1), N, K)
 
 
+def stored_groups(per_group, group: int) -> np.ndarray:
+    """[N][K/group] -> [N][K/min(group, 128)]: the packed scale and zero-point arrays hold one entry
+    per group up to 128 input channels and one per 128 input channels above (each group's entry
+    group / 128 times), so that a kernel never meets more than two 64-column blocks per entry.  The
+    paper does not say how other group sizes are stored; this is a choice of the layout."""
+    a = np.asarray(per_group)
+    return np.repeat(a, group // 128, axis=1) if group > 128 else a
+
+
 def pack_zeros(zeros) -> np.ndarray:
     """zeros u8 [N][ng] -> u8 [N/32][ng][16] in the layout of `zeros_location`."""
     zeros = np.asarray(zeros, dtype=np.uint8)
@@ -345,12 +354,13 @@ def search_clip(W, s, group: int, ratios, bits: int = 4) -> np.ndarray:
 
 
 def quantize_pack(W, act_mean_abs, alpha: float, group: int, clip=None, bits: int = 4, symmetric: bool = False):
-    """The whole offline step: returns (qweight u32, scales fp16 [N/16][ng][16], zeros u8 [N/32][ng][16]).
-    3-bit codes (bits = 3) are stored in the same 4-bit fields."""
+    """The whole offline step: returns (qweight u32, scales fp16 [N/16][ng][16], zeros u8 [N/32][ng][16]),
+    ng = K / min(group, 128) stored entries per row (stored_groups).  3-bit codes (bits = 3) are stored
+    in the same 4-bit fields."""
     K = W.shape[1]
     a = np.ones(K, np.float32) if act_mean_abs is None else act_mean_abs
     codes, zeros, scales = quantize(W, channel_scale(a, alpha), group, clip=clip, bits=bits, symmetric=symmetric)
-    return pack_qweight(codes), pack_scales(scales), pack_zeros(zeros)
+    return pack_qweight(codes), pack_scales(stored_groups(scales, group)), pack_zeros(stored_groups(zeros, group))
 
 
 # ----------------------------------------------------------------- dequantize, multiply
@@ -376,10 +386,10 @@ def linear_from_packed(x, qweight, scales_gn, zeros_packed, N: int, K: int, grou
     """Dequantize-then-multiply starting from the packed arrays (optionally only the
     output channels listed in `rows`, for sampled checks at sizes where the full product
     is too slow)."""
-    ng = K // group
+    nsg, rep = K // min(group, 128), max(group // 128, 1)       # stored entries per row; see stored_groups
     codes = unpack_qweight(qweight, N, K)
-    zeros = unpack_zeros(zeros_packed, N, ng)
-    scales = unpack_scales(scales_gn, N, ng)
+    zeros = unpack_zeros(zeros_packed, N, nsg)[:, ::rep]
+    scales = unpack_scales(scales_gn, N, nsg)[:, ::rep]
     if rows is not None:
         codes, zeros, scales = codes[rows], zeros[rows], scales[rows]
     return linear(x, dequantize(codes, zeros, scales, group))

@@ -136,13 +136,14 @@ def inverse_channel_scale(act_mean_abs: Optional[torch.Tensor], alpha: float, K:
 def quantize_pack(W: torch.Tensor, act_mean_abs: Optional[torch.Tensor], alpha: float, group: int,
                   clip_ratio: Optional[torch.Tensor] = None, bits: int = 4, symmetric: bool = False):
     """awq_quantize_pack / awq_quantize_pack_ex: returns (qweight u8 [N*K/2],
-    scales fp16 [N/16][K/group][16], zeros u8 [N/32][K/group][16])."""
+    scales fp16 [N/16][K/g][16], zeros u8 [N/32][K/g][16]), g = min(group, 128)."""
     N, K = W.shape
     qb, sb, zb = packed_sizes(N, K, group)
     dev = W.device
     qweight = torch.empty(qb, dtype=torch.uint8, device=dev)
-    scales = torch.empty((N // 16, K // group, 16), dtype=torch.float16, device=dev)
-    zeros = torch.empty((N // 32, K // group, 16), dtype=torch.uint8, device=dev)
+    stored = min(int(group), 128)                  # groups above 128 columns are stored once per 128 columns
+    scales = torch.empty((N // 16, K // stored, 16), dtype=torch.float16, device=dev)
+    zeros = torch.empty((N // 32, K // stored, 16), dtype=torch.uint8, device=dev)
     a = 0 if act_mean_abs is None else _dev(act_mean_abs, torch.float32, "act_mean_abs")
     if clip_ratio is None and bits == 4 and not symmetric:
         rc = lib().awq_quantize_pack(_dev(W, torch.float16, "W"), a, float(alpha), int(group),

@@ -79,8 +79,12 @@ bool take_packed_written(DeviceState* d) {
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+// Scales and zero points are stored per group up to 128 columns and per 128 columns above (each
+// group's entry group / 128 times), so the layer kernels see groups of 64 or 128 only.
+int stored_group(int group) { return group > 128 ? 128 : group; }
+
 int check_shape(int N, int K, int group) {
-    if (group != 64 && group != 128) return AWQ_ERR_BAD_GROUP;
+    if (group != 64 && group != 128 && group != 256 && group != 512 && group != 1024) return AWQ_ERR_BAD_GROUP;
     if (N < 128 || K < 128 || N % 128 != 0 || K % 128 != 0 || K % group != 0) return AWQ_ERR_BAD_SHAPE;
     if (N / 128 > kMaxSlabs) return AWQ_ERR_BAD_SHAPE;
     if ((long long)N * K > (1LL << 33)) return AWQ_ERR_BAD_SHAPE;
@@ -101,10 +105,10 @@ size_t awq_qweight_bytes(int N, int K) {
     return check_shape(N, K, 128) == AWQ_OK ? (size_t)N * K / 2 : 0;
 }
 size_t awq_scales_bytes(int N, int K, int group) {
-    return check_shape(N, K, group) == AWQ_OK ? (size_t)(K / group) * N * 2 : 0;
+    return check_shape(N, K, group) == AWQ_OK ? (size_t)(K / stored_group(group)) * N * 2 : 0;
 }
 size_t awq_zeros_bytes(int N, int K, int group) {
-    return check_shape(N, K, group) == AWQ_OK ? (size_t)(K / group) * N / 2 : 0;
+    return check_shape(N, K, group) == AWQ_OK ? (size_t)(K / stored_group(group)) * N / 2 : 0;
 }
 
 int awq_channel_scale(const float* act_mean_abs, float alpha, float* s, int K, void* stream) {
@@ -147,6 +151,7 @@ int awq_search_clip(const void* W, const float* act_mean_abs, float alpha, int g
                     const float* ratios, int n_ratios, float* clip_ratio, int N, int K, void* stream) {
     if (!(alpha >= 0.0f && alpha <= 1.0f)) return AWQ_ERR_BAD_ALPHA;
     if (int rc = check_shape(N, K, group)) return rc;
+    if (group > 128) return AWQ_ERR_BAD_GROUP;
     if ((bits != 3 && bits != 4) || n_ratios < 1 || n_ratios > kMaxClipRatios) return AWQ_ERR_BAD_ARGUMENT;
     if (!W || !ratios || !clip_ratio || (!act_mean_abs && alpha != 0.0f)) return AWQ_ERR_NULL_POINTER;
     if ((reinterpret_cast<uintptr_t>(W) & 1u) || (reinterpret_cast<uintptr_t>(act_mean_abs) & 3u) ||
@@ -189,6 +194,7 @@ static int resolve_path(int M, int K, int path) {
 
 size_t awq_workspace_bytes(int M, int N, int K, int group) {
     if (check_shape(N, K, group) != AWQ_OK || M < 1) return 0;
+    group = stored_group(group);
     // optional for the tensor-core kernels: with it they spread their work evenly over the SMs
     int dev = 0, sms = 0;
     if (cudaGetDevice(&dev) != cudaSuccess ||
@@ -227,6 +233,7 @@ int awq_set_workspace(void* dev_ptr, size_t bytes) {
 int awq_linear_path(const void* x, const void* qweight, const void* scales, const void* zeros,
                     void* y, int M, int N, int K, int group, int path, void* stream) {
     if (int rc = check_shape(N, K, group)) return rc;
+    group = stored_group(group);
     if (M < 1 || (long long)M * K > (1LL << 40) || (long long)M * N > (1LL << 40)) return AWQ_ERR_BAD_SHAPE;
     if (!x || !qweight || !scales || !zeros || !y) return AWQ_ERR_NULL_POINTER;
     if (!aligned16(x) || !aligned16(qweight) || !aligned16(scales) || !aligned16(zeros) || !aligned16(y))
@@ -315,6 +322,7 @@ int awq_linear_path(const void* x, const void* qweight, const void* scales, cons
 int awq_linear_gemv_static(const void* x, const void* qweight, const void* scales, const void* zeros,
                             void* y, int M, int N, int K, int group, void* stream) {
     if (int rc = check_shape(N, K, group)) return rc;
+    group = stored_group(group);
     if (M < 1) return AWQ_ERR_BAD_SHAPE;
     if (M > gemv_static_max_m() || K > 65536) return AWQ_ERR_STATIC_LIMIT;
     if (!x || !qweight || !scales || !zeros || !y) return AWQ_ERR_NULL_POINTER;
@@ -367,6 +375,7 @@ int awq_linear_multi(const void* x, const AwqLinearProblem* problems, int count,
             return AWQ_ERR_MISALIGNED;
         total_n += p.N;
     }
+    group = stored_group(group);
     if (M < 1) return AWQ_ERR_BAD_SHAPE;
     if (!aligned16(x)) return AWQ_ERR_MISALIGNED;
     DeviceState* d;
@@ -399,6 +408,7 @@ static bool scaled_call_folds(int M, int total_n, int K, int group, int sms) {
 
 int awq_linear_scaled_needs_scratch(int M, int N, int K, int group) {
     if (check_shape(N, K, group) != AWQ_OK || M < 1) return 1;
+    group = stored_group(group);
     int dev = 0, sms = 0;
     if (cudaGetDevice(&dev) != cudaSuccess ||
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
@@ -421,6 +431,7 @@ int awq_linear_multi_scaled(const void* x, const float* inv_s, void* x_scratch, 
             return AWQ_ERR_MISALIGNED;
         total_n += p.N;
     }
+    group = stored_group(group);
     if (M < 1 || (long long)M * K > (1LL << 40)) return AWQ_ERR_BAD_SHAPE;
     if (!aligned16(x) || !aligned16(inv_s) || !aligned16(x_scratch)) return AWQ_ERR_MISALIGNED;
     DeviceState* d;
@@ -479,6 +490,7 @@ int awq_unpack_int3(const void* qweight3, void* qweight, int N, int K, void* str
 int awq_linear_int3(const void* x, const void* qweight3, const void* scales, const void* zeros, void* y,
                     void* qweight_scratch, int M, int N, int K, int group, void* stream) {
     if (int rc = check_shape(N, K, group)) return rc;
+    group = stored_group(group);
     if (M < 1 || (long long)M * K > (1LL << 40) || (long long)M * N > (1LL << 40)) return AWQ_ERR_BAD_SHAPE;
     if (!x || !qweight3 || !scales || !zeros || !y) return AWQ_ERR_NULL_POINTER;
     if (!aligned16(x) || !aligned16(qweight3) || !aligned16(scales) || !aligned16(zeros) || !aligned16(y) ||
@@ -503,7 +515,7 @@ int awq_inverse_channel_scale(const float* act_mean_abs, float alpha, float* inv
 }
 
 size_t awq_search_scratch_bytes(int M, int N, int K, int group) {
-    if (check_shape(N, K, group) != AWQ_OK || M < 1) return 0;
+    if (check_shape(N, K, group) != AWQ_OK || M < 1 || group > 128) return 0;
     return search_scratch_bytes(M, N, K, group);
 }
 
@@ -511,6 +523,7 @@ int awq_search_alpha(const void* W, const float* act_mean_abs, const void* X, in
                      const float* alphas, int n_alphas, float* losses, int* best_index,
                      void* scratch, size_t scratch_bytes, void* stream) {
     if (int rc = check_shape(N, K, group)) return rc;
+    if (group > 128) return AWQ_ERR_BAD_GROUP;
     if (M < 1) return AWQ_ERR_BAD_SHAPE;
     if (!W || !act_mean_abs || !X || !alphas || !losses || !best_index || !scratch) return AWQ_ERR_NULL_POINTER;
     if (n_alphas < 1 || n_alphas > kMaxSearchAlphas) return AWQ_ERR_BAD_ARGUMENT;

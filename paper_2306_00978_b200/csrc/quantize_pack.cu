@@ -101,24 +101,33 @@ __device__ __forceinline__ float level_fast2(float w, float rd, float zc, float 
     return CLAMP ? fminf(fmaxf(q, 0.0f), top) : q;
 }
 
-constexpr int kQBands = 2;                                // bands (16 rows) per thread block
-constexpr int kQThreads = kQBands * 2 * 32;              // one warp per band and 64-column block
+// One warp per band (16 rows) and 64-column block.  A thread block covers one group of columns (two
+// groups for G = 64) so that the group's min / max meet in shared memory: 2 bands x 2 blocks up to
+// G = 128, 1 band x G / 64 blocks above.  Scales and zero points are stored per 128 columns for
+// G > 128 (each group's entry G / 128 times), so that the layer kernels need no variant for them.
+template <int G> struct QCfg {
+    static constexpr int kBlocks = G < 128 ? 2 : G / 64;            // 64-column blocks per thread block
+    static constexpr int kBands = kBlocks <= 4 ? 4 / kBlocks : 1;   // bands per thread block
+    static constexpr int kThreads = kBlocks * kBands * 32;
+    static constexpr int kStored = G < 128 ? G : 128;               // columns per stored scale / zero point
+};
 
 template <int G, int BITS, bool CLIP, bool SYM>
-__global__ void __launch_bounds__(kQThreads, 1024 / kQThreads)
+__global__ void __launch_bounds__(QCfg<G>::kThreads, 1024 / QCfg<G>::kThreads)
 quantize_pack_tile_kernel(const __half* __restrict__ W, const float* __restrict__ a, float alpha,
                           int mode, const float* __restrict__ clip,
                           uint32_t* __restrict__ qweight, __half* __restrict__ scales,
                           uint8_t* __restrict__ zeros, int N, int K) {
     constexpr float top = (float)((1 << BITS) - 1);       // largest code
-    __shared__ __align__(16) float s_sm[128];
-    __shared__ float2 s_mm[2][kQBands * 16];               // G = 128: [block of the pair][row] (min, max)
+    constexpr int kQBands = QCfg<G>::kBands, kQBlocks = QCfg<G>::kBlocks, kQThreads = QCfg<G>::kThreads;
+    __shared__ __align__(16) float s_sm[kQBlocks * 64];
+    __shared__ float2 s_mm[kQBlocks][kQBands * 16];        // G >= 128: [64-column block][row] (min, max)
     const int kblk = blockIdx.x;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int bw = warp % kQBands, ti = warp / kQBands;
     const int g = lane >> 2, t = lane & 3;
     const int n0 = (blockIdx.y * kQBands + bw) * 16 + g;   // this lane's upper row; lower = n0 + 8
-    const int kbase = kblk * 128;
+    const int kbase = kblk * (kQBlocks * 64);
 
     uint2 raw[2][4];                                       // [row h][word j] = columns 16j + 4t .. +3 of the block
 #pragma unroll
@@ -127,7 +136,7 @@ quantize_pack_tile_kernel(const __half* __restrict__ W, const float* __restrict_
         for (int j = 0; j < 4; ++j)
             raw[h][j] = ldg_stream(reinterpret_cast<const uint2*>(
                 W + (size_t)(n0 + 8 * h) * K + kbase + ti * 64 + 16 * j + 4 * t));
-    for (int i = threadIdx.x; i < 128; i += kQThreads) {
+    for (int i = threadIdx.x; i < kQBlocks * 64; i += kQThreads) {
         const int k = kbase + i;
         s_sm[i] = channel_scale_one(mode == kAlphaZero ? 1.0f : a[k], alpha, mode);
     }
@@ -162,19 +171,21 @@ quantize_pack_tile_kernel(const __half* __restrict__ W, const float* __restrict_
             mn[h] = fminf(mn[h], __shfl_xor_sync(0xFFFFFFFFu, mn[h], off));
             mx[h] = fmaxf(mx[h], __shfl_xor_sync(0xFFFFFFFFu, mx[h], off));
         }
-    if (G == 128) {
-        // the group spans both blocks of the pair: the other half's min / max through shared memory
+    if (G >= 128) {
+        // the group spans all 64-column blocks of the thread block: the others' min / max through shared memory
         if (t == 0) {
             s_mm[ti][bw * 16 + g] = make_float2(mn[0], mx[0]);
             s_mm[ti][bw * 16 + g + 8] = make_float2(mn[1], mx[1]);
         }
         __syncthreads();
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {
-            const float2 o = s_mm[ti ^ 1][bw * 16 + g + 8 * h];
-            mn[h] = fminf(mn[h], o.x);
-            mx[h] = fmaxf(mx[h], o.y);
-        }
+        for (int h = 0; h < 2; ++h)
+#pragma unroll
+            for (int o = 1; o < kQBlocks; ++o) {
+                const float2 v = s_mm[(ti + o) % kQBlocks][bw * 16 + g + 8 * h];
+                mn[h] = fminf(mn[h], v.x);
+                mx[h] = fmaxf(mx[h], v.y);
+            }
     }
     float wabs[2];                                          // largest |w'| of each group (before clipping)
 #pragma unroll
@@ -252,14 +263,17 @@ quantize_pack_tile_kernel(const __half* __restrict__ W, const float* __restrict_
     if (need_clamp) quantize_words(std::true_type{}); else quantize_words(std::false_type{});
     // band-major: block (band, k-tile) is 512 bytes, a band's blocks are contiguous along K
     const size_t band = (size_t)blockIdx.y * kQBands + bw;
-    const size_t block = band * (K / 64) + (size_t)kblk * 2 + ti;
+    const size_t block = band * (K / 64) + (size_t)kblk * kQBlocks + ti;
     uint4* dst = reinterpret_cast<uint4*>(qweight) + block * 32 + lane;
     *dst = make_uint4(words[0], words[1], words[2], words[3]);
-    if (t == 0 && (G == 64 || ti == 0)) {
-        // scales: [band][group][16]; zero bytes: [band pair][group][16], 8 per band
-        scales[(band * ng + gi) * 16 + g] = d16[0];
-        scales[(band * ng + gi) * 16 + g + 8] = d16[1];
-        zeros[((band >> 1) * ng + gi) * 16 + (band & 1) * 8 + g] =
+    if (t == 0 && (G == 64 || (ti & 1) == 0)) {
+        // scales: [band][stored group][16]; zero bytes: [band pair][stored group][16], 8 per band; a
+        // stored group is the group itself up to 128 columns, else each of its runs of 128 columns
+        const size_t nsg = K / QCfg<G>::kStored;
+        const size_t sgi = (G == 64) ? (size_t)gi : (size_t)kblk * (kQBlocks / 2) + ti / 2;
+        scales[(band * nsg + sgi) * 16 + g] = d16[0];
+        scales[(band * nsg + sgi) * 16 + g + 8] = d16[1];
+        zeros[((band >> 1) * nsg + sgi) * 16 + (band & 1) * 8 + g] =
             (uint8_t)((uint32_t)z[0] | ((uint32_t)z[1] << 4));
     }
 }
@@ -357,9 +371,12 @@ __global__ void unpack_kernel(const uint32_t* __restrict__ qweight, const __half
     const int nib = (slot % 2) * 4 + slot / 2;
     codes[idx] = (uint8_t)((w >> (4 * nib)) & 0xFu);
     if (k % group == 0) {
+        // the group's first stored entry (groups above 128 columns are stored once per 128 columns)
         const int gi = k / group, ng = K / group;
-        scales_nk[(size_t)n * ng + gi] = __half_as_ushort(scales[((size_t)band * ng + gi) * 16 + rr]);
-        const uint8_t zb = zeros[((size_t)(band >> 1) * ng + gi) * 16 + (band & 1) * 8 + g];
+        const int stored = group < 128 ? group : 128;
+        const size_t sgi = k / stored, nsg = K / stored;
+        scales_nk[(size_t)n * ng + gi] = __half_as_ushort(scales[((size_t)band * nsg + sgi) * 16 + rr]);
+        const uint8_t zb = zeros[((size_t)(band >> 1) * nsg + sgi) * 16 + (band & 1) * 8 + g];
         zeros_nk[(size_t)n * ng + gi] = (uint8_t)((zb >> (4 * h)) & 0xFu);
     }
 }
@@ -373,10 +390,10 @@ cudaError_t launch_channel_scale(const float* a, float alpha, float* s, int K, c
 cudaError_t launch_quantize_pack(const __half* W, const float* a, float alpha, int group, int bits,
                                  bool symmetric, const float* clip, uint32_t* qweight, __half* scales, uint8_t* zeros,
                                  int N, int K, cudaStream_t st) {
-    const dim3 grid(K / 128, N / (16 * kQBands));
     const int mode = (int)alpha_mode(alpha);
-#define AWQ_QP_LAUNCH(GG, BB, CC, SS) \
-    quantize_pack_tile_kernel<GG, BB, CC, SS><<<grid, kQThreads, 0, st>>>(W, a, alpha, mode, clip, qweight, scales, zeros, N, K)
+#define AWQ_QP_LAUNCH(GG, BB, CC, SS)                                                                           \
+    quantize_pack_tile_kernel<GG, BB, CC, SS><<<dim3(K / (QCfg<GG>::kBlocks * 64), N / (16 * QCfg<GG>::kBands)), \
+                                                QCfg<GG>::kThreads, 0, st>>>(W, a, alpha, mode, clip, qweight, scales, zeros, N, K)
 #define AWQ_QP_PICK2(GG, SS)                                             \
     do {                                                                 \
         if (bits == 4 && !clip) AWQ_QP_LAUNCH(GG, 4, false, SS);         \
@@ -388,7 +405,13 @@ cudaError_t launch_quantize_pack(const __half* W, const float* a, float alpha, i
     do {                                                                 \
         if (symmetric) AWQ_QP_PICK2(GG, true); else AWQ_QP_PICK2(GG, false); \
     } while (0)
-    if (group == 128) AWQ_QP_PICK(128); else AWQ_QP_PICK(64);
+    switch (group) {
+        case 64: AWQ_QP_PICK(64); break;
+        case 128: AWQ_QP_PICK(128); break;
+        case 256: AWQ_QP_PICK(256); break;
+        case 512: AWQ_QP_PICK(512); break;
+        default: AWQ_QP_PICK(1024); break;
+    }
 #undef AWQ_QP_PICK
 #undef AWQ_QP_PICK2
 #undef AWQ_QP_LAUNCH

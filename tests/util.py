@@ -23,8 +23,8 @@ class Case:
         self.x = (x.astype(np.float32) / self.s[None, :]).astype(np.float16)
         self.codes, self.zeros, self.scales = orc.quantize(self.W, self.s, group)
         self.qweight = orc.pack_qweight(self.codes)
-        self.scales_gn = orc.pack_scales(self.scales)
-        self.zeros_packed = orc.pack_zeros(self.zeros)
+        self.scales_gn = orc.pack_scales(orc.stored_groups(self.scales, group))
+        self.zeros_packed = orc.pack_zeros(orc.stored_groups(self.zeros, group))
 
     def y_ref(self, rows=None, tokens=None):
         x = self.x if tokens is None else self.x[tokens]
