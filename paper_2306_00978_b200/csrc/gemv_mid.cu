@@ -12,14 +12,28 @@
 //     per-group sums of x that the zero-point term needs;
 //   * every math warp owns ONE band of the unit: no sums meet between warps, nothing is reduced in
 //     shared memory, the accumulators stay in registers for the whole unit;
-//   * a stage of the ring is 16 bands x 2 k-tiles = 16 KB of packed weights brought by ONE tensor-map
+//   * a stage of the ring is 16 bands x 4 k-tiles = 32 KB of packed weights brought by ONE tensor-map
 //     copy (the bands' runs are K * 8 bytes apart in the band-major layout: sixteen bulk copies of
-//     1 KB would cost sixteen times the copy engine's per-copy overhead); a unit's scales and zero
+//     2 KB would cost sixteen times the copy engine's per-copy overhead); a unit's scales and zero
 //     points come by two more tensor-map copies per unit;
 //   * a unit's sums over ONE chunk are partial: they go to an fp32 workspace [chunk][token][channel],
 //     and a second, tiny kernel adds the chunks in ascending order and rounds to fp16 once -
 //     deterministic, no counters, no fences, no waiting between blocks.
 // Every wait is bounded as in the other kernels.
+//
+// Measured on 8192 -> 28672 at 8 tokens (block start / end times by the global timer, in a working
+// copy): 140 blocks with 6 units take 22.4 us each (3.7 us per 128 KB unit, 4.9 TB/s over all SMs
+// while they run), the 8 blocks with 7 units 25 us, and the 4 of those whose range crosses into the
+// next chunk (a new slice of x) 28.1 us, which is the kernel's 28.4 us.  Two remedies were built,
+// bit-exact, and measured no better:
+//   * equal shares of STAGES per block instead of units (a cut unit's second part in a slot of its
+//     own, a table telling the reduce kernel which units were cut): with all SMs busy to the end
+//     every block slows to 25.3 us (the memory system gives this access pattern about 4.7 TB/s), the
+//     four crossing blocks still end at 29 us, and the reduce kernel's dependent loads cost 2 us;
+//   * the next chunk's slice of x fetched at the start into a second buffer: 31.0 -> 30.1 us here,
+//     but 42.8 -> 47.3 us on 28672 -> 8192 at 16 tokens (a fifth of the blocks cross there and
+//     start later), 0.2 - 0.6 us slower on the 7B shapes.
+// Stages of 32 KB (4 k-tiles per band) instead of 16 KB: 31.7 -> 31.0 us.
 #include "tcgen05.cuh"
 
 namespace awq {
@@ -30,9 +44,9 @@ constexpr int kMidMathWarps = 16;
 constexpr int kMidThreads = (kMidMathWarps + 1) * 32;   // + producer warp
 constexpr int kMidSmem = 220 * 1024;
 constexpr int kMidChunkTiles = 16;                       // k-tiles (64 columns) per chunk: 16, or 8 where that fills the SMs better
-constexpr int kMidStageTiles = 2;                        // k-tiles per stage and band
+constexpr int kMidStageTiles = 4;                        // k-tiles per stage and band
 constexpr int kMidStageBytes = kMidMathWarps * kMidStageTiles * 512;
-constexpr int kMidStages = 8;
+constexpr int kMidStages = 4;
 
 // the same product starting a new accumulation (C = 0)
 __device__ __forceinline__ void mid_mma_first(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
@@ -133,8 +147,8 @@ gemv_mid_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
             for (int j = 0; j < nt; j += kMidStageTiles) {
                 if (!mbar_wait_relaxed(bars + 64u + 8u * stage, phase ^ 1u, ctl)) { ok = false; break; }
                 mbar_arrive_expect_tx(bars + 8u * stage, kMidStageBytes);
-                // 16 bands x 2 k-tiles (256 words) at (word kt * 128 of the band's run, first band)
-                tma_load_2d(sbase + stage * kMidStageBytes, &w_map, (kt0 + j) * 128, bg * kMidMathWarps, bars + 8u * stage);
+                // 16 bands x 4 k-tiles at (64-bit element kt * 64 of the band's run, first band)
+                tma_load_2d(sbase + stage * kMidStageBytes, &w_map, (kt0 + j) * 64, bg * kMidMathWarps, bars + 8u * stage);
                 ++issued;
                 if (++stage == S) { stage = 0; phase ^= 1u; }
             }
@@ -216,6 +230,7 @@ gemv_mid_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
             // the stage's two k-tiles are one group (G = 128) or two (G = 64)
 #pragma unroll
             for (int q = 0; q < kMidStageTiles / TPG; ++q) {
+                if (j + q * TPG >= nt) break;                       // a ragged last stage of the chunk
                 // one accumulation chain per k-tile of the group and token fragment, interleaved word by
                 // word, so that no product waits for the one before it
                 float ca[TPG][MT][4];
@@ -340,11 +355,12 @@ cudaError_t launch_gemv_mid(const void* x, const void* qweight, const void* scal
     const cuuint32_t estr[2] = {1, 1};
     CUtensorMap wmap, scmap, zmap;
     {
-        // packed weights: one row of K * 2 words per band; boxes of 16 bands x 2 k-tiles (256 words)
-        const cuuint64_t dims[2] = {(cuuint64_t)K * 2, (cuuint64_t)(N / 16)};
+        // packed weights: one row of K * 8 bytes per band, as 64-bit elements (a box side is at most
+        // 256 elements); boxes of 16 bands x 4 k-tiles (256 elements = 2 KB)
+        const cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)(N / 16)};
         const cuuint64_t strides[1] = {(cuuint64_t)K * 8};
-        const cuuint32_t box[2] = {(cuuint32_t)(kMidStageTiles * 128), (cuuint32_t)kMidMathWarps};
-        if (enc(&wmap, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<void*>(qweight), dims, strides, box, estr,
+        const cuuint32_t box[2] = {(cuuint32_t)(kMidStageTiles * 64), (cuuint32_t)kMidMathWarps};
+        if (enc(&wmap, CU_TENSOR_MAP_DATA_TYPE_UINT64, 2, const_cast<void*>(qweight), dims, strides, box, estr,
                 CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
             return cudaErrorInvalidValue;
