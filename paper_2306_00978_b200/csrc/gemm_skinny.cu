@@ -104,8 +104,11 @@ gemm_skinny_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_const
     const int nslabs = N / 128, nkb = K / kBK;
     const int nchunks = (nkb + CK - 1) / CK;
     const int units = nchunks * nslabs;
-    const int u0 = (int)(((long long)units * blockIdx.x) / gridDim.x);
-    const int u1 = (int)(((long long)units * (blockIdx.x + 1)) / gridDim.x);
+    // the blocks with one unit more are the first ones: blocks start in index order, the last ones on
+    // the SMs that the launch in front of this one frees last
+    const int uq = units / (int)gridDim.x, ur = units - uq * (int)gridDim.x;
+    const int u0 = uq * (int)blockIdx.x + min((int)blockIdx.x, ur);
+    const int u1 = u0 + uq + ((int)blockIdx.x < ur ? 1 : 0);
     // unit u = chunk * nslabs + slab; a chunk has nt k-blocks = nt / 2 stages (K is a multiple of 128)
     auto chunk_of = [&](int u) { return u / nslabs; };
     auto tiles_of = [&](int c) { return min(CK, nkb - c * CK); };

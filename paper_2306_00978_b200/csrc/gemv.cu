@@ -356,8 +356,11 @@ gemv_band_kernel(const BandProblems probs, const __half* __restrict__ x, int M, 
     const int ktiles = K / 64, ng = K / G;
     const int upb = XREG ? 1 : (ktiles + UT - 1) / UT;                // units (stages) per band
     const int nbands = probs.first_band[probs.count];
-    const int b0 = (int)(((unsigned)nbands * blockIdx.x) / gridDim.x);
-    const int b1 = (int)(((unsigned)nbands * (blockIdx.x + 1)) / gridDim.x);
+    // the blocks with one band more are the first ones: blocks start in index order, the last ones
+    // on the SMs that the launch in front of this one frees last
+    const int bq = nbands / (int)gridDim.x, br = nbands - bq * (int)gridDim.x;
+    const int b0 = bq * (int)blockIdx.x + min((int)blockIdx.x, br);
+    const int b1 = b0 + bq + ((int)blockIdx.x < br ? 1 : 0);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x < (unsigned)S) {

@@ -87,13 +87,42 @@ inline MidLayout mid_layout(int M, int group, int chunk_tiles = kMidChunkTiles) 
     return l;
 }
 
+// First unit of every block (and the end of the last one).  Blocks start in index order, the last
+// ones on the SMs that the launch in front of this one frees last, so the blocks that hold one unit
+// more than the others are the first ones - except where the longer range would cross into the next
+// chunk, which costs a second slice of x (measured on 28672 -> 8192 at 8 tokens: 6 units 22.4 us, 7
+// units 25 us, 7 units and a crossing 28 us; with the longer ranges simply in front 28672 -> 8192 went
+// 32.3 -> 34.3 us while 8192 -> 28672 went 31.0 -> 28.7 us).
+constexpr int kMidMaxBlocks = 256;
+struct MidStarts {
+    int v[kMidMaxBlocks + 1];
+};
+inline MidStarts mid_starts(int units, int nbg, int blocks) {
+    MidStarts s;
+    int size[kMidMaxBlocks];
+    const int q = units / blocks;
+    int extra = units - q * blocks, pos = 0;
+    for (int b = 0; b < blocks; ++b) {
+        const bool crosses = q > 0 && pos / nbg != (pos + q) / nbg;      // with q + 1 units
+        size[b] = q + ((extra > 0 && !crosses) ? 1 : 0);
+        extra -= size[b] - q;
+        pos += size[b];
+    }
+    for (int b = blocks - 1; b >= 0 && extra > 0; --b)                  // what could not be placed so
+        if (size[b] == q) { ++size[b]; --extra; }
+    s.v[0] = 0;
+    for (int b = 0; b < blocks; ++b) s.v[b + 1] = s.v[b] + size[b];
+    for (int b = blocks + 1; b <= kMidMaxBlocks; ++b) s.v[b] = s.v[blocks];
+    return s;
+}
+
 // MT = 8-token B fragments per product (tokens rounded up to 8 MT); CT = k-tiles per chunk.
 template <int G, int MT, int CT>
 __global__ void __launch_bounds__(kMidThreads, 1)
 gemv_mid_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant__ CUtensorMap sc_map,
                 const __grid_constant__ CUtensorMap z_map, const __half* __restrict__ x,
                 float* __restrict__ partial, int M, int N, int K, const MidLayout lay,
-                unsigned int* status_word) {
+                const __grid_constant__ MidStarts starts, unsigned int* status_word) {
     extern __shared__ __align__(1024) unsigned char smem[];
     __shared__ unsigned int s_abort;
     constexpr int TPG = G / 64;                          // k-tiles per group
@@ -106,8 +135,8 @@ gemv_mid_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
     const int nbg = (nbands + kMidMathWarps - 1) / kMidMathWarps;
     const int nchunks = (ktiles + CT - 1) / CT;
     const int units = nchunks * nbg;
-    const int u0 = (int)(((long long)units * blockIdx.x) / gridDim.x);
-    const int u1 = (int)(((long long)units * (blockIdx.x + 1)) / gridDim.x);
+    const int u0 = starts.v[blockIdx.x], u1 = starts.v[blockIdx.x + 1];
+    (void)units;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x < (unsigned)S) {
@@ -184,12 +213,27 @@ gemv_mid_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
             // of x over each group and token, times 2^-24 (the products carry that factor)
             cur_chunk = c;
             named_barrier_sync(1, kMidMathWarps * 32);              // everybody is done with the old slice
-            const int pieces_per_row = nt * 8;
-            for (int i = threadIdx.x; i < lay.mtok * pieces_per_row; i += kMidMathWarps * 32) {
-                const int m = i / pieces_per_row, p = i - m * pieces_per_row;
-                uint4 v = make_uint4(0u, 0u, 0u, 0u);
-                if (m < M) v = __ldg(reinterpret_cast<const uint4*>(x + (size_t)m * K + (size_t)kt0 * 64) + p);
-                *reinterpret_cast<uint4*>(xs + m * lay.x_row + p * 16) = v;
+            // From three token fragments on, all of a thread's loads leave before its first store (one
+            // after the other they are a chain of latencies: 8192 -> 28672 at 24 tokens 55.8 -> 52.3 us;
+            // with one or two fragments a thread has two or four loads, and the registers of a batch
+            // cost the main loop more than the chain: 40.0 -> 41.0 us at 16 tokens).
+            constexpr int FB = MT >= 3 ? 8 : 1;
+            const int pieces_per_row = nt * 8, total = lay.mtok * pieces_per_row;
+            for (int i0 = threadIdx.x; i0 < total; i0 += FB * kMidMathWarps * 32) {
+                uint4 v[FB];
+#pragma unroll
+                for (int q = 0; q < FB; ++q) {
+                    const int i = i0 + q * kMidMathWarps * 32;
+                    const int m = i / pieces_per_row, p = i - m * pieces_per_row;
+                    v[q] = make_uint4(0u, 0u, 0u, 0u);
+                    if (i < total && m < M) v[q] = __ldg(reinterpret_cast<const uint4*>(x + (size_t)m * K + (size_t)kt0 * 64) + p);
+                }
+#pragma unroll
+                for (int q = 0; q < FB; ++q) {
+                    const int i = i0 + q * kMidMathWarps * 32;
+                    const int m = i / pieces_per_row, p = i - m * pieces_per_row;
+                    if (i < total) *reinterpret_cast<uint4*>(xs + m * lay.x_row + p * 16) = v[q];
+                }
             }
             named_barrier_sync(1, kMidMathWarps * 32);
             const int ngr = nt / TPG;
@@ -392,7 +436,10 @@ cudaError_t launch_gemv_mid(const void* x, const void* qweight, const void* scal
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.gridDim = dim3((unsigned)(units < sms ? units : sms));
+    int blocks = units < sms ? units : sms;
+    if (blocks > kMidMaxBlocks) blocks = kMidMaxBlocks;
+    const MidStarts starts = mid_starts(units, (N / 16 + kMidMathWarps - 1) / kMidMathWarps, blocks);
+    cfg.gridDim = dim3((unsigned)blocks);
     cfg.blockDim = dim3(kMidThreads);
     cfg.dynamicSmemBytes = lay.total;
     cfg.stream = st;
@@ -415,7 +462,7 @@ cudaError_t launch_gemv_mid(const void* x, const void* qweight, const void* scal
             done[dev & 63] = true;                                                                  \
         }                                                                                           \
         e = cudaLaunchKernelEx(&cfg, gemv_mid_kernel<GG, MTT, CTT>, wmap, scmap, zmap,                   \
-                               reinterpret_cast<const __half*>(x), partial, M, N, K, lay, status_word); \
+                               reinterpret_cast<const __half*>(x), partial, M, N, K, lay, starts, status_word); \
         if (e != cudaSuccess) return e;                                                             \
     } while (0)
 #define AWQ_MID_PICK(GG)                                                                            \
