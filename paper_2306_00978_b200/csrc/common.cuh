@@ -81,6 +81,36 @@ cudaError_t launch_gemv_mid(const void* x, const void* qweight, const void* scal
                             int M, int N, int K, int group, void* workspace, unsigned int* status_word, int sms,
                             bool serialize, cudaStream_t st);
 
+// The chunked kernels (gemv_mid.cu, gemm_skinny.cu): first unit of every block (and the end of the
+// last one); units are in chunk-major order, `per_chunk` of them per chunk of K.  Blocks start in index order, the last
+// ones on the SMs that the launch in front of this one frees last, so the blocks that hold one unit
+// more than the others are the first ones - except where the longer range would cross into the next
+// chunk, which costs a second slice of x (measured on 28672 -> 8192 at 8 tokens: 6 units 22.4 us, 7
+// units 25 us, 7 units and a crossing 28 us; with the longer ranges simply in front 28672 -> 8192 went
+// 32.3 -> 34.3 us while 8192 -> 28672 went 31.0 -> 28.7 us).
+constexpr int kUnitMaxBlocks = 256;
+struct UnitStarts {
+    int v[kUnitMaxBlocks + 1];
+};
+inline UnitStarts unit_starts(int units, int per_chunk, int blocks) {
+    UnitStarts s;
+    int size[kUnitMaxBlocks];
+    const int q = units / blocks;
+    int extra = units - q * blocks, pos = 0;
+    for (int b = 0; b < blocks; ++b) {
+        const bool crosses = q > 0 && pos / per_chunk != (pos + q) / per_chunk;      // with q + 1 units
+        size[b] = q + ((extra > 0 && !crosses) ? 1 : 0);
+        extra -= size[b] - q;
+        pos += size[b];
+    }
+    for (int b = blocks - 1; b >= 0 && extra > 0; --b)                  // what could not be placed so
+        if (size[b] == q) { ++size[b]; --extra; }
+    s.v[0] = 0;
+    for (int b = 0; b < blocks; ++b) s.v[b + 1] = s.v[b] + size[b];
+    for (int b = blocks + 1; b <= kUnitMaxBlocks; ++b) s.v[b] = s.v[blocks];
+    return s;
+}
+
 // y[m][n] = fp16(sum over the chunks, ascending, of partial[c][m][n]), mn = M * N a multiple of 4;
 // launched with programmatic stream serialization behind the kernel that wrote the partial sums
 cudaError_t launch_chunk_reduce(const float* partial, void* y, int chunks, size_t mn, cudaStream_t st);

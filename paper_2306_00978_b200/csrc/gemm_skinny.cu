@@ -69,7 +69,8 @@ template <int G, int BN>
 __global__ void __launch_bounds__(kSkThreads, 1)
 gemm_skinny_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ CUtensorMap w_map,
                    const __grid_constant__ CUtensorMap sc_map, const __grid_constant__ CUtensorMap z_map,
-                   float* __restrict__ partial, int M, int N, int K, int CK, unsigned int* status_word) {
+                   float* __restrict__ partial, int M, int N, int K, int CK,
+                   const __grid_constant__ UnitStarts starts, unsigned int* status_word) {
     constexpr int S = SkCfg<BN>::kStages, R = kSkRing, A0 = SkCfg<BN>::kAColumn0;
     constexpr int GS = S / 2;                        // the A slots are released in two groups per turn of the ring
     constexpr int KPG = G / kBK;                     // k-blocks per group
@@ -104,11 +105,8 @@ gemm_skinny_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_const
     const int nslabs = N / 128, nkb = K / kBK;
     const int nchunks = (nkb + CK - 1) / CK;
     const int units = nchunks * nslabs;
-    // the blocks with one unit more are the first ones: blocks start in index order, the last ones on
-    // the SMs that the launch in front of this one frees last
-    const int uq = units / (int)gridDim.x, ur = units - uq * (int)gridDim.x;
-    const int u0 = uq * (int)blockIdx.x + min((int)blockIdx.x, ur);
-    const int u1 = u0 + uq + ((int)blockIdx.x < ur ? 1 : 0);
+    const int u0 = starts.v[blockIdx.x], u1 = starts.v[blockIdx.x + 1];
+    (void)units;
     // unit u = chunk * nslabs + slab; a chunk has nt k-blocks = nt / 2 stages (K is a multiple of 128)
     auto chunk_of = [&](int u) { return u / nslabs; };
     auto tiles_of = [&](int c) { return min(CK, nkb - c * CK); };
@@ -454,7 +452,10 @@ cudaError_t launch_gemm_skinny(const void* x, const void* qweight, const void* s
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.gridDim = dim3((unsigned)(units < sms ? units : sms));
+    int blocks = units < sms ? units : sms;
+    if (blocks > kUnitMaxBlocks) blocks = kUnitMaxBlocks;
+    const UnitStarts starts = unit_starts(units, N / 128, blocks);
+    cfg.gridDim = dim3((unsigned)blocks);
     cfg.blockDim = dim3(kSkThreads);
     cfg.dynamicSmemBytes = kSkSmem;
     cfg.stream = st;
@@ -473,7 +474,7 @@ cudaError_t launch_gemm_skinny(const void* x, const void* qweight, const void* s
             done[dev & 63] = true;                                                                  \
         }                                                                                           \
         e = cudaLaunchKernelEx(&cfg, gemm_skinny_kernel<GG, BNN>, xmap, wmap, scmap, zmap,          \
-                               partial, M, N, K, ck, status_word);                                  \
+                               partial, M, N, K, ck, starts, status_word);                          \
         if (e != cudaSuccess) return e;                                                             \
     } while (0)
 #define AWQ_SK_PICK(GG)                                                                             \

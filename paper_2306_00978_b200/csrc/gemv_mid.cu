@@ -87,42 +87,13 @@ inline MidLayout mid_layout(int M, int group, int chunk_tiles = kMidChunkTiles) 
     return l;
 }
 
-// First unit of every block (and the end of the last one).  Blocks start in index order, the last
-// ones on the SMs that the launch in front of this one frees last, so the blocks that hold one unit
-// more than the others are the first ones - except where the longer range would cross into the next
-// chunk, which costs a second slice of x (measured on 28672 -> 8192 at 8 tokens: 6 units 22.4 us, 7
-// units 25 us, 7 units and a crossing 28 us; with the longer ranges simply in front 28672 -> 8192 went
-// 32.3 -> 34.3 us while 8192 -> 28672 went 31.0 -> 28.7 us).
-constexpr int kMidMaxBlocks = 256;
-struct MidStarts {
-    int v[kMidMaxBlocks + 1];
-};
-inline MidStarts mid_starts(int units, int nbg, int blocks) {
-    MidStarts s;
-    int size[kMidMaxBlocks];
-    const int q = units / blocks;
-    int extra = units - q * blocks, pos = 0;
-    for (int b = 0; b < blocks; ++b) {
-        const bool crosses = q > 0 && pos / nbg != (pos + q) / nbg;      // with q + 1 units
-        size[b] = q + ((extra > 0 && !crosses) ? 1 : 0);
-        extra -= size[b] - q;
-        pos += size[b];
-    }
-    for (int b = blocks - 1; b >= 0 && extra > 0; --b)                  // what could not be placed so
-        if (size[b] == q) { ++size[b]; --extra; }
-    s.v[0] = 0;
-    for (int b = 0; b < blocks; ++b) s.v[b + 1] = s.v[b] + size[b];
-    for (int b = blocks + 1; b <= kMidMaxBlocks; ++b) s.v[b] = s.v[blocks];
-    return s;
-}
-
 // MT = 8-token B fragments per product (tokens rounded up to 8 MT); CT = k-tiles per chunk.
 template <int G, int MT, int CT>
 __global__ void __launch_bounds__(kMidThreads, 1)
 gemv_mid_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant__ CUtensorMap sc_map,
                 const __grid_constant__ CUtensorMap z_map, const __half* __restrict__ x,
                 float* __restrict__ partial, int M, int N, int K, const MidLayout lay,
-                const __grid_constant__ MidStarts starts, unsigned int* status_word) {
+                const __grid_constant__ UnitStarts starts, unsigned int* status_word) {
     extern __shared__ __align__(1024) unsigned char smem[];
     __shared__ unsigned int s_abort;
     constexpr int TPG = G / 64;                          // k-tiles per group
@@ -437,8 +408,8 @@ cudaError_t launch_gemv_mid(const void* x, const void* qweight, const void* scal
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     int blocks = units < sms ? units : sms;
-    if (blocks > kMidMaxBlocks) blocks = kMidMaxBlocks;
-    const MidStarts starts = mid_starts(units, (N / 16 + kMidMathWarps - 1) / kMidMathWarps, blocks);
+    if (blocks > kUnitMaxBlocks) blocks = kUnitMaxBlocks;
+    const UnitStarts starts = unit_starts(units, (N / 16 + kMidMathWarps - 1) / kMidMathWarps, blocks);
     cfg.gridDim = dim3((unsigned)blocks);
     cfg.blockDim = dim3(kMidThreads);
     cfg.dynamicSmemBytes = lay.total;
