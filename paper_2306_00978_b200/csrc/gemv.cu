@@ -595,7 +595,7 @@ gemv_band_kernel(const BandProblems probs, const __half* __restrict__ x, int M, 
         // over each group (G / 8 lanes) into the table (times 2^-24: the products carry that
         // factor).  Nobody else reads these columns, so a warp-level barrier is enough.
         constexpr int LPG = G / 8;                              // lanes per group
-        constexpr int MT = ONE ? 1 : 4;
+        constexpr int MT = ONE ? 1 : 2;                         // the resident form is taken for M <= 2 only
         unsigned char* xb = smem + lay.xsum_off;
         float* xg = reinterpret_cast<float*>(smem + lay.xg_off);
         for (int j0 = 0; j0 < upb; j0 += JB) {
@@ -637,11 +637,7 @@ gemv_band_kernel(const BandProblems probs, const __half* __restrict__ x, int M, 
                 }
                 if (valid && (lane & (LPG - 1)) == 0) {
                     float4 o = make_float4(sum[0] * (1.0f / 16777216.0f), 0.0f, 0.0f, 0.0f);
-                    if constexpr (!ONE) {
-                        o.y = sum[1] * (1.0f / 16777216.0f);
-                        o.z = sum[2] * (1.0f / 16777216.0f);
-                        o.w = sum[3] * (1.0f / 16777216.0f);
-                    }
+                    if constexpr (!ONE) o.y = sum[1] * (1.0f / 16777216.0f);
                     *reinterpret_cast<float4*>(xg + (col / G) * 4) = o;
                 }
             }
