@@ -71,7 +71,7 @@ typedef enum AwqPath {
     AWQ_PATH_AUTO = 0,          /* what awq_linear does: the matrix-vector kernels for M <= 8; the
                                    chunked matrix-vector kernel for 9 <= M <= 16 (up to 24 where
                                    N * K >= 2^25), and where K > 4096 already from 3 tokens
-                                   (N * K >= 2^26) or 5 tokens (N * K >= 2^25), and the chunked
+                                   (N * K >= 2^26; from 2 where K >= 12288) or 5 tokens (N * K >= 2^25), and the chunked
                                    tensor-core kernel for the other M <= 64 (N a multiple of 128), if
                                    a workspace of awq_workspace_bytes is registered; else the
                                    tensor-core prefill kernels */

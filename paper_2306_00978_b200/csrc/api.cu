@@ -181,7 +181,8 @@ int awq_search_clip(const void* W, const float* act_mean_abs, float alpha, int g
 // (4096 -> 11008 at 8 tokens: 11.7 / 9.8; 4096 -> 4096: 6.5 / 6.9).
 static bool mid_kernel_preferred(int M, int N, int K) {
     const long long nk = (long long)N * K;
-    if (M <= 2) return false;
+    if (M < 2) return false;
+    if (M == 2) return K >= 12288 && nk >= (1LL << 26);   // 13824 -> 5120: 13.6 / 14.2 us, 28672 -> 8192: 32.3 / 33.5 us
     if (M <= 8) return K > 4096 && nk >= (M <= 4 ? (1LL << 26) : (1LL << 25));
     if (M <= 16) return true;
     return M <= 24 && nk >= (1LL << 25);
