@@ -158,27 +158,28 @@ int awq_channel_scale(const float* act_mean_abs, float alpha, float* s, int K, v
  *   y[m][n] = sum_g Delta[g][n] * sum_{k in g} (q[n][k] - z[g][n]) * x[m][k],  stored as fp16.
  * x must already be divided by s (the paper folds diag(s)^-1 into the previous operator).
  * x: in, fp16 [M][K].  y: out, fp16 [M][N], fully overwritten; must not alias an input.
- * M <= 8 runs a matrix-vector kernel (HBM-bound; the 4-bit codes enter warp-level tensor-core
- * products exactly, accumulation, zero point and Delta in fp32, one rounding to fp16 at the
- * end), and so does 8 < M <= 16 (<= 24 where N * K >= 2^25) when the registered workspace holds
- * awq_workspace_bytes (the chunked kernel, AWQ_PATH_GEMV_MID: same arithmetic, partial sums per
- * chunk of 1024 input channels added in a fixed order by a second small kernel); everything else the tcgen05 kernel
- * ((q - z) * Delta rounded once to fp16, fp32 accumulation in tensor memory).  Results are
+ * Which kernel runs is listed under AWQ_PATH_AUTO.  The matrix-vector kernels (M <= 8, and the
+ * chunked one up to 24 tokens) are HBM-bound: the 4-bit codes enter warp-level tensor-core products
+ * exactly, accumulation, zero point and Delta are fp32, one rounding to fp16 at the end.  The
+ * tcgen05 kernels (the chunked one up to 64 tokens, the prefill kernels above) round
+ * (q - z) * Delta once to fp16 and accumulate in fp32 in tensor memory.  Results are
  * bit-reproducible.
- * The split-K matrix-vector kernel (used when N is small or M > 8) combines partial sums in a
- * fixed order through the registered workspace; calls that use the workspace must not
+ * Workspace.  The split-K matrix-vector kernel (small N, M <= 16) needs the registered workspace;
+ * the chunked kernels (partial sums per chunk of K, added in ascending order by a second small
+ * kernel) and the prefill kernels' split-K / stream-K use it when it holds awq_workspace_bytes,
+ * else awq_linear falls back to a kernel that needs none.  Calls that use the workspace must not
  * overlap on the GPU (issue them on one stream).
  * Stream order.  x and y follow plain stream order.  The packed arrays are treated as constants
- * of the layer: the band matrix-vector kernel (M <= 8, N / 16 not far below the SM count) is
- * launched with programmatic stream serialization and starts copying qweight, scales and zeros
- * into shared memory BEFORE the work in front of it in the stream has completed; only its reads
- * of x and its writes of y wait for that work.  The library covers its own writers: the first
+ * of the layer: the band and chunked kernels are launched with programmatic stream serialization
+ * and start copying qweight, scales and zeros into shared memory BEFORE the work in front of them
+ * in the stream has completed; only their reads of x and their writes of y and of the workspace
+ * wait for that work.  The library covers its own writers: the first
  * layer call after an awq_quantize_pack / awq_quantize_pack_ex on the same device is launched
  * fully serialized.  A caller who produces packed arrays by other means (its own kernel, a
  * copy) must make sure they are complete before the operation that directly precedes
  * awq_linear in the stream begins - a stream or event synchronization, or any other kernel in
  * between that does not itself signal programmatic launch completion early, is enough.
- * Errors: AWQ_ERR_NO_WORKSPACE if M <= 8, that kernel is chosen and
+ * Errors: AWQ_ERR_NO_WORKSPACE if the split-K matrix-vector kernel is chosen (M <= 8, small N) and
  * awq_workspace_bytes(M,N,K,group) exceeds the registered size; shape / pointer errors as listed
  * in AwqStatus.
  */
@@ -322,14 +323,20 @@ int awq_search_alpha(const void* W, const float* act_mean_abs, const void* X, in
 
 /* Workspace (scratch for partial sums and arrival counters).
  * awq_workspace_bytes: bytes awq_linear can use for this problem (0 if none).  For M <= 16 the
- * split-K matrix-vector kernel REQUIRES them.  Where the SM-pair tensor-core kernel runs (see AWQ_PATH_GEMM) they are
- * OPTIONAL: with a workspace of at least this size the tensor-core kernel cuts the tiles' K loops
- * into equal ranges over all SM pairs (stream-K) and sums split tiles in a fixed order through the
- * workspace; without one, or with a smaller one, whole tiles go round-robin (same result up to
- * fp32 summation order, slower when the tile count is not a multiple of the pair count).
- * For M <= 128 they are OPTIONAL as well: with them the tensor-core kernel splits each tile's K
- * loop over several SMs (up to 16 splits, fp32 partial sums added in split order by whichever SM
- * finishes a tile last), which is what keeps all SMs busy when N / 128 is below the SM count.
+ * split-K matrix-vector kernel (small N) REQUIRES them.  For everything else they are OPTIONAL and
+ * decide which kernel awq_linear takes:
+ *  - the chunked kernels (AWQ_PATH_GEMV_MID up to 24 tokens, AWQ_PATH_GEMM_SKINNY up to 64) keep one
+ *    fp32 [M][N] array of partial sums per chunk of K there; a second small kernel adds the chunks
+ *    in ascending order.  Without a workspace of this size awq_linear takes the band
+ *    matrix-vector kernel (M <= 8) or the prefill kernels instead (same result within the
+ *    tolerance, slower);
+ *  - the one-SM prefill kernel (M <= 128) splits each tile's K loop over several SMs (up to 16
+ *    splits, fp32 partial sums added in split order by whichever SM finishes a tile last), which
+ *    keeps all SMs busy when N / 128 is below the SM count;
+ *  - the SM-pair prefill kernel (see AWQ_PATH_GEMM) cuts the tiles' K loops into equal ranges over
+ *    all SM pairs (stream-K) and sums split tiles in a fixed order; without a workspace whole tiles
+ *    go round-robin (same result up to fp32 summation order, slower when the tile count is not a
+ *    multiple of the pair count).
  * awq_set_workspace: registers caller-owned device memory for the current device; the first
  * 4096 bytes are cleared with a synchronous cudaMemset.  Pass (NULL, 0) to unregister.
  * The memory must stay valid until it is unregistered or replaced. */
